@@ -1,0 +1,127 @@
+/* saf.h - C ABI of the B200 (sm_100a) hybrid causal attention layer of Selective Attention Freezing.
+ *
+ * One layer call runs ordinary query-key softmax heads and "frozen" heads side by side.
+ *   ordinary head (Appendix A, Eq. "standard-head"):  S = Q K^T * scale, A = softmax_causal(S), O = A V
+ *   frozen head   (Sec. 3.1; Sec. 3.2, Eq. "compact-prior"):  O = P^ V with
+ *        P^(i,j) = exp(alpha(j) + rho(i-j)) / Z(i)  for j <= i,  0 for j > i,
+ *        Z(i)    = sum_{k<=i} exp(alpha(k) + rho(i-k)),
+ *     rebuilt tile by tile from the two length-Tp vectors; the T x T pattern is never stored.
+ *   backward      (Sec. 3.3; Appendix E.2): frozen heads give dV = P^T dO and no query/key gradient
+ *     (their dQ/dK slots are written with zeros); ordinary heads give dQ, dK, dV.
+ * Indices are 0-based: alpha[j] for key j in [0,T), rho[d] for distance d = i-j in [0,T).
+ *
+ * Conventions (all entry points):
+ *   - "dev" pointers are device pointers owned by the caller; "host" pointers are host pointers.
+ *     The library never frees or reallocates caller memory.
+ *   - Q, K, V, O, dO are bf16 tensors indexed [b][h][t][c] through element strides (c has stride 1);
+ *     base addresses and strides must be multiples of 8 elements (16 bytes).
+ *   - frozen_mask_host is a host array uint8[H]; nonzero = frozen head.  It is read during the call.
+ *   - alpha, rho, logZ are fp32 [H][Tp] row-major device arrays; rows of ordinary heads are ignored.
+ *     They may be NULL when no head is frozen.  Q/K/LSE rows of frozen heads are never read.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *     The return value covers host-side validation and launch errors.  A kernel whose bounded wait
+ *     gave up reports through saf_last_device_status() after the stream has been synchronised.
+ *   - One context serves one stream at a time; contexts are not thread-safe.
+ *   - Every function returns SAF_OK (0) or one of the SAF_ERR_* codes; nothing is launched on error.
+ */
+#ifndef SAF_H_
+#define SAF_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct saf_ctx saf_ctx; /* opaque: workspace, cached work lists, device status word */
+
+enum {
+  SAF_OK = 0,
+  SAF_ERR_INVALID_ARG = 1,    /* NULL pointer, bad shape, T > Tp, misaligned pointer or stride */
+  SAF_ERR_UNSUPPORTED = 2,    /* head dimension or dtype outside the supported set */
+  SAF_ERR_CUDA = 3,           /* a CUDA runtime/driver call failed */
+  SAF_ERR_DEVICE_TIMEOUT = 4, /* a bounded wait inside a kernel gave up */
+  SAF_ERR_ARCH = 5,           /* device is not compute capability 10.x */
+  SAF_ERR_NOMEM = 6
+};
+enum { SAF_BF16 = 0, SAF_F32 = 1 };
+
+typedef struct {
+  int32_t B, H, T, D;          /* square causal attention: T queries and T keys; D in {64, 128} */
+  int32_t Tp;                  /* stored pattern length (row length of alpha/rho/logZ); T <= Tp */
+  float softmax_scale;         /* <= 0 selects 1/sqrt(D) (Appendix A) */
+  int32_t grad_dtype;          /* dtype of dQ/dK/dV: SAF_F32 or SAF_BF16 */
+  int32_t reserved;
+  int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3]; /* elements: batch, head, seq */
+} saf_problem;                 /* dO uses o_strides; O is bf16; LSE, dQ, dK, dV are contiguous */
+
+/* Library version (major*100 + minor). */
+int saf_version(void);
+const char* saf_status_string(int code);
+
+/* Create / destroy a context on CUDA device `device`.  Creation allocates a small status word and
+ * queries the device; SAF_ERR_ARCH if it is not sm_100-class. */
+int saf_create(saf_ctx** out, int device);
+int saf_destroy(saf_ctx* ctx);
+
+/* Row normalisers of the compact pattern (Sec. 3.2, Eq. "compact-prior"; Algorithm 1 stores
+ * (alpha, rho, log Z) per replaced head):
+ *   logZ_dev_out[h][i] = log sum_{k<=i} exp(alpha[h][k] + rho[h][i-k]),  i in [0,Tp), frozen h only.
+ * Row i uses alpha[0..i] and rho[0..i] only, so the result serves every T <= Tp.  alpha_dev, rho_dev,
+ * logZ_dev_out: device fp32 [H][Tp].  Call again whenever alpha or rho change. */
+int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* frozen_mask_host,
+                        const float* alpha_dev, const float* rho_dev, float* logZ_dev_out, void* stream);
+
+/* Forward of the hybrid layer (Sec. 3.3 "Fused computation"; Appendix E.2): one persistent launch.
+ *   Q, K, V : device bf16, strided as in `p`.
+ *   logZ    : device fp32 [H][Tp] from saf_pattern_prepare, or NULL to have it computed into
+ *             context-owned memory on every call (slower).
+ *   O       : device bf16, strided by p->o_strides, every head in its original slot.
+ *   LSE     : device fp32 [B][H][T]; natural-log sum of exp of the scaled causal scores for ordinary
+ *             heads, 0 for frozen heads (they have no softmax).  May be NULL if every head is frozen. */
+int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const void* K, const void* V,
+                        const uint8_t* frozen_mask_host, const float* alpha, const float* rho,
+                        const float* logZ, void* O, float* LSE, void* stream);
+
+/* Backward of the hybrid layer (Sec. 3.3; Appendix E.2).  Inputs as in the forward plus O and LSE as
+ * the forward wrote them and dO (device bf16, strided by p->o_strides).
+ *   dQ, dK, dV : device, contiguous [B][H][T][D], fp32 or bf16 per p->grad_dtype.
+ *                Frozen heads: dV = P^^T dO, dQ and dK written with zeros.
+ * dQ is accumulated with floating-point atomics across key blocks, so its low-order bits can vary
+ * from run to run.  Head dimension 64 only (SAF_ERR_UNSUPPORTED otherwise). */
+int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const void* K, const void* V,
+                        const void* O, const void* dO, const float* LSE, const uint8_t* frozen_mask_host,
+                        const float* alpha, const float* rho, const float* logZ, void* dQ, void* dK,
+                        void* dV, void* stream);
+
+/* Whole step through HOST buffers: copies the inputs to context-owned device memory, runs
+ * saf_pattern_prepare (only when `prepare` is nonzero; otherwise the normalisers of the previous
+ * call on this context are reused), the forward and - when dO_host is not NULL - the backward, and
+ * copies the results back.  Tensors are contiguous [B][H][T][D] (strides in `p` are ignored);
+ * alpha_host/rho_host are [H][Tp].  Any output pointer may be NULL to skip its copy.  Synchronous. */
+int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_host, const void* K_host,
+                              const void* V_host, const void* dO_host, const uint8_t* frozen_mask_host,
+                              const float* alpha_host, const float* rho_host, int32_t prepare, void* O_host,
+                              float* LSE_host, void* dQ_host, void* dK_host, void* dV_host);
+
+/* Device-side status of the most recent launches on this context: SAF_OK or SAF_ERR_DEVICE_TIMEOUT.
+ * Synchronises the context's device status word with the host (blocks until the stream used by the
+ * last call has drained).  `detail_out` (may be NULL) receives the raw word: site and CTA that gave up. */
+int saf_last_device_status(saf_ctx* ctx, int32_t* detail_out);
+
+/* Head scheduler (host only, no GPU needed).  Builds the per-CTA work lists the persistent kernels
+ * walk: one item per (batch, head, 128-row block); ordinary and frozen items are packed into the
+ * same grid, longest-processing-time first, with a frozen tile weighted `frozen_weight_pct` percent
+ * of an ordinary one.  `backward` = 0: block is a query block and costs (block+1) key tiles;
+ * 1: block is a key block and costs (nblocks-block) query tiles.
+ *   items_out   : host int32[n_items*4] = (b, h, block, kind) with kind 0 ordinary / 1 frozen,
+ *                 grouped by CTA; n_items = B*H*ceil(T/128)
+ *   offsets_out : host int32[n_ctas+1], CSR offsets into items_out
+ * Returns SAF_OK or SAF_ERR_INVALID_ARG. */
+int saf_build_worklist(int32_t B, int32_t H, int32_t T, const uint8_t* frozen_mask_host, int32_t backward,
+                       int32_t n_ctas, int32_t frozen_weight_pct, int32_t* items_out, int32_t* offsets_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAF_H_ */

@@ -1,0 +1,543 @@
+// Host side of the C ABI: argument validation, context (workspace, cached work lists, device status
+// word), TMA tensor maps, the head scheduler and the launches.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <queue>
+#include <vector>
+
+#include "../../include/saf.h"
+#include "saf_internal.h"
+
+using namespace saf;
+
+#define SAF_VERSION_NUM 100
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct WorklistEntry {
+  int B, H, T, backward, grid;
+  std::vector<uint8_t> mask;
+  WorkItem* items_dev = nullptr;
+  int* offsets_dev = nullptr;
+  int n_items = 0;
+};
+
+struct DevBuf {
+  void* ptr = nullptr;
+  size_t bytes = 0;
+};
+
+}  // namespace
+
+struct saf_ctx {
+  int device = 0;
+  int num_sms = 0;
+  int* status_dev = nullptr;
+  cudaStream_t last_stream = nullptr;
+  EncodeTiledFn encode = nullptr;
+  unsigned long long wait_limit_ns = 2000000000ull;
+  int frozen_weight_pct = 60;
+  std::vector<WorklistEntry> worklists;
+  DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf;
+  // staging for the host-buffer entry point
+  DevBuf hq, hk, hv, hdo, ho, hlse, hdq, hdk, hdv, halpha, hrho, hlogz;
+};
+
+namespace {
+
+int ensure(DevBuf& b, size_t bytes) {
+  if (b.bytes >= bytes && b.ptr) return SAF_OK;
+  if (b.ptr) cudaFree(b.ptr);
+  b.ptr = nullptr;
+  b.bytes = 0;
+  if (cudaMalloc(&b.ptr, bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return SAF_ERR_NOMEM;
+  }
+  b.bytes = bytes;
+  return SAF_OK;
+}
+void release(DevBuf& b) {
+  if (b.ptr) cudaFree(b.ptr);
+  b.ptr = nullptr;
+  b.bytes = 0;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// [B][H][T][D] bf16 tensor with element strides (batch, head, seq); box = 64 features x 128 rows,
+// 128-byte swizzle; rows beyond T read as zero.
+int make_map(saf_ctx* ctx, CUtensorMap* out, const void* base, const saf_problem* p, const int64_t* strides) {
+  cuuint64_t dims[4] = {static_cast<cuuint64_t>(p->D), static_cast<cuuint64_t>(p->T), static_cast<cuuint64_t>(p->H),
+                        static_cast<cuuint64_t>(p->B)};
+  cuuint64_t gs[3] = {static_cast<cuuint64_t>(strides[2]) * 2, static_cast<cuuint64_t>(strides[1]) * 2,
+                      static_cast<cuuint64_t>(strides[0]) * 2};
+  cuuint32_t box[4] = {64, BLK, 1, 1};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, gs, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SAF_OK : SAF_ERR_CUDA;
+}
+
+int check_strides(const int64_t* s, int D) {
+  for (int i = 0; i < 3; ++i)
+    if (s[i] <= 0 || (s[i] % 8) != 0) return SAF_ERR_INVALID_ARG;
+  if (s[2] < D) return SAF_ERR_INVALID_ARG;
+  return SAF_OK;
+}
+
+int validate(const saf_problem* p, const uint8_t* mask, int* n_frozen) {
+  if (!p || !mask) return SAF_ERR_INVALID_ARG;
+  if (p->B < 1 || p->H < 1 || p->T < 1 || p->Tp < 1) return SAF_ERR_INVALID_ARG;
+  if (p->T > p->Tp) return SAF_ERR_INVALID_ARG;
+  if (p->D != 64 && p->D != 128) return SAF_ERR_UNSUPPORTED;
+  if (p->grad_dtype != SAF_F32 && p->grad_dtype != SAF_BF16) return SAF_ERR_UNSUPPORTED;
+  int nf = 0;
+  for (int h = 0; h < p->H; ++h) nf += mask[h] ? 1 : 0;
+  *n_frozen = nf;
+  return SAF_OK;
+}
+
+int upload_mask(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st) {
+  int rc = ensure(ctx->mask_buf, std::max(H, 256));
+  if (rc) return rc;
+  // pageable source: the copy is staged before the call returns, so the caller's array may change
+  if (cudaMemcpyAsync(ctx->mask_buf.ptr, mask, H, cudaMemcpyHostToDevice, st) != cudaSuccess) return SAF_ERR_CUDA;
+  return SAF_OK;
+}
+
+void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward, int n_ctas, int frozen_pct,
+                         std::vector<WorkItem>& items, std::vector<int>& offsets) {
+  const int nblk = (T + BLK - 1) / BLK;
+  struct Cand { WorkItem w; long long cost; };
+  std::vector<Cand> cand;
+  cand.reserve(static_cast<size_t>(B) * H * nblk);
+  for (int b = 0; b < B; ++b)
+    for (int h = 0; h < H; ++h)
+      for (int k = 0; k < nblk; ++k) {
+        const int kind = mask[h] ? KIND_FROZEN : KIND_ORDINARY;
+        const long long tiles = backward ? (nblk - k) : (k + 1);
+        const long long cost = tiles * (kind == KIND_FROZEN ? frozen_pct : 100) + 20;   // + fixed per-item overhead
+        cand.push_back({{b, h, k, kind}, cost});
+      }
+  std::stable_sort(cand.begin(), cand.end(), [](const Cand& a, const Cand& b) { return a.cost > b.cost; });
+  // longest processing time first onto the least loaded CTA
+  typedef std::pair<long long, int> Load;   // (load, cta)
+  std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+  for (int c = 0; c < n_ctas; ++c) heap.push({0, c});
+  std::vector<std::vector<WorkItem>> per(n_ctas);
+  for (const Cand& c : cand) {
+    Load l = heap.top();
+    heap.pop();
+    per[l.second].push_back(c.w);
+    heap.push({l.first + c.cost, l.second});
+  }
+  items.clear();
+  offsets.assign(n_ctas + 1, 0);
+  for (int c = 0; c < n_ctas; ++c) {
+    offsets[c] = static_cast<int>(items.size());
+    items.insert(items.end(), per[c].begin(), per[c].end());
+  }
+  offsets[n_ctas] = static_cast<int>(items.size());
+}
+
+int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int backward, int grid, cudaStream_t st,
+                 const WorklistEntry** out) {
+  for (const WorklistEntry& e : ctx->worklists)
+    if (e.B == B && e.H == H && e.T == T && e.backward == backward && e.grid == grid &&
+        std::memcmp(e.mask.data(), mask, H) == 0) {
+      *out = &e;
+      return SAF_OK;
+    }
+  if (ctx->worklists.size() >= 32) {   // bounded cache: drop the oldest
+    cudaStreamSynchronize(st);
+    cudaFree(ctx->worklists.front().items_dev);
+    cudaFree(ctx->worklists.front().offsets_dev);
+    ctx->worklists.erase(ctx->worklists.begin());
+  }
+  std::vector<WorkItem> items;
+  std::vector<int> offsets;
+  build_worklist_host(B, H, T, mask, backward, grid, ctx->frozen_weight_pct, items, offsets);
+  WorklistEntry e;
+  e.B = B; e.H = H; e.T = T; e.backward = backward; e.grid = grid;
+  e.mask.assign(mask, mask + H);
+  e.n_items = static_cast<int>(items.size());
+  if (cudaMalloc(&e.items_dev, items.size() * sizeof(WorkItem)) != cudaSuccess) return SAF_ERR_NOMEM;
+  if (cudaMalloc(&e.offsets_dev, offsets.size() * sizeof(int)) != cudaSuccess) {
+    cudaFree(e.items_dev);
+    return SAF_ERR_NOMEM;
+  }
+  // synchronous copies from pageable memory: the vectors die at the end of this scope
+  if (cudaMemcpy(e.items_dev, items.data(), items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(e.offsets_dev, offsets.data(), offsets.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaFree(e.items_dev);
+    cudaFree(e.offsets_dev);
+    return SAF_ERR_CUDA;
+  }
+  ctx->worklists.push_back(std::move(e));
+  *out = &ctx->worklists.back();
+  return SAF_OK;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+}  // namespace
+
+extern "C" {
+
+int saf_version(void) { return SAF_VERSION_NUM; }
+
+const char* saf_status_string(int code) {
+  switch (code) {
+    case SAF_OK: return "ok";
+    case SAF_ERR_INVALID_ARG: return "invalid argument";
+    case SAF_ERR_UNSUPPORTED: return "unsupported head dimension or dtype";
+    case SAF_ERR_CUDA: return "CUDA call failed";
+    case SAF_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel gave up";
+    case SAF_ERR_ARCH: return "device is not sm_100-class";
+    case SAF_ERR_NOMEM: return "out of device memory";
+    default: return "unknown status";
+  }
+}
+
+int saf_create(saf_ctx** out, int device) {
+  if (!out) return SAF_ERR_INVALID_ARG;
+  *out = nullptr;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
+    cudaGetLastError();
+    return SAF_ERR_CUDA;
+  }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SAF_ERR_CUDA;
+  if (prop.major != 10) return SAF_ERR_ARCH;
+  DeviceGuard g(device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  saf_ctx* ctx = new saf_ctx();
+  ctx->device = device;
+  ctx->num_sms = prop.multiProcessorCount;
+  cudaDriverEntryPointQueryResult q;
+  void* fn = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) {
+    delete ctx;
+    return SAF_ERR_CUDA;
+  }
+  ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (cudaMalloc(&ctx->status_dev, sizeof(int)) != cudaSuccess || cudaMemset(ctx->status_dev, 0, sizeof(int)) != cudaSuccess) {
+    delete ctx;
+    return SAF_ERR_NOMEM;
+  }
+  if (const char* e = std::getenv("SAF_WAIT_LIMIT_MS")) {
+    long v = std::atol(e);
+    if (v > 0) ctx->wait_limit_ns = static_cast<unsigned long long>(v) * 1000000ull;
+  }
+  if (const char* e = std::getenv("SAF_FROZEN_WEIGHT_PCT")) {
+    long v = std::atol(e);
+    if (v > 0 && v <= 400) ctx->frozen_weight_pct = static_cast<int>(v);
+  }
+  *out = ctx;
+  return SAF_OK;
+}
+
+int saf_destroy(saf_ctx* ctx) {
+  if (!ctx) return SAF_OK;
+  DeviceGuard g(ctx->device);
+  cudaDeviceSynchronize();
+  for (WorklistEntry& e : ctx->worklists) {
+    cudaFree(e.items_dev);
+    cudaFree(e.offsets_dev);
+  }
+  DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->hq, &ctx->hk, &ctx->hv,
+                    &ctx->hdo, &ctx->ho, &ctx->hlse, &ctx->hdq, &ctx->hdk, &ctx->hdv, &ctx->halpha, &ctx->hrho,
+                    &ctx->hlogz};
+  for (DevBuf* b : bufs) release(*b);
+  if (ctx->status_dev) cudaFree(ctx->status_dev);
+  delete ctx;
+  return SAF_OK;
+}
+
+int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* frozen_mask_host, const float* alpha_dev,
+                        const float* rho_dev, float* logZ_dev_out, void* stream) {
+  if (!ctx || !frozen_mask_host || H < 1 || Tp < 1) return SAF_ERR_INVALID_ARG;
+  int nf = 0;
+  for (int h = 0; h < H; ++h) nf += frozen_mask_host[h] ? 1 : 0;
+  if (nf == 0) return SAF_OK;
+  if (!alpha_dev || !rho_dev || !logZ_dev_out) return SAF_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = upload_mask(ctx, frozen_mask_host, H, st);
+  if (rc) return rc;
+  ctx->last_stream = st;
+  if (launch_logz(alpha_dev, rho_dev, logZ_dev_out, static_cast<const uint8_t*>(ctx->mask_buf.ptr), H, Tp, st) !=
+      cudaSuccess)
+    return SAF_ERR_CUDA;
+  return SAF_OK;
+}
+
+int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const void* K, const void* V,
+                        const uint8_t* frozen_mask_host, const float* alpha, const float* rho, const float* logZ,
+                        void* O, float* LSE, void* stream) {
+  if (!ctx) return SAF_ERR_INVALID_ARG;
+  int nf = 0;
+  int rc = validate(p, frozen_mask_host, &nf);
+  if (rc) return rc;
+  const int no = p->H - nf;
+  if (!V || !O) return SAF_ERR_INVALID_ARG;
+  if (no > 0 && (!Q || !K || !LSE)) return SAF_ERR_INVALID_ARG;
+  if (nf > 0 && (!alpha || !rho)) return SAF_ERR_INVALID_ARG;
+  if (!aligned16(V) || !aligned16(O) || (no > 0 && (!aligned16(Q) || !aligned16(K)))) return SAF_ERR_INVALID_ARG;
+  if (check_strides(p->v_strides, p->D) || check_strides(p->o_strides, p->D)) return SAF_ERR_INVALID_ARG;
+  if (no > 0 && (check_strides(p->q_strides, p->D) || check_strides(p->k_strides, p->D))) return SAF_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ctx->last_stream = st;
+
+  if (nf > 0 && !logZ) {
+    rc = ensure(ctx->logz_buf, static_cast<size_t>(p->H) * p->Tp * sizeof(float));
+    if (rc) return rc;
+    rc = saf_pattern_prepare(ctx, p->H, p->Tp, frozen_mask_host, alpha, rho, static_cast<float*>(ctx->logz_buf.ptr),
+                             stream);
+    if (rc) return rc;
+    logZ = static_cast<const float*>(ctx->logz_buf.ptr);
+  }
+  const int nblk = (p->T + BLK - 1) / BLK;
+  const long long n_items = static_cast<long long>(p->B) * p->H * nblk;
+  const int grid = static_cast<int>(std::min<long long>(2LL * ctx->num_sms, n_items));
+  const WorklistEntry* wl = nullptr;
+  rc = get_worklist(ctx, p->B, p->H, p->T, frozen_mask_host, 0, grid, st, &wl);
+  if (rc) return rc;
+
+  CUtensorMap mq, mk, mv;
+  // frozen-only layers never touch Q/K: any valid map will do
+  rc = make_map(ctx, &mv, V, p, p->v_strides);
+  if (rc) return rc;
+  if (no > 0) {
+    rc = make_map(ctx, &mq, Q, p, p->q_strides);
+    if (rc) return rc;
+    rc = make_map(ctx, &mk, K, p, p->k_strides);
+    if (rc) return rc;
+  } else {
+    mq = mv;
+    mk = mv;
+  }
+  FwdParams fp;
+  fp.B = p->B; fp.H = p->H; fp.T = p->T; fp.Tp = p->Tp;
+  const float scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
+  fp.scale_log2 = scale * 1.4426950408889634f;
+  fp.alpha = alpha; fp.rho = rho; fp.logZ = logZ;
+  fp.O = O;
+  for (int i = 0; i < 3; ++i) fp.o_strides[i] = p->o_strides[i];
+  fp.LSE = LSE;
+  fp.items = wl->items_dev;
+  fp.cta_offsets = wl->offsets_dev;
+  fp.status = ctx->status_dev;
+  fp.wait_limit_ns = ctx->wait_limit_ns;
+  if (launch_fwd(p->D, mq, mk, mv, fp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+  return SAF_OK;
+}
+
+int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const void* K, const void* V,
+                        const void* O, const void* dO, const float* LSE, const uint8_t* frozen_mask_host,
+                        const float* alpha, const float* rho, const float* logZ, void* dQ, void* dK, void* dV,
+                        void* stream) {
+  if (!ctx) return SAF_ERR_INVALID_ARG;
+  int nf = 0;
+  int rc = validate(p, frozen_mask_host, &nf);
+  if (rc) return rc;
+  if (p->D != 64) return SAF_ERR_UNSUPPORTED;
+  const int no = p->H - nf;
+  if (!dO || !dQ || !dK || !dV) return SAF_ERR_INVALID_ARG;
+  if (no > 0 && (!Q || !K || !V || !O || !LSE)) return SAF_ERR_INVALID_ARG;
+  if (nf > 0 && (!alpha || !rho)) return SAF_ERR_INVALID_ARG;
+  if (!aligned16(dO) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV)) return SAF_ERR_INVALID_ARG;
+  if (no > 0 && (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O))) return SAF_ERR_INVALID_ARG;
+  if (check_strides(p->o_strides, p->D)) return SAF_ERR_INVALID_ARG;
+  if (no > 0 && (check_strides(p->q_strides, p->D) || check_strides(p->k_strides, p->D) ||
+                 check_strides(p->v_strides, p->D)))
+    return SAF_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ctx->last_stream = st;
+
+  if (nf > 0 && !logZ) {
+    rc = ensure(ctx->logz_buf, static_cast<size_t>(p->H) * p->Tp * sizeof(float));
+    if (rc) return rc;
+    rc = saf_pattern_prepare(ctx, p->H, p->Tp, frozen_mask_host, alpha, rho, static_cast<float*>(ctx->logz_buf.ptr),
+                             stream);
+    if (rc) return rc;
+    logZ = static_cast<const float*>(ctx->logz_buf.ptr);
+  }
+  rc = upload_mask(ctx, frozen_mask_host, p->H, st);
+  if (rc) return rc;
+
+  const int nblk = (p->T + BLK - 1) / BLK;
+  const int Tpad = nblk * BLK;
+  const size_t nelem = static_cast<size_t>(p->B) * p->H * p->T * p->D;
+  rc = ensure(ctx->delta_buf, static_cast<size_t>(p->B) * p->H * Tpad * sizeof(float));
+  if (rc) return rc;
+  const int grad_f32 = p->grad_dtype == SAF_F32;
+  float* dqacc = static_cast<float*>(dQ);
+  if (!grad_f32) {
+    rc = ensure(ctx->dqacc_buf, nelem * sizeof(float));
+    if (rc) return rc;
+    dqacc = static_cast<float*>(ctx->dqacc_buf.ptr);
+  }
+  // O is only read for ordinary heads; a frozen-only layer may pass O = NULL
+  if (launch_bwd_prep(O, dO, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr),
+                      static_cast<float*>(ctx->delta_buf.ptr), Tpad, dqacc, dK, grad_f32, p->B, p->H, p->T, p->D,
+                      st) != cudaSuccess)
+    return SAF_ERR_CUDA;
+
+  const long long n_items = static_cast<long long>(p->B) * p->H * nblk;
+  const int grid = static_cast<int>(std::min<long long>(ctx->num_sms, n_items));
+  const WorklistEntry* wl = nullptr;
+  rc = get_worklist(ctx, p->B, p->H, p->T, frozen_mask_host, 1, grid, st, &wl);
+  if (rc) return rc;
+
+  CUtensorMap mq, mk, mv, mdo;
+  rc = make_map(ctx, &mdo, dO, p, p->o_strides);
+  if (rc) return rc;
+  if (no > 0) {
+    if ((rc = make_map(ctx, &mq, Q, p, p->q_strides))) return rc;
+    if ((rc = make_map(ctx, &mk, K, p, p->k_strides))) return rc;
+    if ((rc = make_map(ctx, &mv, V, p, p->v_strides))) return rc;
+  } else {
+    mq = mdo; mk = mdo; mv = mdo;
+  }
+  BwdParams bp;
+  bp.B = p->B; bp.H = p->H; bp.T = p->T; bp.Tp = p->Tp;
+  bp.scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
+  bp.scale_log2 = bp.scale * 1.4426950408889634f;
+  bp.alpha = alpha; bp.rho = rho; bp.logZ = logZ;
+  bp.LSE = LSE;
+  bp.delta = static_cast<const float*>(ctx->delta_buf.ptr);
+  bp.Tpad = Tpad;
+  bp.dQacc = dqacc;
+  bp.dK = dK; bp.dV = dV;
+  bp.grad_f32 = grad_f32;
+  bp.items = wl->items_dev;
+  bp.cta_offsets = wl->offsets_dev;
+  bp.status = ctx->status_dev;
+  bp.wait_limit_ns = ctx->wait_limit_ns;
+  if (launch_bwd(p->D, mq, mk, mv, mdo, bp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+  if (!grad_f32 && launch_bwd_finalize(dqacc, dQ, nelem, st) != cudaSuccess) return SAF_ERR_CUDA;
+  return SAF_OK;
+}
+
+int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_host, const void* K_host,
+                              const void* V_host, const void* dO_host, const uint8_t* frozen_mask_host,
+                              const float* alpha_host, const float* rho_host, int32_t prepare, void* O_host,
+                              float* LSE_host, void* dQ_host, void* dK_host, void* dV_host) {
+  if (!ctx) return SAF_ERR_INVALID_ARG;
+  int nf = 0;
+  int rc = validate(p, frozen_mask_host, &nf);
+  if (rc) return rc;
+  const int no = p->H - nf;
+  if (!V_host || (no > 0 && (!Q_host || !K_host)) || (nf > 0 && (!alpha_host || !rho_host))) return SAF_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  const size_t nelem = static_cast<size_t>(p->B) * p->H * p->T * p->D;
+  const size_t tb = nelem * 2;
+  const size_t gb = nelem * (p->grad_dtype == SAF_F32 ? 4 : 2);
+  const size_t pb = static_cast<size_t>(p->H) * p->Tp * sizeof(float);
+  const size_t lb = static_cast<size_t>(p->B) * p->H * p->T * sizeof(float);
+  const bool bwd = dO_host != nullptr;
+  if ((rc = ensure(ctx->hq, tb)) || (rc = ensure(ctx->hk, tb)) || (rc = ensure(ctx->hv, tb)) ||
+      (rc = ensure(ctx->ho, tb)) || (rc = ensure(ctx->hlse, lb)) || (rc = ensure(ctx->halpha, pb)) ||
+      (rc = ensure(ctx->hrho, pb)) || (rc = ensure(ctx->hlogz, pb)))
+    return rc;
+  if (bwd && ((rc = ensure(ctx->hdo, tb)) || (rc = ensure(ctx->hdq, gb)) || (rc = ensure(ctx->hdk, gb)) ||
+              (rc = ensure(ctx->hdv, gb))))
+    return rc;
+  cudaStream_t st = nullptr;
+  saf_problem q = *p;
+  const int64_t s2 = p->D, s1 = static_cast<int64_t>(p->T) * p->D, s0 = s1 * p->H;
+  int64_t* sets[4] = {q.q_strides, q.k_strides, q.v_strides, q.o_strides};
+  for (int64_t* s : sets) { s[0] = s0; s[1] = s1; s[2] = s2; }
+  bool okc = true;
+  if (no > 0) {
+    okc &= cudaMemcpyAsync(ctx->hq.ptr, Q_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    okc &= cudaMemcpyAsync(ctx->hk.ptr, K_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  okc &= cudaMemcpyAsync(ctx->hv.ptr, V_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (bwd) okc &= cudaMemcpyAsync(ctx->hdo.ptr, dO_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (nf > 0 && prepare) {
+    okc &= cudaMemcpyAsync(ctx->halpha.ptr, alpha_host, pb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    okc &= cudaMemcpyAsync(ctx->hrho.ptr, rho_host, pb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  if (!okc) return SAF_ERR_CUDA;
+  const float* a = static_cast<const float*>(ctx->halpha.ptr);
+  const float* r = static_cast<const float*>(ctx->hrho.ptr);
+  float* z = static_cast<float*>(ctx->hlogz.ptr);
+  if (nf > 0 && prepare && (rc = saf_pattern_prepare(ctx, p->H, p->Tp, frozen_mask_host, a, r, z, st))) return rc;
+  rc = saf_hybrid_attn_fwd(ctx, &q, ctx->hq.ptr, ctx->hk.ptr, ctx->hv.ptr, frozen_mask_host, a, r, z, ctx->ho.ptr,
+                           static_cast<float*>(ctx->hlse.ptr), st);
+  if (rc) return rc;
+  if (bwd) {
+    rc = saf_hybrid_attn_bwd(ctx, &q, ctx->hq.ptr, ctx->hk.ptr, ctx->hv.ptr, ctx->ho.ptr, ctx->hdo.ptr,
+                             static_cast<const float*>(ctx->hlse.ptr), frozen_mask_host, a, r, z, ctx->hdq.ptr,
+                             ctx->hdk.ptr, ctx->hdv.ptr, st);
+    if (rc) return rc;
+  }
+  if (O_host) okc &= cudaMemcpyAsync(O_host, ctx->ho.ptr, tb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (LSE_host) okc &= cudaMemcpyAsync(LSE_host, ctx->hlse.ptr, lb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (bwd) {
+    if (dQ_host) okc &= cudaMemcpyAsync(dQ_host, ctx->hdq.ptr, gb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (dK_host) okc &= cudaMemcpyAsync(dK_host, ctx->hdk.ptr, gb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (dV_host) okc &= cudaMemcpyAsync(dV_host, ctx->hdv.ptr, gb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  }
+  if (!okc) return SAF_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SAF_ERR_CUDA;
+  return saf_last_device_status(ctx, nullptr);
+}
+
+int saf_last_device_status(saf_ctx* ctx, int32_t* detail_out) {
+  if (!ctx) return SAF_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  if (cudaStreamSynchronize(ctx->last_stream) != cudaSuccess) return SAF_ERR_CUDA;
+  int word = 0;
+  if (cudaMemcpy(&word, ctx->status_dev, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SAF_ERR_CUDA;
+  if (detail_out) *detail_out = word;
+  if (word != 0) {
+    cudaMemset(ctx->status_dev, 0, sizeof(int));
+    return SAF_ERR_DEVICE_TIMEOUT;
+  }
+  return SAF_OK;
+}
+
+int saf_build_worklist(int32_t B, int32_t H, int32_t T, const uint8_t* frozen_mask_host, int32_t backward,
+                       int32_t n_ctas, int32_t frozen_weight_pct, int32_t* items_out, int32_t* offsets_out) {
+  if (B < 1 || H < 1 || T < 1 || n_ctas < 1 || !frozen_mask_host || !items_out || !offsets_out ||
+      frozen_weight_pct < 1)
+    return SAF_ERR_INVALID_ARG;
+  std::vector<WorkItem> items;
+  std::vector<int> offsets;
+  build_worklist_host(B, H, T, frozen_mask_host, backward ? 1 : 0, n_ctas, frozen_weight_pct, items, offsets);
+  std::memcpy(items_out, items.data(), items.size() * sizeof(WorkItem));
+  std::memcpy(offsets_out, offsets.data(), offsets.size() * sizeof(int));
+  return SAF_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,436 @@
+// Forward of the hybrid causal attention layer on sm_100a: one persistent kernel for ordinary
+// (flash-style online softmax) and frozen (pattern rebuilt from alpha/rho/logZ) heads.
+//
+// Per CTA (192 threads): warps 0-3 = compute (one query row per thread = one TMEM lane),
+// warp 4 = TMA producer, warp 5 = tcgen05 issuer and TMEM owner.  Two CTAs share an SM, so one CTA's
+// softmax overlaps the other's MMAs.  TMEM columns: [0,128) S (fp32) / P (bf16 pairs in [0,64)),
+// [128,128+D) O accumulator.
+//
+// Ordinary item (b,h,I): for J = 0..I: S = Q_I K_J^T (tcgen05, operands in 128B-swizzled smem via TMA),
+//   row max / lazy rescale / exp2 / row sum in registers, P -> TMEM as bf16, O += P V_J (A from TMEM,
+//   V as MN-major B); epilogue O / l and LSE.
+// Frozen item (b,h,I): for J = 0..I: P^(i,j) = exp(alpha(j) + rho(i-j) - logZ(i)) for j <= i
+//   (Eq. "compact-prior" with the stored normaliser) generated into TMEM, O += P^ V_J.  No Q/K loads,
+//   no score MMA, no max/sum.  The exponential is factorised per tile as
+//   w(i) * a(j) * r(i-j) with a = exp(alpha - max_tile alpha), r = exp(rho - max_band rho),
+//   w = exp(max alpha + max rho - logZ(i)); a tile whose exponent range would leave fp32 falls back to
+//   one exp per element.
+#include <cuda_bf16.h>
+#include "ptx.cuh"
+#include "saf_internal.h"
+
+namespace saf {
+
+constexpr float LOG2E_F = 1.4426950408889634f;
+constexpr float LN2_F = 0.6931471805599453f;
+
+template <int D>
+struct FwdCfg {
+  static constexpr int NPANEL = D / 64;                 // 64-column bf16 panels: 128-byte rows, one swizzle atom
+  static constexpr int PANEL_BYTES = 128 * 64 * 2;      // 16 KB
+  static constexpr int TILE_BYTES = NPANEL * PANEL_BYTES;
+  static constexpr int NS = (D == 64) ? 2 : 1;          // K and V ring depth
+  static constexpr int OFF_Q = 0;
+  static constexpr int OFF_K = TILE_BYTES;
+  static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
+  static constexpr int OFF_TAB = OFF_V + NS * TILE_BYTES;
+  static constexpr int TAB_FLOATS = 128 + 256 + 128 + 256 + 16;
+  static constexpr int OFF_BAR = OFF_TAB + TAB_FLOATS * 4;
+  static constexpr int NBAR = 2 + 4 * NS + 4;
+  static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;   // + slack for 1024-byte alignment
+  static constexpr int TMEM_COLS = 256;
+  static constexpr int COL_S = 0, COL_P = 0, COL_O = 128;
+};
+
+enum FwdSite { SITE_Q_EMPTY = 1, SITE_K_EMPTY, SITE_V_EMPTY, SITE_Q_FULL, SITE_K_FULL, SITE_P_FULL, SITE_V_FULL,
+               SITE_O_FREE, SITE_S_FULL, SITE_PV_DONE };
+
+template <int D>
+__global__ void __launch_bounds__(192, 2)
+saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
+               const __grid_constant__ CUtensorMap mv, const FwdParams p) {
+  using C = FwdCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR);
+  uint64_t* q_full = bars;
+  uint64_t* q_empty = bars + 1;
+  uint64_t* k_full = bars + 2;
+  uint64_t* k_empty = k_full + C::NS;
+  uint64_t* v_full = k_empty + C::NS;
+  uint64_t* v_empty = v_full + C::NS;
+  uint64_t* s_full = v_empty + C::NS;
+  uint64_t* p_full = s_full + 1;
+  uint64_t* pv_done = p_full + 1;
+  uint64_t* o_free = pv_done + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_free + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* tab = reinterpret_cast<float*>(smem + C::OFF_TAB);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const WaitCtx wc{abort_flag, p.status, p.wait_limit_ns};
+
+  if (tid == 0) {
+    *abort_flag = 0;
+    mbar_init(q_full, 1);
+    mbar_init(q_empty, 1);
+    for (int s = 0; s < C::NS; ++s) {
+      mbar_init(k_full + s, 1);
+      mbar_init(k_empty + s, 1);
+      mbar_init(v_full + s, 1);
+      mbar_init(v_empty + s, 1);
+    }
+    mbar_init(s_full, 1);
+    mbar_init(p_full, 128);
+    mbar_init(pv_done, 1);
+    mbar_init(o_free, 128);
+    mbar_fence_init();
+  }
+  if (warp == 5) {
+    tmem_alloc(tmem_slot, C::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  const int it_begin = p.cta_offsets[blockIdx.x], it_end = p.cta_offsets[blockIdx.x + 1];
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&mq);
+      tma_prefetch_desc(&mk);
+      tma_prefetch_desc(&mv);
+      uint32_t nq = 0, nk = 0, nv = 0;
+      bool ok = true;
+      for (int it = it_begin; it < it_end && ok; ++it) {
+        const WorkItem w = p.items[it];
+        const int ntiles = w.blk + 1;
+        if (w.kind == KIND_ORDINARY) {
+          ok = mbar_wait(q_empty, (nq & 1) ^ 1, wc, SITE_Q_EMPTY);
+          if (!ok) break;
+          mbar_expect_tx(q_full, C::TILE_BYTES);
+          for (int pn = 0; pn < C::NPANEL; ++pn)
+            tma_load_4d(smem + C::OFF_Q + pn * C::PANEL_BYTES, &mq, q_full, pn * 64, w.blk * BLK, w.h, w.b);
+          ++nq;
+        }
+        for (int j = 0; j < ntiles && ok; ++j) {
+          if (w.kind == KIND_ORDINARY) {
+            const int s = nk % C::NS;
+            ok = mbar_wait(k_empty + s, ((nk / C::NS) & 1) ^ 1, wc, SITE_K_EMPTY);
+            if (!ok) break;
+            mbar_expect_tx(k_full + s, C::TILE_BYTES);
+            for (int pn = 0; pn < C::NPANEL; ++pn)
+              tma_load_4d(smem + C::OFF_K + s * C::TILE_BYTES + pn * C::PANEL_BYTES, &mk, k_full + s, pn * 64,
+                          j * BLK, w.h, w.b);
+            ++nk;
+          }
+          const int s = nv % C::NS;
+          ok = mbar_wait(v_empty + s, ((nv / C::NS) & 1) ^ 1, wc, SITE_V_EMPTY);
+          if (!ok) break;
+          mbar_expect_tx(v_full + s, C::TILE_BYTES);
+          for (int pn = 0; pn < C::NPANEL; ++pn)
+            tma_load_4d(smem + C::OFF_V + s * C::TILE_BYTES + pn * C::PANEL_BYTES, &mv, v_full + s, pn * 64,
+                        j * BLK, w.h, w.b);
+          ++nv;
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ tcgen05 issuer
+    if (lane == 0) {
+      const uint32_t sb = smem_u32(smem);
+      constexpr uint32_t idesc_s = umma_idesc_bf16(128, 128, 0, 0);
+      constexpr uint32_t idesc_o = umma_idesc_bf16(128, D, 0, 1);
+      uint32_t nq = 0, nk = 0, nv = 0, np = 0, nitem = 0;
+      bool ok = true;
+      for (int it = it_begin; it < it_end && ok; ++it, ++nitem) {
+        const WorkItem w = p.items[it];
+        const int ntiles = w.blk + 1;
+        if (w.kind == KIND_ORDINARY) {
+          ok = mbar_wait(q_full, nq & 1, wc, SITE_Q_FULL);
+          if (!ok) break;
+          ++nq;
+        }
+        for (int j = 0; j < ntiles && ok; ++j) {
+          if (w.kind == KIND_ORDINARY) {
+            const int s = nk % C::NS;
+            ok = mbar_wait(k_full + s, (nk / C::NS) & 1, wc, SITE_K_FULL);
+            if (!ok) break;
+            ++nk;
+            tc_fence_after();
+#pragma unroll
+            for (int kc = 0; kc < D / 16; ++kc) {
+              const uint32_t off = (kc >> 2) * C::PANEL_BYTES + (kc & 3) * 32;
+              umma_ss(tmem + C::COL_S, umma_smem_desc(sb + C::OFF_Q + off, 16, 1024, UMMA_LAYOUT_SW128),
+                      umma_smem_desc(sb + C::OFF_K + s * C::TILE_BYTES + off, 16, 1024, UMMA_LAYOUT_SW128), idesc_s,
+                      kc > 0);
+            }
+            umma_commit(s_full);
+            umma_commit(k_empty + s);
+            if (j == ntiles - 1) umma_commit(q_empty);
+          }
+          ok = mbar_wait(p_full, np & 1, wc, SITE_P_FULL);
+          if (!ok) break;
+          ++np;
+          const int s = nv % C::NS;
+          ok = mbar_wait(v_full + s, (nv / C::NS) & 1, wc, SITE_V_FULL);
+          if (!ok) break;
+          ++nv;
+          if (j == 0) {
+            ok = mbar_wait(o_free, (nitem & 1) ^ 1, wc, SITE_O_FREE);
+            if (!ok) break;
+          }
+          tc_fence_after();
+#pragma unroll
+          for (int kc = 0; kc < 8; ++kc)
+            umma_ts(tmem + C::COL_O, tmem + C::COL_P + 8 * kc,
+                    umma_smem_desc(sb + C::OFF_V + s * C::TILE_BYTES + kc * 2048, C::PANEL_BYTES, 1024,
+                                   UMMA_LAYOUT_SW128),
+                    idesc_o, (j > 0 || kc > 0) ? 1u : 0u);
+          umma_commit(v_empty + s);
+          umma_commit(pv_done);
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ compute warps (128 threads)
+    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    const uint32_t t_s = tmem + lane_base + C::COL_S;
+    const uint32_t t_p = tmem + lane_base + C::COL_P;
+    const uint32_t t_o = tmem + lane_base + C::COL_O;
+    float* aJ = tab;
+    float* rband = tab + 128;
+    float* a2raw = tab + 384;
+    float* r2raw = tab + 512;
+    float* red = tab + 768;
+    uint32_t ns = 0, npv = 0;
+    bool ok = true;
+    for (int it = it_begin; it < it_end && ok; ++it) {
+      const WorkItem w = p.items[it];
+      const int ntiles = w.blk + 1;
+      const int row = w.blk * BLK + tid;
+      float inv_l = 1.0f, lse = 0.0f;
+      if (w.kind == KIND_ORDINARY) {
+        float m_ref = -INFINITY, l = 0.0f;
+        const float c = p.scale_log2;
+        for (int j = 0; j < ntiles; ++j) {
+          ok = mbar_wait_warp(s_full, ns & 1, wc, SITE_S_FULL);
+          if (!ok) break;
+          ++ns;
+          if (j > 0) {
+            ok = mbar_wait_warp(pv_done, npv & 1, wc, SITE_PV_DONE);
+            if (!ok) break;
+            ++npv;
+          }
+          tc_fence_after();
+          const bool diag = (j == w.blk);
+          float mx = -INFINITY;
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) {
+            uint32_t r[32];
+            tmem_ld32(t_s + 32 * cc, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              float s = __uint_as_float(r[e]);
+              if (diag && (32 * cc + e > tid)) s = -INFINITY;
+              mx = fmaxf(mx, s);
+            }
+          }
+          const float m_new = fmaxf(m_ref, mx * c);
+          if (j == 0) {
+            m_ref = m_new;
+          } else {
+            const bool need = (m_new - m_ref) > 8.0f;
+            if (__any_sync(0xffffffffu, need)) {
+              const float f = need ? ex2_approx(m_ref - m_new) : 1.0f;
+              l *= f;
+              if (need) m_ref = m_new;
+#pragma unroll
+              for (int cc = 0; cc < D / 32; ++cc) {
+                uint32_t r[32];
+                tmem_ld32(t_o + 32 * cc, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
+                tmem_st32(t_o + 32 * cc, r);
+              }
+            }
+          }
+          const float neg_m = -m_ref;
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) {
+            uint32_t r[32];
+            tmem_ld32(t_s + 32 * cc, r);
+            tmem_wait_ld();
+            uint32_t pk[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              float s0 = __uint_as_float(r[2 * e]), s1 = __uint_as_float(r[2 * e + 1]);
+              float p0 = ex2_approx(fmaf(s0, c, neg_m)), p1 = ex2_approx(fmaf(s1, c, neg_m));
+              if (diag) {
+                if (32 * cc + 2 * e > tid) p0 = 0.0f;
+                if (32 * cc + 2 * e + 1 > tid) p1 = 0.0f;
+              }
+              l += p0 + p1;
+              pk[e] = pack_bf16x2(p0, p1);
+            }
+            tmem_st16(t_p + 16 * cc, pk);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(p_full);
+        }
+        if (!ok) break;
+        inv_l = 1.0f / l;
+        lse = (m_ref + log2f(l)) * LN2_F;
+      } else {
+        // ---------------- frozen head: generate P^ tiles
+        const float* alpha_h = p.alpha + static_cast<size_t>(w.h) * p.Tp;
+        const float* rho_h = p.rho + static_cast<size_t>(w.h) * p.Tp;
+        const float z2 = (row < p.T) ? p.logZ[static_cast<size_t>(w.h) * p.Tp + row] * LOG2E_F : INFINITY;
+        for (int j = 0; j < ntiles; ++j) {
+          // previous tile's table readers are done; the compute warps also agree here whether a
+          // wait has been abandoned, so that none of them is left alone at a later barrier
+          if (named_bar_or(1, 128, !ok)) {
+            ok = false;
+            break;
+          }
+          const int key = j * BLK + tid;
+          const float a2 = (key < p.T) ? alpha_h[key] * LOG2E_F : -INFINITY;
+          const int d0 = (w.blk - j) * BLK - 127;      // band covers distances d0 .. d0+254
+          const int da = d0 + tid, db = d0 + 128 + tid;
+          const float r2a = (da >= 0 && da < p.T) ? rho_h[da] * LOG2E_F : -INFINITY;
+          const float r2b = (tid < 127 && db >= 0 && db < p.T) ? rho_h[db] * LOG2E_F : -INFINITY;
+          float ma = a2, mr = fmaxf(r2a, r2b);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            ma = fmaxf(ma, __shfl_xor_sync(0xffffffffu, ma, o));
+            mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, o));
+          }
+          if (lane == 0) {
+            red[warp] = ma;
+            red[4 + warp] = mr;
+          }
+          a2raw[tid] = a2;
+          r2raw[tid] = r2a;
+          r2raw[128 + tid] = r2b;
+          named_bar_sync(1, 128);
+          ma = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+          mr = fmaxf(fmaxf(red[4], red[5]), fmaxf(red[6], red[7]));
+          const float ew = ma + mr - z2;               // -inf for rows beyond T
+          const bool bad = ew > 100.0f;                // factorised form would overflow / flush: use exact form
+          const unsigned anybad = __any_sync(0xffffffffu, bad);
+          if (lane == 0) red[8 + warp] = anybad ? 1.0f : 0.0f;
+          aJ[tid] = ex2_approx(a2 - ma);
+          rband[tid] = ex2_approx(r2a - mr);
+          rband[128 + tid] = ex2_approx(r2b - mr);
+          named_bar_sync(1, 128);
+          const bool exact = (red[8] + red[9] + red[10] + red[11]) > 0.0f;
+          if (j > 0) {
+            ok = mbar_wait_warp(pv_done, npv & 1, wc, SITE_PV_DONE);   // previous P^ tile consumed
+            ++npv;
+            tc_fence_after();
+          }
+          if (!exact) {
+            const float wv = ex2_approx(ew);
+            const float* rb = rband + tid + 127;       // rb[-k] = r(distance of key k in this tile)
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+              uint32_t pk[16];
+#pragma unroll
+              for (int e4 = 0; e4 < 8; ++e4) {
+                const int k0 = 32 * cc + 4 * e4;
+                const float4 a4 = *reinterpret_cast<const float4*>(aJ + k0);
+                const float p0 = wv * a4.x * rb[-k0], p1 = wv * a4.y * rb[-k0 - 1];
+                const float p2 = wv * a4.z * rb[-k0 - 2], p3 = wv * a4.w * rb[-k0 - 3];
+                pk[2 * e4] = pack_bf16x2(p0, p1);
+                pk[2 * e4 + 1] = pack_bf16x2(p2, p3);
+              }
+              tmem_st16(t_p + 16 * cc, pk);
+            }
+          } else {
+            const float* rb = r2raw + tid + 127;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+              uint32_t pk[16];
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                const int k0 = 32 * cc + 2 * e;
+                const float p0 = ex2_approx(a2raw[k0] + rb[-k0] - z2);
+                const float p1 = ex2_approx(a2raw[k0 + 1] + rb[-k0 - 1] - z2);
+                pk[e] = pack_bf16x2(p0, p1);
+              }
+              tmem_st16(t_p + 16 * cc, pk);
+            }
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(p_full);
+        }
+        if (!ok) break;
+      }
+      // ---------------- epilogue: wait for the last P V, scale, store
+      ok = mbar_wait_warp(pv_done, npv & 1, wc, SITE_PV_DONE);
+      if (!ok) break;
+      ++npv;
+      tc_fence_after();
+      __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + w.b * p.o_strides[0] + w.h * p.o_strides[1] +
+                            static_cast<int64_t>(row) * p.o_strides[2];
+#pragma unroll
+      for (int cc = 0; cc < D / 32; ++cc) {
+        uint32_t r[32];
+        tmem_ld32(t_o + 32 * cc, r);
+        tmem_wait_ld();
+        if (row < p.T) {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint4 o;
+            o.x = pack_bf16x2(__uint_as_float(r[8 * q4 + 0]) * inv_l, __uint_as_float(r[8 * q4 + 1]) * inv_l);
+            o.y = pack_bf16x2(__uint_as_float(r[8 * q4 + 2]) * inv_l, __uint_as_float(r[8 * q4 + 3]) * inv_l);
+            o.z = pack_bf16x2(__uint_as_float(r[8 * q4 + 4]) * inv_l, __uint_as_float(r[8 * q4 + 5]) * inv_l);
+            o.w = pack_bf16x2(__uint_as_float(r[8 * q4 + 6]) * inv_l, __uint_as_float(r[8 * q4 + 7]) * inv_l);
+            *reinterpret_cast<uint4*>(orow + 32 * cc + 8 * q4) = o;
+          }
+        }
+      }
+      if (p.LSE != nullptr && row < p.T)
+        p.LSE[(static_cast<size_t>(w.b) * p.H + w.h) * p.T + row] = lse;
+      tc_fence_before();
+      mbar_arrive(o_free);
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  if (*abort_flag) {
+    // A wait gave up: let copies and MMAs that are still in flight land before the CTA's
+    // shared memory and TMEM are released.
+    for (int i = 0; i < 64; ++i) __nanosleep(20000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, C::TMEM_COLS);
+}
+
+int fwd_smem_bytes(int D) { return D == 64 ? FwdCfg<64>::SMEM : FwdCfg<128>::SMEM; }
+
+cudaError_t launch_fwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                       const FwdParams& p, int grid, cudaStream_t st) {
+  cudaError_t e;
+  if (D == 64) {
+    e = cudaFuncSetAttribute(saf_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<64>::SMEM);
+    if (e != cudaSuccess) return e;
+    saf_fwd_kernel<64><<<grid, 192, FwdCfg<64>::SMEM, st>>>(mq, mk, mv, p);
+  } else {
+    e = cudaFuncSetAttribute(saf_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128>::SMEM);
+    if (e != cudaSuccess) return e;
+    saf_fwd_kernel<128><<<grid, 192, FwdCfg<128>::SMEM, st>>>(mq, mk, mv, p);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace saf
