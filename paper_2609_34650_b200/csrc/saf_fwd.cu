@@ -208,21 +208,22 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     float* red = tab + 768;
     uint32_t ns = 0, npv = 0;
     bool ok = true;
-    for (int it = it_begin; it < it_end && ok; ++it) {
+    // A compute warp whose wait was abandoned keeps walking (without storing) until the next
+    // agreement barrier, where all four leave together; none is ever left alone at a barrier.
+    for (int it = it_begin; it < it_end; ++it) {
       const WorkItem w = p.items[it];
       const int ntiles = w.blk + 1;
       const int row = w.blk * BLK + tid;
       float inv_l = 1.0f, lse = 0.0f;
+      if (named_bar_or(1, 128, !ok)) break;
       if (w.kind == KIND_ORDINARY) {
         float m_ref = -INFINITY, l = 0.0f;
         const float c = p.scale_log2;
         for (int j = 0; j < ntiles; ++j) {
-          ok = mbar_wait_warp(s_full, ns & 1, wc, SITE_S_FULL);
-          if (!ok) break;
+          if (!mbar_wait_warp(s_full, ns & 1, wc, SITE_S_FULL)) ok = false;
           ++ns;
           if (j > 0) {
-            ok = mbar_wait_warp(pv_done, npv & 1, wc, SITE_PV_DONE);
-            if (!ok) break;
+            if (!mbar_wait_warp(pv_done, npv & 1, wc, SITE_PV_DONE)) ok = false;
             ++npv;
           }
           tc_fence_after();
@@ -284,7 +285,6 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           tc_fence_before();
           mbar_arrive(p_full);
         }
-        if (!ok) break;
         inv_l = 1.0f / l;
         lse = (m_ref + log2f(l)) * LN2_F;
       } else {
@@ -293,12 +293,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         const float* rho_h = p.rho + static_cast<size_t>(w.h) * p.Tp;
         const float z2 = (row < p.T) ? p.logZ[static_cast<size_t>(w.h) * p.Tp + row] * LOG2E_F : INFINITY;
         for (int j = 0; j < ntiles; ++j) {
-          // previous tile's table readers are done; the compute warps also agree here whether a
-          // wait has been abandoned, so that none of them is left alone at a later barrier
-          if (named_bar_or(1, 128, !ok)) {
-            ok = false;
-            break;
-          }
+          named_bar_sync(1, 128);                      // previous tile's table readers are done
           const int key = j * BLK + tid;
           const float a2 = (key < p.T) ? alpha_h[key] * LOG2E_F : -INFINITY;
           const int d0 = (w.blk - j) * BLK - 127;      // band covers distances d0 .. d0+254
@@ -331,7 +326,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           named_bar_sync(1, 128);
           const bool exact = (red[8] + red[9] + red[10] + red[11]) > 0.0f;
           if (j > 0) {
-            ok = mbar_wait_warp(pv_done, npv & 1, wc, SITE_PV_DONE);   // previous P^ tile consumed
+            if (!mbar_wait_warp(pv_done, npv & 1, wc, SITE_PV_DONE)) ok = false;   // previous P^ tile consumed
             ++npv;
             tc_fence_after();
           }
@@ -371,11 +366,9 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           tc_fence_before();
           mbar_arrive(p_full);
         }
-        if (!ok) break;
       }
       // ---------------- epilogue: wait for the last P V, scale, store
-      ok = mbar_wait_warp(pv_done, npv & 1, wc, SITE_PV_DONE);
-      if (!ok) break;
+      if (!mbar_wait_warp(pv_done, npv & 1, wc, SITE_PV_DONE)) ok = false;
       ++npv;
       tc_fence_after();
       __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + w.b * p.o_strides[0] + w.h * p.o_strides[1] +
@@ -385,7 +378,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         uint32_t r[32];
         tmem_ld32(t_o + 32 * cc, r);
         tmem_wait_ld();
-        if (row < p.T) {
+        if (row < p.T && ok) {
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             uint4 o;
@@ -397,7 +390,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           }
         }
       }
-      if (p.LSE != nullptr && row < p.T)
+      if (p.LSE != nullptr && row < p.T && ok)
         p.LSE[(static_cast<size_t>(w.b) * p.H + w.h) * p.T + row] = lse;
       tc_fence_before();
       mbar_arrive(o_free);
