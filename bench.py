@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Benchmark of the hybrid causal attention layer (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 1|2]
+
+One step = one pass of the whole hot path over one synthetic batch: forward kernel, backward
+preparation (delta, zero-fill) and backward kernel, for the GPT-2-124M-shaped layer
+(batch 8, 12 heads of which 3 frozen, T = 4096, head dim 64, bf16).  Pattern normalisers are static
+per layer (the method installs them once), so they are prepared once before the timed steps; the
+time of that preparation is reported in `config`.
+
+Prints ONE JSON line (rank 0).  `value` is TFLOP/s on the layer's algorithmic FLOPs
+(B*D*T*(T+1)*(7*Ho + 2*Hf)), whole job over all ranks, inputs resident in HBM; `e2e` is the same
+metric through the host-buffer entry point with every input copied to the device and every output
+copied back inside the timed region.  `--impl reference` times the fp64 CPU oracle on a bounded
+sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import saf_inputs as si  # noqa: E402
+
+METRIC = "hybrid_attn_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d.get("bf16_tflops_sustained"),
+                "hbm_gbs": d["hbm_gbs"], "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax = float(parts[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm_sorted = sorted(sm)
+        # "under load": the upper half of the samples (idle samples before/after the region drop out)
+        load = sm_sorted[len(sm_sorted) // 2:] if sm_sorted else []
+        return {"sm_mhz": (load[len(load) // 2] if load else None), "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(wl: si.Workload, budget_s: float = 12.0):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload: whole (b,h) units,
+    alternating ordinary and frozen, until the budget is used.  Returns (TFLOP/s, description, threads)."""
+    from oracle import saf_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    rng = np.random.default_rng(wl.seed)
+    T, D = wl.T, wl.D
+    scale = 1.0 / np.sqrt(D)
+    ord_heads = [h for h in range(wl.H) if h not in wl.frozen_heads]
+    kinds = []
+    if ord_heads:
+        kinds.append(False)
+    if wl.frozen_heads:
+        kinds.append(True)
+    unit = D * T * (T + 1)
+    flops, t_used, n_units, i = 0.0, 0.0, {False: 0, True: 0}, 0
+    while t_used < budget_s:
+        fr = kinds[i % len(kinds)]
+        i += 1
+        q, k, v, do = (si.bf16_bits_to_f64(si.f32_to_bf16_bits(rng.standard_normal((T, D), dtype=np.float32)))
+                       for _ in range(4))
+        alpha = rng.standard_normal(T)
+        rho = wl.rho_slope * np.arange(T) + 0.1 * rng.standard_normal(T)
+        t0 = time.perf_counter()
+        orc.head_fwd_panels(fr, q, k, v, alpha, rho, scale, 1024)
+        if wl.backward:
+            orc.head_bwd_panels(fr, q, k, v, do, alpha, rho, scale, 1024)
+        t_used += time.perf_counter() - t0
+        n_units[fr] += 1
+        flops += unit * ((2 if fr else 7) if wl.backward else (1 if fr else 2))
+    desc = (f"{n_units[False]} ordinary + {n_units[True]} frozen (b,h) units of {wl.name} "
+            f"(T={T}, D={D}), fwd{'+bwd' if wl.backward else ''}, dense fp64 numpy, of {wl.B * wl.H} units")
+    return flops / t_used / 1e12, desc, threads, t_used
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", 0))
+    if rank != 0:
+        return
+    wl = si.config(args.config)
+    vals, descs = [], None
+    for _ in range(args.warmup):
+        oracle_sample(wl, budget_s=1.0)
+    t_all = 0.0
+    for _ in range(args.steps):
+        v, descs, threads, t = oracle_sample(wl, budget_s=args.ref_budget)
+        vals.append(v)
+        t_all += t
+    value = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_all / max(args.steps, 1),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "Hf": len(wl.frozen_heads), "T": wl.T, "D": wl.D,
+                       "note": "each step is a bounded sample of the workload run by the CPU oracle"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": descs},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- GPU arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_34650_b200 as saf
+    from paper_2609_34650_b200 import dist as sd
+
+    rank, local_rank, world = sd.env_world()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (sm_100a); there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+
+    wl = si.config(args.config, seed=sd.rank_seed(0, rank))
+    inp = si.generate(wl)
+
+    def t16(bits):
+        return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+
+    hostQ, hostK, hostV, hostdO = (t16(x).pin_memory() for x in (inp.q, inp.k, inp.v, inp.do))
+    Q, K, V, dO = (x.to(dev) for x in (hostQ, hostK, hostV, hostdO))
+    alpha_h, rho_h = torch.from_numpy(inp.alpha).pin_memory(), torch.from_numpy(inp.rho).pin_memory()
+    alpha, rho = alpha_h.to(dev), rho_h.to(dev)
+    logZ = torch.zeros_like(alpha)
+    O = torch.empty_like(Q)
+    LSE = torch.empty(wl.B, wl.H, wl.T, device=dev)
+    dQ, dK, dV = (torch.empty(Q.shape, device=dev, dtype=torch.float32) for _ in range(3))
+    ctx = saf.Context(local_rank)
+    prob = saf.make_problem(Q, wl.stored_len)
+    mask = inp.mask
+    mask0 = np.zeros_like(mask)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    # pattern preparation: once, timed on its own
+    e0, e1 = ev(), ev()
+    ctx.saf_pattern_prepare(mask, alpha, rho, logZ)
+    torch.cuda.synchronize()
+    e0.record()
+    ctx.saf_pattern_prepare(mask, alpha, rho, logZ)
+    e1.record()
+    torch.cuda.synchronize()
+    prepare_ms = e0.elapsed_time(e1)
+
+    def step(m):
+        ctx.saf_hybrid_attn_fwd(prob, Q, K, V, m, alpha, rho, logZ, O, LSE)
+        ctx.saf_hybrid_attn_bwd(prob, Q, K, V, O, dO, LSE, m, alpha, rho, logZ, dQ, dK, dV)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(m, steps):
+        barrier()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(steps):
+            step(m)
+        b.record()
+        barrier()
+        return a.elapsed_time(b) / steps
+
+    for _ in range(max(args.warmup, 3)):
+        step(mask)
+        step(mask0)
+    torch.cuda.synchronize()
+
+    # ---- headline: exactly K timed steps, clocks sampled during the region, per-kernel events on
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ctx.saf_set_profiling(True)
+    ctx.saf_get_kernel_time(saf.SAF_KERNEL_FWD)
+    ctx.saf_get_kernel_time(saf.SAF_KERNEL_BWD)
+    ctx.saf_get_kernel_time(saf.SAF_KERNEL_BWD_PREP)
+    ms_local = timed(mask, args.steps)
+    k_fwd = ctx.saf_get_kernel_time(saf.SAF_KERNEL_FWD)
+    k_bwd = ctx.saf_get_kernel_time(saf.SAF_KERNEL_BWD)
+    k_prep = ctx.saf_get_kernel_time(saf.SAF_KERNEL_BWD_PREP)
+    ctx.saf_set_profiling(False)
+    code, detail = ctx.saf_last_device_status()
+    if code != saf.SAF_OK:
+        raise RuntimeError(f"device status {code} detail {detail:#x}")
+
+    flops_local = wl.flops()
+    rate, ms = sd.whole_job_rate(flops_local * 1.0, ms_local, dev)       # FLOP per step over all ranks / max ms
+    value = rate / 1e12
+
+    # ---- speedup vs the same library with zero frozen heads: interleaved A B B A, plus an A/A control
+    reps = max(3, args.steps // 4)
+    a1 = timed(mask, reps)
+    b1 = timed(mask0, reps)
+    b2 = timed(mask0, reps)
+    a2 = timed(mask, reps)
+    c1 = timed(mask, reps)
+    c2 = timed(mask, reps)
+    speedup = (b1 + b2) / (a1 + a2)
+    aa_control = c1 / c2
+    # the sampler ran through the K timed steps and the interleaved repeats of the same step
+    clocks = sampler.stop() if rank == 0 else None
+    fwd_only = None
+    if True:
+        barrier()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(reps):
+            ctx.saf_hybrid_attn_fwd(prob, Q, K, V, mask, alpha, rho, logZ, O, LSE)
+        b.record()
+        barrier()
+        fwd_only = a.elapsed_time(b) / reps
+    ctx.saf_hybrid_attn_fwd(prob, Q, K, V, mask, alpha, rho, logZ, O, LSE)   # leave O/LSE consistent with `mask`
+
+    # ---- end to end through host buffers (pinned): inputs copied in, every output copied back
+    hO = torch.empty_like(hostQ).pin_memory()
+    hLSE = torch.empty(wl.B, wl.H, wl.T).pin_memory()
+    hdQ, hdK, hdV = (torch.empty(Q.shape, dtype=torch.float32).pin_memory() for _ in range(3))
+    ctx2 = saf.Context(local_rank)
+    probh = saf.make_problem(hostQ, wl.stored_len)
+
+    def step_host(prepare):
+        ctx2.saf_hybrid_attn_step_host(probh, hostQ, hostK, hostV, hostdO, mask, alpha_h, rho_h, prepare, hO, hLSE,
+                                       hdQ, hdK, hdV)
+
+    step_host(1)
+    step_host(0)
+    e2e_steps = max(2, min(args.steps, 5))
+    barrier()
+    t0 = time.perf_counter()
+    a, b = ev(), ev()
+    a.record()
+    for _ in range(e2e_steps):
+        step_host(0)
+    b.record()
+    barrier()
+    e2e_ms_local = a.elapsed_time(b) / e2e_steps
+    e2e_rate, e2e_ms = sd.whole_job_rate(flops_local, e2e_ms_local, dev)
+    nel = wl.B * wl.H * wl.T * wl.D
+    h2d = 4 * nel * 2
+    d2h = nel * 2 + wl.B * wl.H * wl.T * 4 + 3 * nel * 4
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    bwd_flops = wl.B * wl.D * wl.T * (wl.T + 1) * (5 * (wl.H - len(wl.frozen_heads)) + len(wl.frozen_heads))
+    fwd_flops = wl.flops(backward=False)
+    bwd_ms = k_bwd[0] / max(k_bwd[1], 1)
+    fwd_ms = k_fwd[0] / max(k_fwd[1], 1)
+    prep_ms = k_prep[0] / max(k_prep[1], 1)
+    achieved = bwd_flops / (bwd_ms * 1e-3) / 1e12
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "roofline_traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get(f"saf_bwd_kernel@{wl.name}")
+    roofline = {"bound": "tensor", "kernel": "saf_bwd_kernel", "achieved": achieved, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": traffic,
+                "peak_source": f"{peaks['source']} bf16 burst (MEASURED_PEAKS.json)" if peaks["source"] == "measured"
+                else "fallback 1590 TFLOP/s",
+                "launch_ms": bwd_ms, "flops_per_launch": bwd_flops,
+                "other_kernels": {"saf_fwd_kernel": {"launch_ms": fwd_ms, "achieved": fwd_flops / (fwd_ms * 1e-3) / 1e12,
+                                                      "frac": fwd_flops / (fwd_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]},
+                                  "saf_bwd_prep_kernel": {"launch_ms": prep_ms}}}
+
+    cpu_v, cpu_desc, cpu_threads, _ = oracle_sample(si.config(args.config), budget_s=args.ref_budget)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "B_per_gpu": wl.B, "H": wl.H, "Hf": len(wl.frozen_heads), "T": wl.T, "D": wl.D,
+                   "grad_dtype": "f32", "frozen_fraction": len(wl.frozen_heads) / wl.H,
+                   "flops_per_step_per_gpu": flops_local,
+                   "l2": "inputs+outputs per step (0.55 GB) exceed the 126 MB L2; no explicit flush",
+                   "pattern_prepare": "once before the timed steps (static per layer)", "pattern_prepare_ms": prepare_ms,
+                   "parallelism": f"dp{world} (independent batches, no collective in the layer)"},
+        "pct_of_bf16_peak": 100.0 * value / (peaks["bf16_tflops"] * world),
+        "speedup_vs_0pct_frozen": speedup, "aa_control": aa_control,
+        "ms_0pct_frozen": 0.5 * (b1 + b2), "ms_fwd_only": fwd_only,
+        "e2e": {"value": e2e_rate / 1e12, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h},
+        "gpu_launches": 3 * args.steps,
+        "clocks": clocks,
+        "roofline": roofline,
+        "cpu_baseline": {"value": cpu_v, "unit": UNIT, "cores": cpu_threads, "kind": "oracle", "sample": cpu_desc},
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3])
+    ap.add_argument("--ref-budget", type=float, default=12.0, help="seconds of CPU-oracle work per sample")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

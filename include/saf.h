@@ -109,6 +109,21 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
  * last call has drained).  `detail_out` (may be NULL) receives the raw word: site and CTA that gave up. */
 int saf_last_device_status(saf_ctx* ctx, int32_t* detail_out);
 
+/* Kernel timing for benchmarks.  With profiling enabled, every kernel the library launches is
+ * bracketed by a CUDA event pair on the launching stream.  saf_get_kernel_time() waits for the pairs
+ * of kernel `which` recorded since its last call, returns their summed duration and count, and
+ * forgets them.  Off by default (the events cost a few microseconds per launch). */
+enum {
+  SAF_KERNEL_FWD = 0,          /* persistent forward kernel */
+  SAF_KERNEL_BWD = 1,          /* persistent backward kernel */
+  SAF_KERNEL_BWD_PREP = 2,     /* delta = rowsum(dO o O), zero-fill of dQ and of frozen heads' dK */
+  SAF_KERNEL_BWD_FINALIZE = 3, /* fp32 -> bf16 conversion of dQ (bf16 gradients only) */
+  SAF_KERNEL_LOGZ = 4,         /* pattern normalisers */
+  SAF_KERNEL_COUNT = 5
+};
+int saf_set_profiling(saf_ctx* ctx, int32_t enable);
+int saf_get_kernel_time(saf_ctx* ctx, int32_t which, float* total_ms_out, int32_t* launches_out);
+
 /* Head scheduler (host only, no GPU needed).  Builds the per-CTA work lists the persistent kernels
  * walk: one item per (batch, head, 128-row block); ordinary and frozen items are packed into the
  * same grid, longest-processing-time first, with a frozen tile weighted `frozen_weight_pct` percent

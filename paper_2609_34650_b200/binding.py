@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libsaf_b200.so")
 SAF_OK = 0
 SAF_ERR_INVALID_ARG, SAF_ERR_UNSUPPORTED, SAF_ERR_CUDA, SAF_ERR_DEVICE_TIMEOUT, SAF_ERR_ARCH, SAF_ERR_NOMEM = range(1, 7)
 SAF_BF16, SAF_F32 = 0, 1
+SAF_KERNEL_FWD, SAF_KERNEL_BWD, SAF_KERNEL_BWD_PREP, SAF_KERNEL_BWD_FINALIZE, SAF_KERNEL_LOGZ = range(5)
 
 
 class SafProblem(C.Structure):
@@ -55,9 +56,12 @@ def load_library() -> C.CDLL:
     lib.saf_hybrid_attn_bwd.argtypes = [vp, pp, vp, vp, vp, vp, vp, f32p, u8p, f32p, f32p, f32p, vp, vp, vp, vp]
     lib.saf_hybrid_attn_step_host.argtypes = [vp, pp, vp, vp, vp, vp, u8p, f32p, f32p, i32, vp, f32p, vp, vp, vp]
     lib.saf_last_device_status.argtypes = [vp, C.POINTER(C.c_int32)]
+    lib.saf_set_profiling.argtypes = [vp, i32]
+    lib.saf_get_kernel_time.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.saf_build_worklist.argtypes = [i32, i32, i32, u8p, i32, i32, i32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     for name in ("saf_create", "saf_destroy", "saf_pattern_prepare", "saf_hybrid_attn_fwd", "saf_hybrid_attn_bwd",
-                 "saf_hybrid_attn_step_host", "saf_last_device_status", "saf_build_worklist"):
+                 "saf_hybrid_attn_step_host", "saf_last_device_status", "saf_build_worklist", "saf_set_profiling",
+                 "saf_get_kernel_time"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -162,6 +166,15 @@ class Context:
         _check(self._lib.saf_hybrid_attn_step_host(self._h, C.byref(prob), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), mp,
                                                    _ptr(alpha), _ptr(rho), int(prepare), _ptr(O), _ptr(LSE), _ptr(dQ),
                                                    _ptr(dK), _ptr(dV)), "saf_hybrid_attn_step_host")
+
+    def saf_set_profiling(self, enable: bool):
+        _check(self._lib.saf_set_profiling(self._h, int(enable)), "saf_set_profiling")
+
+    def saf_get_kernel_time(self, which: int):
+        """(total milliseconds, launches) of kernel `which` since the previous query."""
+        ms, n = C.c_float(0.0), C.c_int32(0)
+        _check(self._lib.saf_get_kernel_time(self._h, which, C.byref(ms), C.byref(n)), "saf_get_kernel_time")
+        return ms.value, n.value
 
     def saf_last_device_status(self):
         detail = C.c_int32(0)

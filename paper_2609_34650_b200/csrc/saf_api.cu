@@ -33,6 +33,11 @@ struct DevBuf {
   size_t bytes = 0;
 };
 
+struct TimedLaunch {
+  int which;
+  cudaEvent_t beg, end;
+};
+
 }  // namespace
 
 struct saf_ctx {
@@ -45,6 +50,9 @@ struct saf_ctx {
   int frozen_weight_pct = 60;
   std::vector<WorklistEntry> worklists;
   DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf;
+  bool profiling = false;
+  std::vector<TimedLaunch> timed;          // event pairs recorded since the last query
+  std::vector<cudaEvent_t> event_pool;
   // staging for the host-buffer entry point
   DevBuf hq, hk, hv, hdo, ho, hlse, hdq, hdk, hdv, halpha, hrho, hlogz;
 };
@@ -186,6 +194,36 @@ int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int bac
   return SAF_OK;
 }
 
+// Kernel timing (opt-in): an event pair on the launching stream around one kernel.
+cudaEvent_t take_event(saf_ctx* ctx) {
+  if (!ctx->event_pool.empty()) {
+    cudaEvent_t e = ctx->event_pool.back();
+    ctx->event_pool.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+struct ScopedTimer {
+  saf_ctx* ctx;
+  cudaStream_t st;
+  TimedLaunch t{};
+  bool on;
+  ScopedTimer(saf_ctx* c, int which, cudaStream_t s) : ctx(c), st(s), on(c->profiling && c->timed.size() < 65536) {
+    if (!on) return;
+    t.which = which;
+    t.beg = take_event(ctx);
+    t.end = take_event(ctx);
+    cudaEventRecord(t.beg, st);
+  }
+  ~ScopedTimer() {
+    if (!on) return;
+    cudaEventRecord(t.end, st);
+    ctx->timed.push_back(t);
+  }
+};
+
 struct DeviceGuard {
   int prev = -1;
   bool ok = true;
@@ -270,6 +308,11 @@ int saf_destroy(saf_ctx* ctx) {
                     &ctx->hlogz};
   for (DevBuf* b : bufs) release(*b);
   if (ctx->status_dev) cudaFree(ctx->status_dev);
+  for (TimedLaunch& t : ctx->timed) {
+    cudaEventDestroy(t.beg);
+    cudaEventDestroy(t.end);
+  }
+  for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
   delete ctx;
   return SAF_OK;
 }
@@ -287,6 +330,7 @@ int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* froz
   int rc = upload_mask(ctx, frozen_mask_host, H, st);
   if (rc) return rc;
   ctx->last_stream = st;
+  ScopedTimer timer(ctx, SAF_KERNEL_LOGZ, st);
   if (launch_logz(alpha_dev, rho_dev, logZ_dev_out, static_cast<const uint8_t*>(ctx->mask_buf.ptr), H, Tp, st) !=
       cudaSuccess)
     return SAF_ERR_CUDA;
@@ -352,6 +396,7 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   fp.cta_offsets = wl->offsets_dev;
   fp.status = ctx->status_dev;
   fp.wait_limit_ns = ctx->wait_limit_ns;
+  ScopedTimer timer(ctx, SAF_KERNEL_FWD, st);
   if (launch_fwd(p->D, mq, mk, mv, fp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
   return SAF_OK;
 }
@@ -404,10 +449,13 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     dqacc = static_cast<float*>(ctx->dqacc_buf.ptr);
   }
   // O is only read for ordinary heads; a frozen-only layer may pass O = NULL
-  if (launch_bwd_prep(O, dO, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr),
-                      static_cast<float*>(ctx->delta_buf.ptr), Tpad, dqacc, dK, grad_f32, p->B, p->H, p->T, p->D,
-                      st) != cudaSuccess)
-    return SAF_ERR_CUDA;
+  {
+    ScopedTimer timer(ctx, SAF_KERNEL_BWD_PREP, st);
+    if (launch_bwd_prep(O, dO, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr),
+                        static_cast<float*>(ctx->delta_buf.ptr), Tpad, dqacc, dK, grad_f32, p->B, p->H, p->T, p->D,
+                        st) != cudaSuccess)
+      return SAF_ERR_CUDA;
+  }
 
   const long long n_items = static_cast<long long>(p->B) * p->H * nblk;
   const int grid = static_cast<int>(std::min<long long>(ctx->num_sms, n_items));
@@ -440,8 +488,14 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   bp.cta_offsets = wl->offsets_dev;
   bp.status = ctx->status_dev;
   bp.wait_limit_ns = ctx->wait_limit_ns;
-  if (launch_bwd(p->D, mq, mk, mv, mdo, bp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
-  if (!grad_f32 && launch_bwd_finalize(dqacc, dQ, nelem, st) != cudaSuccess) return SAF_ERR_CUDA;
+  {
+    ScopedTimer timer(ctx, SAF_KERNEL_BWD, st);
+    if (launch_bwd(p->D, mq, mk, mv, mdo, bp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+  }
+  if (!grad_f32) {
+    ScopedTimer timer(ctx, SAF_KERNEL_BWD_FINALIZE, st);
+    if (launch_bwd_finalize(dqacc, dQ, nelem, st) != cudaSuccess) return SAF_ERR_CUDA;
+  }
   return SAF_OK;
 }
 
@@ -524,6 +578,38 @@ int saf_last_device_status(saf_ctx* ctx, int32_t* detail_out) {
     cudaMemset(ctx->status_dev, 0, sizeof(int));
     return SAF_ERR_DEVICE_TIMEOUT;
   }
+  return SAF_OK;
+}
+
+int saf_set_profiling(saf_ctx* ctx, int32_t enable) {
+  if (!ctx) return SAF_ERR_INVALID_ARG;
+  ctx->profiling = enable != 0;
+  return SAF_OK;
+}
+
+int saf_get_kernel_time(saf_ctx* ctx, int32_t which, float* total_ms_out, int32_t* launches_out) {
+  if (!ctx || !total_ms_out || !launches_out || which < 0 || which >= SAF_KERNEL_COUNT) return SAF_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  double total = 0.0;
+  int n = 0;
+  std::vector<TimedLaunch> keep;
+  for (const TimedLaunch& t : ctx->timed) {
+    if (t.which != which) {
+      keep.push_back(t);
+      continue;
+    }
+    float ms = 0.0f;
+    if (cudaEventSynchronize(t.end) != cudaSuccess || cudaEventElapsedTime(&ms, t.beg, t.end) != cudaSuccess)
+      return SAF_ERR_CUDA;
+    total += ms;
+    ++n;
+    ctx->event_pool.push_back(t.beg);
+    ctx->event_pool.push_back(t.end);
+  }
+  ctx->timed.swap(keep);
+  *total_ms_out = static_cast<float>(total);
+  *launches_out = n;
   return SAF_OK;
 }
 

@@ -1,0 +1,272 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the fp64 oracle on the same
+seeded inputs.  Tolerance (bf16 inputs, fp32 accumulation): max-abs 2e-2, relative L2 1e-2."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_34650_b200 as saf
+import saf_inputs as si
+from oracle import saf_oracle as orc
+
+from gpu_util import Layer, assert_close, errors, f64, bf16_tensor, MAX_ABS, REL_L2
+
+pytestmark = pytest.mark.gpu
+
+
+def check_units(L: Layer, units, backward=True, rows=None, panel=512):
+    """Compare the (b,h) units in `units` (all rows, or the row slice `rows` of the forward)."""
+    inp, wl = L.inp, L.inp.wl
+    q, k, v, do = f64(inp)
+    scale = 1.0 / np.sqrt(wl.D)
+    O, LSE = L.host(L.O), L.host(L.LSE)
+    G = [L.host(g) for g in L.grads] if backward else None
+    worst = {}
+    for b, h in units:
+        fr = bool(inp.mask[h])
+        eO, eL = orc.head_fwd_panels(fr, q[b, h], k[b, h], v[b, h], inp.alpha[h], inp.rho[h], scale, panel, rows)
+        sl = rows or slice(0, wl.T)
+        worst[("O", fr)] = assert_close(O[b, h][sl], eO, f"O[{b},{h}] frozen={fr}")
+        if fr:
+            assert not LSE[b, h].any(), "LSE slot of a frozen head must be zero"
+        else:
+            assert np.abs(LSE[b, h][sl] - eL).max() < 1e-4, f"LSE[{b},{h}]"
+        if backward:
+            e = orc.head_bwd_panels(fr, q[b, h], k[b, h], v[b, h], do[b, h], inp.alpha[h], inp.rho[h], scale, panel)
+            for name, g, ee in zip(("dQ", "dK", "dV"), G, e):
+                if fr and name != "dV":
+                    assert not g[b, h].any(), f"{name}[{b},{h}] of a frozen head must be exactly zero"
+                else:
+                    assert_close(g[b, h], ee, f"{name}[{b},{h}] frozen={fr}")
+    return worst
+
+
+def all_units(wl):
+    return [(b, h) for b in range(wl.B) for h in range(wl.H)]
+
+
+# --------------------------------------------------------------------------- small, exhaustive
+def test_config0_tiny_all_units():
+    L = Layer(si.generate(si.config(0))).run()
+    check_units(L, all_units(L.inp.wl))
+
+
+def test_paper_test_shape_T129_stored_192():
+    """Batch 2, T=129, 4 heads x 64, stored pattern length 192, heads 1 and 3 frozen (Appendix E.2)."""
+    wl = si.Workload("paper-shape", 2, 4, 129, 64, (1, 3), -0.05, Tp=192, seed=3)
+    L = Layer(si.generate(wl)).run()
+    check_units(L, all_units(wl))
+
+
+@pytest.mark.parametrize("T", [1, 2, 127, 128, 255, 257, 384])
+def test_ragged_lengths(T):
+    wl = si.Workload(f"ragged{T}", 1, 3, T, 64, (1,), -0.05, seed=T)
+    L = Layer(si.generate(wl)).run()
+    check_units(L, all_units(wl))
+
+
+@pytest.mark.parametrize("frozen", [(), (0, 1, 2, 3)])
+def test_empty_and_full_frozen_sets(frozen):
+    wl = si.Workload("sets", 2, 4, 320, 64, frozen, -0.05, seed=11)
+    L = Layer(si.generate(wl)).run()
+    check_units(L, all_units(wl))
+
+
+def test_head_dim_128_forward():
+    wl = si.Workload("d128", 2, 4, 640, 128, (2,), -0.01, alpha0_spike=4.0, backward=False, seed=5)
+    L = Layer(si.generate(wl), backward=False).run(backward=False)
+    check_units(L, all_units(wl), backward=False)
+
+
+def test_backward_head_dim_128_is_reported_unsupported():
+    wl = si.Workload("d128b", 1, 2, 128, 128, (), -0.01, seed=5)
+    L = Layer(si.generate(wl))
+    with pytest.raises(saf.SafError) as e:
+        L.run()
+    assert e.value.code == 2
+
+
+def test_multi_tile_scheduler_mix():
+    """Several items per CTA of both kinds: 8 x 6 heads x 9 blocks = 432 forward items on 296 CTAs."""
+    wl = si.Workload("mix", 8, 6, 1100, 64, (0, 3, 4), -0.05, seed=21)
+    L = Layer(si.generate(wl)).run()
+    check_units(L, [(0, 0), (7, 5), (3, 3), (5, 1), (2, 4), (6, 2)])
+
+
+# --------------------------------------------------------------------------- invariants on the GPU
+def test_frozen_heads_never_read_q_k_and_get_zero_grads():
+    wl = si.Workload("poison", 2, 4, 300, 64, (0, 2), -0.05, seed=8)
+    inp = si.generate(wl)
+    clean = Layer(inp).run()
+    L = Layer(inp)
+    for h in wl.frozen_heads:
+        L.Q[:, h] = float("nan")
+        L.K[:, h] = float("nan")
+    L.run()
+    assert torch.equal(L.O, clean.O)
+    assert torch.equal(L.grads[2], clean.grads[2])
+    for h in wl.frozen_heads:
+        assert not L.grads[0][:, h].any() and not L.grads[1][:, h].any()
+    for h in (1, 3):
+        assert L.grads[0][:, h].abs().max() > 0 and L.grads[1][:, h].abs().max() > 0
+
+
+def test_frozen_head_equals_engineered_ordinary_head_on_gpu():
+    """S[i,j] = alpha[j] + lambda j (+ row constant) makes an ordinary head equal the frozen head
+    (alpha, rho = -lambda d); all values exactly representable in bf16."""
+    T, D, lam, scale = 256, 64, 2.0 ** -4, 0.125
+    rng = np.random.default_rng(0)
+    alpha = si.bf16_bits_to_f32(si.f32_to_bf16_bits(rng.standard_normal(T).astype(np.float32)))
+    wl = si.Workload("p6", 1, 2, T, D, (1,), -lam, seed=1)
+    inp = si.generate(wl)
+    q = np.zeros((T, D), np.float32)
+    k = np.zeros((T, D), np.float32)
+    q[:, 0] = q[:, 1] = 1.0 / scale
+    k[:, 0] = alpha
+    k[:, 1] = lam * np.arange(T)
+    inp.q[0, 0], inp.k[0, 0] = si.f32_to_bf16_bits(q), si.f32_to_bf16_bits(k)
+    inp.v[0, 1], inp.do[0, 1] = inp.v[0, 0], inp.do[0, 0]
+    inp.alpha[1] = alpha
+    inp.rho[1] = -lam * np.arange(T)
+    L = Layer(inp).run()
+    O, dV = L.host(L.O), L.host(L.grads[2])
+    assert np.abs(O[0, 0] - O[0, 1]).max() < MAX_ABS         # two bf16-rounded outputs of values up to ~3
+    ma, rl = errors(dV[0, 0], dV[0, 1])
+    assert ma < MAX_ABS and rl < REL_L2
+
+
+def test_exact_exponent_fallback_for_wide_range_patterns():
+    """alpha / rho ranges far beyond fp32's factorised range (rho rising 0.9 per step) still match."""
+    T = 300
+    wl = si.Workload("wide", 1, 2, T, 64, (0, 1), 0.9, seed=4)
+    inp = si.generate(wl)
+    inp.alpha[1] = (40.0 * np.sin(np.arange(T))).astype(np.float32)
+    # such a pattern puts every row's mass on the earliest keys, so dV[0] sums ~T output gradients;
+    # dO / 16 (exact in bf16) keeps the gradient in the value range the absolute tolerance is meant for
+    inp.do[...] = si.f32_to_bf16_bits(si.bf16_bits_to_f32(inp.do) / 16.0)
+    L = Layer(inp).run()
+    check_units(L, all_units(wl))
+
+
+def test_stale_state_fuzz_on_one_context():
+    """Mask / pattern / shape changes on one context (cached work lists, workspaces) stay correct."""
+    ctx = saf.Context(0)
+    rng = np.random.default_rng(99)
+    for step in range(12):
+        H = int(rng.integers(1, 5))
+        T = int(rng.choice([64, 129, 200, 256, 300]))
+        nf = int(rng.integers(0, H + 1))
+        frozen = tuple(sorted(rng.choice(H, nf, replace=False).tolist()))
+        wl = si.Workload(f"fuzz{step}", int(rng.integers(1, 3)), H, T, 64, frozen, -0.05, Tp=T + int(rng.integers(0, 40)),
+                         seed=100 + step)
+        L = Layer(si.generate(wl), ctx=ctx).run()
+        check_units(L, all_units(wl))
+
+
+def test_strided_views_bthd_layout():
+    """Q/K/V/O/dO given as [B,T,H,D] storage viewed as [B,H,T,D] (non-contiguous heads)."""
+    wl = si.Workload("strided", 2, 3, 260, 64, (1,), -0.05, seed=13)
+    inp = si.generate(wl)
+    L = Layer(inp)
+    for name in ("Q", "K", "V", "dO", "O"):
+        t = getattr(L, name)
+        setattr(L, name, t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3))
+    L.prob = saf.make_problem(L.Q, wl.stored_len, k_like=L.K, v_like=L.V, o_like=L.O)
+    L.run()
+    check_units(L, all_units(wl))
+
+
+def test_bf16_gradients():
+    """grad_dtype = bf16: one extra rounding of the result; |dV| reaches ~8 for concentrated
+    patterns, where half a bf16 ulp is 1.6e-2, so the max-abs bound is 2e-2 + 1.6e-2."""
+    inp = si.generate(si.config(0))
+    L = Layer(inp, grad_dtype=saf.SAF_BF16).run()
+    ref = Layer(inp).run()
+    for g16, g32 in zip(L.grads, ref.grads):
+        ma, rl = errors(L.host(g16), L.host(g32))
+        assert ma <= 3.2e-2 and rl <= 5e-3
+
+
+def test_forward_is_deterministic_and_internal_prepare_matches():
+    inp = si.generate(si.Workload("det", 2, 4, 400, 64, (2,), -0.05, seed=17))
+    A = Layer(inp).run()
+    B = Layer(inp)
+    B.logZ = None                      # library computes the normalisers itself
+    B.run(prepare=False)
+    assert torch.equal(A.O, B.O) and torch.equal(A.LSE, B.LSE)
+    assert torch.equal(A.grads[1], B.grads[1]) and torch.equal(A.grads[2], B.grads[2])
+    ez = orc.pattern_logZ(inp.alpha[2], inp.rho[2], 400)
+    assert np.abs(A.logZ[2].cpu().numpy() - ez).max() < 5e-6
+
+
+def test_host_buffer_step_matches_device_path():
+    inp = si.generate(si.Workload("host", 2, 3, 200, 64, (1,), -0.05, seed=23))
+    D = Layer(inp).run()
+    wl = inp.wl
+    ctx = saf.Context(0)
+    pin = lambda t: t.pin_memory()
+    Q, K, V, dO = (pin(bf16_tensor(x)) for x in (inp.q, inp.k, inp.v, inp.do))
+    alpha, rho = pin(torch.from_numpy(inp.alpha)), pin(torch.from_numpy(inp.rho))
+    O = pin(torch.empty_like(Q))
+    LSE = pin(torch.empty(wl.B, wl.H, wl.T))
+    dQ, dK, dV = (pin(torch.empty(Q.shape, dtype=torch.float32)) for _ in range(3))
+    prob = saf.make_problem(Q, wl.stored_len)
+    for prepare in (1, 0):
+        ctx.saf_hybrid_attn_step_host(prob, Q, K, V, dO, inp.mask, alpha, rho, prepare, O, LSE, dQ, dK, dV)
+        assert torch.equal(O, D.O.cpu()) and torch.equal(LSE, D.LSE.cpu())
+        assert torch.equal(dK, D.grads[1].cpu()) and torch.equal(dV, D.grads[2].cpu())
+        ma, rl = errors(dQ.numpy().astype(np.float64), D.host(D.grads[0]))
+        assert ma < 1e-4                       # atomics order only
+
+
+def test_invalid_arguments_are_rejected():
+    inp = si.generate(si.Workload("bad", 1, 2, 64, 64, (1,), -0.05))
+    L = Layer(inp)
+    L.prob.Tp = 32                             # T > Tp
+    with pytest.raises(saf.SafError) as e:
+        L.run()
+    assert e.value.code == 1
+    L = Layer(inp)
+    L.prob.D = 96
+    with pytest.raises(saf.SafError) as e:
+        L.run()
+    assert e.value.code == 2
+    L = Layer(inp)
+    L.prob.q_strides[2] = 60                   # not a multiple of 8 elements
+    with pytest.raises(saf.SafError) as e:
+        L.run()
+    assert e.value.code == 1
+
+
+# --------------------------------------------------------------------------- full sizes, sampled
+def test_config1_full_size_sampled_units():
+    wl = si.config(1)
+    L = Layer(si.generate(wl)).run()
+    fh, oh = wl.frozen_heads[0], [h for h in range(wl.H) if h not in wl.frozen_heads][0]
+    check_units(L, [(0, fh), (wl.B - 1, oh), (3, wl.frozen_heads[-1])], panel=1024)
+
+
+@pytest.mark.parametrize("nf", [0, 6, 9, 12])
+def test_config3_sweep_full_size_sampled_units(nf):
+    wl = si.config(3, nf)
+    L = Layer(si.generate(wl)).run()
+    units = []
+    if nf > 0:
+        units.append((nf % wl.B, wl.frozen_heads[nf // 2]))
+    if nf < wl.H:
+        units.append(((nf + 1) % wl.B, [h for h in range(wl.H) if h not in wl.frozen_heads][0]))
+    check_units(L, units, panel=1024)
+
+
+def test_config2_full_size_sampled_units():
+    wl = si.config(2)
+    L = Layer(si.generate(wl)).run()
+    oh = [h for h in range(wl.H) if h not in wl.frozen_heads][-1]
+    check_units(L, [(1, wl.frozen_heads[3]), (2, oh)], panel=1024)
+
+
+def test_config4_long_prefill_sampled_row_panels():
+    wl = si.config(4)
+    L = Layer(si.generate(wl), backward=False).run(backward=False)
+    oh = [h for h in range(wl.H) if h not in wl.frozen_heads][5]
+    for rows in (slice(0, 256), slice(16300, 16500), slice(wl.T - 256, wl.T)):
+        check_units(L, [(0, wl.frozen_heads[0]), (0, oh)], backward=False, rows=rows, panel=256)
