@@ -151,7 +151,8 @@ def run_reference(args):
         oracle_sample(wl, budget_s=1.0)
     t_all = 0.0
     for _ in range(args.steps):
-        v, descs, threads, t = oracle_sample(wl, budget_s=args.ref_budget)
+        # keep the whole run within a few minutes whatever K is
+        v, descs, threads, t = oracle_sample(wl, budget_s=min(args.ref_budget, 150.0 / max(args.steps, 1)))
         vals.append(v)
         t_all += t
     value = float(np.mean(vals))
