@@ -437,10 +437,13 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   if (rc) return rc;
 
   const int nblk = (p->T + BLK - 1) / BLK;
-  const int Tpad = nblk * BLK;
   const size_t nelem = static_cast<size_t>(p->B) * p->H * p->T * p->D;
-  rc = ensure(ctx->delta_buf, static_cast<size_t>(p->B) * p->H * Tpad * sizeof(float));
+  const size_t ext_bytes = static_cast<size_t>(p->B) * p->H * nblk * 4096;   // one 4 KB image per 128-row block
+  rc = ensure(ctx->delta_buf, 2 * ext_bytes);                 // q_ext images followed by do_ext images
   if (rc) return rc;
+  uint8_t* q_ext = static_cast<uint8_t*>(ctx->delta_buf.ptr);
+  uint8_t* do_ext = q_ext + ext_bytes;
+  const float scale_v = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   const int grad_f32 = p->grad_dtype == SAF_F32;
   float* dqacc = static_cast<float*>(dQ);
   if (!grad_f32) {
@@ -451,9 +454,8 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   // O is only read for ordinary heads; a frozen-only layer may pass O = NULL
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_PREP, st);
-    if (launch_bwd_prep(O, dO, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr),
-                        static_cast<float*>(ctx->delta_buf.ptr), Tpad, dqacc, dK, grad_f32, p->B, p->H, p->T, p->D,
-                        st) != cudaSuccess)
+    if (launch_bwd_prep(O, dO, LSE, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr), q_ext, do_ext,
+                        1.0f / scale_v, dqacc, dK, grad_f32, p->B, p->H, p->T, p->D, st) != cudaSuccess)
       return SAF_ERR_CUDA;
   }
 
@@ -473,15 +475,26 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   } else {
     mq = mdo; mk = mdo; mv = mdo;
   }
+  // fp32 dQ accumulator [B][H][T][64] as a 4-D tensor for tiled reduce-adds: box = 32 floats x 128 rows
+  CUtensorMap mdq;
+  {
+    cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(p->T), static_cast<cuuint64_t>(p->H), static_cast<cuuint64_t>(p->B)};
+    cuuint64_t gs[3] = {64 * 4, static_cast<cuuint64_t>(p->T) * 64 * 4, static_cast<cuuint64_t>(p->T) * 64 * 4 * p->H};
+    cuuint32_t box[4] = {32, BLK, 1, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    if (ctx->encode(&mdq, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, dqacc, dims, gs, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return SAF_ERR_CUDA;
+  }
   BwdParams bp;
   bp.B = p->B; bp.H = p->H; bp.T = p->T; bp.Tp = p->Tp;
   bp.scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   bp.scale_log2 = bp.scale * 1.4426950408889634f;
   bp.alpha = alpha; bp.rho = rho; bp.logZ = logZ;
-  bp.LSE = LSE;
-  bp.delta = static_cast<const float*>(ctx->delta_buf.ptr);
-  bp.Tpad = Tpad;
-  bp.dQacc = dqacc;
+  bp.q_ext = q_ext;
+  bp.do_ext = do_ext;
+  bp.nblk = nblk;
   bp.dK = dK; bp.dV = dV;
   bp.grad_f32 = grad_f32;
   bp.items = wl->items_dev;
@@ -490,7 +503,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   bp.wait_limit_ns = ctx->wait_limit_ns;
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD, st);
-    if (launch_bwd(p->D, mq, mk, mv, mdo, bp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+    if (launch_bwd(p->D, mq, mk, mv, mdo, mdq, bp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
   }
   if (!grad_f32) {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_FINALIZE, st);

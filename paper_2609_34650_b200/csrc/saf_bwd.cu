@@ -1,24 +1,46 @@
 // Backward of the hybrid causal attention layer on sm_100a (head dimension 64): one persistent
 // kernel, one work item per (batch, head, 128-key block J), looping over query blocks I >= J.
 //
-// CTA = 320 threads: warps 0-7 compute (TMEM lane = key row; warps 0-3 own query columns 0-63 of a
-// tile, warps 4-7 columns 64-127), warp 8 TMA producer, warp 9 tcgen05 issuer / TMEM owner.
+// CTA = 448 threads:
+//   warps 0-3  compute group 0: even 64-query half tiles (TMEM buffer 0); TMEM lane = key row
+//   warps 4-7  compute group 1: odd half tiles (TMEM buffer 1)
+//   warps 8-11 dQ drain: TMEM -> swizzled smem -> TMA reduce-add into the fp32 dQ accumulator
+//   warp 12    TMA producer, warp 13 tcgen05 issuer and TMEM owner
 //
-// Ordinary item, per tile (Appendix E.2: key-block programs accumulate dV and dK; dQ here is produced
-// by the same tile loop and accumulated across key blocks with fp32 atomics instead of a second pass):
-//   S^T  = K_J Q_I^T,  dP^T = V_J dO_I^T                       (tcgen05, smem operands)
-//   P^T  = exp(S^T * scale - LSE_i),  dS^T = P^T o (dP^T - delta_i)   (registers; bf16 to TMEM, dS^T also to smem)
-//   dV_J += P^T dO_I,  dK_J += dS^T Q_I                        (A from TMEM, dO / Q as MN-major B)
-//   dQ_I  = dS K_J                                             (A = dS^T tile in smem read M-major, B = K_J)
-// Frozen item, per tile (Sec. 3.3: dV = P^^T dO, no query/key gradients):
+// Ordinary item (Appendix E.2: key-block programs accumulate dV and dK; dQ here comes out of the same
+// tile loop and is accumulated across key blocks by reduce-adds instead of a second pass).  The tile
+// loop is software-pipelined over half tiles u with S^T/dP^T double-buffered in TMEM:
+//   A(u): S'^T[u&1]  = K_J Q_u^T  + 1 (-LSE_i/scale)^T,   dP'^T[u&1] = V_J dO_u^T + 1 (-delta_i)^T
+//         (the row terms ride on one extra 16-wide reduction step: a constant tile of ones times a
+//          three-way bf16 split of the fp32 row value, so S' and dP' leave the tensor core ready)
+//   compute(u): P^T = exp2(c S'^T) = exp(scale S - LSE),  dS^T = P^T o dP'^T   (bf16 to TMEM; dS^T also to smem)
+//   B(u): dV_J += P^T dO_u,  dK_J += dS^T Q_u                  (A from TMEM, dO / Q rows as MN-major B)
+//   C(t), once per full tile: dQ_t = dS K_J                    (A = smem dS^T tile read M-major, B = K_J)
+// Frozen item (Sec. 3.3: dV = P^^T dO, no query/key gradients), full tiles alternating between the
+// two compute groups:
 //   P^^T(j,i) = exp(alpha(j) + rho(i-j) - logZ(i)) for i >= j, generated into TMEM (factorised as in
 //   the forward), dV_J += P^^T dO_I.
 //
-// TMEM columns: [0,128) S^T / P^T (bf16 pairs in [0,64); frozen P^^T double-buffered in [0,64),[64,128)),
-// [128,256) dP^T / dS^T (bf16 pairs in [128,192)), [256,320) dV, [320,384) dK, [384,448) dQ.
+// TMEM columns: [0,64) dV, [64,128) dK, [128,192)/[192,256) S^T buffers (bf16 P^T pairs re-use the
+// consumed columns; frozen P^^T tiles use the two 64-column buffers whole), [256,320)/[320,384) dP^T
+// buffers (bf16 dS^T likewise), [384,448) dQ.
 #include <cuda_bf16.h>
 #include "ptx.cuh"
 #include "saf_internal.h"
+
+#ifdef SAF_TRACE
+__device__ unsigned long long g_saf_trace[4][16384];
+#define TR(role, id)                                                                                   \
+  do {                                                                                                 \
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && tr_n < 16380)                                    \
+      g_saf_trace[role][tr_n++] = (static_cast<unsigned long long>(id) << 48) | (clock64() & 0xffffffffffffULL); \
+  } while (0)
+extern "C" int saf_debug_read_trace(unsigned long long* out) {
+  return static_cast<int>(cudaMemcpyFromSymbol(out, g_saf_trace, sizeof(g_saf_trace)));
+}
+#else
+#define TR(role, id)
+#endif
 
 namespace saf {
 
@@ -33,62 +55,56 @@ struct BwdCfg {
   static constexpr int OFF_V = PANEL;
   static constexpr int OFF_Q = 2 * PANEL;            // NS stages
   static constexpr int OFF_DO = OFF_Q + NS * PANEL;  // NS stages
-  static constexpr int OFF_DS = OFF_DO + NS * PANEL; // two panels: queries 0-63, 64-127
-  static constexpr int OFF_TAB = OFF_DS + 2 * PANEL;
-  // floats: lse2[128] delta[128] wq[128] z2s[128] rband[256] r2raw[256] red[32]
-  static constexpr int TAB_FLOATS = 128 * 4 + 256 * 2 + 32;
-  static constexpr int OFF_BAR = OFF_TAB + TAB_FLOATS * 4;
-  static constexpr int NBAR = 2 + 2 * NS + 6 + 2;
+  static constexpr int OFF_DS = OFF_DO + NS * PANEL; // 2 buffers x 2 panels (queries 0-63, 64-127)
+  static constexpr int OFF_DQ = OFF_DS + 4 * PANEL;  // fp32 staging: 2 boxes [128 rows][32 floats], 128B swizzle
+  static constexpr int OFF_QX = OFF_DQ + 2 * PANEL;  // NS x 4 KB row-term images of Q
+  static constexpr int OFF_DOX = OFF_QX + NS * 4096; // NS x 4 KB row-term images of dO
+  static constexpr int OFF_ONES = OFF_DOX + NS * 4096;   // 4 KB constant tile: columns 0..2 one, rest zero
+  static constexpr int OFF_TAB = OFF_ONES + 4096;
+  // per compute group: wq[128] z2s[128] rband[256] r2raw[256] red[16]
+  static constexpr int TAB_FLOATS = 128 * 2 + 256 * 2 + 16;
+  static constexpr int OFF_BAR = OFF_TAB + 2 * TAB_FLOATS * 4;
+  static constexpr int NBAR = 2 + 2 * NS + 2 + 2 + 4 + 2;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
   static constexpr int TMEM_COLS = 512;
-  static constexpr int COL_S = 0, COL_DP = 128, COL_DV = 256, COL_DK = 320, COL_DQ = 384;
-  static constexpr int NCT = 256;                    // compute threads
+  static constexpr int COL_DV = 0, COL_DK = 64, COL_S = 128, COL_DP = 256, COL_DQ = 384;
+  static constexpr int NTHREADS = 448;
 };
 
 enum BwdSite { B_KV_EMPTY = 21, B_QDO_EMPTY, B_KV_FULL, B_QDO_FULL, B_PDS_FULL, B_ACC_FREE, B_DQ_FREE, B_SDP_FULL,
                B_DQ_FULL, B_ACC_FULL, B_PFREE };
 
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
 }  // namespace
 
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(BwdCfg::NTHREADS, 1)
 saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
-               const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mdo, const BwdParams p) {
+               const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mdo,
+               const __grid_constant__ CUtensorMap mdq, const BwdParams p) {
   using C = BwdCfg;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR);
   uint64_t* kv_full = bars;
   uint64_t* kv_empty = bars + 1;
-  uint64_t* qdo_full = bars + 2;
-  uint64_t* qdo_empty = qdo_full + C::NS;
-  uint64_t* sdp_full = qdo_empty + C::NS;
-  uint64_t* pds_full = sdp_full + 1;
-  uint64_t* dq_full = pds_full + 1;
+  uint64_t* qdo_full = bars + 2;                 // [NS]
+  uint64_t* qdo_empty = qdo_full + C::NS;        // [NS]
+  uint64_t* sdp_full = qdo_empty + C::NS;        // [2]
+  uint64_t* pds_full = sdp_full + 2;             // [2]
+  uint64_t* dq_full = pds_full + 2;
   uint64_t* dq_free = dq_full + 1;
   uint64_t* acc_full = dq_free + 1;
   uint64_t* acc_free = acc_full + 1;
-  uint64_t* pfree = acc_free + 1;   // [2]
+  uint64_t* pfree = acc_free + 1;                // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pfree + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* tab = reinterpret_cast<float*>(smem + C::OFF_TAB);
-  float* lse2s = tab;
-  float* dels = tab + 128;
-  float* wq = tab + 256;
-  float* z2s = tab + 384;
-  float* rband = tab + 512;
-  float* r2raw = tab + 768;
-  float* red = tab + 1024;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const WaitCtx wc{abort_flag, p.status, p.wait_limit_ns};
-  const int nblk = (p.T + BLK - 1) / BLK;
+  const int nblk = p.nblk;
 
   if (tid == 0) {
     *abort_flag = 0;
@@ -98,27 +114,39 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       mbar_init(qdo_full + s, 1);
       mbar_init(qdo_empty + s, 1);
     }
-    mbar_init(sdp_full, 1);
-    mbar_init(pds_full, C::NCT);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(sdp_full + b, 1);
+      mbar_init(pds_full + b, 4);                // one arrival per warp of the group
+      mbar_init(pfree + b, 1);
+    }
     mbar_init(dq_full, 1);
-    mbar_init(dq_free, C::NCT);
+    mbar_init(dq_free, 4);
     mbar_init(acc_full, 1);
-    mbar_init(acc_free, C::NCT);
-    mbar_init(pfree, 1);
-    mbar_init(pfree + 1, 1);
+    mbar_init(acc_free, 8);
     mbar_fence_init();
   }
-  if (warp == 9) {
+  // constant tile of ones (columns 0..2) in the no-swizzle K-major core-matrix layout
+  for (int i = tid; i < 256; i += C::NTHREADS) {
+    const int k8 = (i >> 3) & 1;                 // 16-byte unit i: row group i>>4, k-half k8, row-in-group i&7
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (k8 == 0) {
+      v.x = 0x3F803F80u;                         // bf16 1.0, 1.0
+      v.y = 0x00003F80u;                         // bf16 1.0, 0
+    }
+    reinterpret_cast<uint4*>(smem + C::OFF_ONES)[i] = v;
+  }
+  if (warp == 13) {
     tmem_alloc(tmem_slot, C::TMEM_COLS);
     tmem_relinquish();
   }
+  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const int it_begin = p.cta_offsets[blockIdx.x], it_end = p.cta_offsets[blockIdx.x + 1];
 
-  if (warp == 8) {
+  if (warp == 12) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&mq);
@@ -130,6 +158,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       for (int it = it_begin; it < it_end && ok; ++it) {
         const WorkItem w = p.items[it];
         const bool ord = w.kind == KIND_ORDINARY;
+        const size_t bh = static_cast<size_t>(w.b) * p.H + w.h;
         if (ord) {
           ok = mbar_wait(kv_empty, (nkv & 1) ^ 1, wc, B_KV_EMPTY);
           if (!ok) break;
@@ -142,176 +171,289 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           const int s = nqdo % C::NS;
           ok = mbar_wait(qdo_empty + s, ((nqdo / C::NS) & 1) ^ 1, wc, B_QDO_EMPTY);
           if (!ok) break;
-          mbar_expect_tx(qdo_full + s, ord ? 2 * C::PANEL : C::PANEL);
-          if (ord) tma_load_4d(smem + C::OFF_Q + s * C::PANEL, &mq, qdo_full + s, 0, I * BLK, w.h, w.b);
+          mbar_expect_tx(qdo_full + s, ord ? 2 * C::PANEL + 8192 : C::PANEL);
+          if (ord) {
+            tma_load_4d(smem + C::OFF_Q + s * C::PANEL, &mq, qdo_full + s, 0, I * BLK, w.h, w.b);
+            const size_t img = (bh * nblk + I) * 4096;
+            bulk_load(smem + C::OFF_QX + s * 4096, static_cast<const uint8_t*>(p.q_ext) + img, 4096, qdo_full + s);
+            bulk_load(smem + C::OFF_DOX + s * 4096, static_cast<const uint8_t*>(p.do_ext) + img, 4096, qdo_full + s);
+          }
           tma_load_4d(smem + C::OFF_DO + s * C::PANEL, &mdo, qdo_full + s, 0, I * BLK, w.h, w.b);
           ++nqdo;
         }
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == 13) {
     // ------------------------------------------------------------------ tcgen05 issuer
-    if (lane == 0) {
-      const uint32_t sb = smem_u32(smem);
-      constexpr uint32_t id_s = umma_idesc_bf16(128, 128, 0, 0);     // S^T, dP^T: both operands K-major
-      constexpr uint32_t id_acc = umma_idesc_bf16(128, 64, 0, 1);    // dV, dK: A from TMEM, B MN-major
-      constexpr uint32_t id_dq = umma_idesc_bf16(128, 64, 1, 1);     // dQ: A (dS^T tile) M-major, B MN-major
-      uint32_t nkv = 0, nqdo = 0, npds = 0, nitem = 0, ndq = 0;
-      bool ok = true;
-      for (int it = it_begin; it < it_end && ok; ++it, ++nitem) {
-        const WorkItem w = p.items[it];
-        const bool ord = w.kind == KIND_ORDINARY;
-        if (ord) {
-          ok = mbar_wait(kv_full, nkv & 1, wc, B_KV_FULL);
-          if (!ok) break;
-          ++nkv;
-        }
-        int t = 0;
-        for (int I = w.blk; I < nblk; ++I, ++t) {
-          const int s = nqdo % C::NS;
-          ok = mbar_wait(qdo_full + s, (nqdo / C::NS) & 1, wc, B_QDO_FULL);
-          if (!ok) break;
-          ++nqdo;
-          tc_fence_after();
-          const uint32_t q_s = sb + C::OFF_Q + s * C::PANEL, do_s = sb + C::OFF_DO + s * C::PANEL;
-          if (ord) {
-#pragma unroll
-            for (int kc = 0; kc < 4; ++kc)
-              umma_ss(tmem + C::COL_S, umma_smem_desc(sb + C::OFF_K + 32 * kc, 16, 1024, UMMA_LAYOUT_SW128),
-                      umma_smem_desc(q_s + 32 * kc, 16, 1024, UMMA_LAYOUT_SW128), id_s, kc > 0);
-#pragma unroll
-            for (int kc = 0; kc < 4; ++kc)
-              umma_ss(tmem + C::COL_DP, umma_smem_desc(sb + C::OFF_V + 32 * kc, 16, 1024, UMMA_LAYOUT_SW128),
-                      umma_smem_desc(do_s + 32 * kc, 16, 1024, UMMA_LAYOUT_SW128), id_s, kc > 0);
-            umma_commit(sdp_full);
+    // The whole warp walks the loops (warp-uniform operands); one elected lane issues.
+    const bool leader = elect_one() != 0;
+    const uint32_t sb = smem_u32(smem);
+    constexpr uint32_t id_s = umma_idesc_bf16(128, 64, 0, 0);      // S^T, dP^T half tiles: both operands K-major
+    constexpr uint32_t id_acc = umma_idesc_bf16(128, 64, 0, 1);    // dV, dK: A from TMEM, B MN-major
+    constexpr uint32_t id_dq = umma_idesc_bf16(128, 64, 1, 1);     // dQ: A (dS^T tile) M-major, B MN-major
+    // descriptor halves for smem offset 0: 128B-swizzled K-major (k-step +32 B), 128B-swizzled MN-major
+    // (k-step +2048 B, LBO = panel) and the no-swizzle K-major row-term tiles (LBO 128 B, SBO 256 B)
+    const uint64_t d_k = umma_smem_desc(sb, 16, 1024, UMMA_LAYOUT_SW128);
+    const uint64_t d_m = umma_smem_desc(sb, C::PANEL, 1024, UMMA_LAYOUT_SW128);
+    const uint64_t d_x = umma_smem_desc(sb, 128, 256, UMMA_LAYOUT_NONE);
+    const uint32_t lo_k = desc_lo(d_k), hi_k = desc_hi(d_k), lo_m = desc_lo(d_m), hi_m = desc_hi(d_m);
+    const uint32_t lo_x = desc_lo(d_x), hi_x = desc_hi(d_x);
+    const uint32_t k_lo = lo_k + (C::OFF_K >> 4), v_lo = lo_k + (C::OFF_V >> 4);
+    const uint32_t ones_lo = lo_x + (C::OFF_ONES >> 4), km_lo = lo_m + (C::OFF_K >> 4);
+    uint32_t nkv = 0, nqdo = 0, nitem = 0, ndq = 0, ntile_ord = 0;
+    uint32_t npds0 = 0, npds1 = 0;
+    int tr_n = 0;
+    (void)tr_n;
+    bool ok = true;
+    for (int it = it_begin; it < it_end && ok; ++it, ++nitem) {
+      const WorkItem w = p.items[it];
+      const bool ord = w.kind == KIND_ORDINARY;
+      const int ntiles = nblk - w.blk;
+      if (ord) {
+        ok = mbar_wait_warp(kv_full, nkv & 1, wc, B_KV_FULL);
+        if (!ok) break;
+        ++nkv;
+        const int U = 2 * ntiles;
+        const uint32_t stage0 = nqdo;                   // ring position of this item's first tile
+        // A(u): augmented scores and dP of half tile u into TMEM buffer u&1
+        auto issue_a = [&](int u) -> bool {
+          const uint32_t pos = stage0 + (u >> 1);
+          const uint32_t s = pos % C::NS;
+          const uint32_t b = u & 1;
+          if (b == 0) {
+            if (!mbar_wait_warp(qdo_full + s, (pos / C::NS) & 1, wc, B_QDO_FULL)) return false;
+            tc_fence_after();
           }
-          ok = mbar_wait(pds_full, npds & 1, wc, B_PDS_FULL);
+          const uint32_t q_lo = lo_k + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
+          const uint32_t do_lo = lo_k + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
+          const uint32_t qx_lo = lo_x + ((C::OFF_QX + s * 4096 + b * 2048) >> 4);
+          const uint32_t dox_lo = lo_x + ((C::OFF_DOX + s * 4096 + b * 2048) >> 4);
+          const uint32_t t_s = tmem + C::COL_S + 64 * b, t_dp = tmem + C::COL_DP + 64 * b;
+          if (leader) {
+#pragma unroll
+            for (int kc = 0; kc < 4; ++kc) umma_ss2(t_s, k_lo + 2 * kc, hi_k, q_lo + 2 * kc, hi_k, id_s, kc > 0);
+            umma_ss2(t_s, ones_lo, hi_x, qx_lo, hi_x, id_s, 1);
+#pragma unroll
+            for (int kc = 0; kc < 4; ++kc) umma_ss2(t_dp, v_lo + 2 * kc, hi_k, do_lo + 2 * kc, hi_k, id_s, kc > 0);
+            umma_ss2(t_dp, ones_lo, hi_x, dox_lo, hi_x, id_s, 1);
+            umma_commit(sdp_full + b);
+          }
+          __syncwarp();
+          return true;
+        };
+        ok = issue_a(0);
+        for (int u = 0; u < U && ok; ++u) {
+          const uint32_t b = u & 1;
+          if (u + 1 < U) {
+            ok = issue_a(u + 1);
+            if (!ok) break;
+          }
+          TR(0, 4);
+          if (b == 0) {
+            ok = mbar_wait_warp(pds_full, npds0 & 1, wc, B_PDS_FULL);
+            ++npds0;
+          } else {
+            ok = mbar_wait_warp(pds_full + 1, npds1 & 1, wc, B_PDS_FULL);
+            ++npds1;
+          }
           if (!ok) break;
-          ++npds;
-          if (t == 0) {
-            ok = mbar_wait(acc_free, (nitem & 1) ^ 1, wc, B_ACC_FREE);
+          TR(0, 5);
+          if (u == 0) {
+            ok = mbar_wait_warp(acc_free, (nitem & 1) ^ 1, wc, B_ACC_FREE);
             if (!ok) break;
           }
           tc_fence_after();
-          // ordinary: P^T pairs sit in columns [0,32) and [64,96); frozen: contiguous in buffer t&1
-          const uint32_t pcol = ord ? C::COL_S : (t & 1) * 64;
-          const uint32_t hstep = ord ? 32u : 0u;     // extra column offset of k-steps 4..7
+          const uint32_t pos = stage0 + (u >> 1);
+          const uint32_t s = pos % C::NS;
+          const uint32_t q_lo = lo_m + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
+          const uint32_t do_lo = lo_m + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
+          const uint32_t acc0 = u > 0 ? 1u : 0u;
+          const uint32_t t_p = tmem + C::COL_S + 64 * b, t_ds = tmem + C::COL_DP + 64 * b;
+          if (leader) {
 #pragma unroll
-          for (int kc = 0; kc < 8; ++kc)
-            umma_ts(tmem + C::COL_DV, tmem + pcol + 8 * kc + (kc >= 4 ? hstep : 0u),
-                    umma_smem_desc(do_s + 2048 * kc, C::PANEL, 1024, UMMA_LAYOUT_SW128), id_acc,
-                    (t > 0 || kc > 0) ? 1u : 0u);
-          if (ord) {
+            for (int kc = 0; kc < 4; ++kc)
+              umma_ts2(tmem + C::COL_DV, t_p + 8 * kc, do_lo + 128 * kc, hi_m, id_acc, kc > 0 ? 1u : acc0);
 #pragma unroll
-            for (int kc = 0; kc < 8; ++kc)
-              umma_ts(tmem + C::COL_DK, tmem + C::COL_DP + 8 * kc + (kc >= 4 ? 32u : 0u),
-                      umma_smem_desc(q_s + 2048 * kc, C::PANEL, 1024, UMMA_LAYOUT_SW128), id_acc,
-                      (t > 0 || kc > 0) ? 1u : 0u);
-            umma_commit(qdo_empty + s);
-            ok = mbar_wait(dq_free, (ndq & 1) ^ 1, wc, B_DQ_FREE);
+            for (int kc = 0; kc < 4; ++kc)
+              umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc, q_lo + 128 * kc, hi_m, id_acc, kc > 0 ? 1u : acc0);
+          }
+          TR(0, 6);
+          if (b == 1) {
+            // full tile done: its Q/dO stage can be refilled, and dQ of the tile follows
+            if (leader) umma_commit(qdo_empty + s);
+            ok = mbar_wait_warp(dq_free, (ndq & 1) ^ 1, wc, B_DQ_FREE);
             if (!ok) break;
             ++ndq;
             tc_fence_after();
+            const uint32_t ds_lo = lo_m + ((C::OFF_DS + (ntile_ord & 1) * 2 * C::PANEL) >> 4);
+            if (leader) {
 #pragma unroll
-            for (int kc = 0; kc < 8; ++kc)
-              umma_ss(tmem + C::COL_DQ, umma_smem_desc(sb + C::OFF_DS + 2048 * kc, C::PANEL, 1024, UMMA_LAYOUT_SW128),
-                      umma_smem_desc(sb + C::OFF_K + 2048 * kc, C::PANEL, 1024, UMMA_LAYOUT_SW128), id_dq, kc > 0);
-            umma_commit(dq_full);
-          } else {
-            umma_commit(qdo_empty + s);
-            umma_commit(pfree + (t & 1));
+              for (int kc = 0; kc < 8; ++kc)
+                umma_ss2(tmem + C::COL_DQ, ds_lo + 128 * kc, hi_m, km_lo + 128 * kc, hi_m, id_dq, kc > 0);
+              umma_commit(dq_full);
+            }
+            TR(0, 9);
+            ++ntile_ord;
           }
+          __syncwarp();
         }
         if (!ok) break;
-        if (ord) umma_commit(kv_empty);
-        umma_commit(acc_full);
+        nqdo += ntiles;
+        if (leader) umma_commit(kv_empty);
+      } else {
+        for (int t = 0; t < ntiles; ++t) {
+          const uint32_t s = nqdo % C::NS;
+          ok = mbar_wait_warp(qdo_full + s, (nqdo / C::NS) & 1, wc, B_QDO_FULL);
+          if (!ok) break;
+          ++nqdo;
+          const uint32_t b = t & 1;
+          if (b == 0) {
+            ok = mbar_wait_warp(pds_full, npds0 & 1, wc, B_PDS_FULL);
+            ++npds0;
+          } else {
+            ok = mbar_wait_warp(pds_full + 1, npds1 & 1, wc, B_PDS_FULL);
+            ++npds1;
+          }
+          if (!ok) break;
+          if (t == 0) {
+            ok = mbar_wait_warp(acc_free, (nitem & 1) ^ 1, wc, B_ACC_FREE);
+            if (!ok) break;
+          }
+          tc_fence_after();
+          const uint32_t do_lo = lo_m + ((C::OFF_DO + s * C::PANEL) >> 4);
+          const uint32_t acc0 = t > 0 ? 1u : 0u;
+          if (leader) {
+#pragma unroll
+            for (int kc = 0; kc < 8; ++kc)
+              umma_ts2(tmem + C::COL_DV, tmem + C::COL_S + 64 * b + 8 * kc, do_lo + 128 * kc, hi_m, id_acc,
+                       kc > 0 ? 1u : acc0);
+            umma_commit(qdo_empty + s);
+            umma_commit(pfree + b);
+          }
+          __syncwarp();
+        }
+        if (!ok) break;
       }
+      if (leader) umma_commit(acc_full);
+      __syncwarp();
     }
-  } else {
-    // ------------------------------------------------------------------ compute warps (256 threads)
-    const int q4 = warp & 3, half = warp >> 2;
-    const int rowl = q4 * 32 + lane;                     // TMEM lane: key row (tile loop) / query row (dQ drain)
+  } else if (warp >= 8) {
+    // ------------------------------------------------------------------ dQ drain warps (128 threads)
+    const int q4 = warp & 3;                            // TMEM lane quarter of this warp
+    const int rowl = q4 * 32 + lane;                    // query row within the tile
     const uint32_t lane_base = static_cast<uint32_t>(q4 * 32) << 16;
-    uint32_t nsdp = 0, ndq = 0, nacc = 0, npf0 = 0, npf1 = 0;
+    uint32_t ndq = 0;
     bool ok = true;
+    const uint32_t stage_row = smem_u32(smem + C::OFF_DQ) + rowl * 128;
+    for (int it = it_begin; it < it_end; ++it) {
+      const WorkItem w = p.items[it];
+      if (w.kind != KIND_ORDINARY) continue;
+      bool leave = false;
+      for (int I = w.blk; I < nblk; ++I) {
+        // the previous tile's reduce has finished reading the staging buffer (thread 256 waits for it
+        // before arriving here); the drain warps also agree here whether a wait has been abandoned
+        if (named_bar_or(2, 128, !ok)) {
+          leave = true;
+          break;
+        }
+        if (!mbar_wait_warp(dq_full, ndq & 1, wc, B_DQ_FULL)) ok = false;
+        ++ndq;
+        tc_fence_after();
+        uint32_t r0[32], r1[32];
+        tmem_ld32(tmem + lane_base + C::COL_DQ, r0);
+        tmem_ld32(tmem + lane_base + C::COL_DQ + 32, r1);
+        tmem_wait_ld();
+        tc_fence_before();
+        warp_arrive(dq_free);                           // the tensor core may overwrite dQ
+        // fp32 rows -> two [128][32] boxes, 128-byte swizzle (16-byte chunk index ^= row & 7)
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const uint32_t chunk = static_cast<uint32_t>(g ^ (rowl & 7)) * 16;
+          st_shared_v4(stage_row + chunk, __float_as_uint(__uint_as_float(r0[4 * g]) * p.scale),
+                       __float_as_uint(__uint_as_float(r0[4 * g + 1]) * p.scale),
+                       __float_as_uint(__uint_as_float(r0[4 * g + 2]) * p.scale),
+                       __float_as_uint(__uint_as_float(r0[4 * g + 3]) * p.scale));
+          st_shared_v4(stage_row + C::PANEL + chunk, __float_as_uint(__uint_as_float(r1[4 * g]) * p.scale),
+                       __float_as_uint(__uint_as_float(r1[4 * g + 1]) * p.scale),
+                       __float_as_uint(__uint_as_float(r1[4 * g + 2]) * p.scale),
+                       __float_as_uint(__uint_as_float(r1[4 * g + 3]) * p.scale));
+        }
+        fence_proxy_async_smem();
+        named_bar_sync(3, 128);
+        if (tid == 256 && ok) {
+          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 0, I * BLK, w.h, w.b);
+          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ + C::PANEL, 32, I * BLK, w.h, w.b);
+          bulk_commit_group();
+          bulk_wait_group_read0();
+        }
+      }
+      if (leave) break;
+    }
+    if (tid == 256) bulk_wait_group0();                 // all reduce-adds have landed before the kernel ends
+  } else {
+    // ------------------------------------------------------------------ compute groups (2 x 128 threads)
+    const int grp = warp >> 2, q4 = warp & 3;
+    const int gtid = tid & 127;                          // thread index within the group
+    const int rowl = q4 * 32 + lane;                     // TMEM lane = key row of the block
+    const uint32_t lane_base = static_cast<uint32_t>(q4 * 32) << 16;
+    float* tab = reinterpret_cast<float*>(smem + C::OFF_TAB) + grp * C::TAB_FLOATS;
+    float* wq = tab;
+    float* z2s = tab + 128;
+    float* rband = tab + 256;
+    float* r2raw = tab + 512;
+    float* red = tab + 768;
+    const int bar_id = 4 + grp;                          // named barrier of this group
+    uint32_t nacc = 0, ntile_ord = 0, nsdp = 0, npf = 0;
+    bool ok = true;
+    int tr_n = 0;
+    (void)tr_n;
+    // A warp whose wait was abandoned keeps walking (without storing) to the next agreement barrier,
+    // where the warps of its group leave together; none is ever left alone at a named barrier.
     for (int it = it_begin; it < it_end; ++it) {
       const WorkItem w = p.items[it];
       const bool ord = w.kind == KIND_ORDINARY;
       const int ntiles = nblk - w.blk;
       const int key = w.blk * BLK + rowl;
       const size_t bh = static_cast<size_t>(w.b) * p.H + w.h;
-      bool leave = false;
+      if (named_bar_or(bar_id, 128, !ok)) break;
+
       if (ord) {
         const float c = p.scale_log2;
         for (int t = 0; t < ntiles; ++t) {
-          const int I = w.blk + t;
-          if (named_bar_or(1, C::NCT, !ok)) {   // uniform over the compute warps: leave together
-            ok = false;
-            leave = true;
-            break;
-          }
-          if (tid < 128) {
-            const int qi = I * BLK + tid;
-            lse2s[tid] = (qi < p.T) ? p.LSE[bh * p.T + qi] * LOG2E_B : INFINITY;
-            dels[tid] = (qi < p.T) ? p.delta[bh * p.Tpad + qi] : 0.0f;
-          }
-          // drain dQ of the previous tile while the tensor core works on this tile's S^T / dP^T
-          if (t > 0) {
-            if (mbar_wait_warp(dq_full, ndq & 1, wc, B_DQ_FULL)) {
-              ++ndq;
-              tc_fence_after();
-              uint32_t r[32];
-              tmem_ld32(tmem + lane_base + C::COL_DQ + 32 * half, r);
-              tmem_wait_ld();
-              const int qi = (I - 1) * BLK + rowl;
-              if (qi < p.T && ok) {
-                float* dst = p.dQacc + (bh * p.T + qi) * 64 + 32 * half;
-#pragma unroll
-                for (int e = 0; e < 8; ++e)
-                  red_add_v4(dst + 4 * e, __uint_as_float(r[4 * e]) * p.scale, __uint_as_float(r[4 * e + 1]) * p.scale,
-                             __uint_as_float(r[4 * e + 2]) * p.scale, __uint_as_float(r[4 * e + 3]) * p.scale);
-              }
-              tc_fence_before();
-              mbar_arrive(dq_free);
-            } else {
-              ok = false;
-            }
-          }
-          named_bar_sync(1, C::NCT);
-          if (!mbar_wait_warp(sdp_full, nsdp & 1, wc, B_SDP_FULL)) ok = false;
+          // this group's half tile of tile t: queries 64*grp .. 64*grp+63
+          TR(1 + grp, 11);
+          if (!mbar_wait_warp(sdp_full + grp, nsdp & 1, wc, B_SDP_FULL)) ok = false;
           ++nsdp;
           tc_fence_after();
+          TR(1 + grp, 12);
+          const uint32_t t_s = tmem + lane_base + C::COL_S + 64 * grp;
+          const uint32_t t_dp = tmem + lane_base + C::COL_DP + 64 * grp;
+          const uint32_t rowaddr =
+              smem_u32(smem + C::OFF_DS + ((ntile_ord + t) & 1) * 2 * C::PANEL + grp * C::PANEL) + rowl * 128;
           const bool diag = (t == 0);
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
-            const int q0 = 64 * half + 32 * cc;          // first query column of this chunk
             uint32_t rs[32], rd[32];
-            tmem_ld32(tmem + lane_base + C::COL_S + q0, rs);
-            tmem_ld32(tmem + lane_base + C::COL_DP + q0, rd);
+            tmem_ld32(t_s + 32 * cc, rs);
+            tmem_ld32(t_dp + 32 * cc, rd);
             tmem_wait_ld();
             uint32_t pk[16], dk[16];
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              const int qa = q0 + 2 * e;
-              const float2 l2 = *reinterpret_cast<const float2*>(lse2s + qa);
-              const float2 de = *reinterpret_cast<const float2*>(dels + qa);
-              float p0 = ex2_approx(fmaf(__uint_as_float(rs[2 * e]), c, -l2.x));
-              float p1 = ex2_approx(fmaf(__uint_as_float(rs[2 * e + 1]), c, -l2.y));
-              if (diag) {                                // causal: query index >= key index
+              float p0 = ex2_approx(__uint_as_float(rs[2 * e]) * c);
+              float p1 = ex2_approx(__uint_as_float(rs[2 * e + 1]) * c);
+              if (diag) {                                  // causal: query index >= key index
+                const int qa = 64 * grp + 32 * cc + 2 * e;
                 if (qa < rowl) p0 = 0.0f;
                 if (qa + 1 < rowl) p1 = 0.0f;
               }
-              const float d0 = p0 * (__uint_as_float(rd[2 * e]) - de.x);
-              const float d1 = p1 * (__uint_as_float(rd[2 * e + 1]) - de.y);
               pk[e] = pack_bf16x2(p0, p1);
-              dk[e] = pack_bf16x2(d0, d1);
+              dk[e] = pack_bf16x2(p0 * __uint_as_float(rd[2 * e]), p1 * __uint_as_float(rd[2 * e + 1]));
             }
-            // bf16 pairs go where this warp has already consumed the fp32 values: queries 0-63 in
-            // columns +[0,32), queries 64-127 in columns +[64,96) (the other half's columns are still live)
-            tmem_st16(tmem + lane_base + C::COL_S + 64 * half + 16 * cc, pk);
-            tmem_st16(tmem + lane_base + C::COL_DP + 64 * half + 16 * cc, dk);
-            // dS^T row (this key) -> smem panel `half`, 128-byte swizzle: 16-byte chunk index ^= row & 7
-            const uint32_t rowaddr = smem_u32(smem + C::OFF_DS + half * C::PANEL + rowl * 128);
+            // bf16 pairs re-use columns this warp has already consumed
+            tmem_st16(t_s + 16 * cc, pk);
+            tmem_st16(t_dp + 16 * cc, dk);
+            // dS^T row (this key) -> smem panel of this half tile, 128-byte swizzle (chunk ^= row & 7)
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
               const uint32_t chunk = static_cast<uint32_t>((4 * cc + g) ^ (rowl & 7));
@@ -321,29 +463,12 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           tmem_wait_st();
           fence_proxy_async_smem();
           tc_fence_before();
-          mbar_arrive(pds_full);
+          warp_arrive(pds_full + grp);
+          TR(1 + grp, 16);
         }
-        // last tile's dQ
-        {
-          if (!mbar_wait_warp(dq_full, ndq & 1, wc, B_DQ_FULL)) ok = false;
-          ++ndq;
-          tc_fence_after();
-          uint32_t r[32];
-          tmem_ld32(tmem + lane_base + C::COL_DQ + 32 * half, r);
-          tmem_wait_ld();
-          const int qi = (nblk - 1) * BLK + rowl;
-          if (qi < p.T && ok) {
-            float* dst = p.dQacc + (bh * p.T + qi) * 64 + 32 * half;
-#pragma unroll
-            for (int e = 0; e < 8; ++e)
-              red_add_v4(dst + 4 * e, __uint_as_float(r[4 * e]) * p.scale, __uint_as_float(r[4 * e + 1]) * p.scale,
-                         __uint_as_float(r[4 * e + 2]) * p.scale, __uint_as_float(r[4 * e + 3]) * p.scale);
-          }
-          tc_fence_before();
-          mbar_arrive(dq_free);
-        }
+        ntile_ord += ntiles;
       } else {
-        // ---------------- frozen head: P^^T tiles
+        // ---------------- frozen head: P^^T tiles; group g generates tiles t = g, g+2, ...
         const float* alpha_h = p.alpha + static_cast<size_t>(w.h) * p.Tp;
         const float* rho_h = p.rho + static_cast<size_t>(w.h) * p.Tp;
         const float* logz_h = p.logZ + static_cast<size_t>(w.h) * p.Tp;
@@ -352,66 +477,52 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ma = fmaxf(ma, __shfl_xor_sync(0xffffffffu, ma, o));
         // block maximum of alpha over the 128 keys: exchanged once per item through `red`
-        if (named_bar_or(1, C::NCT, !ok)) {
-          ok = false;
-          break;
-        }
-        if (lane == 0 && half == 0) red[16 + q4] = ma;
-        named_bar_sync(1, C::NCT);
-        ma = fmaxf(fmaxf(red[16], red[17]), fmaxf(red[18], red[19]));
+        if (lane == 0) red[12 + q4] = ma;
+        named_bar_sync(bar_id, 128);
+        ma = fmaxf(fmaxf(red[12], red[13]), fmaxf(red[14], red[15]));
         const float aj = ex2_approx(a2 - ma);
-        for (int t = 0; t < ntiles; ++t) {
+        bool leave = false;
+        int nmine = 0;
+        for (int t = grp; t < ntiles; t += 2, ++nmine) {
           const int I = w.blk + t;
-          if (named_bar_or(1, C::NCT, !ok)) {   // uniform over the compute warps: leave together
+          if (named_bar_or(bar_id, 128, !ok)) {          // uniform over the group: leave together
             ok = false;
             leave = true;
             break;
           }
-          const int d0 = t * BLK - 127;                // band: distances d0 .. d0+254, index x = q - row + 127
-          float r2v = -INFINITY;
-          {
-            const int d = d0 + tid;                    // tid in [0,256): one band entry per compute thread
-            if (tid < 255 && d >= 0 && d < p.T) r2v = rho_h[d] * LOG2E_B;
-            r2raw[tid] = r2v;
-            float mr = r2v;
+          const int d0 = t * BLK - 127;                  // band: distances d0 .. d0+254, index x = q - row + 127
+          const int da = d0 + gtid, db = d0 + 128 + gtid;
+          const float r2a = (da >= 0 && da < p.T) ? rho_h[da] * LOG2E_B : -INFINITY;
+          const float r2b = (gtid < 127 && db >= 0 && db < p.T) ? rho_h[db] * LOG2E_B : -INFINITY;
+          r2raw[gtid] = r2a;
+          r2raw[128 + gtid] = r2b;
+          float mr = fmaxf(r2a, r2b);
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, o));
-            if (lane == 0) red[warp] = mr;
-          }
-          float z2 = INFINITY;
-          if (tid < 128) {
-            const int qi = I * BLK + tid;
-            if (qi < p.T) z2 = logz_h[qi] * LOG2E_B;
-            z2s[tid] = z2;
-          }
-          named_bar_sync(1, C::NCT);
-          float mr = red[0];
-#pragma unroll
-          for (int k = 1; k < 8; ++k) mr = fmaxf(mr, red[k]);
-          rband[tid] = ex2_approx(r2v - mr);
-          bool bad = false;
-          if (tid < 128) {
-            const float ew = ma + mr - z2;
-            bad = ew > 100.0f;
-            wq[tid] = ex2_approx(ew);
-          }
-          const unsigned anybad = __any_sync(0xffffffffu, bad);
-          if (lane == 0) red[8 + warp] = anybad ? 1.0f : 0.0f;
-          named_bar_sync(1, C::NCT);
-          bool exact = false;
-#pragma unroll
-          for (int k = 0; k < 4; ++k) exact |= red[8 + k] > 0.0f;
-          // buffer (t&1) must have been consumed by the dV MMA of tile t-2
-          if (t >= 2) {
-            uint32_t& n = (t & 1) ? npf1 : npf0;
-            if (!mbar_wait_warp(pfree + (t & 1), n & 1, wc, B_PFREE)) ok = false;
-            ++n;
+          for (int o = 16; o > 0; o >>= 1) mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, o));
+          if (lane == 0) red[q4] = mr;
+          const int qi = I * BLK + gtid;
+          const float z2 = (qi < p.T) ? logz_h[qi] * LOG2E_B : INFINITY;
+          z2s[gtid] = z2;
+          named_bar_sync(bar_id, 128);
+          mr = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+          rband[gtid] = ex2_approx(r2a - mr);
+          rband[128 + gtid] = ex2_approx(r2b - mr);
+          const float ew = ma + mr - z2;
+          wq[gtid] = ex2_approx(ew);
+          const unsigned anybad = __any_sync(0xffffffffu, ew > 100.0f);
+          if (lane == 0) red[4 + q4] = anybad ? 1.0f : 0.0f;
+          named_bar_sync(bar_id, 128);
+          const bool exact = (red[4] + red[5] + red[6] + red[7]) > 0.0f;
+          // this group's buffer must have been consumed by the dV MMA of its previous tile
+          if (nmine > 0) {
+            if (!mbar_wait_warp(pfree + grp, npf & 1, wc, B_PFREE)) ok = false;
+            ++npf;
             tc_fence_after();
           }
-          const uint32_t t_p = tmem + lane_base + (t & 1) * 64;
+          const uint32_t t_p = tmem + lane_base + C::COL_S + grp * 64;
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            const int q0 = 64 * half + 32 * cc;
+          for (int cc = 0; cc < 4; ++cc) {
+            const int q0 = 32 * cc;
             uint32_t pk[16];
             if (!exact) {
               const float* rb = rband + (q0 - rowl + 127);
@@ -432,37 +543,27 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
                 pk[e] = pack_bf16x2(p0, p1);
               }
             }
-            tmem_st16(t_p + (q0 >> 1), pk);
+            tmem_st16(t_p + 16 * cc, pk);
           }
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(pds_full);
+          warp_arrive(pds_full + grp);
+        }
+        if (leave) break;
+        // keep the buffer barrier in step: absorb the completion of this group's last tile
+        if (nmine > 0) {
+          if (!mbar_wait_warp(pfree + grp, npf & 1, wc, B_PFREE)) ok = false;
+          ++npf;
         }
       }
-      if (leave) break;
-      // ---------------- epilogue: dV (warps 0-3) and dK (warps 4-7) of this key block
-      // (a warp whose wait was abandoned keeps walking - without storing - to the next agreement
-      // barrier, so that no other compute warp is left waiting for it)
+      // ---------------- epilogue: dV (group 0) and dK (group 1) of this key block
       if (!mbar_wait_warp(acc_full, nacc & 1, wc, B_ACC_FULL)) ok = false;
       ++nacc;
       tc_fence_after();
-      if (!ord) {
-        // keep the double-buffer barriers in step: absorb the completions not waited for in the loop
-        const int left0 = (ntiles + 1) / 2 - ((ntiles > 2) ? (ntiles - 1) / 2 : 0);   // buffer 0: tiles 0,2,4,..
-        const int left1 = ntiles / 2 - ((ntiles > 3) ? (ntiles - 2) / 2 : 0);          // buffer 1: tiles 1,3,5,..
-        for (int k = 0; k < left0; ++k) {
-          if (!mbar_wait_warp(pfree, npf0 & 1, wc, B_PFREE)) ok = false;
-          ++npf0;
-        }
-        for (int k = 0; k < left1; ++k) {
-          if (!mbar_wait_warp(pfree + 1, npf1 & 1, wc, B_PFREE)) ok = false;
-          ++npf1;
-        }
-      }
-      if (half == 0 || ord) {
-        const uint32_t col = half == 0 ? C::COL_DV : C::COL_DK;
-        const float mul = half == 0 ? 1.0f : p.scale;
-        void* base = half == 0 ? p.dV : p.dK;
+      if (grp == 0 || ord) {
+        const uint32_t col = grp == 0 ? C::COL_DV : C::COL_DK;
+        const float mul = grp == 0 ? 1.0f : p.scale;
+        void* base = grp == 0 ? p.dV : p.dK;
         const size_t off = (bh * p.T + key) * 64;
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
@@ -489,28 +590,30 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         }
       }
       tc_fence_before();
-      mbar_arrive(acc_free);
+      warp_arrive(acc_free);
     }
   }
 
   // ------------------------------------------------------------------ teardown
   __syncwarp();
   if (*abort_flag) {
+    // A wait gave up: let copies and MMAs that are still in flight land before the CTA's
+    // shared memory and TMEM are released.
     for (int i = 0; i < 64; ++i) __nanosleep(20000);
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) tmem_dealloc(tmem, C::TMEM_COLS);
+  if (warp == 13) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
 int bwd_smem_bytes(int) { return BwdCfg::SMEM; }
 
 cudaError_t launch_bwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t st) {
+                       const CUtensorMap& mdo, const CUtensorMap& mdq, const BwdParams& p, int grid, cudaStream_t st) {
   if (D != 64) return cudaErrorNotSupported;
   cudaError_t e = cudaFuncSetAttribute(saf_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg::SMEM);
   if (e != cudaSuccess) return e;
-  saf_bwd_kernel<<<grid, 320, BwdCfg::SMEM, st>>>(mq, mk, mv, mdo, p);
+  saf_bwd_kernel<<<grid, BwdCfg::NTHREADS, BwdCfg::SMEM, st>>>(mq, mk, mv, mdo, mdq, p);
   return cudaGetLastError();
 }
 

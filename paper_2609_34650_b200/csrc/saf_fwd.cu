@@ -81,9 +81,9 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       mbar_init(v_empty + s, 1);
     }
     mbar_init(s_full, 1);
-    mbar_init(p_full, 128);
+    mbar_init(p_full, 4);
     mbar_init(pv_done, 1);
-    mbar_init(o_free, 128);
+    mbar_init(o_free, 4);
     mbar_fence_init();
   }
   if (warp == 5) {
@@ -146,6 +146,11 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       constexpr uint32_t idesc_o = umma_idesc_bf16(128, D, 0, 1);
       uint32_t nq = 0, nk = 0, nv = 0, np = 0, nitem = 0;
       bool ok = true;
+      // descriptor halves for smem offset 0: K-major tiles (k-step +32 B within a 64-column panel) and
+      // the MN-major V tile (k-step +2048 B, LBO = panel stride)
+      const uint64_t d_kmaj = umma_smem_desc(sb, 16, 1024, UMMA_LAYOUT_SW128);
+      const uint64_t d_mn = umma_smem_desc(sb, C::PANEL_BYTES, 1024, UMMA_LAYOUT_SW128);
+      const uint32_t lo_k = desc_lo(d_kmaj), hi_k = desc_hi(d_kmaj), lo_m = desc_lo(d_mn), hi_m = desc_hi(d_mn);
       for (int it = it_begin; it < it_end && ok; ++it, ++nitem) {
         const WorkItem w = p.items[it];
         const int ntiles = w.blk + 1;
@@ -161,12 +166,11 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             if (!ok) break;
             ++nk;
             tc_fence_after();
+            const uint32_t q_lo = lo_k + (C::OFF_Q >> 4), k_lo = lo_k + ((C::OFF_K + s * C::TILE_BYTES) >> 4);
 #pragma unroll
             for (int kc = 0; kc < D / 16; ++kc) {
-              const uint32_t off = (kc >> 2) * C::PANEL_BYTES + (kc & 3) * 32;
-              umma_ss(tmem + C::COL_S, umma_smem_desc(sb + C::OFF_Q + off, 16, 1024, UMMA_LAYOUT_SW128),
-                      umma_smem_desc(sb + C::OFF_K + s * C::TILE_BYTES + off, 16, 1024, UMMA_LAYOUT_SW128), idesc_s,
-                      kc > 0);
+              const uint32_t off = ((kc >> 2) * C::PANEL_BYTES + (kc & 3) * 32) >> 4;
+              umma_ss2(tmem + C::COL_S, q_lo + off, hi_k, k_lo + off, hi_k, idesc_s, kc > 0);
             }
             umma_commit(s_full);
             umma_commit(k_empty + s);
@@ -184,12 +188,11 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             if (!ok) break;
           }
           tc_fence_after();
+          const uint32_t v_lo = lo_m + ((C::OFF_V + s * C::TILE_BYTES) >> 4);
+          const uint32_t acc0 = j > 0 ? 1u : 0u;
 #pragma unroll
           for (int kc = 0; kc < 8; ++kc)
-            umma_ts(tmem + C::COL_O, tmem + C::COL_P + 8 * kc,
-                    umma_smem_desc(sb + C::OFF_V + s * C::TILE_BYTES + kc * 2048, C::PANEL_BYTES, 1024,
-                                   UMMA_LAYOUT_SW128),
-                    idesc_o, (j > 0 || kc > 0) ? 1u : 0u);
+            umma_ts2(tmem + C::COL_O, tmem + C::COL_P + 8 * kc, v_lo + 128 * kc, hi_m, idesc_o, kc > 0 ? 1u : acc0);
           umma_commit(v_empty + s);
           umma_commit(pv_done);
         }
@@ -283,7 +286,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           }
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(p_full);
+          warp_arrive(p_full);
         }
         inv_l = 1.0f / l;
         lse = (m_ref + log2f(l)) * LN2_F;
@@ -364,7 +367,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           }
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(p_full);
+          warp_arrive(p_full);
         }
       }
       // ---------------- epilogue: wait for the last P V, scale, store
@@ -393,7 +396,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       if (p.LSE != nullptr && row < p.T && ok)
         p.LSE[(static_cast<size_t>(w.b) * p.H + w.h) * p.T + row] = lse;
       tc_fence_before();
-      mbar_arrive(o_free);
+      warp_arrive(o_free);
     }
   }
 

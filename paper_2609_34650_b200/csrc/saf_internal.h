@@ -33,10 +33,12 @@ struct BwdParams {
   const float* alpha;
   const float* rho;
   const float* logZ;
-  const float* LSE;                 // [B][H][T]
-  const float* delta;               // [B][H][Tpad] workspace, rowsum(dO o O) for ordinary heads
-  int Tpad;
-  float* dQacc;                     // fp32 [B][H][T][D], zeroed before the launch (atomically accumulated)
+  // Workspace images of the extra reduction step that folds the row terms into the score MMAs
+  // (ordinary heads): per (b,h,128-row block) a 4 KB no-swizzle K-major tile [128 rows][16] bf16 whose
+  // first three columns hold a three-way bf16 split of -LSE/scale (q_ext) or of -delta (do_ext).
+  const void* q_ext;
+  const void* do_ext;
+  int nblk;
   void* dK;                         // [B][H][T][D] grad dtype
   void* dV;
   int grad_f32;
@@ -52,11 +54,12 @@ cudaError_t launch_logz(const float* alpha, const float* rho, float* logZ, const
 cudaError_t launch_fwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                        const FwdParams& p, int grid, cudaStream_t st);
 cudaError_t launch_bwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t st);
-// delta = rowsum(dO o O) for ordinary heads; also zeroes dQacc (all heads) and dK of frozen heads.
-cudaError_t launch_bwd_prep(const void* O, const void* dO, const int64_t* o_strides, const uint8_t* mask_dev,
-                            float* delta, int Tpad, float* dQacc, void* dK, int grad_f32, int B, int H, int T,
-                            int D, cudaStream_t st);
+                       const CUtensorMap& mdo, const CUtensorMap& mdq, const BwdParams& p, int grid, cudaStream_t st);
+// Row terms of ordinary heads (q_ext / do_ext images, see BwdParams); also zeroes dQacc (all heads) and
+// dK of frozen heads.
+cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* o_strides,
+                            const uint8_t* mask_dev, void* q_ext, void* do_ext, float inv_scale, float* dQacc,
+                            void* dK, int grad_f32, int B, int H, int T, int D, cudaStream_t st);
 // dQ (grad dtype) = scale-free copy/convert of dQacc (fp32) for the bf16-gradient case.
 cudaError_t launch_bwd_finalize(const float* dQacc, void* dQ, size_t n, cudaStream_t st);
 int fwd_smem_bytes(int D);

@@ -43,32 +43,54 @@ cudaError_t launch_logz(const float* alpha, const float* rho, float* logZ, const
   return cudaGetLastError();
 }
 
+// Three-way bf16 split of an fp32 value: hi + mid + lo reproduces x to ~24 bits.
+__device__ __forceinline__ uint4 split3_bf16(float x) {
+  const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+  const float r1 = x - __bfloat162float(hi);
+  const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+  const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+  uint4 v = make_uint4(0, 0, 0, 0);
+  v.x = static_cast<uint32_t>(__bfloat16_as_ushort(hi)) | (static_cast<uint32_t>(__bfloat16_as_ushort(mid)) << 16);
+  v.y = static_cast<uint32_t>(__bfloat16_as_ushort(lo));
+  return v;
+}
+
 // Backward preparation.  Eight threads per (b,h,row) with D = 64 (sixteen with D = 128), each owning
-// eight consecutive features:
-//   ordinary head: delta[b][h][row] = sum_c dO*O  (the row term of the softmax Jacobian)
-//   every head   : dQacc row = 0 (it is accumulated atomically by the main kernel)
+// eight consecutive features; rows run to a multiple of 128 so that the row-term images are complete:
+//   ordinary head: delta = sum_c dO*O (the row term of the softmax Jacobian);
+//                  q_ext row  = split3(-LSE/scale)  (so that S - LSE/scale comes out of the score MMA),
+//                  do_ext row = split3(-delta)      (so that dP - delta comes out of the dP MMA);
+//                  rows beyond T: q_ext = most negative bf16 (their probabilities become 0), do_ext = 0
+//   every head   : dQacc row = 0 (it is accumulated by reduce-adds of the main kernel)
 //   frozen head  : dK row = 0 (no key gradient; Sec. 3.3)
+// Image layout per 128-row block (4 KB): byte (n/8)*256 + (k/8)*128 + (n%8)*16 + (k%8)*2 for row n, column k < 16.
 template <int D>
 __global__ void __launch_bounds__(256) saf_bwd_prep_kernel(const __nv_bfloat16* __restrict__ O,
-                                                           const __nv_bfloat16* __restrict__ dO, int64_t os0, int64_t os1,
+                                                           const __nv_bfloat16* __restrict__ dO,
+                                                           const float* __restrict__ LSE, int64_t os0, int64_t os1,
                                                            int64_t os2, const uint8_t* __restrict__ mask,
-                                                           float* __restrict__ delta, int Tpad, float* __restrict__ dQacc,
+                                                           uint8_t* __restrict__ q_ext, uint8_t* __restrict__ do_ext,
+                                                           float inv_scale, float* __restrict__ dQacc,
                                                            void* __restrict__ dK, int grad_f32, int B, int H, int T) {
   constexpr int TPR = D / 8;                       // threads per row
+  const int Tpad = (T + 127) / 128 * 128;
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
-  const long long rowid = gid / TPR;
+  const long long rowid = gid / TPR;               // over [B][H][Tpad]
   const int part = static_cast<int>(gid % TPR);
-  const long long nrows = static_cast<long long>(B) * H * T;
-  const bool valid = rowid < nrows;
+  const long long nrows = static_cast<long long>(B) * H * Tpad;
+  const bool inrange = rowid < nrows;
   float acc = 0.0f;
   int b = 0, h = 0, t = 0;
-  bool frozen = false;
-  if (valid) {
-    t = static_cast<int>(rowid % T);
-    h = static_cast<int>((rowid / T) % H);
-    b = static_cast<int>(rowid / (static_cast<long long>(T) * H));
+  bool frozen = false, valid = false;
+  if (inrange) {
+    t = static_cast<int>(rowid % Tpad);
+    h = static_cast<int>((rowid / Tpad) % H);
+    b = static_cast<int>(rowid / (static_cast<long long>(Tpad) * H));
     frozen = mask[h] != 0;
-    const size_t grow = static_cast<size_t>(rowid) * D + part * 8;
+    valid = t < T;
+  }
+  if (valid) {
+    const size_t grow = ((static_cast<size_t>(b) * H + h) * T + t) * D + part * 8;
     float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
     *reinterpret_cast<float4*>(dQacc + grow) = z;
     *reinterpret_cast<float4*>(dQacc + grow + 4) = z;
@@ -95,22 +117,41 @@ __global__ void __launch_bounds__(256) saf_bwd_prep_kernel(const __nv_bfloat16* 
   }
 #pragma unroll
   for (int o = TPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-  if (valid && part == 0 && !frozen) delta[(static_cast<size_t>(b) * H + h) * Tpad + t] = acc;
+  if (inrange && part == 0 && !frozen) {
+    const size_t bh = static_cast<size_t>(b) * H + h;
+    const size_t img = (bh * (Tpad / 128) + t / 128) * 4096 + ((t % 128) / 8) * 256 + (t % 8) * 16;
+    uint4 qv, dv;
+    if (valid) {
+      qv = split3_bf16(-LSE[bh * T + t] * inv_scale);
+      dv = split3_bf16(-acc);
+    } else {
+      qv = make_uint4(0xFF7Fu, 0, 0, 0);           // bf16 0xFF7F = -3.39e38
+      dv = make_uint4(0, 0, 0, 0);
+    }
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    *reinterpret_cast<uint4*>(q_ext + img) = qv;
+    *reinterpret_cast<uint4*>(q_ext + img + 128) = zero;
+    *reinterpret_cast<uint4*>(do_ext + img) = dv;
+    *reinterpret_cast<uint4*>(do_ext + img + 128) = zero;
+  }
 }
 
-cudaError_t launch_bwd_prep(const void* O, const void* dO, const int64_t* os, const uint8_t* mask_dev, float* delta,
-                            int Tpad, float* dQacc, void* dK, int grad_f32, int B, int H, int T, int D,
-                            cudaStream_t st) {
-  const long long nthreads = static_cast<long long>(B) * H * T * (D / 8);
+cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* os, const uint8_t* mask_dev,
+                            void* q_ext, void* do_ext, float inv_scale, float* dQacc, void* dK, int grad_f32, int B,
+                            int H, int T, int D, cudaStream_t st) {
+  const int Tpad = (T + 127) / 128 * 128;
+  const long long nthreads = static_cast<long long>(B) * H * Tpad * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
   if (D == 64)
     saf_bwd_prep_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
-                                                  static_cast<const __nv_bfloat16*>(dO), os[0], os[1], os[2], mask_dev,
-                                                  delta, Tpad, dQacc, dK, grad_f32, B, H, T);
+                                                  static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2],
+                                                  mask_dev, static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext),
+                                                  inv_scale, dQacc, dK, grad_f32, B, H, T);
   else
     saf_bwd_prep_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
-                                                   static_cast<const __nv_bfloat16*>(dO), os[0], os[1], os[2], mask_dev,
-                                                   delta, Tpad, dQacc, dK, grad_f32, B, H, T);
+                                                   static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2],
+                                                   mask_dev, static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext),
+                                                   inv_scale, dQacc, dK, grad_f32, B, H, T);
   return cudaGetLastError();
 }
 
