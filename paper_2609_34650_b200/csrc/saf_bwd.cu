@@ -5,7 +5,10 @@
 //   warps 0-3  compute group 0: even 64-query half tiles (TMEM buffer 0); TMEM lane = key row
 //   warps 4-7  compute group 1: odd half tiles (TMEM buffer 1)
 //   warps 8-11 dQ drain: TMEM -> swizzled smem -> TMA reduce-add into the fp32 dQ accumulator
-//   warp 12    TMA producer, warp 13 tcgen05 issuer and TMEM owner
+//   warp 12    TMA producer
+//   warp 13    tcgen05 issuer of the score MMAs A(u); warp 14 issuer of the gradient MMAs B(u), C(t) and
+//              TMEM owner.  An issuing thread is stalled while its MMAs queue, so two issuers let one
+//              stream's bookkeeping (barrier waits) overlap the other stream's tensor work.
 //
 // Ordinary item (Appendix E.2: key-block programs accumulate dV and dK; dQ here comes out of the same
 // tile loop and is accumulated across key blocks by reduce-adds instead of a second pass).  The tile
@@ -64,11 +67,11 @@ struct BwdCfg {
   // per compute group: wq[128] z2s[128] rband[256] r2raw[256] red[16]
   static constexpr int TAB_FLOATS = 128 * 2 + 256 * 2 + 16;
   static constexpr int OFF_BAR = OFF_TAB + 2 * TAB_FLOATS * 4;
-  static constexpr int NBAR = 2 + 2 * NS + 2 + 2 + 4 + 2;
+  static constexpr int NBAR = 2 + 2 * NS + 2 + 2 + 4 + 2 + 3;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
   static constexpr int TMEM_COLS = 512;
   static constexpr int COL_DV = 0, COL_DK = 64, COL_S = 128, COL_DP = 256, COL_DQ = 384;
-  static constexpr int NTHREADS = 448;
+  static constexpr int NTHREADS = 480;
 };
 
 enum BwdSite { B_KV_EMPTY = 21, B_QDO_EMPTY, B_KV_FULL, B_QDO_FULL, B_PDS_FULL, B_ACC_FREE, B_DQ_FREE, B_SDP_FULL,
@@ -99,7 +102,9 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   uint64_t* acc_full = dq_free + 1;
   uint64_t* acc_free = acc_full + 1;
   uint64_t* pfree = acc_free + 1;                // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pfree + 2);
+  uint64_t* bdone = pfree + 2;                   // [2] gradient MMAs that read buffer b have completed
+  uint64_t* fdone = bdone + 2;                   // a frozen item's MMAs have completed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fdone + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -109,16 +114,18 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   if (tid == 0) {
     *abort_flag = 0;
     mbar_init(kv_full, 1);
-    mbar_init(kv_empty, 1);
+    mbar_init(kv_empty, 2);                      // both issuers are done with K_J / V_J
     for (int s = 0; s < C::NS; ++s) {
       mbar_init(qdo_full + s, 1);
-      mbar_init(qdo_empty + s, 1);
+      mbar_init(qdo_empty + s, 2);               // both issuers are done with the stage
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(sdp_full + b, 1);
       mbar_init(pds_full + b, 4);                // one arrival per warp of the group
       mbar_init(pfree + b, 1);
+      mbar_init(bdone + b, 1);
     }
+    mbar_init(fdone, 1);
     mbar_init(dq_full, 1);
     mbar_init(dq_free, 4);
     mbar_init(acc_full, 1);
@@ -135,7 +142,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     }
     reinterpret_cast<uint4*>(smem + C::OFF_ONES)[i] = v;
   }
-  if (warp == 13) {
+  if (warp == 14) {
     tmem_alloc(tmem_slot, C::TMEM_COLS);
     tmem_relinquish();
   }
@@ -184,23 +191,87 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       }
     }
   } else if (warp == 13) {
-    // ------------------------------------------------------------------ tcgen05 issuer
+    // ------------------------------------------------------------------ tcgen05 issuer X: score MMAs A(u)
     // The whole warp walks the loops (warp-uniform operands); one elected lane issues.
     const bool leader = elect_one() != 0;
     const uint32_t sb = smem_u32(smem);
     constexpr uint32_t id_s = umma_idesc_bf16(128, 64, 0, 0);      // S^T, dP^T half tiles: both operands K-major
+    // descriptor halves for smem offset 0: 128B-swizzled K-major (k-step +32 B) and the no-swizzle
+    // K-major row-term tiles (LBO 128 B, SBO 256 B)
+    const uint64_t d_k = umma_smem_desc(sb, 16, 1024, UMMA_LAYOUT_SW128);
+    const uint64_t d_x = umma_smem_desc(sb, 128, 256, UMMA_LAYOUT_NONE);
+    const uint32_t lo_k = desc_lo(d_k), hi_k = desc_hi(d_k), lo_x = desc_lo(d_x), hi_x = desc_hi(d_x);
+    const uint32_t k_lo = lo_k + (C::OFF_K >> 4), v_lo = lo_k + (C::OFF_V >> 4);
+    const uint32_t ones_lo = lo_x + (C::OFF_ONES >> 4);
+    uint32_t nkv = 0, nqdo = 0, nfd = 0;
+    uint32_t nbd0 = 0, nbd1 = 0;
+    bool ok = true;
+    for (int it = it_begin; it < it_end && ok; ++it) {
+      const WorkItem w = p.items[it];
+      const int ntiles = nblk - w.blk;
+      if (w.kind != KIND_ORDINARY) {
+        // not this issuer's item: hand its stages on, then wait until its MMAs have left the S^T buffers
+        for (int t = 0; t < ntiles && ok; ++t, ++nqdo) {
+          const uint32_t s = nqdo % C::NS;
+          ok = mbar_wait_warp(qdo_full + s, (nqdo / C::NS) & 1, wc, B_QDO_FULL);
+          if (ok && leader) mbar_arrive(qdo_empty + s);
+          __syncwarp();
+        }
+        if (!ok) break;
+        ok = mbar_wait_warp(fdone, nfd & 1, wc, B_ACC_FULL);
+        ++nfd;
+        continue;
+      }
+      ok = mbar_wait_warp(kv_full, nkv & 1, wc, B_KV_FULL);
+      if (!ok) break;
+      ++nkv;
+      const int U = 2 * ntiles;
+      for (int u = 0; u < U && ok; ++u) {
+        const uint32_t pos = nqdo + (u >> 1);
+        const uint32_t s = pos % C::NS;
+        const uint32_t b = u & 1;
+        // buffer b is free once the gradient MMAs of half tile u-2 have read their bf16 operands from it
+        if (b == 0) {
+          ok = mbar_wait_warp(bdone, (nbd0 & 1) ^ 1, wc, B_PFREE);
+          ++nbd0;
+          if (ok) ok = mbar_wait_warp(qdo_full + s, (pos / C::NS) & 1, wc, B_QDO_FULL);
+        } else {
+          ok = mbar_wait_warp(bdone + 1, (nbd1 & 1) ^ 1, wc, B_PFREE);
+          ++nbd1;
+        }
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t q_lo = lo_k + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
+        const uint32_t do_lo = lo_k + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
+        const uint32_t qx_lo = lo_x + ((C::OFF_QX + s * 4096 + b * 2048) >> 4);
+        const uint32_t dox_lo = lo_x + ((C::OFF_DOX + s * 4096 + b * 2048) >> 4);
+        const uint32_t t_s = tmem + C::COL_S + 64 * b, t_dp = tmem + C::COL_DP + 64 * b;
+        if (leader) {
+#pragma unroll
+          for (int kc = 0; kc < 4; ++kc) umma_ss2(t_s, k_lo + 2 * kc, hi_k, q_lo + 2 * kc, hi_k, id_s, kc > 0);
+          umma_ss2(t_s, ones_lo, hi_x, qx_lo, hi_x, id_s, 1);
+#pragma unroll
+          for (int kc = 0; kc < 4; ++kc) umma_ss2(t_dp, v_lo + 2 * kc, hi_k, do_lo + 2 * kc, hi_k, id_s, kc > 0);
+          umma_ss2(t_dp, ones_lo, hi_x, dox_lo, hi_x, id_s, 1);
+          umma_commit(sdp_full + b);
+          if (b == 1) umma_commit(qdo_empty + s);       // this issuer's reads of the stage
+          if (u == U - 1) umma_commit(kv_empty);         // ... and of K_J / V_J
+        }
+        __syncwarp();
+      }
+      nqdo += ntiles;
+    }
+  } else if (warp == 14) {
+    // ------------------------------------------------------------------ tcgen05 issuer Y: gradient MMAs
+    const bool leader = elect_one() != 0;
+    const uint32_t sb = smem_u32(smem);
     constexpr uint32_t id_acc = umma_idesc_bf16(128, 64, 0, 1);    // dV, dK: A from TMEM, B MN-major
     constexpr uint32_t id_dq = umma_idesc_bf16(128, 64, 1, 1);     // dQ: A (dS^T tile) M-major, B MN-major
-    // descriptor halves for smem offset 0: 128B-swizzled K-major (k-step +32 B), 128B-swizzled MN-major
-    // (k-step +2048 B, LBO = panel) and the no-swizzle K-major row-term tiles (LBO 128 B, SBO 256 B)
-    const uint64_t d_k = umma_smem_desc(sb, 16, 1024, UMMA_LAYOUT_SW128);
+    // 128B-swizzled MN-major tiles: k-step +2048 B, LBO = panel
     const uint64_t d_m = umma_smem_desc(sb, C::PANEL, 1024, UMMA_LAYOUT_SW128);
-    const uint64_t d_x = umma_smem_desc(sb, 128, 256, UMMA_LAYOUT_NONE);
-    const uint32_t lo_k = desc_lo(d_k), hi_k = desc_hi(d_k), lo_m = desc_lo(d_m), hi_m = desc_hi(d_m);
-    const uint32_t lo_x = desc_lo(d_x), hi_x = desc_hi(d_x);
-    const uint32_t k_lo = lo_k + (C::OFF_K >> 4), v_lo = lo_k + (C::OFF_V >> 4);
-    const uint32_t ones_lo = lo_x + (C::OFF_ONES >> 4), km_lo = lo_m + (C::OFF_K >> 4);
-    uint32_t nkv = 0, nqdo = 0, nitem = 0, ndq = 0, ntile_ord = 0;
+    const uint32_t lo_m = desc_lo(d_m), hi_m = desc_hi(d_m);
+    const uint32_t km_lo = lo_m + (C::OFF_K >> 4);
+    uint32_t nqdo = 0, nitem = 0, ndq = 0, ntile_ord = 0;
     uint32_t npds0 = 0, npds1 = 0;
     int tr_n = 0;
     (void)tr_n;
@@ -210,44 +281,9 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       const bool ord = w.kind == KIND_ORDINARY;
       const int ntiles = nblk - w.blk;
       if (ord) {
-        ok = mbar_wait_warp(kv_full, nkv & 1, wc, B_KV_FULL);
-        if (!ok) break;
-        ++nkv;
         const int U = 2 * ntiles;
-        const uint32_t stage0 = nqdo;                   // ring position of this item's first tile
-        // A(u): augmented scores and dP of half tile u into TMEM buffer u&1
-        auto issue_a = [&](int u) -> bool {
-          const uint32_t pos = stage0 + (u >> 1);
-          const uint32_t s = pos % C::NS;
-          const uint32_t b = u & 1;
-          if (b == 0) {
-            if (!mbar_wait_warp(qdo_full + s, (pos / C::NS) & 1, wc, B_QDO_FULL)) return false;
-            tc_fence_after();
-          }
-          const uint32_t q_lo = lo_k + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
-          const uint32_t do_lo = lo_k + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
-          const uint32_t qx_lo = lo_x + ((C::OFF_QX + s * 4096 + b * 2048) >> 4);
-          const uint32_t dox_lo = lo_x + ((C::OFF_DOX + s * 4096 + b * 2048) >> 4);
-          const uint32_t t_s = tmem + C::COL_S + 64 * b, t_dp = tmem + C::COL_DP + 64 * b;
-          if (leader) {
-#pragma unroll
-            for (int kc = 0; kc < 4; ++kc) umma_ss2(t_s, k_lo + 2 * kc, hi_k, q_lo + 2 * kc, hi_k, id_s, kc > 0);
-            umma_ss2(t_s, ones_lo, hi_x, qx_lo, hi_x, id_s, 1);
-#pragma unroll
-            for (int kc = 0; kc < 4; ++kc) umma_ss2(t_dp, v_lo + 2 * kc, hi_k, do_lo + 2 * kc, hi_k, id_s, kc > 0);
-            umma_ss2(t_dp, ones_lo, hi_x, dox_lo, hi_x, id_s, 1);
-            umma_commit(sdp_full + b);
-          }
-          __syncwarp();
-          return true;
-        };
-        ok = issue_a(0);
         for (int u = 0; u < U && ok; ++u) {
           const uint32_t b = u & 1;
-          if (u + 1 < U) {
-            ok = issue_a(u + 1);
-            if (!ok) break;
-          }
           TR(0, 4);
           if (b == 0) {
             ok = mbar_wait_warp(pds_full, npds0 & 1, wc, B_PDS_FULL);
@@ -263,7 +299,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             if (!ok) break;
           }
           tc_fence_after();
-          const uint32_t pos = stage0 + (u >> 1);
+          const uint32_t pos = nqdo + (u >> 1);
           const uint32_t s = pos % C::NS;
           const uint32_t q_lo = lo_m + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
           const uint32_t do_lo = lo_m + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
@@ -276,6 +312,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
 #pragma unroll
             for (int kc = 0; kc < 4; ++kc)
               umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc, q_lo + 128 * kc, hi_m, id_acc, kc > 0 ? 1u : acc0);
+            umma_commit(bdone + b);
           }
           TR(0, 6);
           if (b == 1) {
@@ -333,11 +370,12 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           __syncwarp();
         }
         if (!ok) break;
+        if (leader) umma_commit(fdone);
       }
       if (leader) umma_commit(acc_full);
       __syncwarp();
     }
-  } else if (warp >= 8) {
+  } else if (warp >= 8 && warp < 12) {
     // ------------------------------------------------------------------ dQ drain warps (128 threads)
     const int q4 = warp & 3;                            // TMEM lane quarter of this warp
     const int rowl = q4 * 32 + lane;                    // query row within the tile
@@ -603,7 +641,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 13) tmem_dealloc(tmem, C::TMEM_COLS);
+  if (warp == 14) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
 int bwd_smem_bytes(int) { return BwdCfg::SMEM; }
