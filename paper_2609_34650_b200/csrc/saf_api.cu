@@ -121,6 +121,12 @@ int upload_mask(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st) {
   return SAF_OK;
 }
 
+// Work lists of the persistent kernels.  Items of one (batch, head) unit are kept close in time, so that
+// what they share stays in L2 while it is needed: in the backward every key block of a unit adds into
+// the unit's dQ rows and re-reads its Q/dO tiles; in the forward every query block re-reads its K/V
+// tiles.  Units are walked in order, the blocks of a unit alternately from the expensive and the cheap
+// end, and each item goes to the CTA that becomes free first (list scheduling, which is what a dynamic
+// queue would do); only the last items are ordered longest-first so that the tail stays short.
 void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward, int n_ctas, int frozen_pct,
                          std::vector<WorkItem>& items, std::vector<int>& offsets) {
   const int nblk = (T + BLK - 1) / BLK;
@@ -128,15 +134,20 @@ void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward,
   std::vector<Cand> cand;
   cand.reserve(static_cast<size_t>(B) * H * nblk);
   for (int b = 0; b < B; ++b)
-    for (int h = 0; h < H; ++h)
-      for (int k = 0; k < nblk; ++k) {
-        const int kind = mask[h] ? KIND_FROZEN : KIND_ORDINARY;
+    for (int h = 0; h < H; ++h) {
+      const int kind = mask[h] ? KIND_FROZEN : KIND_ORDINARY;
+      for (int z = 0; z < nblk; ++z) {
+        // zig-zag over the blocks: most expensive, cheapest, second most expensive, ...
+        const int r = (z & 1) ? (nblk - 1 - z / 2) : (z / 2);        // rank by cost, 0 = most expensive
+        const int k = backward ? r : (nblk - 1 - r);
         const long long tiles = backward ? (nblk - k) : (k + 1);
         const long long cost = tiles * (kind == KIND_FROZEN ? frozen_pct : 100) + 20;   // + fixed per-item overhead
         cand.push_back({{b, h, k, kind}, cost});
       }
-  std::stable_sort(cand.begin(), cand.end(), [](const Cand& a, const Cand& b) { return a.cost > b.cost; });
-  // longest processing time first onto the least loaded CTA
+    }
+  // the tail (about two items per CTA) longest-first
+  const size_t tail = std::min(cand.size(), static_cast<size_t>(2) * n_ctas);
+  std::stable_sort(cand.end() - tail, cand.end(), [](const Cand& a, const Cand& b) { return a.cost > b.cost; });
   typedef std::pair<long long, int> Load;   // (load, cta)
   std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
   for (int c = 0; c < n_ctas; ++c) heap.push({0, c});

@@ -65,11 +65,25 @@ def test_worklist_covers_every_item_once_and_balances(lib, backward, B, H, T, fr
     tiles = np.where(backward, nblk - items[:, 2], items[:, 2] + 1)
     cost = tiles * np.where(items[:, 3] == 1, pct, 100) + 20
     loads = np.array([cost[offs[c]:offs[c + 1]].sum() for c in range(ncta)])
-    # longest-processing-time-first: no CTA exceeds the mean by more than one largest item
+    # list scheduling: no CTA exceeds the mean by more than one largest item
     assert loads.max() <= cost.sum() / ncta + cost.max()
-    # within a CTA, items come in non-increasing cost order
-    for c in range(ncta):
-        assert np.all(np.diff(cost[offs[c]:offs[c + 1]]) <= 0)
+    # locality: the items of one (batch, head) unit start close together in time.  With the load
+    # of the items placed before it as each item's start time, a unit's items all start within about
+    # the time the grid needs for two units' worth of work.
+    if B * H * nblk >= 4 * ncta:
+        start = np.zeros(len(items))
+        for c in range(ncta):
+            seg = slice(offs[c], offs[c + 1])
+            start[seg] = np.concatenate([[0], np.cumsum(cost[seg])[:-1]])
+        unit_cost = cost.sum() / (B * H)
+        span_limit = 2 * unit_cost / ncta * 2 + 2 * cost.max()
+        tail_from = len(items) - 2 * ncta          # the tail is re-ordered longest-first
+        for b in range(B):
+            for h in range(H):
+                sel = (items[:, 0] == b) & (items[:, 1] == h)
+                st = start[sel]
+                if (b * H + h + 1) * nblk <= tail_from:
+                    assert st.max() - st.min() <= span_limit, (b, h, st.max() - st.min(), span_limit)
 
 
 def test_worklist_rejects_bad_arguments(lib):
