@@ -118,8 +118,9 @@ enum {
   SAF_KERNEL_BWD = 1,          /* persistent backward kernel */
   SAF_KERNEL_BWD_PREP = 2,     /* delta = rowsum(dO o O), zero-fill of dQ and of frozen heads' dK */
   SAF_KERNEL_BWD_FINALIZE = 3, /* fp32 -> bf16 conversion of dQ (bf16 gradients only) */
-  SAF_KERNEL_LOGZ = 4,         /* pattern normalisers */
-  SAF_KERNEL_COUNT = 5
+  SAF_KERNEL_LOGZ = 4,         /* pattern normalisers and tables (saf_pattern_prepare) */
+  SAF_KERNEL_SCALE = 5,        /* per-call row scaling of the frozen heads' V (forward) / dO (backward) */
+  SAF_KERNEL_COUNT = 6
 };
 int saf_set_profiling(saf_ctx* ctx, int32_t enable);
 int saf_get_kernel_time(saf_ctx* ctx, int32_t which, float* total_ms_out, int32_t* launches_out);

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libsaf_b200.so")
 SAF_OK = 0
 SAF_ERR_INVALID_ARG, SAF_ERR_UNSUPPORTED, SAF_ERR_CUDA, SAF_ERR_DEVICE_TIMEOUT, SAF_ERR_ARCH, SAF_ERR_NOMEM = range(1, 7)
 SAF_BF16, SAF_F32 = 0, 1
-SAF_KERNEL_FWD, SAF_KERNEL_BWD, SAF_KERNEL_BWD_PREP, SAF_KERNEL_BWD_FINALIZE, SAF_KERNEL_LOGZ = range(5)
+SAF_KERNEL_FWD, SAF_KERNEL_BWD, SAF_KERNEL_BWD_PREP, SAF_KERNEL_BWD_FINALIZE, SAF_KERNEL_LOGZ, SAF_KERNEL_SCALE = range(6)
 
 
 class SafProblem(C.Structure):

@@ -33,6 +33,16 @@ struct DevBuf {
   size_t bytes = 0;
 };
 
+// Which (alpha, rho, logZ) the context's tensor-core pattern tables were built from.
+struct PatternCache {
+  bool valid = false;
+  const float* alpha = nullptr;
+  const float* rho = nullptr;
+  const float* logZ = nullptr;
+  int H = 0, Tp = 0, Hf = 0;
+  std::vector<uint8_t> mask;
+};
+
 struct TimedLaunch {
   int which;
   cudaEvent_t beg, end;
@@ -47,9 +57,14 @@ struct saf_ctx {
   cudaStream_t last_stream = nullptr;
   EncodeTiledFn encode = nullptr;
   unsigned long long wait_limit_ns = 2000000000ull;
-  int frozen_weight_pct = 60;
+  int frozen_weight_pct = 30;              // cost of a frozen tile relative to an ordinary one, forward
+  int frozen_weight_bwd_pct = 20;          // ... and backward
   std::vector<WorklistEntry> worklists;
   DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf;
+  // tensor-core form of frozen heads: tables built by saf_pattern_prepare, scaled V / dO per call
+  PatternCache pat;
+  bool tensor_pattern = true;              // SAF_DISABLE_TENSOR_PATTERN=1 turns the form off
+  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, vt_buf, dot_buf, ok_fwd, ok_bwd;
   bool profiling = false;
   std::vector<TimedLaunch> timed;          // event pairs recorded since the last query
   std::vector<cudaEvent_t> event_pool;
@@ -81,17 +96,34 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 // [B][H][T][D] bf16 tensor with element strides (batch, head, seq); box = 64 features x 128 rows,
 // 128-byte swizzle; rows beyond T read as zero.
-int make_map(saf_ctx* ctx, CUtensorMap* out, const void* base, const saf_problem* p, const int64_t* strides) {
+int make_map(saf_ctx* ctx, CUtensorMap* out, const void* base, const saf_problem* p, const int64_t* strides,
+             CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) {
   cuuint64_t dims[4] = {static_cast<cuuint64_t>(p->D), static_cast<cuuint64_t>(p->T), static_cast<cuuint64_t>(p->H),
                         static_cast<cuuint64_t>(p->B)};
   cuuint64_t gs[3] = {static_cast<cuuint64_t>(strides[2]) * 2, static_cast<cuuint64_t>(strides[1]) * 2,
                       static_cast<cuuint64_t>(strides[0]) * 2};
   cuuint32_t box[4] = {64, BLK, 1, 1};
   cuuint32_t es[4] = {1, 1, 1, 1};
-  CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, gs, box, es,
+  CUresult r = ctx->encode(out, dtype, 4, const_cast<void*>(base), dims, gs, box, es,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? SAF_OK : SAF_ERR_CUDA;
+}
+
+// The tables in the context describe exactly these vectors and this mask.
+bool pattern_matches(const saf_ctx* ctx, const saf_problem* p, const uint8_t* mask, const float* alpha,
+                     const float* rho, const float* logZ) {
+  const PatternCache& c = ctx->pat;
+  return ctx->tensor_pattern && c.valid && c.alpha == alpha && c.rho == rho && c.logZ == logZ && c.H == p->H &&
+         c.Tp == p->Tp && std::memcmp(c.mask.data(), mask, p->H) == 0;
+}
+
+// map of a contiguous [B][Hn][T][D] fp16 workspace
+int make_map_contig(saf_ctx* ctx, CUtensorMap* out, const void* base, const saf_problem* p, int Hn) {
+  saf_problem q = *p;
+  q.H = Hn;
+  const int64_t st[3] = {static_cast<int64_t>(Hn) * p->T * p->D, static_cast<int64_t>(p->T) * p->D, p->D};
+  return make_map(ctx, out, base, &q, st, CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
 }
 
 int check_strides(const int64_t* s, int D) {
@@ -183,7 +215,8 @@ int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int bac
   }
   std::vector<WorkItem> items;
   std::vector<int> offsets;
-  build_worklist_host(B, H, T, mask, backward, grid, ctx->frozen_weight_pct, items, offsets);
+  build_worklist_host(B, H, T, mask, backward, grid, backward ? ctx->frozen_weight_bwd_pct : ctx->frozen_weight_pct,
+                      items, offsets);
   WorklistEntry e;
   e.B = B; e.H = H; e.T = T; e.backward = backward; e.grid = grid;
   e.mask.assign(mask, mask + H);
@@ -298,9 +331,14 @@ int saf_create(saf_ctx** out, int device) {
     long v = std::atol(e);
     if (v > 0) ctx->wait_limit_ns = static_cast<unsigned long long>(v) * 1000000ull;
   }
+  if (const char* e = std::getenv("SAF_DISABLE_TENSOR_PATTERN")) ctx->tensor_pattern = std::atoi(e) == 0;
   if (const char* e = std::getenv("SAF_FROZEN_WEIGHT_PCT")) {
     long v = std::atol(e);
     if (v > 0 && v <= 400) ctx->frozen_weight_pct = static_cast<int>(v);
+  }
+  if (const char* e = std::getenv("SAF_FROZEN_WEIGHT_BWD_PCT")) {
+    long v = std::atol(e);
+    if (v > 0 && v <= 400) ctx->frozen_weight_bwd_pct = static_cast<int>(v);
   }
   *out = ctx;
   return SAF_OK;
@@ -314,6 +352,9 @@ int saf_destroy(saf_ctx* ctx) {
     cudaFree(e.items_dev);
     cudaFree(e.offsets_dev);
   }
+  DevBuf* pbufs[] = {&ctx->pat_consts, &ctx->pat_ok, &ctx->pat_avec, &ctx->pat_wvec, &ctx->pat_bandf, &ctx->pat_bandb,
+                     &ctx->pat_hord, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd};
+  for (DevBuf* b : pbufs) release(*b);
   DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->hq, &ctx->hk, &ctx->hv,
                     &ctx->hdo, &ctx->ho, &ctx->hlse, &ctx->hdq, &ctx->hdk, &ctx->hdv, &ctx->halpha, &ctx->hrho,
                     &ctx->hlogz};
@@ -341,10 +382,46 @@ int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* froz
   int rc = upload_mask(ctx, frozen_mask_host, H, st);
   if (rc) return rc;
   ctx->last_stream = st;
-  ScopedTimer timer(ctx, SAF_KERNEL_LOGZ, st);
-  if (launch_logz(alpha_dev, rho_dev, logZ_dev_out, static_cast<const uint8_t*>(ctx->mask_buf.ptr), H, Tp, st) !=
+  {
+    ScopedTimer timer(ctx, SAF_KERNEL_LOGZ, st);
+    if (launch_logz(alpha_dev, rho_dev, logZ_dev_out, static_cast<const uint8_t*>(ctx->mask_buf.ptr), H, Tp, st) !=
+        cudaSuccess)
+      return SAF_ERR_CUDA;
+  }
+  ctx->pat.valid = false;
+  if (!ctx->tensor_pattern) return SAF_OK;
+  // tables of the tensor-core form (Hankel bands of exp(rho), key scale a, row scale w, per-head flag)
+  const int nblkp = (Tp + 127) / 128;
+  const size_t vecb = static_cast<size_t>(H) * Tp * sizeof(float);
+  const size_t bandb = static_cast<size_t>(H) * nblkp * 4096;
+  if ((rc = ensure(ctx->pat_consts, static_cast<size_t>(H) * 2 * sizeof(float))) ||
+      (rc = ensure(ctx->pat_ok, static_cast<size_t>(H) * sizeof(int))) || (rc = ensure(ctx->pat_avec, vecb)) ||
+      (rc = ensure(ctx->pat_wvec, vecb)) || (rc = ensure(ctx->pat_bandf, bandb)) ||
+      (rc = ensure(ctx->pat_bandb, bandb)) || (rc = ensure(ctx->pat_hord, static_cast<size_t>(H) * sizeof(int))))
+    return rc;
+  std::vector<int> hord(H, -1);
+  int ord = 0;
+  for (int h = 0; h < H; ++h)
+    if (frozen_mask_host[h]) hord[h] = ord++;
+  if (cudaMemcpyAsync(ctx->pat_hord.ptr, hord.data(), static_cast<size_t>(H) * sizeof(int), cudaMemcpyHostToDevice, st) !=
       cudaSuccess)
     return SAF_ERR_CUDA;
+  {
+    ScopedTimer timer(ctx, SAF_KERNEL_LOGZ, st);
+    if (launch_pattern_tables(alpha_dev, rho_dev, logZ_dev_out, static_cast<const uint8_t*>(ctx->mask_buf.ptr), H, Tp,
+                              static_cast<float*>(ctx->pat_consts.ptr), static_cast<int*>(ctx->pat_ok.ptr),
+                              static_cast<float*>(ctx->pat_avec.ptr), static_cast<float*>(ctx->pat_wvec.ptr),
+                              ctx->pat_bandf.ptr, ctx->pat_bandb.ptr, st) != cudaSuccess)
+      return SAF_ERR_CUDA;
+  }
+  ctx->pat.valid = true;
+  ctx->pat.alpha = alpha_dev;
+  ctx->pat.rho = rho_dev;
+  ctx->pat.logZ = logZ_dev_out;
+  ctx->pat.H = H;
+  ctx->pat.Tp = Tp;
+  ctx->pat.Hf = nf;
+  ctx->pat.mask.assign(frozen_mask_host, frozen_mask_host + H);
   return SAF_OK;
 }
 
@@ -396,6 +473,33 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     mk = mv;
   }
   FwdParams fp;
+  CUtensorMap mvt = mv;
+  fp.band_f = nullptr; fp.wvec = nullptr; fp.fast_ok = nullptr; fp.hord = nullptr; fp.nblkp = (p->Tp + 127) / 128;
+  if (nf > 0 && pattern_matches(ctx, p, frozen_mask_host, alpha, rho, logZ)) {
+    // tensor-core form: V of the frozen heads scaled by a(j) once per call
+    const size_t vtb = static_cast<size_t>(p->B) * nf * p->T * p->D * 2;
+    rc = ensure(ctx->vt_buf, vtb);
+    if (rc) return rc;
+    rc = ensure(ctx->ok_fwd, static_cast<size_t>(p->H) * sizeof(int));
+    if (rc) return rc;
+    // per-call copy of the per-head flags; the scaling kernel clears a head whose values leave fp16's range
+    if (cudaMemcpyAsync(ctx->ok_fwd.ptr, ctx->pat_ok.ptr, static_cast<size_t>(p->H) * sizeof(int),
+                        cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return SAF_ERR_CUDA;
+    {
+      ScopedTimer timer(ctx, SAF_KERNEL_SCALE, st);
+      if (launch_scale_rows(V, p->v_strides, static_cast<const float*>(ctx->pat_avec.ptr), p->Tp,
+                            static_cast<const int*>(ctx->pat_hord.ptr), static_cast<int*>(ctx->ok_fwd.ptr),
+                            ctx->vt_buf.ptr, p->B, p->H, nf, p->T, p->D, st) != cudaSuccess)
+        return SAF_ERR_CUDA;
+    }
+    rc = make_map_contig(ctx, &mvt, ctx->vt_buf.ptr, p, nf);
+    if (rc) return rc;
+    fp.band_f = ctx->pat_bandf.ptr;
+    fp.wvec = static_cast<const float*>(ctx->pat_wvec.ptr);
+    fp.fast_ok = static_cast<const int*>(ctx->ok_fwd.ptr);
+    fp.hord = static_cast<const int*>(ctx->pat_hord.ptr);
+  }
   fp.B = p->B; fp.H = p->H; fp.T = p->T; fp.Tp = p->Tp;
   const float scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   fp.scale_log2 = scale * 1.4426950408889634f;
@@ -408,7 +512,7 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   fp.status = ctx->status_dev;
   fp.wait_limit_ns = ctx->wait_limit_ns;
   ScopedTimer timer(ctx, SAF_KERNEL_FWD, st);
-  if (launch_fwd(p->D, mq, mk, mv, fp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+  if (launch_fwd(p->D, mq, mk, mv, mvt, fp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
   return SAF_OK;
 }
 
@@ -499,6 +603,32 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
       return SAF_ERR_CUDA;
   }
   BwdParams bp;
+  CUtensorMap mdot = mdo;
+  bp.band_b = nullptr; bp.avec = nullptr; bp.fast_ok = nullptr; bp.hord = nullptr; bp.nblkp = (p->Tp + 127) / 128;
+  if (nf > 0 && pattern_matches(ctx, p, frozen_mask_host, alpha, rho, logZ)) {
+    // tensor-core form: dO of the frozen heads scaled by w(i) once per call
+    const size_t dob = static_cast<size_t>(p->B) * nf * p->T * p->D * 2;
+    rc = ensure(ctx->dot_buf, dob);
+    if (rc) return rc;
+    rc = ensure(ctx->ok_bwd, static_cast<size_t>(p->H) * sizeof(int));
+    if (rc) return rc;
+    if (cudaMemcpyAsync(ctx->ok_bwd.ptr, ctx->pat_ok.ptr, static_cast<size_t>(p->H) * sizeof(int),
+                        cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return SAF_ERR_CUDA;
+    {
+      ScopedTimer timer(ctx, SAF_KERNEL_SCALE, st);
+      if (launch_scale_rows(dO, p->o_strides, static_cast<const float*>(ctx->pat_wvec.ptr), p->Tp,
+                            static_cast<const int*>(ctx->pat_hord.ptr), static_cast<int*>(ctx->ok_bwd.ptr),
+                            ctx->dot_buf.ptr, p->B, p->H, nf, p->T, p->D, st) != cudaSuccess)
+        return SAF_ERR_CUDA;
+    }
+    rc = make_map_contig(ctx, &mdot, ctx->dot_buf.ptr, p, nf);
+    if (rc) return rc;
+    bp.band_b = ctx->pat_bandb.ptr;
+    bp.avec = static_cast<const float*>(ctx->pat_avec.ptr);
+    bp.fast_ok = static_cast<const int*>(ctx->ok_bwd.ptr);
+    bp.hord = static_cast<const int*>(ctx->pat_hord.ptr);
+  }
   bp.B = p->B; bp.H = p->H; bp.T = p->T; bp.Tp = p->Tp;
   bp.scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   bp.scale_log2 = bp.scale * 1.4426950408889634f;
@@ -514,7 +644,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   bp.wait_limit_ns = ctx->wait_limit_ns;
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD, st);
-    if (launch_bwd(p->D, mq, mk, mv, mdo, mdq, bp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+    if (launch_bwd(p->D, mq, mk, mv, mdo, mdq, mdot, bp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
   }
   if (!grad_f32) {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_FINALIZE, st);

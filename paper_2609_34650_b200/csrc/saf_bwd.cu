@@ -24,6 +24,11 @@
 //   P^^T(j,i) = exp(alpha(j) + rho(i-j) - logZ(i)) for i >= j, generated into TMEM (factorised as in
 //   the forward), dV_J += P^^T dO_I.
 //
+// Frozen item, tensor-core form (pattern tables prepared and the head's flag set):
+//   dV = diag(a) R^T (diag(w) dO).  A tile of R^T with reversed rows is a Hankel matrix read by the tensor
+//   core from a 4 KB band table; per tile one bulk copy of the band, one TMA load of the w-scaled dO tile
+//   and 8 MMAs.  The compute warps only scale the finished rows by a(j) (lane m holds key 127-m).
+//
 // TMEM columns: [0,64) dV, [64,128) dK, [128,192)/[192,256) S^T buffers (bf16 P^T pairs re-use the
 // consumed columns; frozen P^^T tiles use the two 64-column buffers whole), [256,320)/[320,384) dP^T
 // buffers (bf16 dS^T likewise), [384,448) dQ.
@@ -86,7 +91,8 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 __global__ void __launch_bounds__(BwdCfg::NTHREADS, 1)
 saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mdo,
-               const __grid_constant__ CUtensorMap mdq, const BwdParams p) {
+               const __grid_constant__ CUtensorMap mdq, const __grid_constant__ CUtensorMap mdot,
+               const BwdParams p) {
   using C = BwdCfg;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -160,6 +166,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       tma_prefetch_desc(&mk);
       tma_prefetch_desc(&mv);
       tma_prefetch_desc(&mdo);
+      tma_prefetch_desc(&mdot);
       uint32_t nkv = 0, nqdo = 0;
       bool ok = true;
       for (int it = it_begin; it < it_end && ok; ++it) {
@@ -173,6 +180,22 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           tma_load_4d(smem + C::OFF_K, &mk, kv_full, 0, w.blk * BLK, w.h, w.b);
           tma_load_4d(smem + C::OFF_V, &mv, kv_full, 0, w.blk * BLK, w.h, w.b);
           ++nkv;
+        }
+        const bool fast = !ord && p.band_b != nullptr && p.fast_ok[w.h] != 0;
+        if (fast) {
+          // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled dO tile
+          const int fo = p.hord[w.h];
+          const uint8_t* bands = static_cast<const uint8_t*>(p.band_b) + static_cast<size_t>(w.h) * p.nblkp * 4096;
+          for (int I = w.blk; I < nblk; ++I) {
+            const int s = nqdo % C::NS;
+            ok = mbar_wait(qdo_empty + s, ((nqdo / C::NS) & 1) ^ 1, wc, B_QDO_EMPTY);
+            if (!ok) break;
+            mbar_expect_tx(qdo_full + s, C::PANEL + 4096);
+            bulk_load(smem + C::OFF_QX + s * 4096, bands + static_cast<size_t>(I - w.blk) * 4096, 4096, qdo_full + s);
+            tma_load_4d(smem + C::OFF_DO + s * C::PANEL, &mdot, qdo_full + s, 0, I * BLK, fo, w.b);
+            ++nqdo;
+          }
+          continue;
         }
         for (int I = w.blk; I < nblk; ++I) {
           const int s = nqdo % C::NS;
@@ -337,6 +360,34 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         if (!ok) break;
         nqdo += ntiles;
         if (leader) umma_commit(kv_empty);
+      } else if (p.band_b != nullptr && p.fast_ok[w.h] != 0) {
+        // tensor-core form of a frozen head: A = Hankel band (no-swizzle, both strides 128 B), B = scaled dO
+        constexpr uint32_t id_hk = umma_idesc_f16(128, 64, 0, 1);   // fp16 band x fp16 scaled dO
+        const uint64_t d_band = umma_smem_desc(sb, 128, 128, UMMA_LAYOUT_NONE);
+        const uint32_t lo_b = desc_lo(d_band), hi_b = desc_hi(d_band);
+        for (int t = 0; t < ntiles; ++t) {
+          const uint32_t s = nqdo % C::NS;
+          ok = mbar_wait_warp(qdo_full + s, (nqdo / C::NS) & 1, wc, B_QDO_FULL);
+          if (!ok) break;
+          ++nqdo;
+          if (t == 0) {
+            ok = mbar_wait_warp(acc_free, (nitem & 1) ^ 1, wc, B_ACC_FREE);
+            if (!ok) break;
+          }
+          tc_fence_after();
+          const uint32_t band_lo = lo_b + ((C::OFF_QX + s * 4096) >> 4);
+          const uint32_t do_lo = lo_m + ((C::OFF_DO + s * C::PANEL) >> 4);
+          const uint32_t acc0 = t > 0 ? 1u : 0u;
+          if (leader) {
+#pragma unroll
+            for (int kc = 0; kc < 8; ++kc)
+              umma_ss2(tmem + C::COL_DV, band_lo + 16 * kc, hi_b, do_lo + 128 * kc, hi_m, id_hk, kc > 0 ? 1u : acc0);
+            umma_commit(qdo_empty + s);
+          }
+          __syncwarp();
+        }
+        if (!ok) break;
+        if (leader) umma_commit(fdone);
       } else {
         for (int t = 0; t < ntiles; ++t) {
           const uint32_t s = nqdo % C::NS;
@@ -451,11 +502,16 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       const WorkItem w = p.items[it];
       const bool ord = w.kind == KIND_ORDINARY;
       const int ntiles = nblk - w.blk;
-      const int key = w.blk * BLK + rowl;
+      int key = w.blk * BLK + rowl;
       const size_t bh = static_cast<size_t>(w.b) * p.H + w.h;
+      float dv_mul = 1.0f;
       if (named_bar_or(bar_id, 128, !ok)) break;
 
-      if (ord) {
+      if (!ord && p.band_b != nullptr && p.fast_ok[w.h] != 0) {
+        // tensor-core form: nothing to do per tile; lane m holds key 127-m, scaled by a(j) below
+        key = w.blk * BLK + 127 - rowl;
+        dv_mul = (key < p.T) ? p.avec[static_cast<size_t>(w.h) * p.Tp + key] : 0.0f;
+      } else if (ord) {
         const float c = p.scale_log2;
         for (int t = 0; t < ntiles; ++t) {
           // this group's half tile of tile t: queries 64*grp .. 64*grp+63
@@ -600,7 +656,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       tc_fence_after();
       if (grp == 0 || ord) {
         const uint32_t col = grp == 0 ? C::COL_DV : C::COL_DK;
-        const float mul = grp == 0 ? 1.0f : p.scale;
+        const float mul = grp == 0 ? dv_mul : p.scale;
         void* base = grp == 0 ? p.dV : p.dK;
         const size_t off = (bh * p.T + key) * 64;
 #pragma unroll
@@ -647,11 +703,12 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
 int bwd_smem_bytes(int) { return BwdCfg::SMEM; }
 
 cudaError_t launch_bwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const CUtensorMap& mdo, const CUtensorMap& mdq, const BwdParams& p, int grid, cudaStream_t st) {
+                       const CUtensorMap& mdo, const CUtensorMap& mdq, const CUtensorMap& mdot, const BwdParams& p,
+                       int grid, cudaStream_t st) {
   if (D != 64) return cudaErrorNotSupported;
   cudaError_t e = cudaFuncSetAttribute(saf_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg::SMEM);
   if (e != cudaSuccess) return e;
-  saf_bwd_kernel<<<grid, BwdCfg::NTHREADS, BwdCfg::SMEM, st>>>(mq, mk, mv, mdo, mdq, p);
+  saf_bwd_kernel<<<grid, BwdCfg::NTHREADS, BwdCfg::SMEM, st>>>(mq, mk, mv, mdo, mdq, mdot, p);
   return cudaGetLastError();
 }
 

@@ -17,6 +17,11 @@
 //   w(i) * a(j) * r(i-j) with a = exp(alpha - max_tile alpha), r = exp(rho - max_band rho),
 //   w = exp(max alpha + max rho - logZ(i)); a tile whose exponent range would leave fp32 falls back to
 //   one exp per element.
+// Frozen item, tensor-core form (pattern tables prepared and the head's flag set): with global maxima,
+//   O = diag(w) R (diag(a) V), R(i,j) = r(i-j).  A tile of R with reversed rows is a Hankel matrix that the
+//   tensor core reads straight from a 4 KB band table (no-swizzle descriptor, both strides 128 bytes), so
+//   a tile is one bulk copy of the band, one TMA load of the a-scaled V tile and 8 MMAs; the compute warps
+//   only scale the finished rows by w(i) (TMEM lane m holds query 127-m of the block).
 #include <cuda_bf16.h>
 #include "ptx.cuh"
 #include "saf_internal.h"
@@ -69,7 +74,7 @@ enum FwdSite { SITE_Q_EMPTY = 1, SITE_K_EMPTY, SITE_V_EMPTY, SITE_Q_FULL, SITE_K
 template <int D>
 __global__ void __launch_bounds__(320, 2)
 saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
-               const __grid_constant__ CUtensorMap mv, const FwdParams p) {
+               const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mvt, const FwdParams p) {
   using C = FwdCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -126,11 +131,35 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       tma_prefetch_desc(&mq);
       tma_prefetch_desc(&mk);
       tma_prefetch_desc(&mv);
+      tma_prefetch_desc(&mvt);
       uint32_t nq = 0, nk = 0, nv = 0;
       bool ok = true;
       for (int it = it_begin; it < it_end && ok; ++it) {
         const WorkItem w = p.items[it];
         const int ntiles = w.blk + 1;
+        if (w.kind == KIND_FROZEN && p.band_f != nullptr && p.fast_ok[w.h] != 0) {
+          // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled V tile
+          const int ord = p.hord[w.h];
+          const uint8_t* bands = static_cast<const uint8_t*>(p.band_f) + static_cast<size_t>(w.h) * p.nblkp * 4096;
+          for (int j = 0; j < ntiles; ++j) {
+            const int sk = nk % C::NS;
+            ok = mbar_wait(k_empty + sk, ((nk / C::NS) & 1) ^ 1, wc, SITE_K_EMPTY);
+            if (!ok) break;
+            mbar_expect_tx(k_full + sk, 4096);
+            bulk_load(smem + C::OFF_K + sk * C::TILE_BYTES, bands + static_cast<size_t>(w.blk - j) * 4096, 4096,
+                      k_full + sk);
+            ++nk;
+            const int sv = nv % C::NS;
+            ok = mbar_wait(v_empty + sv, ((nv / C::NS) & 1) ^ 1, wc, SITE_V_EMPTY);
+            if (!ok) break;
+            mbar_expect_tx(v_full + sv, C::TILE_BYTES);
+            for (int pn = 0; pn < C::NPANEL; ++pn)
+              tma_load_4d(smem + C::OFF_V + sv * C::TILE_BYTES + pn * C::PANEL_BYTES, &mvt, v_full + sv, pn * 64,
+                          j * BLK, ord, w.b);
+            ++nv;
+          }
+          continue;
+        }
         if (w.kind == KIND_ORDINARY) {
           ok = mbar_wait(q_empty, (nq & 1) ^ 1, wc, SITE_Q_EMPTY);
           if (!ok) break;
@@ -168,6 +197,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     const uint32_t sb = smem_u32(smem);
     constexpr uint32_t idesc_s = umma_idesc_bf16(128, 128, 0, 0);
     constexpr uint32_t idesc_o = umma_idesc_bf16(128, D, 0, 1);
+    constexpr uint32_t idesc_hk = umma_idesc_f16(128, D, 0, 1);    // tensor-core frozen form: fp16 band x fp16 scaled V
     uint32_t nq = 0, nk = 0, nv = 0, np = 0, nitem = 0;
     bool ok = true;
     // descriptor halves for smem offset 0: K-major tiles (k-step +32 B within a 64-column panel) and
@@ -176,10 +206,42 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     const uint64_t d_mn = umma_smem_desc(sb, C::PANEL_BYTES, 1024, UMMA_LAYOUT_SW128);
     const uint32_t lo_k = desc_lo(d_kmaj), hi_k = desc_hi(d_kmaj), lo_m = desc_lo(d_mn), hi_m = desc_hi(d_mn);
     const uint32_t q_lo = lo_k + (C::OFF_Q >> 4);
+    // Hankel band: no-swizzle K-major, core matrices 128 bytes apart in both directions
+    const uint64_t d_band = umma_smem_desc(sb, 128, 128, UMMA_LAYOUT_NONE);
+    const uint32_t lo_b = desc_lo(d_band), hi_b = desc_hi(d_band);
     for (int it = it_begin; it < it_end && ok; ++it, ++nitem) {
       const WorkItem w = p.items[it];
       const int ntiles = w.blk + 1;
       const bool ord = w.kind == KIND_ORDINARY;
+      if (w.kind == KIND_FROZEN && p.band_f != nullptr && p.fast_ok[w.h] != 0) {
+        for (int j = 0; j < ntiles && ok; ++j) {
+          const uint32_t sk = nk % C::NS, sv = nv % C::NS;
+          ok = mbar_wait_warp(k_full + sk, (nk / C::NS) & 1, wc, SITE_K_FULL);
+          if (!ok) break;
+          ++nk;
+          ok = mbar_wait_warp(v_full + sv, (nv / C::NS) & 1, wc, SITE_V_FULL);
+          if (!ok) break;
+          ++nv;
+          if (j == 0) {
+            ok = mbar_wait_warp(o_free, (nitem & 1) ^ 1, wc, SITE_O_FREE);
+            if (!ok) break;
+          }
+          tc_fence_after();
+          const uint32_t band_lo = lo_b + ((C::OFF_K + sk * C::TILE_BYTES) >> 4);
+          const uint32_t v_lo = lo_m + ((C::OFF_V + sv * C::TILE_BYTES) >> 4);
+          const uint32_t acc0 = j > 0 ? 1u : 0u;
+          if (leader) {
+#pragma unroll
+            for (int kc = 0; kc < 8; ++kc)
+              umma_ss2(tmem + C::COL_O, band_lo + 16 * kc, hi_b, v_lo + 128 * kc, hi_m, idesc_hk, kc > 0 ? 1u : acc0);
+            umma_commit(k_empty + sk);
+            umma_commit(v_empty + sv);
+            if (j == ntiles - 1) umma_commit(pv_done);
+          }
+          __syncwarp();
+        }
+        continue;
+      }
       if (ord) {
         ok = mbar_wait_warp(q_full, nq & 1, wc, SITE_Q_FULL);
         if (!ok) break;
@@ -262,10 +324,14 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     for (int it = it_begin; it < it_end; ++it) {
       const WorkItem w = p.items[it];
       const int ntiles = w.blk + 1;
-      const int row = w.blk * BLK + rowl;
+      int row = w.blk * BLK + rowl;
       float inv_l = 1.0f, lse = 0.0f;
       if (named_bar_or(5, 256, !ok)) break;
-      if (w.kind == KIND_ORDINARY) {
+      if (w.kind == KIND_FROZEN && p.band_f != nullptr && p.fast_ok[w.h] != 0) {
+        // tensor-core form: nothing to do per tile; lane m holds query 127-m, scaled by w(i) below
+        row = w.blk * BLK + 127 - rowl;
+        inv_l = (row < p.T) ? p.wvec[static_cast<size_t>(w.h) * p.Tp + row] : 0.0f;
+      } else if (w.kind == KIND_ORDINARY) {
         float m_ref = -INFINITY, l = 0.0f;
         const float c = p.scale_log2;
         for (int j = 0; j < ntiles; ++j) {
@@ -529,16 +595,16 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
 int fwd_smem_bytes(int D) { return D == 64 ? FwdCfg<64>::SMEM : FwdCfg<128>::SMEM; }
 
 cudaError_t launch_fwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const FwdParams& p, int grid, cudaStream_t st) {
+                       const CUtensorMap& mvt, const FwdParams& p, int grid, cudaStream_t st) {
   cudaError_t e;
   if (D == 64) {
     e = cudaFuncSetAttribute(saf_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<64>::SMEM);
     if (e != cudaSuccess) return e;
-    saf_fwd_kernel<64><<<grid, 320, FwdCfg<64>::SMEM, st>>>(mq, mk, mv, p);
+    saf_fwd_kernel<64><<<grid, 320, FwdCfg<64>::SMEM, st>>>(mq, mk, mv, mvt, p);
   } else {
     e = cudaFuncSetAttribute(saf_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128>::SMEM);
     if (e != cudaSuccess) return e;
-    saf_fwd_kernel<128><<<grid, 320, FwdCfg<128>::SMEM, st>>>(mq, mk, mv, p);
+    saf_fwd_kernel<128><<<grid, 320, FwdCfg<128>::SMEM, st>>>(mq, mk, mv, mvt, p);
   }
   return cudaGetLastError();
 }

@@ -21,6 +21,14 @@ struct FwdParams {
   void* O;                          // bf16, strided
   int64_t o_strides[3];             // elements: batch, head, seq
   float* LSE;                       // [B][H][T]
+  // Tensor-core form of frozen heads (all NULL when the pattern tables are not prepared): band_f is the
+  // forward Hankel band table [H][nblkp][2048] fp16, wvec the row scale w(i) [H][Tp], fast_ok[h] != 0
+  // where the form may be used, hord[h] the head's ordinal among the frozen heads (-1 otherwise).
+  const void* band_f;
+  const float* wvec;
+  const int* fast_ok;
+  const int* hord;
+  int nblkp;
   const WorkItem* items;            // grouped by CTA
   const int* cta_offsets;           // [grid+1]
   int* status;                      // device status word
@@ -42,6 +50,12 @@ struct BwdParams {
   void* dK;                         // [B][H][T][D] grad dtype
   void* dV;
   int grad_f32;
+  // tensor-core form of frozen heads (see FwdParams): backward band table and the key scale a(j)
+  const void* band_b;
+  const float* avec;
+  const int* fast_ok;
+  const int* hord;
+  int nblkp;
   const WorkItem* items;
   const int* cta_offsets;
   int* status;
@@ -51,10 +65,18 @@ struct BwdParams {
 // Launchers (defined in the .cu files).  All return the launch error.
 cudaError_t launch_logz(const float* alpha, const float* rho, float* logZ, const uint8_t* mask_dev, int H,
                         int Tp, cudaStream_t st);
+cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const float* logZ, const uint8_t* mask_dev,
+                                  int H, int Tp, float* consts, int* fast_ok, float* avec, float* wvec, void* band_f,
+                                  void* band_b, cudaStream_t st);
+cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, int Tp, const int* hord,
+                              int* call_ok, void* dst, int B, int H, int Hf, int T, int D, cudaStream_t st);
+// mvt: map of the a-scaled V of the frozen heads [B][Hf][T][D] (any valid map when band_f is NULL)
 cudaError_t launch_fwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const FwdParams& p, int grid, cudaStream_t st);
+                       const CUtensorMap& mvt, const FwdParams& p, int grid, cudaStream_t st);
+// mdot: map of the w-scaled dO of the frozen heads [B][Hf][T][D] (any valid map when band_b is NULL)
 cudaError_t launch_bwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const CUtensorMap& mdo, const CUtensorMap& mdq, const BwdParams& p, int grid, cudaStream_t st);
+                       const CUtensorMap& mdo, const CUtensorMap& mdq, const CUtensorMap& mdot, const BwdParams& p,
+                       int grid, cudaStream_t st);
 // Row terms of ordinary heads (q_ext / do_ext images, see BwdParams); also zeroes dQacc (all heads) and
 // dK of frozen heads.
 cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* o_strides,

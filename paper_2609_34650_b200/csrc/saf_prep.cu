@@ -1,6 +1,7 @@
 // Small memory-bound helper kernels: the pattern's row normalisers, the backward's delta / zero-fill
 // pass and the fp32 -> bf16 conversion of the accumulated query gradient.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include "saf_internal.h"
 
 namespace saf {
@@ -40,6 +41,161 @@ cudaError_t launch_logz(const float* alpha, const float* rho, float* logZ, const
                         cudaStream_t st) {
   dim3 grid((Tp + 7) / 8, H);
   saf_logz_kernel<<<grid, 256, 0, st>>>(alpha, rho, logZ, mask_dev, Tp);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Tables of the tensor-core form of a frozen head.  With c_a = max alpha, c_r = max rho,
+//   a(j) = exp(alpha(j) - c_a),  r(d) = exp(rho(d) - c_r),  w(i) = exp(c_a + c_r - logZ(i)),
+// Eq. "compact-prior" reads  P^(i,j) = w(i) r(i-j) a(j):  O = diag(w) R (diag(a) V) with the Toeplitz
+// matrix R(i,j) = r(i-j) [j <= i], and dV = diag(a) R^T (diag(w) dO).  A 128x128 tile of R (or R^T)
+// with its rows in reverse order is a Hankel matrix g[m + k]; stored as 31 overlapping 8x8 core
+// matrices (chunk c, row ri, element e = g[8c + ri + e], 128 bytes per chunk) it is a valid no-swizzle
+// K-major UMMA operand with both descriptor strides equal to 128 bytes, so the tensor core reads the
+// pattern tile straight from a 4 KB band of the relative-distance vector.
+//   band_f[h][D][x] : g[x] = r(128 D + 127 - x)   (forward,  rows = queries reversed)
+//   band_b[h][D][x] : g[x] = r(128 D - 127 + x)   (backward, rows = keys reversed)
+// The band and the scaled V / dO tiles are fp16 (the tensor core needs one 16-bit type for both operands;
+// fp16 keeps 11 significant bits, so the form adds less rounding than the bf16 pattern tile of the
+// general path).  It is used for a head only if max_i (c_a + c_r - logZ(i)) <= 5 (fast_ok): then w <= e^5,
+// every r below fp16's normal range weighs less than 1 % of its row, and w dO stays in range.
+__global__ void __launch_bounds__(256) saf_pattern_consts_kernel(const float* __restrict__ alpha,
+                                                                 const float* __restrict__ rho,
+                                                                 const float* __restrict__ logZ,
+                                                                 const uint8_t* __restrict__ mask, int Tp,
+                                                                 float* __restrict__ consts, int* __restrict__ fast_ok) {
+  const int h = blockIdx.x;
+  if (!mask[h]) {
+    if (threadIdx.x == 0) fast_ok[h] = 0;
+    return;
+  }
+  __shared__ float red[3][8];
+  const float* a = alpha + static_cast<size_t>(h) * Tp;
+  const float* r = rho + static_cast<size_t>(h) * Tp;
+  const float* z = logZ + static_cast<size_t>(h) * Tp;
+  float ma = -INFINITY, mr = -INFINITY, mz = INFINITY;
+  for (int t = threadIdx.x; t < Tp; t += 256) {
+    ma = fmaxf(ma, a[t]);
+    mr = fmaxf(mr, r[t]);
+    mz = fminf(mz, z[t]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    ma = fmaxf(ma, __shfl_xor_sync(0xffffffffu, ma, o));
+    mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, o));
+    mz = fminf(mz, __shfl_xor_sync(0xffffffffu, mz, o));
+  }
+  const int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0) {
+    red[0][warp] = ma;
+    red[1][warp] = mr;
+    red[2][warp] = mz;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int k = 1; k < 8; ++k) {
+      ma = fmaxf(ma, red[0][k]);
+      mr = fmaxf(mr, red[1][k]);
+      mz = fminf(mz, red[2][k]);
+    }
+    consts[2 * h] = ma;
+    consts[2 * h + 1] = mr;
+    const float wmax = ma + mr - mz;
+    fast_ok[h] = (wmax <= 5.0f && wmax > -1e30f && ma < 1e30f && mr < 1e30f) ? 1 : 0;
+  }
+}
+
+__global__ void __launch_bounds__(256) saf_pattern_tables_kernel(const float* __restrict__ alpha,
+                                                                 const float* __restrict__ rho,
+                                                                 const float* __restrict__ logZ,
+                                                                 const uint8_t* __restrict__ mask, int Tp,
+                                                                 const float* __restrict__ consts,
+                                                                 float* __restrict__ avec, float* __restrict__ wvec,
+                                                                 __half* __restrict__ band_f,
+                                                                 __half* __restrict__ band_b, int nblkp) {
+  const int h = blockIdx.y, dblk = blockIdx.x;
+  if (!mask[h]) return;
+  const float ca = consts[2 * h], cr = consts[2 * h + 1];
+  const size_t row = static_cast<size_t>(h) * Tp;
+  const int t = dblk * 128 + threadIdx.x;
+  if (threadIdx.x < 128 && t < Tp) {
+    avec[row + t] = __expf(alpha[row + t] - ca);
+    wvec[row + t] = __expf(ca + cr - logZ[row + t]);
+  }
+  const size_t band = (static_cast<size_t>(h) * nblkp + dblk) * 2048;
+  for (int idx = threadIdx.x; idx < 2048; idx += 256) {
+    const int c = idx >> 6, ri = (idx >> 3) & 7, e = idx & 7;
+    const int x = 8 * c + ri + e;
+    const int df = dblk * 128 + 127 - x, db = dblk * 128 - 127 + x;
+    const bool used = c < 31;
+    const float vf = (used && df >= 0 && df < Tp) ? __expf(rho[row + df] - cr) : 0.0f;
+    const float vb = (used && db >= 0 && db < Tp) ? __expf(rho[row + db] - cr) : 0.0f;
+    band_f[band + idx] = __float2half_rn(vf);
+    band_b[band + idx] = __float2half_rn(vb);
+  }
+}
+
+cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const float* logZ, const uint8_t* mask_dev, int H,
+                                  int Tp, float* consts, int* fast_ok, float* avec, float* wvec, void* band_f,
+                                  void* band_b, cudaStream_t st) {
+  const int nblkp = (Tp + 127) / 128;
+  saf_pattern_consts_kernel<<<H, 256, 0, st>>>(alpha, rho, logZ, mask_dev, Tp, consts, fast_ok);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  saf_pattern_tables_kernel<<<dim3(nblkp, H), 256, 0, st>>>(alpha, rho, logZ, mask_dev, Tp, consts, avec, wvec,
+                                                            static_cast<__half*>(band_f),
+                                                            static_cast<__half*>(band_b), nblkp);
+  return cudaGetLastError();
+}
+
+// dst[b][ord(h)][t][:] = fp16(vec[h][t] * src[b][h][t][:]) for the frozen heads whose tensor-core form is
+// enabled (V scaled by a, or dO scaled by w).  Eight features per thread.  call_ok[h] starts as a copy of
+// fast_ok[h]; a product that leaves fp16's range clears it, which sends that head down the general path
+// in the kernel that follows.
+template <int D>
+__global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16* __restrict__ src, int64_t s0, int64_t s1,
+                                                             int64_t s2, const float* __restrict__ vec, int Tp,
+                                                             const int* __restrict__ hord, int* __restrict__ call_ok,
+                                                             __half* __restrict__ dst, int B, int H, int Hf, int T) {
+  constexpr int TPR = D / 8;
+  const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
+  const long long rowid = gid / TPR;
+  const int part = static_cast<int>(gid % TPR);
+  if (rowid >= static_cast<long long>(B) * H * T) return;
+  const int t = static_cast<int>(rowid % T);
+  const int h = static_cast<int>((rowid / T) % H);
+  const int b = static_cast<int>(rowid / (static_cast<long long>(T) * H));
+  const int ord = hord[h];
+  if (ord < 0 || !call_ok[h]) return;
+  const float f = vec[static_cast<size_t>(h) * Tp + t];
+  const uint4 v4 = *reinterpret_cast<const uint4*>(src + b * s0 + h * s1 + static_cast<int64_t>(t) * s2 + part * 8);
+  const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&v4);
+  __half2 o[4];
+  bool bad = false;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 x = __bfloat1622float2(v2[e]);
+    const float y0 = x.x * f, y1 = x.y * f;
+    bad |= !(fabsf(y0) <= 65504.0f) || !(fabsf(y1) <= 65504.0f);     // also catches NaN
+    o[e] = __floats2half2_rn(y0, y1);
+  }
+  if (bad) atomicExch(call_ok + h, 0);
+  *reinterpret_cast<uint4*>(dst + ((static_cast<size_t>(b) * Hf + ord) * T + t) * D + part * 8) =
+      *reinterpret_cast<uint4*>(o);
+}
+
+cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, int Tp, const int* hord,
+                              int* call_ok, void* dst, int B, int H, int Hf, int T, int D, cudaStream_t st) {
+  const long long nthreads = static_cast<long long>(B) * H * T * (D / 8);
+  const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
+  if (D == 64)
+    saf_scale_rows_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
+                                                    strides[2], vec, Tp, hord, call_ok, static_cast<__half*>(dst), B,
+                                                    H, Hf, T);
+  else
+    saf_scale_rows_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
+                                                     strides[2], vec, Tp, hord, call_ok, static_cast<__half*>(dst), B,
+                                                     H, Hf, T);
   return cudaGetLastError();
 }
 

@@ -147,6 +147,29 @@ def test_exact_exponent_fallback_for_wide_range_patterns():
     check_units(L, all_units(wl))
 
 
+def test_values_beyond_fp16_range_take_the_general_frozen_path():
+    """The tensor-core form of a frozen head stages a V and w dO in fp16; tensors that would overflow there
+    must be detected per call and handled by the general (bf16 pattern tile) path.  V and dO scaled by 2^17
+    (exact in bf16) must give O and dV scaled by 2^17."""
+    wl = si.Workload("range", 1, 2, 300, 64, (0,), -0.05, seed=31)
+    inp = si.generate(wl)
+    ref = Layer(inp).run()
+    big = si.generate(wl)
+    k = 2.0 ** 17
+    big.v[...] = si.f32_to_bf16_bits(si.bf16_bits_to_f32(big.v) * k)
+    big.do[...] = si.f32_to_bf16_bits(si.bf16_bits_to_f32(big.do) * k)
+    L = Layer(big).run()
+    q, kk, v, do = f64(inp)
+    scale = 1.0 / np.sqrt(wl.D)
+    eO, _ = orc.head_fwd_panels(True, q[0, 0], kk[0, 0], v[0, 0], inp.alpha[0], inp.rho[0], scale)
+    _, _, edV = orc.head_bwd_panels(True, q[0, 0], kk[0, 0], v[0, 0], do[0, 0], inp.alpha[0], inp.rho[0], scale)
+    assert_close(L.host(L.O)[0, 0] / k, eO, "O of the scaled problem")
+    assert_close(L.host(L.grads[2])[0, 0] / k, edV, "dV of the scaled problem")
+    # and the unscaled problem went through the tensor-core form with much smaller error on dV
+    ma, rl = errors(ref.host(ref.grads[2])[0, 0], edV)
+    assert rl < 1e-3
+
+
 def test_stale_state_fuzz_on_one_context():
     """Mask / pattern / shape changes on one context (cached work lists, workspaces) stay correct."""
     ctx = saf.Context(0)
