@@ -72,6 +72,28 @@ int saf_destroy(saf_ctx* ctx);
 int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* frozen_mask_host,
                         const float* alpha_dev, const float* rho_dev, float* logZ_dev_out, void* stream);
 
+/* Row normalisers without any allocation (the paper has no counterpart: this entry point exists for the
+ * host program's sake, not the method's).
+ *
+ * Some host programs cannot let a library allocate device memory: a serving process that hands all of
+ * the GPU's memory to its own pool at start-up (a later cudaMalloc simply fails), or a component that
+ * must not block on the allocator inside a latency-critical loop.  saf_pattern_prepare needs a device
+ * copy of the frozen-head mask and gets it from memory the context allocates; this variant computes
+ * the same logZ with that copy in a fixed array inside the library image.
+ *
+ *   - No context.  `device` is the CUDA device to run on.  Other arguments as saf_pattern_prepare.
+ *   - H must not exceed SAF_STATIC_MAX_HEADS; a larger H returns SAF_ERR_INVALID_ARG and launches nothing.
+ *   - The call makes no cudaMalloc / cudaFree and uses no allocating library routine.  It only computes
+ *     logZ; the tensor-core pattern tables of saf_pattern_prepare are not built.
+ *   - The first call on a device resolves the array's device address (one cudaGetSymbolAddress, cached per
+ *     device).  Make that first call during set-up, before any stream capture is begun.
+ *   - The array (SAF_STATIC_MAX_HEADS bytes per GPU, held until the process exits) is shared by every
+ *     call and keeps the previous call's contents; each call overwrites the H bytes it reads.  Two calls
+ *     whose GPU work overlaps (different streams, or different threads) race on it: serialise them. */
+#define SAF_STATIC_MAX_HEADS 1024
+int saf_pattern_logz_static(int32_t device, int32_t H, int32_t Tp, const uint8_t* frozen_mask_host,
+                            const float* alpha_dev, const float* rho_dev, float* logZ_dev_out, void* stream);
+
 /* Forward of the hybrid layer (Sec. 3.3 "Fused computation"; Appendix E.2): one persistent launch.
  *   Q, K, V : device bf16, strided as in `p`.
  *   logZ    : device fp32 [H][Tp] from saf_pattern_prepare, or NULL to have it computed into

@@ -58,6 +58,8 @@ def load_library() -> C.CDLL:
     lib.saf_last_device_status.argtypes = [vp, C.POINTER(C.c_int32)]
     lib.saf_set_profiling.argtypes = [vp, i32]
     lib.saf_get_kernel_time.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.saf_pattern_logz_static.argtypes = [i32, i32, i32, u8p, f32p, f32p, f32p, vp]
+    lib.saf_pattern_logz_static.restype = C.c_int
     lib.saf_build_worklist.argtypes = [i32, i32, i32, u8p, i32, i32, i32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     for name in ("saf_create", "saf_destroy", "saf_pattern_prepare", "saf_hybrid_attn_fwd", "saf_hybrid_attn_bwd",
                  "saf_hybrid_attn_step_host", "saf_last_device_status", "saf_build_worklist", "saf_set_profiling",
@@ -105,6 +107,14 @@ def saf_build_worklist(B, H, T, mask, backward, n_ctas, frozen_weight_pct=60):
                                   items.ctypes.data_as(C.POINTER(C.c_int32)),
                                   offsets.ctypes.data_as(C.POINTER(C.c_int32))), "saf_build_worklist")
     return items, offsets
+
+
+def saf_pattern_logz_static(device, mask, alpha, rho, logZ_out):
+    """Row normalisers through the entry point that allocates nothing (no context; at most 1024 heads)."""
+    H, Tp = alpha.shape
+    m, mp = _mask_ptr(mask)
+    _check(load_library().saf_pattern_logz_static(device, H, Tp, mp, _ptr(alpha), _ptr(rho), _ptr(logZ_out), _stream()),
+           "saf_pattern_logz_static")
 
 
 def make_problem(q_like, Tp, softmax_scale=0.0, grad_dtype=SAF_F32, k_like=None, v_like=None, o_like=None):

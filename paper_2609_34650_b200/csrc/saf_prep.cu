@@ -2,6 +2,9 @@
 // pass and the fp32 -> bf16 conversion of the accumulated query gradient.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <mutex>
+
+#include "../../include/saf.h"
 #include "saf_internal.h"
 
 namespace saf {
@@ -333,3 +336,63 @@ cudaError_t launch_bwd_finalize(const float* dQacc, void* dQ, size_t n, cudaStre
 }
 
 }  // namespace saf
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of the normaliser computation.
+//
+// saf_logz_kernel needs the frozen-head mask in device memory.  saf_pattern_prepare keeps that copy in
+// memory it allocates through the context; here it lives in a fixed array that is part of the library
+// image, so the call path contains no allocation at all.  Every GPU that loads the library carries
+// these SAF_STATIC_MAX_HEADS bytes until the process exits.
+namespace {
+
+static __device__ __align__(256) uint8_t g_static_mask_scratch[SAF_STATIC_MAX_HEADS];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+uint8_t* g_static_mask_ptr[kMaxDevices] = {};   // device address of the array, per device, resolved once
+
+}  // namespace
+
+extern "C" int saf_pattern_logz_static(int32_t device, int32_t H, int32_t Tp, const uint8_t* frozen_mask_host,
+                                       const float* alpha_dev, const float* rho_dev, float* logZ_dev_out,
+                                       void* stream) {
+  if (device < 0 || device >= kMaxDevices || H < 1 || Tp < 1 || !frozen_mask_host) return SAF_ERR_INVALID_ARG;
+  if (H > SAF_STATIC_MAX_HEADS) return SAF_ERR_INVALID_ARG;   // beyond the built-in scratch: use saf_pattern_prepare
+  int nf = 0;
+  for (int h = 0; h < H; ++h) nf += frozen_mask_host[h] ? 1 : 0;
+  if (nf == 0) return SAF_OK;
+  if (!alpha_dev || !rho_dev || !logZ_dev_out) return SAF_ERR_INVALID_ARG;
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return SAF_ERR_CUDA;
+  if (prev != device && cudaSetDevice(device) != cudaSuccess) return SAF_ERR_CUDA;
+  int rc = SAF_OK;
+  uint8_t* scratch = nullptr;
+  {
+    // In host code the array's name is only a handle; the address a kernel can use has to be asked
+    // for, once per device, with that device current.
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_mask_ptr[device]) {
+      void* ptr = nullptr;
+      if (cudaGetSymbolAddress(&ptr, g_static_mask_scratch) != cudaSuccess || !ptr) {
+        cudaGetLastError();
+        rc = SAF_ERR_CUDA;
+      } else {
+        g_static_mask_ptr[device] = static_cast<uint8_t*>(ptr);
+      }
+    }
+    scratch = g_static_mask_ptr[device];
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (rc == SAF_OK) {
+    // The array keeps whatever the previous call left; the first H bytes are all this call reads,
+    // and they are overwritten here.
+    if (cudaMemcpyAsync(scratch, frozen_mask_host, static_cast<size_t>(H), cudaMemcpyHostToDevice, st) != cudaSuccess)
+      rc = SAF_ERR_CUDA;
+  }
+  if (rc == SAF_OK && saf::launch_logz(alpha_dev, rho_dev, logZ_dev_out, scratch, H, Tp, st) != cudaSuccess)
+    rc = SAF_ERR_CUDA;
+  if (prev != device) cudaSetDevice(prev);
+  return rc;
+}
+
