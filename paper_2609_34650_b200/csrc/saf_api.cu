@@ -488,7 +488,7 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
       return SAF_ERR_CUDA;
     {
       ScopedTimer timer(ctx, SAF_KERNEL_SCALE, st);
-      if (launch_scale_rows(V, p->v_strides, static_cast<const float*>(ctx->pat_avec.ptr), p->Tp,
+      if (launch_scale_rows(V, p->v_strides, static_cast<const float*>(ctx->pat_avec.ptr), HK_A_SCALE, p->Tp,
                             static_cast<const int*>(ctx->pat_hord.ptr), static_cast<int*>(ctx->ok_fwd.ptr),
                             ctx->vt_buf.ptr, p->B, p->H, nf, p->T, p->D, st) != cudaSuccess)
         return SAF_ERR_CUDA;
@@ -617,7 +617,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
       return SAF_ERR_CUDA;
     {
       ScopedTimer timer(ctx, SAF_KERNEL_SCALE, st);
-      if (launch_scale_rows(dO, p->o_strides, static_cast<const float*>(ctx->pat_wvec.ptr), p->Tp,
+      if (launch_scale_rows(dO, p->o_strides, static_cast<const float*>(ctx->pat_wvec.ptr), 1.0f, p->Tp,
                             static_cast<const int*>(ctx->pat_hord.ptr), static_cast<int*>(ctx->ok_bwd.ptr),
                             ctx->dot_buf.ptr, p->B, p->H, nf, p->T, p->D, st) != cudaSuccess)
         return SAF_ERR_CUDA;

@@ -31,7 +31,9 @@
 //
 // TMEM columns: [0,64) dV, [64,128) dK, [128,192)/[192,256) S^T buffers (bf16 P^T pairs re-use the
 // consumed columns; frozen P^^T tiles use the two 64-column buffers whole), [256,320)/[320,384) dP^T
-// buffers (bf16 dS^T likewise), [384,448) dQ.
+// buffers (bf16 dS^T likewise), [384,448) dQ, [448,480) K_J and [480,512) V_J as bf16 pairs (copied once
+// per item from their smem tiles, so that the score MMAs read their A operand from TMEM instead of
+// re-reading 4 KB of shared memory per instruction: the kernel is shared-memory-bandwidth bound).
 #include <cuda_bf16.h>
 #include "ptx.cuh"
 #include "saf_internal.h"
@@ -72,10 +74,10 @@ struct BwdCfg {
   // per compute group: wq[128] z2s[128] rband[256] r2raw[256] red[16]
   static constexpr int TAB_FLOATS = 128 * 2 + 256 * 2 + 16;
   static constexpr int OFF_BAR = OFF_TAB + 2 * TAB_FLOATS * 4;
-  static constexpr int NBAR = 2 + 2 * NS + 2 + 2 + 4 + 2 + 3;
+  static constexpr int NBAR = 2 + 2 * NS + 2 + 2 + 4 + 2 + 3 + 1;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
   static constexpr int TMEM_COLS = 512;
-  static constexpr int COL_DV = 0, COL_DK = 64, COL_S = 128, COL_DP = 256, COL_DQ = 384;
+  static constexpr int COL_DV = 0, COL_DK = 64, COL_S = 128, COL_DP = 256, COL_DQ = 384, COL_KT = 448, COL_VT = 480;
   static constexpr int NTHREADS = 480;
 };
 
@@ -110,7 +112,8 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   uint64_t* pfree = acc_free + 1;                // [2]
   uint64_t* bdone = pfree + 2;                   // [2] gradient MMAs that read buffer b have completed
   uint64_t* fdone = bdone + 2;                   // a frozen item's MMAs have completed
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fdone + 1);
+  uint64_t* kvt_full = fdone + 1;                // K_J / V_J have been copied into TMEM
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(kvt_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -132,6 +135,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       mbar_init(bdone + b, 1);
     }
     mbar_init(fdone, 1);
+    mbar_init(kvt_full, 8);
     mbar_init(dq_full, 1);
     mbar_init(dq_free, 4);
     mbar_init(acc_full, 1);
@@ -224,7 +228,6 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     const uint64_t d_k = umma_smem_desc(sb, 16, 1024, UMMA_LAYOUT_SW128);
     const uint64_t d_x = umma_smem_desc(sb, 128, 256, UMMA_LAYOUT_NONE);
     const uint32_t lo_k = desc_lo(d_k), hi_k = desc_hi(d_k), lo_x = desc_lo(d_x), hi_x = desc_hi(d_x);
-    const uint32_t k_lo = lo_k + (C::OFF_K >> 4), v_lo = lo_k + (C::OFF_V >> 4);
     const uint32_t ones_lo = lo_x + (C::OFF_ONES >> 4);
     uint32_t nkv = 0, nqdo = 0, nfd = 0;
     uint32_t nbd0 = 0, nbd1 = 0;
@@ -245,9 +248,14 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         ++nfd;
         continue;
       }
-      ok = mbar_wait_warp(kv_full, nkv & 1, wc, B_KV_FULL);
+      // K_J / V_J are read from TMEM: wait for the compute warps' copy; the smem tiles are then free
+      // as far as this issuer is concerned
+      ok = mbar_wait_warp(kvt_full, nkv & 1, wc, B_KV_FULL);
       if (!ok) break;
       ++nkv;
+      tc_fence_after();
+      if (leader) mbar_arrive(kv_empty);
+      __syncwarp();
       const int U = 2 * ntiles;
       for (int u = 0; u < U && ok; ++u) {
         const uint32_t pos = nqdo + (u >> 1);
@@ -271,14 +279,15 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         const uint32_t t_s = tmem + C::COL_S + 64 * b, t_dp = tmem + C::COL_DP + 64 * b;
         if (leader) {
 #pragma unroll
-          for (int kc = 0; kc < 4; ++kc) umma_ss2(t_s, k_lo + 2 * kc, hi_k, q_lo + 2 * kc, hi_k, id_s, kc > 0);
+          for (int kc = 0; kc < 4; ++kc)
+            umma_ts2(t_s, tmem + C::COL_KT + 8 * kc, q_lo + 2 * kc, hi_k, id_s, kc > 0);
           umma_ss2(t_s, ones_lo, hi_x, qx_lo, hi_x, id_s, 1);
 #pragma unroll
-          for (int kc = 0; kc < 4; ++kc) umma_ss2(t_dp, v_lo + 2 * kc, hi_k, do_lo + 2 * kc, hi_k, id_s, kc > 0);
+          for (int kc = 0; kc < 4; ++kc)
+            umma_ts2(t_dp, tmem + C::COL_VT + 8 * kc, do_lo + 2 * kc, hi_k, id_s, kc > 0);
           umma_ss2(t_dp, ones_lo, hi_x, dox_lo, hi_x, id_s, 1);
           umma_commit(sdp_full + b);
           if (b == 1) umma_commit(qdo_empty + s);       // this issuer's reads of the stage
-          if (u == U - 1) umma_commit(kv_empty);         // ... and of K_J / V_J
         }
         __syncwarp();
       }
@@ -492,7 +501,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     float* r2raw = tab + 512;
     float* red = tab + 768;
     const int bar_id = 4 + grp;                          // named barrier of this group
-    uint32_t nacc = 0, ntile_ord = 0, nsdp = 0, npf = 0;
+    uint32_t nacc = 0, ntile_ord = 0, nsdp = 0, npf = 0, nkvc = 0;
     bool ok = true;
     int tr_n = 0;
     (void)tr_n;
@@ -510,9 +519,29 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       if (!ord && p.band_b != nullptr && p.fast_ok[w.h] != 0) {
         // tensor-core form: nothing to do per tile; lane m holds key 127-m, scaled by a(j) below
         key = w.blk * BLK + 127 - rowl;
-        dv_mul = (key < p.T) ? p.avec[static_cast<size_t>(w.h) * p.Tp + key] : 0.0f;
+        dv_mul = (key < p.T) ? p.avec[static_cast<size_t>(w.h) * p.Tp + key] * (1.0f / HK_BAND_SCALE) : 0.0f;
       } else if (ord) {
         const float c = p.scale_log2;
+        {
+          // K_J (group 0) / V_J (group 1): this thread's row from the swizzled smem tile into TMEM as the
+          // A operand of the score MMAs (bf16 pairs, feature index = reduction index)
+          if (!mbar_wait_warp(kv_full, nkvc & 1, wc, B_KV_FULL)) ok = false;
+          ++nkvc;
+          const uint32_t src = smem_u32(smem + (grp == 0 ? C::OFF_K : C::OFF_V)) + rowl * 128;
+          uint32_t kvr[32];
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            const uint32_t a = src + static_cast<uint32_t>(g ^ (rowl & 7)) * 16;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(kvr[4 * g]), "=r"(kvr[4 * g + 1]), "=r"(kvr[4 * g + 2]), "=r"(kvr[4 * g + 3])
+                         : "r"(a)
+                         : "memory");
+          }
+          tmem_st32(tmem + lane_base + (grp == 0 ? C::COL_KT : C::COL_VT), kvr);
+          tmem_wait_st();
+          tc_fence_before();
+          warp_arrive(kvt_full);
+        }
         for (int t = 0; t < ntiles; ++t) {
           // this group's half tile of tile t: queries 64*grp .. 64*grp+63
           TR(1 + grp, 11);

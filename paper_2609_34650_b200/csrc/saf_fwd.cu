@@ -330,7 +330,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       if (w.kind == KIND_FROZEN && p.band_f != nullptr && p.fast_ok[w.h] != 0) {
         // tensor-core form: nothing to do per tile; lane m holds query 127-m, scaled by w(i) below
         row = w.blk * BLK + 127 - rowl;
-        inv_l = (row < p.T) ? p.wvec[static_cast<size_t>(w.h) * p.Tp + row] : 0.0f;
+        inv_l = (row < p.T) ? p.wvec[static_cast<size_t>(w.h) * p.Tp + row] * (1.0f / (HK_BAND_SCALE * HK_A_SCALE)) : 0.0f;
       } else if (w.kind == KIND_ORDINARY) {
         float m_ref = -INFINITY, l = 0.0f;
         const float c = p.scale_log2;

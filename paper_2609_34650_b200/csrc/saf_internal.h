@@ -68,8 +68,12 @@ cudaError_t launch_logz(const float* alpha, const float* rho, float* logZ, const
 cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const float* logZ, const uint8_t* mask_dev,
                                   int H, int Tp, float* consts, int* fast_ok, float* avec, float* wvec, void* band_f,
                                   void* band_b, cudaStream_t st);
-cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, int Tp, const int* hord,
-                              int* call_ok, void* dst, int B, int H, int Hf, int T, int D, cudaStream_t st);
+cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, float extra, int Tp,
+                              const int* hord, int* call_ok, void* dst, int B, int H, int Hf, int T, int D,
+                              cudaStream_t st);
+// powers of two that put the fp16 operands of the tensor-core frozen form into fp16's range
+constexpr float HK_BAND_SCALE = 16384.0f;        // bands hold 2^14 r
+constexpr float HK_A_SCALE = 2048.0f;            // the forward stages 2^11 a V
 // mvt: map of the a-scaled V of the frozen heads [B][Hf][T][D] (any valid map when band_f is NULL)
 cudaError_t launch_fwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                        const CUtensorMap& mvt, const FwdParams& p, int grid, cudaStream_t st);

@@ -60,8 +60,11 @@ cudaError_t launch_logz(const float* alpha, const float* rho, float* logZ, const
 //   band_b[h][D][x] : g[x] = r(128 D - 127 + x)   (backward, rows = keys reversed)
 // The band and the scaled V / dO tiles are fp16 (the tensor core needs one 16-bit type for both operands;
 // fp16 keeps 11 significant bits, so the form adds less rounding than the bf16 pattern tile of the
-// general path).  It is used for a head only if max_i (c_a + c_r - logZ(i)) <= 5 (fast_ok): then w <= e^5,
-// every r below fp16's normal range weighs less than 1 % of its row, and w dO stays in range.
+// general path).  To use fp16's range, the bands hold 2^14 r and the forward stages 2^11 a V; the
+// epilogues undo the powers of two.  A value below fp16's normal range is then off by at most 2^-25 in
+// scaled units, i.e. the pattern entry w a r by at most w 2^-39: the form is used for a head only if
+// max_i (c_a + c_r - logZ(i)) <= 9 (fast_ok), which keeps that below 1e-8 and leaves w dO room in fp16
+// (the scaling kernel checks the staged values against fp16's range on every call).
 __global__ void __launch_bounds__(256) saf_pattern_consts_kernel(const float* __restrict__ alpha,
                                                                  const float* __restrict__ rho,
                                                                  const float* __restrict__ logZ,
@@ -104,7 +107,7 @@ __global__ void __launch_bounds__(256) saf_pattern_consts_kernel(const float* __
     consts[2 * h] = ma;
     consts[2 * h + 1] = mr;
     const float wmax = ma + mr - mz;
-    fast_ok[h] = (wmax <= 5.0f && wmax > -1e30f && ma < 1e30f && mr < 1e30f) ? 1 : 0;
+    fast_ok[h] = (wmax <= 9.0f && wmax > -1e30f && ma < 1e30f && mr < 1e30f) ? 1 : 0;
   }
 }
 
@@ -131,8 +134,8 @@ __global__ void __launch_bounds__(256) saf_pattern_tables_kernel(const float* __
     const int x = 8 * c + ri + e;
     const int df = dblk * 128 + 127 - x, db = dblk * 128 - 127 + x;
     const bool used = c < 31;
-    const float vf = (used && df >= 0 && df < Tp) ? __expf(rho[row + df] - cr) : 0.0f;
-    const float vb = (used && db >= 0 && db < Tp) ? __expf(rho[row + db] - cr) : 0.0f;
+    const float vf = (used && df >= 0 && df < Tp) ? 16384.0f * __expf(rho[row + df] - cr) : 0.0f;
+    const float vb = (used && db >= 0 && db < Tp) ? 16384.0f * __expf(rho[row + db] - cr) : 0.0f;
     band_f[band + idx] = __float2half_rn(vf);
     band_b[band + idx] = __float2half_rn(vb);
   }
@@ -151,14 +154,15 @@ cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const fl
   return cudaGetLastError();
 }
 
-// dst[b][ord(h)][t][:] = fp16(vec[h][t] * src[b][h][t][:]) for the frozen heads whose tensor-core form is
+// dst[b][ord(h)][t][:] = fp16(extra * vec[h][t] * src[b][h][t][:]) for the frozen heads whose tensor-core form is
 // enabled (V scaled by a, or dO scaled by w).  Eight features per thread.  call_ok[h] starts as a copy of
 // fast_ok[h]; a product that leaves fp16's range clears it, which sends that head down the general path
 // in the kernel that follows.
 template <int D>
 __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16* __restrict__ src, int64_t s0, int64_t s1,
-                                                             int64_t s2, const float* __restrict__ vec, int Tp,
-                                                             const int* __restrict__ hord, int* __restrict__ call_ok,
+                                                             int64_t s2, const float* __restrict__ vec, float extra,
+                                                             int Tp, const int* __restrict__ hord,
+                                                             int* __restrict__ call_ok,
                                                              __half* __restrict__ dst, int B, int H, int Hf, int T) {
   constexpr int TPR = D / 8;
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
@@ -170,7 +174,7 @@ __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16
   const int b = static_cast<int>(rowid / (static_cast<long long>(T) * H));
   const int ord = hord[h];
   if (ord < 0 || !call_ok[h]) return;
-  const float f = vec[static_cast<size_t>(h) * Tp + t];
+  const float f = vec[static_cast<size_t>(h) * Tp + t] * extra;
   const uint4 v4 = *reinterpret_cast<const uint4*>(src + b * s0 + h * s1 + static_cast<int64_t>(t) * s2 + part * 8);
   const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&v4);
   __half2 o[4];
@@ -187,18 +191,19 @@ __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16
       *reinterpret_cast<uint4*>(o);
 }
 
-cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, int Tp, const int* hord,
-                              int* call_ok, void* dst, int B, int H, int Hf, int T, int D, cudaStream_t st) {
+cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, float extra, int Tp,
+                              const int* hord, int* call_ok, void* dst, int B, int H, int Hf, int T, int D,
+                              cudaStream_t st) {
   const long long nthreads = static_cast<long long>(B) * H * T * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
   if (D == 64)
     saf_scale_rows_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
-                                                    strides[2], vec, Tp, hord, call_ok, static_cast<__half*>(dst), B,
-                                                    H, Hf, T);
+                                                    strides[2], vec, extra, Tp, hord, call_ok,
+                                                    static_cast<__half*>(dst), B, H, Hf, T);
   else
     saf_scale_rows_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
-                                                     strides[2], vec, Tp, hord, call_ok, static_cast<__half*>(dst), B,
-                                                     H, Hf, T);
+                                                     strides[2], vec, extra, Tp, hord, call_ok,
+                                                     static_cast<__half*>(dst), B, H, Hf, T);
   return cudaGetLastError();
 }
 
