@@ -64,7 +64,7 @@ struct saf_ctx {
   // tensor-core form of frozen heads: tables built by saf_pattern_prepare, scaled V / dO per call
   PatternCache pat;
   bool tensor_pattern = true;              // SAF_DISABLE_TENSOR_PATTERN=1 turns the form off
-  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, vt_buf, dot_buf, ok_fwd, ok_bwd;
+  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, vt_buf, dot_buf, ok_fwd, ok_bwd;
   bool profiling = false;
   std::vector<TimedLaunch> timed;          // event pairs recorded since the last query
   std::vector<cudaEvent_t> event_pool;
@@ -353,7 +353,7 @@ int saf_destroy(saf_ctx* ctx) {
     cudaFree(e.offsets_dev);
   }
   DevBuf* pbufs[] = {&ctx->pat_consts, &ctx->pat_ok, &ctx->pat_avec, &ctx->pat_wvec, &ctx->pat_bandf, &ctx->pat_bandb,
-                     &ctx->pat_hord, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd};
+                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd};
   for (DevBuf* b : pbufs) release(*b);
   DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->hq, &ctx->hk, &ctx->hv,
                     &ctx->hdo, &ctx->ho, &ctx->hlse, &ctx->hdq, &ctx->hdk, &ctx->hdv, &ctx->halpha, &ctx->hrho,
@@ -397,14 +397,20 @@ int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* froz
   if ((rc = ensure(ctx->pat_consts, static_cast<size_t>(H) * 2 * sizeof(float))) ||
       (rc = ensure(ctx->pat_ok, static_cast<size_t>(H) * sizeof(int))) || (rc = ensure(ctx->pat_avec, vecb)) ||
       (rc = ensure(ctx->pat_wvec, vecb)) || (rc = ensure(ctx->pat_bandf, bandb)) ||
-      (rc = ensure(ctx->pat_bandb, bandb)) || (rc = ensure(ctx->pat_hord, static_cast<size_t>(H) * sizeof(int))))
+      (rc = ensure(ctx->pat_bandb, bandb)) || (rc = ensure(ctx->pat_hord, static_cast<size_t>(H) * sizeof(int))) ||
+      (rc = ensure(ctx->pat_hlist, static_cast<size_t>(H) * sizeof(int))))
     return rc;
-  std::vector<int> hord(H, -1);
+  std::vector<int> hord(H, -1), hlist(H, 0);
   int ord = 0;
   for (int h = 0; h < H; ++h)
-    if (frozen_mask_host[h]) hord[h] = ord++;
+    if (frozen_mask_host[h]) {
+      hlist[ord] = h;
+      hord[h] = ord++;
+    }
   if (cudaMemcpyAsync(ctx->pat_hord.ptr, hord.data(), static_cast<size_t>(H) * sizeof(int), cudaMemcpyHostToDevice, st) !=
-      cudaSuccess)
+          cudaSuccess ||
+      cudaMemcpyAsync(ctx->pat_hlist.ptr, hlist.data(), static_cast<size_t>(H) * sizeof(int), cudaMemcpyHostToDevice,
+                      st) != cudaSuccess)
     return SAF_ERR_CUDA;
   {
     ScopedTimer timer(ctx, SAF_KERNEL_LOGZ, st);
@@ -489,8 +495,8 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     {
       ScopedTimer timer(ctx, SAF_KERNEL_SCALE, st);
       if (launch_scale_rows(V, p->v_strides, static_cast<const float*>(ctx->pat_avec.ptr), HK_A_SCALE, p->Tp,
-                            static_cast<const int*>(ctx->pat_hord.ptr), static_cast<int*>(ctx->ok_fwd.ptr),
-                            ctx->vt_buf.ptr, p->B, p->H, nf, p->T, p->D, st) != cudaSuccess)
+                            static_cast<const int*>(ctx->pat_hlist.ptr), static_cast<int*>(ctx->ok_fwd.ptr),
+                            ctx->vt_buf.ptr, p->B, nf, p->T, p->D, st) != cudaSuccess)
         return SAF_ERR_CUDA;
     }
     rc = make_map_contig(ctx, &mvt, ctx->vt_buf.ptr, p, nf);
@@ -618,8 +624,8 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     {
       ScopedTimer timer(ctx, SAF_KERNEL_SCALE, st);
       if (launch_scale_rows(dO, p->o_strides, static_cast<const float*>(ctx->pat_wvec.ptr), 1.0f, p->Tp,
-                            static_cast<const int*>(ctx->pat_hord.ptr), static_cast<int*>(ctx->ok_bwd.ptr),
-                            ctx->dot_buf.ptr, p->B, p->H, nf, p->T, p->D, st) != cudaSuccess)
+                            static_cast<const int*>(ctx->pat_hlist.ptr), static_cast<int*>(ctx->ok_bwd.ptr),
+                            ctx->dot_buf.ptr, p->B, nf, p->T, p->D, st) != cudaSuccess)
         return SAF_ERR_CUDA;
     }
     rc = make_map_contig(ctx, &mdot, ctx->dot_buf.ptr, p, nf);

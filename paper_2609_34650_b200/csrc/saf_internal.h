@@ -69,7 +69,7 @@ cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const fl
                                   int H, int Tp, float* consts, int* fast_ok, float* avec, float* wvec, void* band_f,
                                   void* band_b, cudaStream_t st);
 cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, float extra, int Tp,
-                              const int* hord, int* call_ok, void* dst, int B, int H, int Hf, int T, int D,
+                              const int* hlist, int* call_ok, void* dst, int B, int Hf, int T, int D,
                               cudaStream_t st);
 // powers of two that put the fp16 operands of the tensor-core frozen form into fp16's range
 constexpr float HK_BAND_SCALE = 16384.0f;        // bands hold 2^14 r

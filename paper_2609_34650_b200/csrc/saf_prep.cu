@@ -154,26 +154,26 @@ cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const fl
   return cudaGetLastError();
 }
 
-// dst[b][ord(h)][t][:] = fp16(extra * vec[h][t] * src[b][h][t][:]) for the frozen heads whose tensor-core form is
+// dst[b][ord][t][:] = fp16(extra * vec[h][t] * src[b][h][t][:]), h = hlist[ord], for the frozen heads whose tensor-core form is
 // enabled (V scaled by a, or dO scaled by w).  Eight features per thread.  call_ok[h] starts as a copy of
 // fast_ok[h]; a product that leaves fp16's range clears it, which sends that head down the general path
 // in the kernel that follows.
 template <int D>
 __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16* __restrict__ src, int64_t s0, int64_t s1,
                                                              int64_t s2, const float* __restrict__ vec, float extra,
-                                                             int Tp, const int* __restrict__ hord,
+                                                             int Tp, const int* __restrict__ hlist,
                                                              int* __restrict__ call_ok,
-                                                             __half* __restrict__ dst, int B, int H, int Hf, int T) {
+                                                             __half* __restrict__ dst, int B, int Hf, int T) {
   constexpr int TPR = D / 8;
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
-  const long long rowid = gid / TPR;
+  const long long rowid = gid / TPR;               // over [B][Hf][T]: frozen heads only
   const int part = static_cast<int>(gid % TPR);
-  if (rowid >= static_cast<long long>(B) * H * T) return;
+  if (rowid >= static_cast<long long>(B) * Hf * T) return;
   const int t = static_cast<int>(rowid % T);
-  const int h = static_cast<int>((rowid / T) % H);
-  const int b = static_cast<int>(rowid / (static_cast<long long>(T) * H));
-  const int ord = hord[h];
-  if (ord < 0 || !call_ok[h]) return;
+  const int ord = static_cast<int>((rowid / T) % Hf);
+  const int b = static_cast<int>(rowid / (static_cast<long long>(T) * Hf));
+  const int h = hlist[ord];
+  if (!call_ok[h]) return;
   const float f = vec[static_cast<size_t>(h) * Tp + t] * extra;
   const uint4 v4 = *reinterpret_cast<const uint4*>(src + b * s0 + h * s1 + static_cast<int64_t>(t) * s2 + part * 8);
   const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&v4);
@@ -187,23 +187,22 @@ __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16
     o[e] = __floats2half2_rn(y0, y1);
   }
   if (bad) atomicExch(call_ok + h, 0);
-  *reinterpret_cast<uint4*>(dst + ((static_cast<size_t>(b) * Hf + ord) * T + t) * D + part * 8) =
-      *reinterpret_cast<uint4*>(o);
+  *reinterpret_cast<uint4*>(dst + (static_cast<size_t>(rowid)) * D + part * 8) = *reinterpret_cast<uint4*>(o);
 }
 
 cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, float extra, int Tp,
-                              const int* hord, int* call_ok, void* dst, int B, int H, int Hf, int T, int D,
+                              const int* hlist, int* call_ok, void* dst, int B, int Hf, int T, int D,
                               cudaStream_t st) {
-  const long long nthreads = static_cast<long long>(B) * H * T * (D / 8);
+  const long long nthreads = static_cast<long long>(B) * Hf * T * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
   if (D == 64)
     saf_scale_rows_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
-                                                    strides[2], vec, extra, Tp, hord, call_ok,
-                                                    static_cast<__half*>(dst), B, H, Hf, T);
+                                                    strides[2], vec, extra, Tp, hlist, call_ok,
+                                                    static_cast<__half*>(dst), B, Hf, T);
   else
     saf_scale_rows_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
-                                                     strides[2], vec, extra, Tp, hord, call_ok,
-                                                     static_cast<__half*>(dst), B, H, Hf, T);
+                                                     strides[2], vec, extra, Tp, hlist, call_ok,
+                                                     static_cast<__half*>(dst), B, Hf, T);
   return cudaGetLastError();
 }
 
