@@ -1,14 +1,17 @@
 // Backward of the hybrid causal attention layer on sm_100a (head dimension 64): one persistent
 // kernel, one work item per (batch, head, 128-key block J), looping over query blocks I >= J.
 //
-// CTA = 448 threads:
-//   warps 0-3  compute group 0: even 64-query half tiles (TMEM buffer 0); TMEM lane = key row
-//   warps 4-7  compute group 1: odd half tiles (TMEM buffer 1)
-//   warps 8-11 dQ drain: TMEM -> swizzled smem -> TMA reduce-add into the fp32 dQ accumulator
-//   warp 12    TMA producer
-//   warp 13    tcgen05 issuer of the score MMAs A(u); warp 14 issuer of the gradient MMAs B(u), C(t) and
-//              TMEM owner.  An issuing thread is stalled while its MMAs queue, so two issuers let one
-//              stream's bookkeeping (barrier waits) overlap the other stream's tensor work.
+// CTA = 736 threads:
+//   warps 0-7   compute group 0: even 64-query half tiles (TMEM buffer 0); TMEM lane = key row, two warps
+//               per lane quarter, each on 32 of the half tile's 64 query columns
+//   warps 8-15  compute group 1: odd half tiles (TMEM buffer 1)
+//   warps 16-19 dQ drain: TMEM -> swizzled smem -> TMA reduce-add into the fp32 dQ accumulator
+//   warp 20     TMA producer
+//   warp 21     tcgen05 issuer of the score MMAs A(u); warp 22 issuer of the gradient MMAs B(u), C(t) and
+//               TMEM owner.  An issuing thread is stalled while its MMAs queue, so two issuers let one
+//               stream's bookkeeping (barrier waits) overlap the other stream's tensor work.
+// The per-tile critical path is a chain (scores -> exponentials -> gradient MMAs -> next scores on the
+// same buffer), so the exponential step is spread over as many warps as the register file allows.
 //
 // Ordinary item (Appendix E.2: key-block programs accumulate dV and dK; dQ here comes out of the same
 // tile loop and is accumulated across key blocks by reduce-adds instead of a second pass).  The tile
@@ -30,7 +33,7 @@
 //   and 8 MMAs.  The compute warps only scale the finished rows by a(j) (lane m holds key 127-m).
 //
 // TMEM columns: [0,64) dV, [64,128) dK, [128,192)/[192,256) S^T buffers (bf16 P^T pairs re-use the
-// consumed columns; frozen P^^T tiles use the two 64-column buffers whole), [256,320)/[320,384) dP^T
+// columns their own warp consumed: [0,16) and [32,48) of the buffer; frozen P^^T tiles use the two 64-column buffers whole), [256,320)/[320,384) dP^T
 // buffers (bf16 dS^T likewise), [384,448) dQ, [448,480) K_J and [480,512) V_J as bf16 pairs (copied once
 // per item from their smem tiles, so that the score MMAs read their A operand from TMEM instead of
 // re-reading 4 KB of shared memory per instruction: the kernel is shared-memory-bandwidth bound).
@@ -78,7 +81,7 @@ struct BwdCfg {
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
   static constexpr int TMEM_COLS = 512;
   static constexpr int COL_DV = 0, COL_DK = 64, COL_S = 128, COL_DP = 256, COL_DQ = 384, COL_KT = 448, COL_VT = 480;
-  static constexpr int NTHREADS = 480;
+  static constexpr int NTHREADS = 736;
 };
 
 enum BwdSite { B_KV_EMPTY = 21, B_QDO_EMPTY, B_KV_FULL, B_QDO_FULL, B_PDS_FULL, B_ACC_FREE, B_DQ_FREE, B_SDP_FULL,
@@ -130,16 +133,16 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(sdp_full + b, 1);
-      mbar_init(pds_full + b, 4);                // one arrival per warp of the group
+      mbar_init(pds_full + b, 8);                // one arrival per warp of the group
       mbar_init(pfree + b, 1);
       mbar_init(bdone + b, 1);
     }
     mbar_init(fdone, 1);
-    mbar_init(kvt_full, 8);
+    mbar_init(kvt_full, 16);
     mbar_init(dq_full, 1);
     mbar_init(dq_free, 4);
     mbar_init(acc_full, 1);
-    mbar_init(acc_free, 8);
+    mbar_init(acc_free, 16);
     mbar_fence_init();
   }
   // constant tile of ones (columns 0..2) in the no-swizzle K-major core-matrix layout
@@ -152,7 +155,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     }
     reinterpret_cast<uint4*>(smem + C::OFF_ONES)[i] = v;
   }
-  if (warp == 14) {
+  if (warp == 22) {
     tmem_alloc(tmem_slot, C::TMEM_COLS);
     tmem_relinquish();
   }
@@ -163,7 +166,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   const uint32_t tmem = *tmem_slot;
   const int it_begin = p.cta_offsets[blockIdx.x], it_end = p.cta_offsets[blockIdx.x + 1];
 
-  if (warp == 12) {
+  if (warp == 20) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&mq);
@@ -217,7 +220,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         }
       }
     }
-  } else if (warp == 13) {
+  } else if (warp == 21) {
     // ------------------------------------------------------------------ tcgen05 issuer X: score MMAs A(u)
     // The whole warp walks the loops (warp-uniform operands); one elected lane issues.
     const bool leader = elect_one() != 0;
@@ -231,6 +234,8 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     const uint32_t ones_lo = lo_x + (C::OFF_ONES >> 4);
     uint32_t nkv = 0, nqdo = 0, nfd = 0;
     uint32_t nbd0 = 0, nbd1 = 0;
+    int tr_n = 0;
+    (void)tr_n;
     bool ok = true;
     for (int it = it_begin; it < it_end && ok; ++it) {
       const WorkItem w = p.items[it];
@@ -261,6 +266,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         const uint32_t pos = nqdo + (u >> 1);
         const uint32_t s = pos % C::NS;
         const uint32_t b = u & 1;
+        TR(3, 1);
         // buffer b is free once the gradient MMAs of half tile u-2 have read their bf16 operands from it
         if (b == 0) {
           ok = mbar_wait_warp(bdone, (nbd0 & 1) ^ 1, wc, B_PFREE);
@@ -271,6 +277,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           ++nbd1;
         }
         if (!ok) break;
+        TR(3, 2);
         tc_fence_after();
         const uint32_t q_lo = lo_k + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
         const uint32_t do_lo = lo_k + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
@@ -289,11 +296,12 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           umma_commit(sdp_full + b);
           if (b == 1) umma_commit(qdo_empty + s);       // this issuer's reads of the stage
         }
+        TR(3, 3);
         __syncwarp();
       }
       nqdo += ntiles;
     }
-  } else if (warp == 14) {
+  } else if (warp == 22) {
     // ------------------------------------------------------------------ tcgen05 issuer Y: gradient MMAs
     const bool leader = elect_one() != 0;
     const uint32_t sb = smem_u32(smem);
@@ -340,10 +348,10 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           if (leader) {
 #pragma unroll
             for (int kc = 0; kc < 4; ++kc)
-              umma_ts2(tmem + C::COL_DV, t_p + 8 * kc, do_lo + 128 * kc, hi_m, id_acc, kc > 0 ? 1u : acc0);
+              umma_ts2(tmem + C::COL_DV, t_p + 8 * kc + (kc >= 2 ? 16 : 0), do_lo + 128 * kc, hi_m, id_acc, kc > 0 ? 1u : acc0);
 #pragma unroll
             for (int kc = 0; kc < 4; ++kc)
-              umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc, q_lo + 128 * kc, hi_m, id_acc, kc > 0 ? 1u : acc0);
+              umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc + (kc >= 2 ? 16 : 0), q_lo + 128 * kc, hi_m, id_acc, kc > 0 ? 1u : acc0);
             umma_commit(bdone + b);
           }
           TR(0, 6);
@@ -435,7 +443,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       if (leader) umma_commit(acc_full);
       __syncwarp();
     }
-  } else if (warp >= 8 && warp < 12) {
+  } else if (warp >= 16 && warp < 20) {
     // ------------------------------------------------------------------ dQ drain warps (128 threads)
     const int q4 = warp & 3;                            // TMEM lane quarter of this warp
     const int rowl = q4 * 32 + lane;                    // query row within the tile
@@ -448,7 +456,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       if (w.kind != KIND_ORDINARY) continue;
       bool leave = false;
       for (int I = w.blk; I < nblk; ++I) {
-        // the previous tile's reduce has finished reading the staging buffer (thread 256 waits for it
+        // the previous tile's reduce has finished reading the staging buffer (thread 512 waits for it
         // before arriving here); the drain warps also agree here whether a wait has been abandoned
         if (named_bar_or(2, 128, !ok)) {
           leave = true;
@@ -478,7 +486,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         }
         fence_proxy_async_smem();
         named_bar_sync(3, 128);
-        if (tid == 256 && ok) {
+        if (tid == 512 && ok) {
           tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 0, I * BLK, w.h, w.b);
           tma_reduce_add_4d(&mdq, smem + C::OFF_DQ + C::PANEL, 32, I * BLK, w.h, w.b);
           bulk_commit_group();
@@ -487,11 +495,12 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       }
       if (leave) break;
     }
-    if (tid == 256) bulk_wait_group0();                 // all reduce-adds have landed before the kernel ends
+    if (tid == 512) bulk_wait_group0();                 // all reduce-adds have landed before the kernel ends
   } else {
-    // ------------------------------------------------------------------ compute groups (2 x 128 threads)
-    const int grp = warp >> 2, q4 = warp & 3;
-    const int gtid = tid & 127;                          // thread index within the group
+    // ------------------------------------------------------------------ compute groups (2 x 256 threads)
+    // warp = 8 grp + 4 sub + q4: two warps per TMEM lane quarter, `sub` picks the 32-column half
+    const int grp = warp >> 3, sub = (warp >> 2) & 1, q4 = warp & 3;
+    const int gtid = tid & 255;                          // thread index within the group
     const int rowl = q4 * 32 + lane;                     // TMEM lane = key row of the block
     const uint32_t lane_base = static_cast<uint32_t>(q4 * 32) << 16;
     float* tab = reinterpret_cast<float*>(smem + C::OFF_TAB) + grp * C::TAB_FLOATS;
@@ -514,7 +523,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       int key = w.blk * BLK + rowl;
       const size_t bh = static_cast<size_t>(w.b) * p.H + w.h;
       float dv_mul = 1.0f;
-      if (named_bar_or(bar_id, 128, !ok)) break;
+      if (named_bar_or(bar_id, 256, !ok)) break;
 
       if (!ord && p.band_b != nullptr && p.fast_ok[w.h] != 0) {
         // tensor-core form: nothing to do per tile; lane m holds key 127-m, scaled by a(j) below
@@ -528,45 +537,46 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           if (!mbar_wait_warp(kv_full, nkvc & 1, wc, B_KV_FULL)) ok = false;
           ++nkvc;
           const uint32_t src = smem_u32(smem + (grp == 0 ? C::OFF_K : C::OFF_V)) + rowl * 128;
-          uint32_t kvr[32];
+          uint32_t kvr[16];
 #pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            const uint32_t a = src + static_cast<uint32_t>(g ^ (rowl & 7)) * 16;
+          for (int g = 0; g < 4; ++g) {
+            const uint32_t a = src + static_cast<uint32_t>((4 * sub + g) ^ (rowl & 7)) * 16;
             asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                          : "=r"(kvr[4 * g]), "=r"(kvr[4 * g + 1]), "=r"(kvr[4 * g + 2]), "=r"(kvr[4 * g + 3])
                          : "r"(a)
                          : "memory");
           }
-          tmem_st32(tmem + lane_base + (grp == 0 ? C::COL_KT : C::COL_VT), kvr);
+          tmem_st16(tmem + lane_base + (grp == 0 ? C::COL_KT : C::COL_VT) + 16 * sub, kvr);
           tmem_wait_st();
           tc_fence_before();
           warp_arrive(kvt_full);
         }
         for (int t = 0; t < ntiles; ++t) {
-          // this group's half tile of tile t: queries 64*grp .. 64*grp+63
-          TR(1 + grp, 11);
+          // this group's half tile of tile t: queries 64*grp .. 64*grp+63; this warp's 32 of them
+          if ((warp & 7) == 0) TR(1 + grp, 11);
           if (!mbar_wait_warp(sdp_full + grp, nsdp & 1, wc, B_SDP_FULL)) ok = false;
           ++nsdp;
           tc_fence_after();
-          TR(1 + grp, 12);
+          if ((warp & 7) == 0) TR(1 + grp, 12);
           const uint32_t t_s = tmem + lane_base + C::COL_S + 64 * grp;
           const uint32_t t_dp = tmem + lane_base + C::COL_DP + 64 * grp;
           const uint32_t rowaddr =
               smem_u32(smem + C::OFF_DS + ((ntile_ord + t) & 1) * 2 * C::PANEL + grp * C::PANEL) + rowl * 128;
           const bool diag = (t == 0);
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            uint32_t rs[32], rd[32];
-            tmem_ld32(t_s + 32 * cc, rs);
-            tmem_ld32(t_dp + 32 * cc, rd);
+          for (int hh = 0; hh < 2; ++hh) {
+            const int c0 = 32 * sub + 16 * hh;             // first of this pass's 16 query columns
+            uint32_t rs[16], rd[16];
+            tmem_ld16(t_s + c0, rs);
+            tmem_ld16(t_dp + c0, rd);
             tmem_wait_ld();
-            uint32_t pk[16], dk[16];
+            uint32_t pk[8], dk[8];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
+            for (int e = 0; e < 8; ++e) {
               float p0 = ex2_approx(__uint_as_float(rs[2 * e]) * c);
               float p1 = ex2_approx(__uint_as_float(rs[2 * e + 1]) * c);
               if (diag) {                                  // causal: query index >= key index
-                const int qa = 64 * grp + 32 * cc + 2 * e;
+                const int qa = 64 * grp + c0 + 2 * e;
                 if (qa < rowl) p0 = 0.0f;
                 if (qa + 1 < rowl) p1 = 0.0f;
               }
@@ -574,12 +584,12 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
               dk[e] = pack_bf16x2(p0 * __uint_as_float(rd[2 * e]), p1 * __uint_as_float(rd[2 * e + 1]));
             }
             // bf16 pairs re-use columns this warp has already consumed
-            tmem_st16(t_s + 16 * cc, pk);
-            tmem_st16(t_dp + 16 * cc, dk);
+            tmem_st8(t_s + 32 * sub + 8 * hh, pk);
+            tmem_st8(t_dp + 32 * sub + 8 * hh, dk);
             // dS^T row (this key) -> smem panel of this half tile, 128-byte swizzle (chunk ^= row & 7)
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              const uint32_t chunk = static_cast<uint32_t>((4 * cc + g) ^ (rowl & 7));
+            for (int g = 0; g < 2; ++g) {
+              const uint32_t chunk = static_cast<uint32_t>((4 * sub + 2 * hh + g) ^ (rowl & 7));
               st_shared_v4(rowaddr + chunk * 16, dk[4 * g], dk[4 * g + 1], dk[4 * g + 2], dk[4 * g + 3]);
             }
           }
@@ -587,7 +597,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           fence_proxy_async_smem();
           tc_fence_before();
           warp_arrive(pds_full + grp);
-          TR(1 + grp, 16);
+          if ((warp & 7) == 0) TR(1 + grp, 16);
         }
         ntile_ord += ntiles;
       } else {
@@ -600,42 +610,41 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ma = fmaxf(ma, __shfl_xor_sync(0xffffffffu, ma, o));
         // block maximum of alpha over the 128 keys: exchanged once per item through `red`
-        if (lane == 0) red[12 + q4] = ma;
-        named_bar_sync(bar_id, 128);
+        if (lane == 0 && sub == 0) red[12 + q4] = ma;
+        named_bar_sync(bar_id, 256);
         ma = fmaxf(fmaxf(red[12], red[13]), fmaxf(red[14], red[15]));
         const float aj = ex2_approx(a2 - ma);
         bool leave = false;
         int nmine = 0;
         for (int t = grp; t < ntiles; t += 2, ++nmine) {
           const int I = w.blk + t;
-          if (named_bar_or(bar_id, 128, !ok)) {          // uniform over the group: leave together
+          if (named_bar_or(bar_id, 256, !ok)) {          // uniform over the group: leave together
             ok = false;
             leave = true;
             break;
           }
           const int d0 = t * BLK - 127;                  // band: distances d0 .. d0+254, index x = q - row + 127
-          const int da = d0 + gtid, db = d0 + 128 + gtid;
-          const float r2a = (da >= 0 && da < p.T) ? rho_h[da] * LOG2E_B : -INFINITY;
-          const float r2b = (gtid < 127 && db >= 0 && db < p.T) ? rho_h[db] * LOG2E_B : -INFINITY;
+          // band entry x = gtid (255 of them); the query terms are built by the first 128 threads
+          const int da = d0 + gtid;
+          const float r2a = (gtid < 255 && da >= 0 && da < p.T) ? rho_h[da] * LOG2E_B : -INFINITY;
           r2raw[gtid] = r2a;
-          r2raw[128 + gtid] = r2b;
-          float mr = fmaxf(r2a, r2b);
+          float mr = r2a;
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, o));
-          if (lane == 0) red[q4] = mr;
-          const int qi = I * BLK + gtid;
+          if (lane == 0) red[4 * sub + q4] = mr;
+          const int qi = I * BLK + (gtid & 127);
           const float z2 = (qi < p.T) ? logz_h[qi] * LOG2E_B : INFINITY;
-          z2s[gtid] = z2;
-          named_bar_sync(bar_id, 128);
-          mr = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+          if (sub == 0) z2s[gtid] = z2;
+          named_bar_sync(bar_id, 256);
+          mr = fmaxf(fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3])),
+                     fmaxf(fmaxf(red[4], red[5]), fmaxf(red[6], red[7])));
           rband[gtid] = ex2_approx(r2a - mr);
-          rband[128 + gtid] = ex2_approx(r2b - mr);
           const float ew = ma + mr - z2;
-          wq[gtid] = ex2_approx(ew);
+          if (sub == 0) wq[gtid] = ex2_approx(ew);
           const unsigned anybad = __any_sync(0xffffffffu, ew > 100.0f);
-          if (lane == 0) red[4 + q4] = anybad ? 1.0f : 0.0f;
-          named_bar_sync(bar_id, 128);
-          const bool exact = (red[4] + red[5] + red[6] + red[7]) > 0.0f;
+          if (lane == 0 && sub == 0) red[8 + q4] = anybad ? 1.0f : 0.0f;
+          named_bar_sync(bar_id, 256);
+          const bool exact = (red[8] + red[9] + red[10] + red[11]) > 0.0f;
           // this group's buffer must have been consumed by the dV MMA of its previous tile
           if (nmine > 0) {
             if (!mbar_wait_warp(pfree + grp, npf & 1, wc, B_PFREE)) ok = false;
@@ -644,7 +653,8 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           }
           const uint32_t t_p = tmem + lane_base + C::COL_S + grp * 64;
 #pragma unroll
-          for (int cc = 0; cc < 4; ++cc) {
+          for (int ch = 0; ch < 2; ++ch) {
+            const int cc = 2 * sub + ch;                  // this warp's 32-query chunks of the tile
             const int q0 = 32 * cc;
             uint32_t pk[16];
             if (!exact) {
@@ -688,8 +698,8 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         const float mul = grp == 0 ? dv_mul : p.scale;
         void* base = grp == 0 ? p.dV : p.dK;
         const size_t off = (bh * p.T + key) * 64;
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
+        {
+          const int cc = sub;                             // this warp's 32 feature columns
           uint32_t r[32];
           tmem_ld32(tmem + lane_base + col + 32 * cc, r);
           tmem_wait_ld();
@@ -726,7 +736,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 14) tmem_dealloc(tmem, C::TMEM_COLS);
+  if (warp == 22) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
 int bwd_smem_bytes(int) { return BwdCfg::SMEM; }
