@@ -142,6 +142,12 @@ __device__ __forceinline__ void tma_reduce_add_4d(const CUtensorMap* map, const 
                "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(src))
                : "memory");
 }
+// 4-D tiled store shared -> global (same coordinate rules as the reduce-add).
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, const void* src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::"l"(map),
+               "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(src))
+               : "memory");
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Wait until the bulk groups of this thread have finished READING their shared-memory sources.
 __device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }

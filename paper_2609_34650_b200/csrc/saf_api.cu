@@ -597,16 +597,22 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     mq = mdo; mk = mdo; mv = mdo;
   }
   // fp32 dQ accumulator [B][H][T][64] as a 4-D tensor for tiled reduce-adds: box = 32 floats x 128 rows
-  CUtensorMap mdq;
+  // (dK and dV get maps of the same shape for the tiled stores of the fp32 epilogue)
+  CUtensorMap mdq, mdk, mdv;
   {
     cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(p->T), static_cast<cuuint64_t>(p->H), static_cast<cuuint64_t>(p->B)};
     cuuint64_t gs[3] = {64 * 4, static_cast<cuuint64_t>(p->T) * 64 * 4, static_cast<cuuint64_t>(p->T) * 64 * 4 * p->H};
     cuuint32_t box[4] = {32, BLK, 1, 1};
     cuuint32_t es[4] = {1, 1, 1, 1};
-    if (ctx->encode(&mdq, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, dqacc, dims, gs, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return SAF_ERR_CUDA;
+    auto enc = [&](CUtensorMap* m, void* base) {
+      return ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, dims, gs, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
+    if (!enc(&mdq, dqacc)) return SAF_ERR_CUDA;
+    mdk = mdq;
+    mdv = mdq;
+    if (grad_f32 && (!enc(&mdk, dK) || !enc(&mdv, dV))) return SAF_ERR_CUDA;
   }
   BwdParams bp;
   CUtensorMap mdot = mdo;
@@ -650,7 +656,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   bp.wait_limit_ns = ctx->wait_limit_ns;
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD, st);
-    if (launch_bwd(p->D, mq, mk, mv, mdo, mdq, mdot, bp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+    if (launch_bwd(p->D, mq, mk, mv, mdo, mdq, mdot, mdk, mdv, bp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
   }
   if (!grad_f32) {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_FINALIZE, st);

@@ -42,10 +42,10 @@
 #include "saf_internal.h"
 
 #ifdef SAF_TRACE
-__device__ unsigned long long g_saf_trace[4][16384];
+__device__ unsigned long long g_saf_trace[24][4096];
 #define TR(role, id)                                                                                   \
   do {                                                                                                 \
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && tr_n < 16380)                                    \
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && tr_n < 4090)                                    \
       g_saf_trace[role][tr_n++] = (static_cast<unsigned long long>(id) << 48) | (clock64() & 0xffffffffffffULL); \
   } while (0)
 extern "C" int saf_debug_read_trace(unsigned long long* out) {
@@ -64,24 +64,24 @@ constexpr float LOG2E_B = 1.4426950408889634f;
 struct BwdCfg {
   static constexpr int PANEL = 128 * 64 * 2;         // one [128][64] bf16 tile, 128-byte rows, 16 KB
   static constexpr int NS = 2;                       // Q/dO ring depth
-  static constexpr int OFF_K = 0;
-  static constexpr int OFF_V = PANEL;
-  static constexpr int OFF_Q = 2 * PANEL;            // NS stages
+  static constexpr int OFF_K = 0;                    // 2 slots: the next item's K_J is prefetched
+  static constexpr int OFF_V = 2 * PANEL;            // 1 slot: V_J is only staged here on its way to TMEM
+  static constexpr int OFF_Q = 3 * PANEL;            // NS stages
   static constexpr int OFF_DO = OFF_Q + NS * PANEL;  // NS stages
   static constexpr int OFF_DS = OFF_DO + NS * PANEL; // 2 buffers x 2 panels (queries 0-63, 64-127)
-  static constexpr int OFF_DQ = OFF_DS + 4 * PANEL;  // fp32 staging: 2 boxes [128 rows][32 floats], 128B swizzle
-  static constexpr int OFF_QX = OFF_DQ + 2 * PANEL;  // NS x 4 KB row-term images of Q
+  static constexpr int OFF_DQ = OFF_DS + 4 * PANEL;  // fp32 staging: one box [128 rows][32 floats], 128B swizzle
+  static constexpr int OFF_QX = OFF_DQ + PANEL;      // NS x 4 KB row-term images of Q
   static constexpr int OFF_DOX = OFF_QX + NS * 4096; // NS x 4 KB row-term images of dO
   static constexpr int OFF_ONES = OFF_DOX + NS * 4096;   // 4 KB constant tile: columns 0..2 one, rest zero
   static constexpr int OFF_TAB = OFF_ONES + 4096;
   // per compute group: wq[128] z2s[128] rband[256] r2raw[256] red[16]
   static constexpr int TAB_FLOATS = 128 * 2 + 256 * 2 + 16;
   static constexpr int OFF_BAR = OFF_TAB + 2 * TAB_FLOATS * 4;
-  static constexpr int NBAR = 2 + 2 * NS + 2 + 2 + 4 + 2 + 3 + 1;
+  static constexpr int NBAR = 4 + 2 * NS + 2 + 2 + 4 + 2 + 1;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
   static constexpr int TMEM_COLS = 512;
   static constexpr int COL_DV = 0, COL_DK = 64, COL_S = 128, COL_DP = 256, COL_DQ = 384, COL_KT = 448, COL_VT = 480;
-  static constexpr int NTHREADS = 736;
+  static constexpr int NTHREADS = 704;
 };
 
 enum BwdSite { B_KV_EMPTY = 21, B_QDO_EMPTY, B_KV_FULL, B_QDO_FULL, B_PDS_FULL, B_ACC_FREE, B_DQ_FREE, B_SDP_FULL,
@@ -91,20 +91,39 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// Work item `it` and whether it takes the tensor-core frozen form, fetched one item ahead of its use so
+// that the two dependent global loads stay off the item-to-item critical path.
+struct ItemView {
+  WorkItem w;
+  bool fast;
+};
+__device__ __forceinline__ ItemView load_item(const BwdParams& p, int it, int it_end) {
+  ItemView v;
+  v.w = WorkItem{0, 0, 0, KIND_ORDINARY};
+  v.fast = false;
+  if (it < it_end) {
+    const int4 raw = __ldg(reinterpret_cast<const int4*>(p.items + it));
+    v.w = WorkItem{raw.x, raw.y, raw.z, raw.w};
+    v.fast = raw.w != KIND_ORDINARY && p.band_b != nullptr && __ldg(p.fast_ok + raw.y) != 0;
+  }
+  return v;
+}
+
 }  // namespace
 
 __global__ void __launch_bounds__(BwdCfg::NTHREADS, 1)
 saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mdo,
                const __grid_constant__ CUtensorMap mdq, const __grid_constant__ CUtensorMap mdot,
+               const __grid_constant__ CUtensorMap mdk, const __grid_constant__ CUtensorMap mdv,
                const BwdParams p) {
   using C = BwdCfg;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR);
-  uint64_t* kv_full = bars;
-  uint64_t* kv_empty = bars + 1;
-  uint64_t* qdo_full = bars + 2;                 // [NS]
+  uint64_t* kv_full = bars;                      // [2] K_J / V_J of an item have landed (index = K slot)
+  uint64_t* kv_empty = bars + 2;                 // [2] the item's MMAs have finished with K slot s
+  uint64_t* qdo_full = bars + 4;                 // [NS]
   uint64_t* qdo_empty = qdo_full + C::NS;        // [NS]
   uint64_t* sdp_full = qdo_empty + C::NS;        // [2]
   uint64_t* pds_full = sdp_full + 2;             // [2]
@@ -113,9 +132,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   uint64_t* acc_full = dq_free + 1;
   uint64_t* acc_free = acc_full + 1;
   uint64_t* pfree = acc_free + 1;                // [2]
-  uint64_t* bdone = pfree + 2;                   // [2] gradient MMAs that read buffer b have completed
-  uint64_t* fdone = bdone + 2;                   // a frozen item's MMAs have completed
-  uint64_t* kvt_full = fdone + 1;                // K_J / V_J have been copied into TMEM
+  uint64_t* kvt_full = pfree + 2;                // K_J / V_J have been copied into TMEM
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(kvt_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -125,19 +142,19 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
 
   if (tid == 0) {
     *abort_flag = 0;
-    mbar_init(kv_full, 1);
-    mbar_init(kv_empty, 2);                      // both issuers are done with K_J / V_J
+    for (int k = 0; k < 2; ++k) {
+      mbar_init(kv_full + k, 1);
+      mbar_init(kv_empty + k, 1);
+    }
     for (int s = 0; s < C::NS; ++s) {
       mbar_init(qdo_full + s, 1);
-      mbar_init(qdo_empty + s, 2);               // both issuers are done with the stage
+      mbar_init(qdo_empty + s, 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(sdp_full + b, 1);
       mbar_init(pds_full + b, 8);                // one arrival per warp of the group
       mbar_init(pfree + b, 1);
-      mbar_init(bdone + b, 1);
     }
-    mbar_init(fdone, 1);
     mbar_init(kvt_full, 16);
     mbar_init(dq_full, 1);
     mbar_init(dq_free, 4);
@@ -155,7 +172,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     }
     reinterpret_cast<uint4*>(smem + C::OFF_ONES)[i] = v;
   }
-  if (warp == 22) {
+  if (warp == 21) {
     tmem_alloc(tmem_slot, C::TMEM_COLS);
     tmem_relinquish();
   }
@@ -176,18 +193,31 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       tma_prefetch_desc(&mdot);
       uint32_t nkv = 0, nqdo = 0;
       bool ok = true;
+      int tr_n = 0;
+      (void)tr_n;
+      // K_J / V_J of the ordinary items run one item ahead of the tile loads: K into the other K slot (free
+      // once the item before the current one has finished), V into the single V slot (free once the
+      // current item's V has been copied to TMEM).
+      int next_kv = it_begin;
+      auto load_next_kv = [&]() {
+        while (next_kv < it_end && p.items[next_kv].kind != KIND_ORDINARY) ++next_kv;
+        if (next_kv >= it_end) return;
+        const WorkItem w2 = p.items[next_kv++];
+        const uint32_t ks = nkv & 1;
+        ok = mbar_wait(kv_empty + ks, ((nkv >> 1) & 1) ^ 1, wc, B_KV_EMPTY);
+        if (ok && nkv > 0) ok = mbar_wait(kvt_full, (nkv - 1) & 1, wc, B_KV_EMPTY);
+        if (!ok) return;
+        TR(2, 31);
+        mbar_expect_tx(kv_full + ks, 2 * C::PANEL);
+        tma_load_4d(smem + C::OFF_K + ks * C::PANEL, &mk, kv_full + ks, 0, w2.blk * BLK, w2.h, w2.b);
+        tma_load_4d(smem + C::OFF_V, &mv, kv_full + ks, 0, w2.blk * BLK, w2.h, w2.b);
+        ++nkv;
+      };
+      load_next_kv();
       for (int it = it_begin; it < it_end && ok; ++it) {
         const WorkItem w = p.items[it];
         const bool ord = w.kind == KIND_ORDINARY;
         const size_t bh = static_cast<size_t>(w.b) * p.H + w.h;
-        if (ord) {
-          ok = mbar_wait(kv_empty, (nkv & 1) ^ 1, wc, B_KV_EMPTY);
-          if (!ok) break;
-          mbar_expect_tx(kv_full, 2 * C::PANEL);
-          tma_load_4d(smem + C::OFF_K, &mk, kv_full, 0, w.blk * BLK, w.h, w.b);
-          tma_load_4d(smem + C::OFF_V, &mv, kv_full, 0, w.blk * BLK, w.h, w.b);
-          ++nkv;
-        }
         const bool fast = !ord && p.band_b != nullptr && p.fast_ok[w.h] != 0;
         if (fast) {
           // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled dO tile
@@ -208,6 +238,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           const int s = nqdo % C::NS;
           ok = mbar_wait(qdo_empty + s, ((nqdo / C::NS) & 1) ^ 1, wc, B_QDO_EMPTY);
           if (!ok) break;
+          TR(2, I == w.blk ? 33 : 32);
           mbar_expect_tx(qdo_full + s, ord ? 2 * C::PANEL + 8192 : C::PANEL);
           if (ord) {
             tma_load_4d(smem + C::OFF_Q + s * C::PANEL, &mq, qdo_full + s, 0, I * BLK, w.h, w.b);
@@ -217,111 +248,83 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           }
           tma_load_4d(smem + C::OFF_DO + s * C::PANEL, &mdo, qdo_full + s, 0, I * BLK, w.h, w.b);
           ++nqdo;
+          // with this item's first tiles under way, fetch K_J / V_J of the next ordinary item
+          if (ord && I == min(w.blk + 1, nblk - 1)) {
+            load_next_kv();
+            if (!ok) break;
+          }
         }
       }
     }
   } else if (warp == 21) {
-    // ------------------------------------------------------------------ tcgen05 issuer X: score MMAs A(u)
-    // The whole warp walks the loops (warp-uniform operands); one elected lane issues.
+    // ------------------------------------------------------------------ tcgen05 issuer
+    // The whole warp walks the loops (warp-uniform operands); one elected lane issues.  MMAs issued by one
+    // thread execute in issue order, which is what lets A(u+2) follow B(u) on the same TMEM buffer with
+    // no completion round trip in between.
     const bool leader = elect_one() != 0;
     const uint32_t sb = smem_u32(smem);
     constexpr uint32_t id_s = umma_idesc_bf16(128, 64, 0, 0);      // S^T, dP^T half tiles: both operands K-major
-    // descriptor halves for smem offset 0: 128B-swizzled K-major (k-step +32 B) and the no-swizzle
-    // K-major row-term tiles (LBO 128 B, SBO 256 B)
-    const uint64_t d_k = umma_smem_desc(sb, 16, 1024, UMMA_LAYOUT_SW128);
-    const uint64_t d_x = umma_smem_desc(sb, 128, 256, UMMA_LAYOUT_NONE);
-    const uint32_t lo_k = desc_lo(d_k), hi_k = desc_hi(d_k), lo_x = desc_lo(d_x), hi_x = desc_hi(d_x);
-    const uint32_t ones_lo = lo_x + (C::OFF_ONES >> 4);
-    uint32_t nkv = 0, nqdo = 0, nfd = 0;
-    uint32_t nbd0 = 0, nbd1 = 0;
-    int tr_n = 0;
-    (void)tr_n;
-    bool ok = true;
-    for (int it = it_begin; it < it_end && ok; ++it) {
-      const WorkItem w = p.items[it];
-      const int ntiles = nblk - w.blk;
-      if (w.kind != KIND_ORDINARY) {
-        // not this issuer's item: hand its stages on, then wait until its MMAs have left the S^T buffers
-        for (int t = 0; t < ntiles && ok; ++t, ++nqdo) {
-          const uint32_t s = nqdo % C::NS;
-          ok = mbar_wait_warp(qdo_full + s, (nqdo / C::NS) & 1, wc, B_QDO_FULL);
-          if (ok && leader) mbar_arrive(qdo_empty + s);
-          __syncwarp();
-        }
-        if (!ok) break;
-        ok = mbar_wait_warp(fdone, nfd & 1, wc, B_ACC_FULL);
-        ++nfd;
-        continue;
-      }
-      // K_J / V_J are read from TMEM: wait for the compute warps' copy; the smem tiles are then free
-      // as far as this issuer is concerned
-      ok = mbar_wait_warp(kvt_full, nkv & 1, wc, B_KV_FULL);
-      if (!ok) break;
-      ++nkv;
-      tc_fence_after();
-      if (leader) mbar_arrive(kv_empty);
-      __syncwarp();
-      const int U = 2 * ntiles;
-      for (int u = 0; u < U && ok; ++u) {
-        const uint32_t pos = nqdo + (u >> 1);
-        const uint32_t s = pos % C::NS;
-        const uint32_t b = u & 1;
-        TR(3, 1);
-        // buffer b is free once the gradient MMAs of half tile u-2 have read their bf16 operands from it
-        if (b == 0) {
-          ok = mbar_wait_warp(bdone, (nbd0 & 1) ^ 1, wc, B_PFREE);
-          ++nbd0;
-          if (ok) ok = mbar_wait_warp(qdo_full + s, (pos / C::NS) & 1, wc, B_QDO_FULL);
-        } else {
-          ok = mbar_wait_warp(bdone + 1, (nbd1 & 1) ^ 1, wc, B_PFREE);
-          ++nbd1;
-        }
-        if (!ok) break;
-        TR(3, 2);
-        tc_fence_after();
-        const uint32_t q_lo = lo_k + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
-        const uint32_t do_lo = lo_k + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
-        const uint32_t qx_lo = lo_x + ((C::OFF_QX + s * 4096 + b * 2048) >> 4);
-        const uint32_t dox_lo = lo_x + ((C::OFF_DOX + s * 4096 + b * 2048) >> 4);
-        const uint32_t t_s = tmem + C::COL_S + 64 * b, t_dp = tmem + C::COL_DP + 64 * b;
-        if (leader) {
-#pragma unroll
-          for (int kc = 0; kc < 4; ++kc)
-            umma_ts2(t_s, tmem + C::COL_KT + 8 * kc, q_lo + 2 * kc, hi_k, id_s, kc > 0);
-          umma_ss2(t_s, ones_lo, hi_x, qx_lo, hi_x, id_s, 1);
-#pragma unroll
-          for (int kc = 0; kc < 4; ++kc)
-            umma_ts2(t_dp, tmem + C::COL_VT + 8 * kc, do_lo + 2 * kc, hi_k, id_s, kc > 0);
-          umma_ss2(t_dp, ones_lo, hi_x, dox_lo, hi_x, id_s, 1);
-          umma_commit(sdp_full + b);
-          if (b == 1) umma_commit(qdo_empty + s);       // this issuer's reads of the stage
-        }
-        TR(3, 3);
-        __syncwarp();
-      }
-      nqdo += ntiles;
-    }
-  } else if (warp == 22) {
-    // ------------------------------------------------------------------ tcgen05 issuer Y: gradient MMAs
-    const bool leader = elect_one() != 0;
-    const uint32_t sb = smem_u32(smem);
     constexpr uint32_t id_acc = umma_idesc_bf16(128, 64, 0, 1);    // dV, dK: A from TMEM, B MN-major
     constexpr uint32_t id_dq = umma_idesc_bf16(128, 64, 1, 1);     // dQ: A (dS^T tile) M-major, B MN-major
-    // 128B-swizzled MN-major tiles: k-step +2048 B, LBO = panel
+    // descriptor halves for smem offset 0: 128B-swizzled K-major (k-step +32 B), the no-swizzle K-major
+    // row-term tiles (LBO 128 B, SBO 256 B) and 128B-swizzled MN-major tiles (k-step +2048 B, LBO = panel)
+    const uint64_t d_k = umma_smem_desc(sb, 16, 1024, UMMA_LAYOUT_SW128);
+    const uint64_t d_x = umma_smem_desc(sb, 128, 256, UMMA_LAYOUT_NONE);
     const uint64_t d_m = umma_smem_desc(sb, C::PANEL, 1024, UMMA_LAYOUT_SW128);
+    const uint32_t lo_k = desc_lo(d_k), hi_k = desc_hi(d_k), lo_x = desc_lo(d_x), hi_x = desc_hi(d_x);
     const uint32_t lo_m = desc_lo(d_m), hi_m = desc_hi(d_m);
-    const uint32_t km_lo = lo_m + (C::OFF_K >> 4);
-    uint32_t nqdo = 0, nitem = 0, ndq = 0, ntile_ord = 0;
+    const uint32_t ones_lo = lo_x + (C::OFF_ONES >> 4);
+    uint32_t nqdo = 0, nitem = 0, ndq = 0, ntile_ord = 0, nkv = 0;
     uint32_t npds0 = 0, npds1 = 0;
     int tr_n = 0;
     (void)tr_n;
     bool ok = true;
+    ItemView nxt = load_item(p, it_begin, it_end);
     for (int it = it_begin; it < it_end && ok; ++it, ++nitem) {
-      const WorkItem w = p.items[it];
+      const WorkItem w = nxt.w;
+      const bool fast = nxt.fast;
+      nxt = load_item(p, it + 1, it_end);
       const bool ord = w.kind == KIND_ORDINARY;
       const int ntiles = nblk - w.blk;
       if (ord) {
+        // K_J / V_J are read from TMEM (copied there by the compute warps); K_J's smem slot feeds dQ
+        const uint32_t km_lo = lo_m + ((C::OFF_K + (nkv & 1) * C::PANEL) >> 4);
+        uint64_t* const kv_done = kv_empty + (nkv & 1);
+        ok = mbar_wait_warp(kvt_full, nkv & 1, wc, B_KV_FULL);
+        if (!ok) break;
+        ++nkv;
+        TR(3, 7);
         const int U = 2 * ntiles;
+        // score MMAs of half tile u into buffer u & 1
+        auto issue_A = [&](int u) {
+          const uint32_t s = (nqdo + (u >> 1)) % C::NS;
+          const uint32_t b = u & 1;
+          const uint32_t q_lo = lo_k + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
+          const uint32_t do_lo = lo_k + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
+          const uint32_t qx_lo = lo_x + ((C::OFF_QX + s * 4096 + b * 2048) >> 4);
+          const uint32_t dox_lo = lo_x + ((C::OFF_DOX + s * 4096 + b * 2048) >> 4);
+          const uint32_t t_s = tmem + C::COL_S + 64 * b, t_dp = tmem + C::COL_DP + 64 * b;
+          if (leader) {
+#pragma unroll
+            for (int kc = 0; kc < 4; ++kc)
+              umma_ts2(t_s, tmem + C::COL_KT + 8 * kc, q_lo + 2 * kc, hi_k, id_s, kc > 0);
+            umma_ss2(t_s, ones_lo, hi_x, qx_lo, hi_x, id_s, 1);
+#pragma unroll
+            for (int kc = 0; kc < 4; ++kc)
+              umma_ts2(t_dp, tmem + C::COL_VT + 8 * kc, do_lo + 2 * kc, hi_k, id_s, kc > 0);
+            umma_ss2(t_dp, ones_lo, hi_x, dox_lo, hi_x, id_s, 1);
+            umma_commit(sdp_full + b);
+          }
+          __syncwarp();
+        };
+        ok = mbar_wait_warp(qdo_full + nqdo % C::NS, (nqdo / C::NS) & 1, wc, B_QDO_FULL);
+        if (!ok) break;
+        tc_fence_after();
+        TR(3, 1);
+        issue_A(0);
+        TR(3, 2);
+        issue_A(1);
+        TR(3, 3);
         for (int u = 0; u < U && ok; ++u) {
           const uint32_t b = u & 1;
           TR(0, 4);
@@ -348,13 +351,25 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           if (leader) {
 #pragma unroll
             for (int kc = 0; kc < 4; ++kc)
-              umma_ts2(tmem + C::COL_DV, t_p + 8 * kc + (kc >= 2 ? 16 : 0), do_lo + 128 * kc, hi_m, id_acc, kc > 0 ? 1u : acc0);
+              umma_ts2(tmem + C::COL_DV, t_p + 8 * kc + (kc >= 2 ? 16 : 0), do_lo + 128 * kc, hi_m, id_acc,
+                       kc > 0 ? 1u : acc0);
 #pragma unroll
             for (int kc = 0; kc < 4; ++kc)
-              umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc + (kc >= 2 ? 16 : 0), q_lo + 128 * kc, hi_m, id_acc, kc > 0 ? 1u : acc0);
-            umma_commit(bdone + b);
+              umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc + (kc >= 2 ? 16 : 0), q_lo + 128 * kc, hi_m, id_acc,
+                       kc > 0 ? 1u : acc0);
           }
+          __syncwarp();
           TR(0, 6);
+          // the buffer's next score MMAs follow its gradient MMAs directly (in-order execution)
+          if (u + 2 < U) {
+            if (b == 0) {
+              ok = mbar_wait_warp(qdo_full + (pos + 1) % C::NS, ((pos + 1) / C::NS) & 1, wc, B_QDO_FULL);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            issue_A(u + 2);
+            TR(3, 3);
+          }
           if (b == 1) {
             // full tile done: its Q/dO stage can be refilled, and dQ of the tile follows
             if (leader) umma_commit(qdo_empty + s);
@@ -371,13 +386,13 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             }
             TR(0, 9);
             ++ntile_ord;
+            __syncwarp();
           }
-          __syncwarp();
         }
         if (!ok) break;
         nqdo += ntiles;
-        if (leader) umma_commit(kv_empty);
-      } else if (p.band_b != nullptr && p.fast_ok[w.h] != 0) {
+        if (leader) umma_commit(kv_done);
+      } else if (fast) {
         // tensor-core form of a frozen head: A = Hankel band (no-swizzle, both strides 128 B), B = scaled dO
         constexpr uint32_t id_hk = umma_idesc_f16(128, 64, 0, 1);   // fp16 band x fp16 scaled dO
         const uint64_t d_band = umma_smem_desc(sb, 128, 128, UMMA_LAYOUT_NONE);
@@ -404,7 +419,6 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           __syncwarp();
         }
         if (!ok) break;
-        if (leader) umma_commit(fdone);
       } else {
         for (int t = 0; t < ntiles; ++t) {
           const uint32_t s = nqdo % C::NS;
@@ -438,7 +452,6 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           __syncwarp();
         }
         if (!ok) break;
-        if (leader) umma_commit(fdone);
       }
       if (leader) umma_commit(acc_full);
       __syncwarp();
@@ -471,7 +484,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         tmem_wait_ld();
         tc_fence_before();
         warp_arrive(dq_free);                           // the tensor core may overwrite dQ
-        // fp32 rows -> two [128][32] boxes, 128-byte swizzle (16-byte chunk index ^= row & 7)
+        // fp32 rows -> one [128][32] box at a time, 128-byte swizzle (16-byte chunk index ^= row & 7)
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
           const uint32_t chunk = static_cast<uint32_t>(g ^ (rowl & 7)) * 16;
@@ -479,7 +492,19 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
                        __float_as_uint(__uint_as_float(r0[4 * g + 1]) * p.scale),
                        __float_as_uint(__uint_as_float(r0[4 * g + 2]) * p.scale),
                        __float_as_uint(__uint_as_float(r0[4 * g + 3]) * p.scale));
-          st_shared_v4(stage_row + C::PANEL + chunk, __float_as_uint(__uint_as_float(r1[4 * g]) * p.scale),
+        }
+        fence_proxy_async_smem();
+        named_bar_sync(3, 128);
+        if (tid == 512 && ok) {
+          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 0, I * BLK, w.h, w.b);
+          bulk_commit_group();
+          bulk_wait_group_read0();
+        }
+        named_bar_sync(6, 128);                         // the first box has been read
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const uint32_t chunk = static_cast<uint32_t>(g ^ (rowl & 7)) * 16;
+          st_shared_v4(stage_row + chunk, __float_as_uint(__uint_as_float(r1[4 * g]) * p.scale),
                        __float_as_uint(__uint_as_float(r1[4 * g + 1]) * p.scale),
                        __float_as_uint(__uint_as_float(r1[4 * g + 2]) * p.scale),
                        __float_as_uint(__uint_as_float(r1[4 * g + 3]) * p.scale));
@@ -487,8 +512,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         fence_proxy_async_smem();
         named_bar_sync(3, 128);
         if (tid == 512 && ok) {
-          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 0, I * BLK, w.h, w.b);
-          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ + C::PANEL, 32, I * BLK, w.h, w.b);
+          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 32, I * BLK, w.h, w.b);
           bulk_commit_group();
           bulk_wait_group_read0();
         }
@@ -514,50 +538,69 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     bool ok = true;
     int tr_n = 0;
     (void)tr_n;
+    // K_J (group 0) / V_J (group 1) of the next ordinary item: this thread's half row from the swizzled
+    // smem tile into TMEM as the A operand of the score MMAs (bf16 pairs, feature index = reduction index)
+    // The fp32 epilogue leaves through TMA stores that read this group's dS^T panels; before the group
+    // writes those panels again (dS^T of a first tile, or the next epilogue) the stores must have read them.
+    bool store_pending = false;                          // uniform over the group
+    auto staging_free = [&]() {
+      if (!store_pending) return;
+      if (gtid == 0) bulk_wait_group_read0();
+      named_bar_sync(bar_id, 256);
+      store_pending = false;
+    };
+    bool kv_in_tmem = false;
+    auto copy_kv = [&]() {
+      const uint32_t ks = nkvc & 1;
+      if (!mbar_wait_warp(kv_full + ks, (nkvc >> 1) & 1, wc, B_KV_FULL)) ok = false;
+      ++nkvc;
+      const uint32_t src = smem_u32(smem + (grp == 0 ? C::OFF_K + ks * C::PANEL : C::OFF_V)) + rowl * 128;
+      uint32_t kvr[16];
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const uint32_t a = src + static_cast<uint32_t>((4 * sub + g) ^ (rowl & 7)) * 16;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(kvr[4 * g]), "=r"(kvr[4 * g + 1]), "=r"(kvr[4 * g + 2]), "=r"(kvr[4 * g + 3])
+                     : "r"(a)
+                     : "memory");
+      }
+      tmem_st16(tmem + lane_base + (grp == 0 ? C::COL_KT : C::COL_VT) + 16 * sub, kvr);
+      tmem_wait_st();
+      tc_fence_before();
+      warp_arrive(kvt_full);
+    };
     // A warp whose wait was abandoned keeps walking (without storing) to the next agreement barrier,
     // where the warps of its group leave together; none is ever left alone at a named barrier.
+    ItemView nxt = load_item(p, it_begin, it_end);
     for (int it = it_begin; it < it_end; ++it) {
-      const WorkItem w = p.items[it];
+      const WorkItem w = nxt.w;
+      const bool fast = nxt.fast;
+      nxt = load_item(p, it + 1, it_end);
       const bool ord = w.kind == KIND_ORDINARY;
       const int ntiles = nblk - w.blk;
       int key = w.blk * BLK + rowl;
       const size_t bh = static_cast<size_t>(w.b) * p.H + w.h;
       float dv_mul = 1.0f;
+      bool rev = false;                                  // tensor-core frozen form: lane m holds key 127-m
+      bool stored = false;                               // this group staged an fp32 block for a TMA store
       if (named_bar_or(bar_id, 256, !ok)) break;
 
-      if (!ord && p.band_b != nullptr && p.fast_ok[w.h] != 0) {
+      if (fast) {
         // tensor-core form: nothing to do per tile; lane m holds key 127-m, scaled by a(j) below
         key = w.blk * BLK + 127 - rowl;
+        rev = true;
         dv_mul = (key < p.T) ? p.avec[static_cast<size_t>(w.h) * p.Tp + key] * (1.0f / HK_BAND_SCALE) : 0.0f;
       } else if (ord) {
         const float c = p.scale_log2;
-        {
-          // K_J (group 0) / V_J (group 1): this thread's row from the swizzled smem tile into TMEM as the
-          // A operand of the score MMAs (bf16 pairs, feature index = reduction index)
-          if (!mbar_wait_warp(kv_full, nkvc & 1, wc, B_KV_FULL)) ok = false;
-          ++nkvc;
-          const uint32_t src = smem_u32(smem + (grp == 0 ? C::OFF_K : C::OFF_V)) + rowl * 128;
-          uint32_t kvr[16];
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const uint32_t a = src + static_cast<uint32_t>((4 * sub + g) ^ (rowl & 7)) * 16;
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(kvr[4 * g]), "=r"(kvr[4 * g + 1]), "=r"(kvr[4 * g + 2]), "=r"(kvr[4 * g + 3])
-                         : "r"(a)
-                         : "memory");
-          }
-          tmem_st16(tmem + lane_base + (grp == 0 ? C::COL_KT : C::COL_VT) + 16 * sub, kvr);
-          tmem_wait_st();
-          tc_fence_before();
-          warp_arrive(kvt_full);
-        }
+        if (!kv_in_tmem) copy_kv();                  // first ordinary item of this CTA
         for (int t = 0; t < ntiles; ++t) {
           // this group's half tile of tile t: queries 64*grp .. 64*grp+63; this warp's 32 of them
-          if ((warp & 7) == 0) TR(1 + grp, 11);
+          TR(4 + warp, 11);
           if (!mbar_wait_warp(sdp_full + grp, nsdp & 1, wc, B_SDP_FULL)) ok = false;
           ++nsdp;
           tc_fence_after();
-          if ((warp & 7) == 0) TR(1 + grp, 12);
+          if (t == 0) staging_free();
+          TR(4 + warp, 12);
           const uint32_t t_s = tmem + lane_base + C::COL_S + 64 * grp;
           const uint32_t t_dp = tmem + lane_base + C::COL_DP + 64 * grp;
           const uint32_t rowaddr =
@@ -597,9 +640,25 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           fence_proxy_async_smem();
           tc_fence_before();
           warp_arrive(pds_full + grp);
-          if ((warp & 7) == 0) TR(1 + grp, 16);
+          TR(4 + warp, 16);
         }
         ntile_ord += ntiles;
+        // K_J / V_J of the next ordinary item go to TMEM now, ahead of this item's epilogue, so that its
+        // score MMAs can start while the epilogue runs.  The last score MMAs of this item (both buffers)
+        // must have read the old copies first.
+        kv_in_tmem = false;
+        for (int nx = it + 1; nx < it_end; ++nx)
+          if (p.items[nx].kind == KIND_ORDINARY) {
+            kv_in_tmem = true;
+            break;
+          }
+        if (kv_in_tmem) {
+          TR(4 + warp, 21);
+          if (!mbar_wait_warp(sdp_full + (grp ^ 1), (nsdp - 1) & 1, wc, B_SDP_FULL)) ok = false;
+          tc_fence_after();
+          copy_kv();
+          TR(4 + warp, 22);
+        }
       } else {
         // ---------------- frozen head: P^^T tiles; group g generates tiles t = g, g+2, ...
         const float* alpha_h = p.alpha + static_cast<size_t>(w.h) * p.Tp;
@@ -693,6 +752,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       if (!mbar_wait_warp(acc_full, nacc & 1, wc, B_ACC_FULL)) ok = false;
       ++nacc;
       tc_fence_after();
+      TR(4 + warp, 23);
       if (grp == 0 || ord) {
         const uint32_t col = grp == 0 ? C::COL_DV : C::COL_DK;
         const float mul = grp == 0 ? dv_mul : p.scale;
@@ -703,28 +763,56 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           uint32_t r[32];
           tmem_ld32(tmem + lane_base + col + 32 * cc, r);
           tmem_wait_ld();
-          if (key < p.T && ok) {
-            if (p.grad_f32) {
-              float4* dst = reinterpret_cast<float4*>(static_cast<float*>(base) + off + 32 * cc);
+          tc_fence_before();
+          warp_arrive(acc_free);                          // the accumulators may be overwritten
+          TR(4 + warp, 25);
+          if (p.grad_f32) {
+            staging_free();
+            // fp32 rows go through the (idle) dS^T buffers as two 128-byte-swizzled [128][32] boxes and
+            // leave with tiled TMA stores (rows beyond T are clipped).  A group stages inside the panels
+            // it writes dS^T to itself, since the other group may already be in the next item.
+            const int srow_i = rev ? 127 - rowl : rowl;
+            const uint32_t srow =
+                smem_u32(smem + C::OFF_DS + (2 * sub + grp) * C::PANEL) + static_cast<uint32_t>(srow_i) * 128;
 #pragma unroll
-              for (int e = 0; e < 8; ++e)
-                dst[e] = make_float4(__uint_as_float(r[4 * e]) * mul, __uint_as_float(r[4 * e + 1]) * mul,
-                                     __uint_as_float(r[4 * e + 2]) * mul, __uint_as_float(r[4 * e + 3]) * mul);
-            } else {
-              uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(base) + off + 32 * cc);
+            for (int g = 0; g < 8; ++g)
+              st_shared_v4(srow + static_cast<uint32_t>(g ^ (srow_i & 7)) * 16,
+                           __float_as_uint(__uint_as_float(r[4 * g]) * mul),
+                           __float_as_uint(__uint_as_float(r[4 * g + 1]) * mul),
+                           __float_as_uint(__uint_as_float(r[4 * g + 2]) * mul),
+                           __float_as_uint(__uint_as_float(r[4 * g + 3]) * mul));
+            TR(4 + warp, 26);
+            fence_proxy_async_smem();
+            TR(4 + warp, 27);
+            stored = true;
+          } else if (key < p.T && ok) {
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(base) + off + 32 * cc);
 #pragma unroll
               for (int e = 0; e < 4; ++e)
                 dst[e] = make_uint4(pack_bf16x2(__uint_as_float(r[8 * e]) * mul, __uint_as_float(r[8 * e + 1]) * mul),
                                     pack_bf16x2(__uint_as_float(r[8 * e + 2]) * mul, __uint_as_float(r[8 * e + 3]) * mul),
                                     pack_bf16x2(__uint_as_float(r[8 * e + 4]) * mul, __uint_as_float(r[8 * e + 5]) * mul),
                                     pack_bf16x2(__uint_as_float(r[8 * e + 6]) * mul, __uint_as_float(r[8 * e + 7]) * mul));
-            }
           }
         }
+      } else {
+        tc_fence_before();
+        warp_arrive(acc_free);
       }
-      tc_fence_before();
-      warp_arrive(acc_free);
+      if (stored) {                                      // uniform over the group
+        named_bar_sync(bar_id, 256);
+        TR(4 + warp, 28);
+        if (gtid == 0 && ok) {
+          const CUtensorMap* m = grp == 0 ? &mdv : &mdk;
+          tma_store_4d(m, smem + C::OFF_DS + grp * C::PANEL, 0, w.blk * BLK, w.h, w.b);
+          tma_store_4d(m, smem + C::OFF_DS + (2 + grp) * C::PANEL, 32, w.blk * BLK, w.h, w.b);
+          bulk_commit_group();
+        }
+        store_pending = true;
+      }
+      TR(4 + warp, 24);
     }
+    if (gtid == 0) bulk_wait_group0();                   // the stores have landed before the kernel ends
   }
 
   // ------------------------------------------------------------------ teardown
@@ -736,18 +824,18 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 22) tmem_dealloc(tmem, C::TMEM_COLS);
+  if (warp == 21) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
 int bwd_smem_bytes(int) { return BwdCfg::SMEM; }
 
 cudaError_t launch_bwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const CUtensorMap& mdo, const CUtensorMap& mdq, const CUtensorMap& mdot, const BwdParams& p,
-                       int grid, cudaStream_t st) {
+                       const CUtensorMap& mdo, const CUtensorMap& mdq, const CUtensorMap& mdot, const CUtensorMap& mdk,
+                       const CUtensorMap& mdv, const BwdParams& p, int grid, cudaStream_t st) {
   if (D != 64) return cudaErrorNotSupported;
   cudaError_t e = cudaFuncSetAttribute(saf_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg::SMEM);
   if (e != cudaSuccess) return e;
-  saf_bwd_kernel<<<grid, BwdCfg::NTHREADS, BwdCfg::SMEM, st>>>(mq, mk, mv, mdo, mdq, mdot, p);
+  saf_bwd_kernel<<<grid, BwdCfg::NTHREADS, BwdCfg::SMEM, st>>>(mq, mk, mv, mdo, mdq, mdot, mdk, mdv, p);
   return cudaGetLastError();
 }
 

@@ -77,10 +77,11 @@ constexpr float HK_A_SCALE = 2048.0f;            // the forward stages 2^11 a V
 // mvt: map of the a-scaled V of the frozen heads [B][Hf][T][D] (any valid map when band_f is NULL)
 cudaError_t launch_fwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                        const CUtensorMap& mvt, const FwdParams& p, int grid, cudaStream_t st);
-// mdot: map of the w-scaled dO of the frozen heads [B][Hf][T][D] (any valid map when band_b is NULL)
+// mdot: map of the w-scaled dO of the frozen heads [B][Hf][T][D] (any valid map when band_b is NULL);
+// mdk / mdv: fp32 maps of dK / dV shaped like mdq (only used when grad_f32 is set)
 cudaError_t launch_bwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const CUtensorMap& mdo, const CUtensorMap& mdq, const CUtensorMap& mdot, const BwdParams& p,
-                       int grid, cudaStream_t st);
+                       const CUtensorMap& mdo, const CUtensorMap& mdq, const CUtensorMap& mdot, const CUtensorMap& mdk,
+                       const CUtensorMap& mdv, const BwdParams& p, int grid, cudaStream_t st);
 // Row terms of ordinary heads (q_ext / do_ext images, see BwdParams); also zeroes dQacc (all heads) and
 // dK of frozen heads.
 cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* o_strides,
