@@ -26,19 +26,7 @@
 #include "ptx.cuh"
 #include "saf_internal.h"
 
-#ifdef SAF_TRACE
-__device__ unsigned long long g_saf_trace_fwd[4][16384];
-#define TRF(role, id)                                                                                  \
-  do {                                                                                                 \
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && tr_n < 16380)                                    \
-      g_saf_trace_fwd[role][tr_n++] = (static_cast<unsigned long long>(id) << 48) | (clock64() & 0xffffffffffffULL); \
-  } while (0)
-extern "C" int saf_debug_read_trace_fwd(unsigned long long* out) {
-  return static_cast<int>(cudaMemcpyFromSymbol(out, g_saf_trace_fwd, sizeof(g_saf_trace_fwd)));
-}
-#else
 #define TRF(role, id)
-#endif
 
 namespace saf {
 
@@ -592,15 +580,13 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   if (warp == 9) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
-int fwd_smem_bytes(int D) { return D == 64 ? FwdCfg<64>::SMEM : FwdCfg<128>::SMEM; }
+int fwd_smem_bytes(int D) { return D == 64 ? fwd64_smem_bytes() : FwdCfg<128>::SMEM; }
 
 cudaError_t launch_fwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                        const CUtensorMap& mvt, const FwdParams& p, int grid, cudaStream_t st) {
   cudaError_t e;
   if (D == 64) {
-    e = cudaFuncSetAttribute(saf_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<64>::SMEM);
-    if (e != cudaSuccess) return e;
-    saf_fwd_kernel<64><<<grid, 320, FwdCfg<64>::SMEM, st>>>(mq, mk, mv, mvt, p);
+    return launch_fwd64(mq, mk, mv, mvt, p, grid, st);   // head dimension 64 has its own kernel
   } else {
     e = cudaFuncSetAttribute(saf_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128>::SMEM);
     if (e != cudaSuccess) return e;

@@ -89,6 +89,10 @@ cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, con
                             void* dK, int grad_f32, int B, int H, int T, int D, cudaStream_t st);
 // dQ (grad dtype) = scale-free copy/convert of dQacc (fp32) for the bf16-gradient case.
 cudaError_t launch_bwd_finalize(const float* dQacc, void* dQ, size_t n, cudaStream_t st);
+// head dimension 64 (saf_fwd64.cu); launch_fwd dispatches to it
+cudaError_t launch_fwd64(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mvt,
+                         const FwdParams& p, int grid, cudaStream_t st);
+int fwd64_smem_bytes();
 int fwd_smem_bytes(int D);
 int bwd_smem_bytes(int D);
 
