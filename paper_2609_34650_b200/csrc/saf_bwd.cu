@@ -542,12 +542,17 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     // smem tile into TMEM as the A operand of the score MMAs (bf16 pairs, feature index = reduction index)
     // The fp32 epilogue leaves through TMA stores that read this group's dS^T panels; before the group
     // writes those panels again (dS^T of a first tile, or the next epilogue) the stores must have read them.
-    bool store_pending = false;                          // uniform over the group
-    auto staging_free = [&]() {
-      if (!store_pending) return;
-      if (gtid == 0) bulk_wait_group_read0();
+    // The two panels leave as separate bulk groups, the one that the next item's first tile writes first,
+    // so that that tile only waits for half of the store.
+    int store_pending = 0;                               // bulk groups possibly unread; uniform over the group
+    auto staging_free = [&](int allow) {
+      if (store_pending <= allow) return;
+      if (gtid == 0) {
+        if (allow == 0) bulk_wait_group_read0();
+        else asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      }
       named_bar_sync(bar_id, 256);
-      store_pending = false;
+      store_pending = allow;
     };
     bool kv_in_tmem = false;
     auto copy_kv = [&]() {
@@ -599,7 +604,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           if (!mbar_wait_warp(sdp_full + grp, nsdp & 1, wc, B_SDP_FULL)) ok = false;
           ++nsdp;
           tc_fence_after();
-          if (t == 0) staging_free();
+          if (t <= 1) staging_free(1 - t);
           TR(4 + warp, 12);
           const uint32_t t_s = tmem + lane_base + C::COL_S + 64 * grp;
           const uint32_t t_dp = tmem + lane_base + C::COL_DP + 64 * grp;
@@ -767,7 +772,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           warp_arrive(acc_free);                          // the accumulators may be overwritten
           TR(4 + warp, 25);
           if (p.grad_f32) {
-            staging_free();
+            staging_free(0);
             // fp32 rows go through the (idle) dS^T buffers as two 128-byte-swizzled [128][32] boxes and
             // leave with tiled TMA stores (rows beyond T are clipped).  A group stages inside the panels
             // it writes dS^T to itself, since the other group may already be in the next item.
@@ -804,11 +809,14 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         TR(4 + warp, 28);
         if (gtid == 0 && ok) {
           const CUtensorMap* m = grp == 0 ? &mdv : &mdk;
-          tma_store_4d(m, smem + C::OFF_DS + grp * C::PANEL, 0, w.blk * BLK, w.h, w.b);
-          tma_store_4d(m, smem + C::OFF_DS + (2 + grp) * C::PANEL, 32, w.blk * BLK, w.h, w.b);
+          const int first = ntile_ord & 1;              // dS^T buffer of the next ordinary tile
+          tma_store_4d(m, smem + C::OFF_DS + (2 * first + grp) * C::PANEL, 32 * first, w.blk * BLK, w.h, w.b);
+          bulk_commit_group();
+          tma_store_4d(m, smem + C::OFF_DS + (2 * (first ^ 1) + grp) * C::PANEL, 32 * (first ^ 1), w.blk * BLK, w.h,
+                       w.b);
           bulk_commit_group();
         }
-        store_pending = true;
+        store_pending = 2;
       }
       TR(4 + warp, 24);
     }
