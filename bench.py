@@ -335,7 +335,7 @@ def run_ours(args):
                 "peak_source": f"{peaks['source']} bf16 burst (MEASURED_PEAKS.json)" if peaks["source"] == "measured"
                 else "fallback 1590 TFLOP/s",
                 "launch_ms": bwd_ms, "flops_per_launch": bwd_flops,
-                "other_kernels": {"saf_fwd_kernel": {"launch_ms": fwd_ms, "achieved": fwd_flops / (fwd_ms * 1e-3) / 1e12,
+                "other_kernels": {"saf_fwd64_kernel" if wl.D == 64 else "saf_fwd_kernel<128>": {"launch_ms": fwd_ms, "achieved": fwd_flops / (fwd_ms * 1e-3) / 1e12,
                                                       "frac": fwd_flops / (fwd_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]},
                                   "saf_bwd_prep_kernel": {"launch_ms": prep_ms}}}
 
