@@ -356,7 +356,7 @@ def run_ours(args):
         "e2e": {"value": e2e_rate / 1e12, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
         # per step: V scaling + forward kernel, dO scaling + backward preparation + backward kernel
-        "gpu_launches": (5 if len(wl.frozen_heads) else 3) * args.steps,
+        "gpu_launches": (4 if len(wl.frozen_heads) else 3) * args.steps,
         "clocks": clocks,
         "roofline": roofline,
         "cpu_baseline": {"value": cpu_v, "unit": UNIT, "cores": cpu_threads, "kind": "oracle", "sample": cpu_desc},

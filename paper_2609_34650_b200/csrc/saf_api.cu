@@ -58,7 +58,8 @@ struct saf_ctx {
   EncodeTiledFn encode = nullptr;
   unsigned long long wait_limit_ns = 2000000000ull;
   int frozen_weight_pct = 30;              // cost of a frozen tile relative to an ordinary one, forward
-  int frozen_weight_bwd_pct = 20;          // ... and backward
+  int frozen_weight_bwd_pct = 25;          // ... and backward
+  int call_counter = 0;                    // ids of the calls that stage fp16 operands (overflow marks)
   std::vector<WorklistEntry> worklists;
   DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf;
   // tensor-core form of frozen heads: tables built by saf_pattern_prepare, scaled V / dO per call
@@ -398,8 +399,14 @@ int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* froz
       (rc = ensure(ctx->pat_ok, static_cast<size_t>(H) * sizeof(int))) || (rc = ensure(ctx->pat_avec, vecb)) ||
       (rc = ensure(ctx->pat_wvec, vecb)) || (rc = ensure(ctx->pat_bandf, bandb)) ||
       (rc = ensure(ctx->pat_bandb, bandb)) || (rc = ensure(ctx->pat_hord, static_cast<size_t>(H) * sizeof(int))) ||
-      (rc = ensure(ctx->pat_hlist, static_cast<size_t>(H) * sizeof(int))))
+      (rc = ensure(ctx->pat_hlist, static_cast<size_t>(H) * sizeof(int))) ||
+      (rc = ensure(ctx->ok_fwd, static_cast<size_t>(H) * sizeof(int))) ||
+      (rc = ensure(ctx->ok_bwd, static_cast<size_t>(H) * sizeof(int))))
     return rc;
+  // per-head overflow marks of the forward / backward staging kernels (a mark is the id of the call that set it)
+  if (cudaMemsetAsync(ctx->ok_fwd.ptr, 0, static_cast<size_t>(H) * sizeof(int), st) != cudaSuccess ||
+      cudaMemsetAsync(ctx->ok_bwd.ptr, 0, static_cast<size_t>(H) * sizeof(int), st) != cudaSuccess)
+    return SAF_ERR_CUDA;
   std::vector<int> hord(H, -1), hlist(H, 0);
   int ord = 0;
   for (int h = 0; h < H; ++h)
@@ -480,30 +487,28 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   }
   FwdParams fp;
   CUtensorMap mvt = mv;
-  fp.band_f = nullptr; fp.wvec = nullptr; fp.fast_ok = nullptr; fp.hord = nullptr; fp.nblkp = (p->Tp + 127) / 128;
+  fp.band_f = nullptr; fp.wvec = nullptr; fp.fast_ok = nullptr; fp.hord = nullptr; fp.ovf = nullptr; fp.call_id = 0; fp.nblkp = (p->Tp + 127) / 128;
   if (nf > 0 && pattern_matches(ctx, p, frozen_mask_host, alpha, rho, logZ)) {
     // tensor-core form: V of the frozen heads scaled by a(j) once per call
     const size_t vtb = static_cast<size_t>(p->B) * nf * p->T * p->D * 2;
     rc = ensure(ctx->vt_buf, vtb);
     if (rc) return rc;
-    rc = ensure(ctx->ok_fwd, static_cast<size_t>(p->H) * sizeof(int));
-    if (rc) return rc;
-    // per-call copy of the per-head flags; the scaling kernel clears a head whose values leave fp16's range
-    if (cudaMemcpyAsync(ctx->ok_fwd.ptr, ctx->pat_ok.ptr, static_cast<size_t>(p->H) * sizeof(int),
-                        cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-      return SAF_ERR_CUDA;
+    // the scaling kernel marks a head whose values leave fp16's range with this call's id
+    fp.call_id = ++ctx->call_counter;
     {
       ScopedTimer timer(ctx, SAF_KERNEL_SCALE, st);
       if (launch_scale_rows(V, p->v_strides, static_cast<const float*>(ctx->pat_avec.ptr), HK_A_SCALE, p->Tp,
-                            static_cast<const int*>(ctx->pat_hlist.ptr), static_cast<int*>(ctx->ok_fwd.ptr),
-                            ctx->vt_buf.ptr, p->B, nf, p->T, p->D, st) != cudaSuccess)
+                            static_cast<const int*>(ctx->pat_hlist.ptr), static_cast<const int*>(ctx->pat_ok.ptr),
+                            static_cast<int*>(ctx->ok_fwd.ptr), fp.call_id, ctx->vt_buf.ptr, p->B, nf, p->T, p->D,
+                            st) != cudaSuccess)
         return SAF_ERR_CUDA;
     }
     rc = make_map_contig(ctx, &mvt, ctx->vt_buf.ptr, p, nf);
     if (rc) return rc;
     fp.band_f = ctx->pat_bandf.ptr;
     fp.wvec = static_cast<const float*>(ctx->pat_wvec.ptr);
-    fp.fast_ok = static_cast<const int*>(ctx->ok_fwd.ptr);
+    fp.fast_ok = static_cast<const int*>(ctx->pat_ok.ptr);
+    fp.ovf = static_cast<const int*>(ctx->ok_fwd.ptr);
     fp.hord = static_cast<const int*>(ctx->pat_hord.ptr);
   }
   fp.B = p->B; fp.H = p->H; fp.T = p->T; fp.Tp = p->Tp;
@@ -572,11 +577,26 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     if (rc) return rc;
     dqacc = static_cast<float*>(ctx->dqacc_buf.ptr);
   }
+  // tensor-core form of the frozen heads: the preparation kernel also stages w(i) dO in fp16
+  const bool tensor_form = nf > 0 && pattern_matches(ctx, p, frozen_mask_host, alpha, rho, logZ);
+  PrepFrozen fz{};
+  if (tensor_form) {
+    rc = ensure(ctx->dot_buf, static_cast<size_t>(p->B) * nf * p->T * p->D * 2);
+    if (rc) return rc;
+    fz.wvec = static_cast<const float*>(ctx->pat_wvec.ptr);
+    fz.hord = static_cast<const int*>(ctx->pat_hord.ptr);
+    fz.pat_ok = static_cast<const int*>(ctx->pat_ok.ptr);
+    fz.ovf = static_cast<int*>(ctx->ok_bwd.ptr);
+    fz.call_id = ++ctx->call_counter;
+    fz.dot_dst = ctx->dot_buf.ptr;
+    fz.Hf = nf;
+    fz.Tp = p->Tp;
+  }
   // O is only read for ordinary heads; a frozen-only layer may pass O = NULL
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_PREP, st);
     if (launch_bwd_prep(O, dO, LSE, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr), q_ext, do_ext,
-                        1.0f / scale_v, dqacc, dK, grad_f32, p->B, p->H, p->T, p->D, st) != cudaSuccess)
+                        1.0f / scale_v, dqacc, dK, grad_f32, fz, p->B, p->H, p->T, p->D, st) != cudaSuccess)
       return SAF_ERR_CUDA;
   }
 
@@ -616,30 +636,16 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   }
   BwdParams bp;
   CUtensorMap mdot = mdo;
-  bp.band_b = nullptr; bp.avec = nullptr; bp.fast_ok = nullptr; bp.hord = nullptr; bp.nblkp = (p->Tp + 127) / 128;
-  if (nf > 0 && pattern_matches(ctx, p, frozen_mask_host, alpha, rho, logZ)) {
-    // tensor-core form: dO of the frozen heads scaled by w(i) once per call
-    const size_t dob = static_cast<size_t>(p->B) * nf * p->T * p->D * 2;
-    rc = ensure(ctx->dot_buf, dob);
-    if (rc) return rc;
-    rc = ensure(ctx->ok_bwd, static_cast<size_t>(p->H) * sizeof(int));
-    if (rc) return rc;
-    if (cudaMemcpyAsync(ctx->ok_bwd.ptr, ctx->pat_ok.ptr, static_cast<size_t>(p->H) * sizeof(int),
-                        cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-      return SAF_ERR_CUDA;
-    {
-      ScopedTimer timer(ctx, SAF_KERNEL_SCALE, st);
-      if (launch_scale_rows(dO, p->o_strides, static_cast<const float*>(ctx->pat_wvec.ptr), 1.0f, p->Tp,
-                            static_cast<const int*>(ctx->pat_hlist.ptr), static_cast<int*>(ctx->ok_bwd.ptr),
-                            ctx->dot_buf.ptr, p->B, nf, p->T, p->D, st) != cudaSuccess)
-        return SAF_ERR_CUDA;
-    }
+  bp.band_b = nullptr; bp.avec = nullptr; bp.fast_ok = nullptr; bp.hord = nullptr; bp.ovf = nullptr; bp.call_id = 0; bp.nblkp = (p->Tp + 127) / 128;
+  if (tensor_form) {
     rc = make_map_contig(ctx, &mdot, ctx->dot_buf.ptr, p, nf);
     if (rc) return rc;
     bp.band_b = ctx->pat_bandb.ptr;
     bp.avec = static_cast<const float*>(ctx->pat_avec.ptr);
-    bp.fast_ok = static_cast<const int*>(ctx->ok_bwd.ptr);
-    bp.hord = static_cast<const int*>(ctx->pat_hord.ptr);
+    bp.fast_ok = fz.pat_ok;
+    bp.hord = fz.hord;
+    bp.ovf = fz.ovf;
+    bp.call_id = fz.call_id;
   }
   bp.B = p->B; bp.H = p->H; bp.T = p->T; bp.Tp = p->Tp;
   bp.scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));

@@ -104,7 +104,8 @@ __device__ __forceinline__ ItemView load_item(const BwdParams& p, int it, int it
   if (it < it_end) {
     const int4 raw = __ldg(reinterpret_cast<const int4*>(p.items + it));
     v.w = WorkItem{raw.x, raw.y, raw.z, raw.w};
-    v.fast = raw.w != KIND_ORDINARY && p.band_b != nullptr && __ldg(p.fast_ok + raw.y) != 0;
+    v.fast = raw.w != KIND_ORDINARY && p.band_b != nullptr && __ldg(p.fast_ok + raw.y) != 0 &&
+             __ldg(p.ovf + raw.y) != p.call_id;
   }
   return v;
 }
@@ -218,7 +219,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         const WorkItem w = p.items[it];
         const bool ord = w.kind == KIND_ORDINARY;
         const size_t bh = static_cast<size_t>(w.b) * p.H + w.h;
-        const bool fast = !ord && p.band_b != nullptr && p.fast_ok[w.h] != 0;
+        const bool fast = !ord && p.band_b != nullptr && p.fast_ok[w.h] != 0 && p.ovf[w.h] != p.call_id;
         if (fast) {
           // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled dO tile
           const int fo = p.hord[w.h];

@@ -125,7 +125,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       for (int it = it_begin; it < it_end && ok; ++it) {
         const WorkItem w = p.items[it];
         const int ntiles = w.blk + 1;
-        if (w.kind == KIND_FROZEN && p.band_f != nullptr && p.fast_ok[w.h] != 0) {
+        if (w.kind == KIND_FROZEN && p.band_f != nullptr && p.fast_ok[w.h] != 0 && p.ovf[w.h] != p.call_id) {
           // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled V tile
           const int ord = p.hord[w.h];
           const uint8_t* bands = static_cast<const uint8_t*>(p.band_f) + static_cast<size_t>(w.h) * p.nblkp * 4096;
@@ -201,7 +201,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       const WorkItem w = p.items[it];
       const int ntiles = w.blk + 1;
       const bool ord = w.kind == KIND_ORDINARY;
-      if (w.kind == KIND_FROZEN && p.band_f != nullptr && p.fast_ok[w.h] != 0) {
+      if (w.kind == KIND_FROZEN && p.band_f != nullptr && p.fast_ok[w.h] != 0 && p.ovf[w.h] != p.call_id) {
         for (int j = 0; j < ntiles && ok; ++j) {
           const uint32_t sk = nk % C::NS, sv = nv % C::NS;
           ok = mbar_wait_warp(k_full + sk, (nk / C::NS) & 1, wc, SITE_K_FULL);
@@ -315,7 +315,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       int row = w.blk * BLK + rowl;
       float inv_l = 1.0f, lse = 0.0f;
       if (named_bar_or(5, 256, !ok)) break;
-      if (w.kind == KIND_FROZEN && p.band_f != nullptr && p.fast_ok[w.h] != 0) {
+      if (w.kind == KIND_FROZEN && p.band_f != nullptr && p.fast_ok[w.h] != 0 && p.ovf[w.h] != p.call_id) {
         // tensor-core form: nothing to do per tile; lane m holds query 127-m, scaled by w(i) below
         row = w.blk * BLK + 127 - rowl;
         inv_l = (row < p.T) ? p.wvec[static_cast<size_t>(w.h) * p.Tp + row] * (1.0f / (HK_BAND_SCALE * HK_A_SCALE)) : 0.0f;

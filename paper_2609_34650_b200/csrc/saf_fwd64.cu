@@ -85,7 +85,8 @@ __device__ __forceinline__ ItemView64 load_item64(const FwdParams& p, int it, in
   if (it < it_end) {
     const int4 raw = __ldg(reinterpret_cast<const int4*>(p.items + it));
     v.w = WorkItem{raw.x, raw.y, raw.z, raw.w};
-    v.fast = raw.w != KIND_ORDINARY && p.band_f != nullptr && __ldg(p.fast_ok + raw.y) != 0;
+    v.fast = raw.w != KIND_ORDINARY && p.band_f != nullptr && __ldg(p.fast_ok + raw.y) != 0 &&
+             __ldg(p.ovf + raw.y) != p.call_id;
   }
   return v;
 }

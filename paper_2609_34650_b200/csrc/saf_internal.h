@@ -28,6 +28,9 @@ struct FwdParams {
   const float* wvec;
   const int* fast_ok;
   const int* hord;
+  // ovf[h] == call_id: a staged fp16 value of head h left fp16's range in this call (general path instead)
+  const int* ovf;
+  int call_id;
   int nblkp;
   const WorkItem* items;            // grouped by CTA
   const int* cta_offsets;           // [grid+1]
@@ -55,6 +58,8 @@ struct BwdParams {
   const float* avec;
   const int* fast_ok;
   const int* hord;
+  const int* ovf;                   // as in FwdParams
+  int call_id;
   int nblkp;
   const WorkItem* items;
   const int* cta_offsets;
@@ -69,8 +74,8 @@ cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const fl
                                   int H, int Tp, float* consts, int* fast_ok, float* avec, float* wvec, void* band_f,
                                   void* band_b, cudaStream_t st);
 cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, float extra, int Tp,
-                              const int* hlist, int* call_ok, void* dst, int B, int Hf, int T, int D,
-                              cudaStream_t st);
+                              const int* hlist, const int* pat_ok, int* ovf, int call_id, void* dst, int B, int Hf,
+                              int T, int D, cudaStream_t st);
 // powers of two that put the fp16 operands of the tensor-core frozen form into fp16's range
 constexpr float HK_BAND_SCALE = 16384.0f;        // bands hold 2^14 r
 constexpr float HK_A_SCALE = 2048.0f;            // the forward stages 2^11 a V
@@ -83,10 +88,20 @@ cudaError_t launch_bwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, cons
                        const CUtensorMap& mdo, const CUtensorMap& mdq, const CUtensorMap& mdot, const CUtensorMap& mdk,
                        const CUtensorMap& mdv, const BwdParams& p, int grid, cudaStream_t st);
 // Row terms of ordinary heads (q_ext / do_ext images, see BwdParams); also zeroes dQacc (all heads) and
-// dK of frozen heads.
+// dK of frozen heads, and (dot_dst != NULL) stages w(i) dO of the frozen heads in fp16 for the tensor-core form.
+struct PrepFrozen {
+  const float* wvec;                // [H][Tp]
+  const int* hord;                  // head -> ordinal among the frozen heads
+  const int* pat_ok;                // per-head flag of the pattern
+  int* ovf;                         // set to call_id when a staged value leaves fp16's range
+  int call_id;
+  void* dot_dst;                    // fp16 [B][Hf][T][D], or NULL
+  int Hf, Tp;
+};
 cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* o_strides,
                             const uint8_t* mask_dev, void* q_ext, void* do_ext, float inv_scale, float* dQacc,
-                            void* dK, int grad_f32, int B, int H, int T, int D, cudaStream_t st);
+                            void* dK, int grad_f32, const PrepFrozen& fz, int B, int H, int T, int D,
+                            cudaStream_t st);
 // dQ (grad dtype) = scale-free copy/convert of dQacc (fp32) for the bf16-gradient case.
 cudaError_t launch_bwd_finalize(const float* dQacc, void* dQ, size_t n, cudaStream_t st);
 // head dimension 64 (saf_fwd64.cu); launch_fwd dispatches to it

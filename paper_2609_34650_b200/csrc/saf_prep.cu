@@ -155,15 +155,16 @@ cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const fl
 }
 
 // dst[b][ord][t][:] = fp16(extra * vec[h][t] * src[b][h][t][:]), h = hlist[ord], for the frozen heads whose tensor-core form is
-// enabled (V scaled by a, or dO scaled by w).  Eight features per thread.  call_ok[h] starts as a copy of
-// fast_ok[h]; a product that leaves fp16's range clears it, which sends that head down the general path
-// in the kernel that follows.
+// enabled (V scaled by a, or dO scaled by w).  Eight features per thread.  A product that leaves fp16's range
+// marks the head (ovf[h] = call_id), which sends it down the general path in the kernel that follows; the
+// mark of an earlier call has another id and needs no reset.
 template <int D>
 __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16* __restrict__ src, int64_t s0, int64_t s1,
                                                              int64_t s2, const float* __restrict__ vec, float extra,
                                                              int Tp, const int* __restrict__ hlist,
-                                                             int* __restrict__ call_ok,
-                                                             __half* __restrict__ dst, int B, int Hf, int T) {
+                                                             const int* __restrict__ pat_ok, int* __restrict__ ovf,
+                                                             int call_id, __half* __restrict__ dst, int B, int Hf,
+                                                             int T) {
   constexpr int TPR = D / 8;
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
   const long long rowid = gid / TPR;               // over [B][Hf][T]: frozen heads only
@@ -173,7 +174,7 @@ __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16
   const int ord = static_cast<int>((rowid / T) % Hf);
   const int b = static_cast<int>(rowid / (static_cast<long long>(T) * Hf));
   const int h = hlist[ord];
-  if (!call_ok[h]) return;
+  if (!pat_ok[h]) return;
   const float f = vec[static_cast<size_t>(h) * Tp + t] * extra;
   const uint4 v4 = *reinterpret_cast<const uint4*>(src + b * s0 + h * s1 + static_cast<int64_t>(t) * s2 + part * 8);
   const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&v4);
@@ -186,22 +187,22 @@ __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16
     bad |= !(fabsf(y0) <= 65504.0f) || !(fabsf(y1) <= 65504.0f);     // also catches NaN
     o[e] = __floats2half2_rn(y0, y1);
   }
-  if (bad) atomicExch(call_ok + h, 0);
+  if (bad) ovf[h] = call_id;
   *reinterpret_cast<uint4*>(dst + (static_cast<size_t>(rowid)) * D + part * 8) = *reinterpret_cast<uint4*>(o);
 }
 
 cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, float extra, int Tp,
-                              const int* hlist, int* call_ok, void* dst, int B, int Hf, int T, int D,
-                              cudaStream_t st) {
+                              const int* hlist, const int* pat_ok, int* ovf, int call_id, void* dst, int B, int Hf,
+                              int T, int D, cudaStream_t st) {
   const long long nthreads = static_cast<long long>(B) * Hf * T * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
   if (D == 64)
     saf_scale_rows_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
-                                                    strides[2], vec, extra, Tp, hlist, call_ok,
+                                                    strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
                                                     static_cast<__half*>(dst), B, Hf, T);
   else
     saf_scale_rows_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
-                                                     strides[2], vec, extra, Tp, hlist, call_ok,
+                                                     strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
                                                      static_cast<__half*>(dst), B, Hf, T);
   return cudaGetLastError();
 }
@@ -225,7 +226,7 @@ __device__ __forceinline__ uint4 split3_bf16(float x) {
 //                  do_ext row = split3(-delta)      (so that dP - delta comes out of the dP MMA);
 //                  rows beyond T: q_ext = most negative bf16 (their probabilities become 0), do_ext = 0
 //   every head   : dQacc row = 0 (it is accumulated by reduce-adds of the main kernel)
-//   frozen head  : dK row = 0 (no key gradient; Sec. 3.3)
+//   frozen head  : dK row = 0 (no key gradient; Sec. 3.3); with the tensor-core form, the row w(i) dO in fp16
 // Image layout per 128-row block (4 KB): byte (n/8)*256 + (k/8)*128 + (n%8)*16 + (k%8)*2 for row n, column k < 16.
 template <int D>
 __global__ void __launch_bounds__(256) saf_bwd_prep_kernel(const __nv_bfloat16* __restrict__ O,
@@ -234,7 +235,8 @@ __global__ void __launch_bounds__(256) saf_bwd_prep_kernel(const __nv_bfloat16* 
                                                            int64_t os2, const uint8_t* __restrict__ mask,
                                                            uint8_t* __restrict__ q_ext, uint8_t* __restrict__ do_ext,
                                                            float inv_scale, float* __restrict__ dQacc,
-                                                           void* __restrict__ dK, int grad_f32, int B, int H, int T) {
+                                                           void* __restrict__ dK, int grad_f32, const PrepFrozen fz,
+                                                           int B, int H, int T) {
   constexpr int TPR = D / 8;                       // threads per row
   const int Tpad = (T + 127) / 128 * 128;
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
@@ -263,6 +265,25 @@ __global__ void __launch_bounds__(256) saf_bwd_prep_kernel(const __nv_bfloat16* 
         *reinterpret_cast<float4*>(static_cast<float*>(dK) + grow + 4) = z;
       } else {
         *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(dK) + grow) = make_uint4(0, 0, 0, 0);
+      }
+      if (fz.dot_dst != nullptr && fz.pat_ok[h] != 0) {
+        const float f = fz.wvec[static_cast<size_t>(h) * fz.Tp + t];
+        const uint4 d4 =
+            *reinterpret_cast<const uint4*>(dO + b * os0 + h * os1 + static_cast<int64_t>(t) * os2 + part * 8);
+        const __nv_bfloat162* d2 = reinterpret_cast<const __nv_bfloat162*>(&d4);
+        __half2 o[4];
+        bool bad = false;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 x = __bfloat1622float2(d2[e]);
+          const float y0 = x.x * f, y1 = x.y * f;
+          bad |= !(fabsf(y0) <= 65504.0f) || !(fabsf(y1) <= 65504.0f);     // also catches NaN
+          o[e] = __floats2half2_rn(y0, y1);
+        }
+        if (bad) fz.ovf[h] = fz.call_id;
+        const size_t drow = (static_cast<size_t>(b) * fz.Hf + fz.hord[h]) * T + t;
+        *reinterpret_cast<uint4*>(static_cast<__half*>(fz.dot_dst) + drow * D + part * 8) =
+            *reinterpret_cast<uint4*>(o);
       }
     } else {
       const int64_t off = b * os0 + h * os1 + static_cast<int64_t>(t) * os2 + part * 8;
@@ -300,8 +321,8 @@ __global__ void __launch_bounds__(256) saf_bwd_prep_kernel(const __nv_bfloat16* 
 }
 
 cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* os, const uint8_t* mask_dev,
-                            void* q_ext, void* do_ext, float inv_scale, float* dQacc, void* dK, int grad_f32, int B,
-                            int H, int T, int D, cudaStream_t st) {
+                            void* q_ext, void* do_ext, float inv_scale, float* dQacc, void* dK, int grad_f32,
+                            const PrepFrozen& fz, int B, int H, int T, int D, cudaStream_t st) {
   const int Tpad = (T + 127) / 128 * 128;
   const long long nthreads = static_cast<long long>(B) * H * Tpad * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
@@ -309,12 +330,12 @@ cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, con
     saf_bwd_prep_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
                                                   static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2],
                                                   mask_dev, static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext),
-                                                  inv_scale, dQacc, dK, grad_f32, B, H, T);
+                                                  inv_scale, dQacc, dK, grad_f32, fz, B, H, T);
   else
     saf_bwd_prep_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
                                                    static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2],
                                                    mask_dev, static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext),
-                                                   inv_scale, dQacc, dK, grad_f32, B, H, T);
+                                                   inv_scale, dQacc, dK, grad_f32, fz, B, H, T);
   return cudaGetLastError();
 }
 
