@@ -110,9 +110,12 @@ def frozen_head_bwd(dO, alpha, rho):
 
 # ----------------------------------------------------------------------------- the layer
 def hybrid_attn_fwd(Q, K, V, mask, alpha, rho, scale=None):
-    """Q,K,V: [B,H,T,D] float64; mask: [H] (nonzero = frozen); alpha,rho: [H,Tp].
+    """Q: [B,H,T,D], K,V: [B,Hkv,T,D] float64 with Hkv dividing H (grouped-query path, Appendix E.2: query head h
+    reads the shared key/value head h // (H/Hkv); Hkv = H is ordinary multi-head attention);
+    mask: [H] (nonzero = frozen); alpha,rho: [H,Tp].
     Returns O [B,H,T,D] and LSE [B,H,T] (0 for frozen heads, which have no softmax)."""
     B, H, T, D = Q.shape
+    g = H // K.shape[1]
     scale = 1.0 / np.sqrt(D) if scale is None else scale
     O = np.zeros((B, H, T, D))
     LSE = np.zeros((B, H, T))
@@ -120,28 +123,35 @@ def hybrid_attn_fwd(Q, K, V, mask, alpha, rho, scale=None):
         if mask[h]:
             P = pattern_dense(alpha[h], rho[h], T)
             for b in range(B):
-                O[b, h] = P @ V[b, h]
+                O[b, h] = P @ V[b, h // g]
         else:
             for b in range(B):
-                O[b, h], LSE[b, h], _ = ordinary_head_fwd(Q[b, h], K[b, h], V[b, h], scale)
+                O[b, h], LSE[b, h], _ = ordinary_head_fwd(Q[b, h], K[b, h // g], V[b, h // g], scale)
     return O, LSE
 
 
 def hybrid_attn_bwd(Q, K, V, dO, mask, alpha, rho, scale=None):
-    """Gradients of sum(O o dO) w.r.t. Q, K, V.  Frozen heads: dQ = dK = 0, dV = P^T dO."""
+    """Gradients of sum(O o dO) w.r.t. Q, K, V.  Frozen heads: dQ = dK = 0, dV = P^T dO.  With shared
+    key/value heads (K, V: [B,Hkv,T,D]) the gradient of a shared head is the sum over the query heads that
+    read it."""
     B, H, T, D = Q.shape
+    Hkv = K.shape[1]
+    g = H // Hkv
     scale = 1.0 / np.sqrt(D) if scale is None else scale
     dQ = np.zeros((B, H, T, D))
-    dK = np.zeros((B, H, T, D))
-    dV = np.zeros((B, H, T, D))
+    dK = np.zeros((B, Hkv, T, D))
+    dV = np.zeros((B, Hkv, T, D))
     for h in range(H):
         if mask[h]:
             P = pattern_dense(alpha[h], rho[h], T)
             for b in range(B):
-                dV[b, h] = P.T @ dO[b, h]
+                dV[b, h // g] += P.T @ dO[b, h]
         else:
             for b in range(B):
-                dQ[b, h], dK[b, h], dV[b, h] = ordinary_head_bwd(Q[b, h], K[b, h], V[b, h], dO[b, h], scale)
+                dq, dk, dv = ordinary_head_bwd(Q[b, h], K[b, h // g], V[b, h // g], dO[b, h], scale)
+                dQ[b, h] = dq
+                dK[b, h // g] += dk
+                dV[b, h // g] += dv
     return dQ, dK, dV
 
 

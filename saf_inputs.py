@@ -54,6 +54,7 @@ class Workload:
     alpha0_spike: float = 0.0     # added to alpha[0] (attention-sink-like)
     backward: bool = True
     seed: int = 0
+    kv_group: int = 1             # grouped-query attention: query heads per shared key/value head
 
     @property
     def stored_len(self) -> int:
@@ -105,7 +106,7 @@ def config(k: int, n_frozen: int | None = None, seed: int = 0) -> Workload:
 class Inputs:
     wl: Workload
     q: np.ndarray       # [B,H,T,D] uint16 (bf16 bits)
-    k: np.ndarray
+    k: np.ndarray       # [B,H/kv_group,T,D]
     v: np.ndarray
     do: np.ndarray      # [B,H,T,D] uint16 (bf16 bits); drawn even for forward-only workloads
     alpha: np.ndarray   # [H,Tp] float32 (rows of ordinary heads are zero)
@@ -124,9 +125,10 @@ def _normal_bf16(rng: np.random.Generator, shape) -> np.ndarray:
 def generate(wl: Workload) -> Inputs:
     rng = np.random.default_rng(wl.seed)
     shape = (wl.B, wl.H, wl.T, wl.D)
+    kv_shape = (wl.B, wl.H // wl.kv_group, wl.T, wl.D)
     q = _normal_bf16(rng, shape)
-    k = _normal_bf16(rng, shape)
-    v = _normal_bf16(rng, shape)
+    k = _normal_bf16(rng, kv_shape)
+    v = _normal_bf16(rng, kv_shape)
     do = _normal_bf16(rng, shape)
     tp = wl.stored_len
     alpha = np.zeros((wl.H, tp), dtype=np.float32)

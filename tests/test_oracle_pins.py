@@ -14,6 +14,9 @@ off-by-one in the relative distance or the causal boundary):
   P7  gradients: frozen dQ = dK = 0; central finite differences of sum(O o dO) on tiny shapes;
       frozen dV against torch autograd through a dense P built with torch ops
   P8  pure-Python triple loops (math.exp) on tiny inputs for every output of the layer
+  P9  grouped-query path (Appendix E.2): shared key/value heads == the multi-head layer on K, V repeated per
+      query head, with the shared heads' gradients summed over their query heads (torch autograd through
+      repeat_interleave; torch's own enable_gqa route for the all-ordinary case; finite differences)
 """
 import math
 
@@ -330,3 +333,75 @@ def test_panel_routes_equal_dense(frozen):
         assert np.abs(LSE - eL).max() < 1e-13
     for g, e in ((O, eO), (gQ, eQ), (gK, eK), (gV, eV)):
         assert np.abs(g - e).max() < 1e-12
+
+
+# ------------------------------------------------------------------ P9 grouped-query path
+@pytest.mark.parametrize("H,g,frozen", [(4, 2, ()), (6, 3, (1, 5)), (4, 4, (0, 2)), (4, 1, (3,))])
+def test_p9_gqa_equals_repeated_kv(H, g, frozen):
+    B, T, D = 2, 21, 8
+    rng = np.random.default_rng(90 + H + g)
+    Q, dO = rng.standard_normal((B, H, T, D)), rng.standard_normal((B, H, T, D))
+    K, V = rng.standard_normal((B, H // g, T, D)), rng.standard_normal((B, H // g, T, D))
+    mask = np.zeros(H, dtype=np.uint8)
+    mask[list(frozen)] = 1
+    alpha, rho = rng.standard_normal((H, T)), -0.1 * np.arange(T)[None, :] + 0.1 * rng.standard_normal((H, T))
+    O, LSE = orc.hybrid_attn_fwd(Q, K, V, mask, alpha, rho)
+    dQ, dK, dV = orc.hybrid_attn_bwd(Q, K, V, dO, mask, alpha, rho)
+    assert dK.shape == K.shape and dV.shape == V.shape
+    # torch: repeat the shared heads, dense attention weights per head, autograd sums the shared gradients
+    tq, tk, tv = (torch.tensor(x, requires_grad=True) for x in (Q, K, V))
+    kr, vr = tk.repeat_interleave(g, dim=1), tv.repeat_interleave(g, dim=1)
+    causal = torch.tril(torch.ones(T, T, dtype=torch.bool))
+    outs = []
+    for h in range(H):
+        if mask[h]:
+            i, j = np.indices((T, T))
+            bias = torch.tensor(alpha[h][j] + rho[h][np.clip(i - j, 0, None)])
+            w = torch.softmax(bias.masked_fill(~causal, -math.inf), dim=-1)
+            outs.append(torch.einsum("ij,bjd->bid", w, vr[:, h]))
+        else:
+            s = torch.einsum("bid,bjd->bij", tq[:, h], kr[:, h]) / math.sqrt(D)
+            w = torch.softmax(s.masked_fill(~causal, -math.inf), dim=-1)
+            outs.append(torch.einsum("bij,bjd->bid", w, vr[:, h]))
+    to = torch.stack(outs, dim=1)
+    to.backward(torch.tensor(dO))
+    assert np.abs(O - to.detach().numpy()).max() < 1e-12
+    assert np.abs(dQ - tq.grad.numpy()).max() < 1e-11
+    assert np.abs(dK - tk.grad.numpy()).max() < 1e-11
+    assert np.abs(dV - tv.grad.numpy()).max() < 1e-11
+    for h in frozen:
+        assert not dQ[:, h].any()
+
+
+def test_p9_gqa_all_ordinary_equals_torch_enable_gqa():
+    B, H, g, T, D = 2, 8, 4, 40, 16
+    rng = np.random.default_rng(99)
+    Q = rng.standard_normal((B, H, T, D))
+    K, V = rng.standard_normal((B, H // g, T, D)), rng.standard_normal((B, H // g, T, D))
+    O, _ = orc.hybrid_attn_fwd(Q, K, V, np.zeros(H, dtype=np.uint8), None, None)
+    to = torch.nn.functional.scaled_dot_product_attention(torch.tensor(Q), torch.tensor(K), torch.tensor(V),
+                                                          is_causal=True, enable_gqa=True)
+    assert np.abs(O - to.numpy()).max() < 1e-12
+
+
+def test_p9_gqa_finite_differences_of_shared_heads():
+    B, H, g, T, D = 1, 4, 2, 7, 3
+    rng = np.random.default_rng(91)
+    Q, dO = rng.standard_normal((B, H, T, D)), rng.standard_normal((B, H, T, D))
+    K, V = rng.standard_normal((B, H // g, T, D)), rng.standard_normal((B, H // g, T, D))
+    mask = np.array([0, 1, 0, 0], dtype=np.uint8)
+    alpha, rho = rng.standard_normal((H, T)), rng.standard_normal((H, T))
+    _, dK, dV = orc.hybrid_attn_bwd(Q, K, V, dO, mask, alpha, rho)
+
+    def loss(Kx, Vx):
+        O, _ = orc.hybrid_attn_fwd(Q, Kx, Vx, mask, alpha, rho)
+        return float((O * dO).sum())
+
+    h = 1e-6
+    for arr, grad, which in ((K, dK, 0), (V, dV, 1)):
+        for idx in [(0, 0, 2, 1), (0, 1, 5, 0), (0, 1, 0, 2), (0, 0, 6, 2)]:
+            ap, am = arr.copy(), arr.copy()
+            ap[idx] += h
+            am[idx] -= h
+            fd = (loss(ap, V) - loss(am, V)) / (2 * h) if which == 0 else (loss(K, ap) - loss(K, am)) / (2 * h)
+            assert abs(fd - grad[idx]) < 1e-7
