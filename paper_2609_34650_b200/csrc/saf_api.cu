@@ -98,9 +98,9 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // [B][H][T][D] bf16 tensor with element strides (batch, head, seq); box = 64 features x 128 rows,
 // 128-byte swizzle; rows beyond T read as zero.
 int make_map(saf_ctx* ctx, CUtensorMap* out, const void* base, const saf_problem* p, const int64_t* strides,
-             CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) {
-  cuuint64_t dims[4] = {static_cast<cuuint64_t>(p->D), static_cast<cuuint64_t>(p->T), static_cast<cuuint64_t>(p->H),
-                        static_cast<cuuint64_t>(p->B)};
+             CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, int heads = 0) {
+  cuuint64_t dims[4] = {static_cast<cuuint64_t>(p->D), static_cast<cuuint64_t>(p->T),
+                        static_cast<cuuint64_t>(heads > 0 ? heads : p->H), static_cast<cuuint64_t>(p->B)};
   cuuint64_t gs[3] = {static_cast<cuuint64_t>(strides[2]) * 2, static_cast<cuuint64_t>(strides[1]) * 2,
                       static_cast<cuuint64_t>(strides[0]) * 2};
   cuuint32_t box[4] = {64, BLK, 1, 1};
@@ -140,11 +140,14 @@ int validate(const saf_problem* p, const uint8_t* mask, int* n_frozen) {
   if (p->T > p->Tp) return SAF_ERR_INVALID_ARG;
   if (p->D != 64 && p->D != 128) return SAF_ERR_UNSUPPORTED;
   if (p->grad_dtype != SAF_F32 && p->grad_dtype != SAF_BF16) return SAF_ERR_UNSUPPORTED;
+  if (p->kv_group < 0 || (p->kv_group > 1 && p->H % p->kv_group != 0)) return SAF_ERR_INVALID_ARG;
   int nf = 0;
   for (int h = 0; h < p->H; ++h) nf += mask[h] ? 1 : 0;
   *n_frozen = nf;
   return SAF_OK;
 }
+
+inline int kv_group_of(const saf_problem* p) { return p->kv_group > 1 ? p->kv_group : 1; }
 
 int upload_mask(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st) {
   int rc = ensure(ctx->mask_buf, std::max(H, 256));
@@ -474,12 +477,13 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
 
   CUtensorMap mq, mk, mv;
   // frozen-only layers never touch Q/K: any valid map will do
-  rc = make_map(ctx, &mv, V, p, p->v_strides);
+  const int kvg = kv_group_of(p);
+  rc = make_map(ctx, &mv, V, p, p->v_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg);
   if (rc) return rc;
   if (no > 0) {
     rc = make_map(ctx, &mq, Q, p, p->q_strides);
     if (rc) return rc;
-    rc = make_map(ctx, &mk, K, p, p->k_strides);
+    rc = make_map(ctx, &mk, K, p, p->k_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg);
     if (rc) return rc;
   } else {
     mq = mv;
@@ -500,7 +504,7 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
       if (launch_scale_rows(V, p->v_strides, static_cast<const float*>(ctx->pat_avec.ptr), HK_A_SCALE, p->Tp,
                             static_cast<const int*>(ctx->pat_hlist.ptr), static_cast<const int*>(ctx->pat_ok.ptr),
                             static_cast<int*>(ctx->ok_fwd.ptr), fp.call_id, ctx->vt_buf.ptr, p->B, nf, p->T, p->D,
-                            st) != cudaSuccess)
+                            kvg, st) != cudaSuccess)
         return SAF_ERR_CUDA;
     }
     rc = make_map_contig(ctx, &mvt, ctx->vt_buf.ptr, p, nf);
@@ -512,6 +516,7 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     fp.hord = static_cast<const int*>(ctx->pat_hord.ptr);
   }
   fp.B = p->B; fp.H = p->H; fp.T = p->T; fp.Tp = p->Tp;
+  fp.kv_group = kvg;
   const float scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   fp.scale_log2 = scale * 1.4426950408889634f;
   fp.alpha = alpha; fp.rho = rho; fp.logZ = logZ;
@@ -571,6 +576,8 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   uint8_t* do_ext = q_ext + ext_bytes;
   const float scale_v = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   const int grad_f32 = p->grad_dtype == SAF_F32;
+  const int kvg = kv_group_of(p);
+  if (kvg > 1 && !grad_f32) return SAF_ERR_UNSUPPORTED;   // shared heads' gradients are accumulated in fp32
   float* dqacc = static_cast<float*>(dQ);
   if (!grad_f32) {
     rc = ensure(ctx->dqacc_buf, nelem * sizeof(float));
@@ -596,7 +603,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_PREP, st);
     if (launch_bwd_prep(O, dO, LSE, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr), q_ext, do_ext,
-                        1.0f / scale_v, dqacc, dK, grad_f32, fz, p->B, p->H, p->T, p->D, st) != cudaSuccess)
+                        1.0f / scale_v, dqacc, dK, dV, grad_f32, kvg, fz, p->B, p->H, p->T, p->D, st) != cudaSuccess)
       return SAF_ERR_CUDA;
   }
 
@@ -611,8 +618,8 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   if (rc) return rc;
   if (no > 0) {
     if ((rc = make_map(ctx, &mq, Q, p, p->q_strides))) return rc;
-    if ((rc = make_map(ctx, &mk, K, p, p->k_strides))) return rc;
-    if ((rc = make_map(ctx, &mv, V, p, p->v_strides))) return rc;
+    if ((rc = make_map(ctx, &mk, K, p, p->k_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg))) return rc;
+    if ((rc = make_map(ctx, &mv, V, p, p->v_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg))) return rc;
   } else {
     mq = mdo; mk = mdo; mv = mdo;
   }
@@ -632,6 +639,9 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     if (!enc(&mdq, dqacc)) return SAF_ERR_CUDA;
     mdk = mdq;
     mdv = mdq;
+    // dK, dV: [B][H/kv_group][T][64]
+    dims[2] = static_cast<cuuint64_t>(p->H / kvg);
+    gs[2] = static_cast<cuuint64_t>(p->T) * 64 * 4 * (p->H / kvg);
     if (grad_f32 && (!enc(&mdk, dK) || !enc(&mdv, dV))) return SAF_ERR_CUDA;
   }
   BwdParams bp;
@@ -648,6 +658,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     bp.call_id = fz.call_id;
   }
   bp.B = p->B; bp.H = p->H; bp.T = p->T; bp.Tp = p->Tp;
+  bp.kv_group = kvg;
   bp.scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   bp.scale_log2 = bp.scale * 1.4426950408889634f;
   bp.alpha = alpha; bp.rho = rho; bp.logZ = logZ;
@@ -683,9 +694,12 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
   if (!V_host || (no > 0 && (!Q_host || !K_host)) || (nf > 0 && (!alpha_host || !rho_host))) return SAF_ERR_INVALID_ARG;
   DeviceGuard g(ctx->device);
   if (!g.ok) return SAF_ERR_CUDA;
+  const int kvg = kv_group_of(p);
   const size_t nelem = static_cast<size_t>(p->B) * p->H * p->T * p->D;
   const size_t tb = nelem * 2;
+  const size_t tkv = tb / kvg;                      // K, V: H / kv_group heads
   const size_t gb = nelem * (p->grad_dtype == SAF_F32 ? 4 : 2);
+  const size_t gkv = gb / kvg;
   const size_t pb = static_cast<size_t>(p->H) * p->Tp * sizeof(float);
   const size_t lb = static_cast<size_t>(p->B) * p->H * p->T * sizeof(float);
   const bool bwd = dO_host != nullptr;
@@ -701,12 +715,13 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
   const int64_t s2 = p->D, s1 = static_cast<int64_t>(p->T) * p->D, s0 = s1 * p->H;
   int64_t* sets[4] = {q.q_strides, q.k_strides, q.v_strides, q.o_strides};
   for (int64_t* s : sets) { s[0] = s0; s[1] = s1; s[2] = s2; }
+  q.k_strides[0] = q.v_strides[0] = s0 / kvg;
   bool okc = true;
   if (no > 0) {
     okc &= cudaMemcpyAsync(ctx->hq.ptr, Q_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    okc &= cudaMemcpyAsync(ctx->hk.ptr, K_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    okc &= cudaMemcpyAsync(ctx->hk.ptr, K_host, tkv, cudaMemcpyHostToDevice, st) == cudaSuccess;
   }
-  okc &= cudaMemcpyAsync(ctx->hv.ptr, V_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  okc &= cudaMemcpyAsync(ctx->hv.ptr, V_host, tkv, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (bwd) okc &= cudaMemcpyAsync(ctx->hdo.ptr, dO_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (nf > 0 && prepare) {
     okc &= cudaMemcpyAsync(ctx->halpha.ptr, alpha_host, pb, cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -730,8 +745,8 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
   if (LSE_host) okc &= cudaMemcpyAsync(LSE_host, ctx->hlse.ptr, lb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   if (bwd) {
     if (dQ_host) okc &= cudaMemcpyAsync(dQ_host, ctx->hdq.ptr, gb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (dK_host) okc &= cudaMemcpyAsync(dK_host, ctx->hdk.ptr, gb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (dV_host) okc &= cudaMemcpyAsync(dV_host, ctx->hdv.ptr, gb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (dK_host) okc &= cudaMemcpyAsync(dK_host, ctx->hdk.ptr, gkv, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (dV_host) okc &= cudaMemcpyAsync(dV_host, ctx->hdv.ptr, gkv, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   }
   if (!okc) return SAF_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return SAF_ERR_CUDA;

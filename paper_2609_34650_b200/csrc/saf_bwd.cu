@@ -210,8 +210,8 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         if (!ok) return;
         TR(2, 31);
         mbar_expect_tx(kv_full + ks, 2 * C::PANEL);
-        tma_load_4d(smem + C::OFF_K + ks * C::PANEL, &mk, kv_full + ks, 0, w2.blk * BLK, w2.h, w2.b);
-        tma_load_4d(smem + C::OFF_V, &mv, kv_full + ks, 0, w2.blk * BLK, w2.h, w2.b);
+        tma_load_4d(smem + C::OFF_K + ks * C::PANEL, &mk, kv_full + ks, 0, w2.blk * BLK, w2.h / p.kv_group, w2.b);
+        tma_load_4d(smem + C::OFF_V, &mv, kv_full + ks, 0, w2.blk * BLK, w2.h / p.kv_group, w2.b);
         ++nkv;
       };
       load_next_kv();
@@ -811,11 +811,21 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         if (gtid == 0 && ok) {
           const CUtensorMap* m = grp == 0 ? &mdv : &mdk;
           const int first = ntile_ord & 1;              // dS^T buffer of the next ordinary tile
-          tma_store_4d(m, smem + C::OFF_DS + (2 * first + grp) * C::PANEL, 32 * first, w.blk * BLK, w.h, w.b);
-          bulk_commit_group();
-          tma_store_4d(m, smem + C::OFF_DS + (2 * (first ^ 1) + grp) * C::PANEL, 32 * (first ^ 1), w.blk * BLK, w.h,
-                       w.b);
-          bulk_commit_group();
+          const uint8_t* src0 = smem + C::OFF_DS + (2 * first + grp) * C::PANEL;
+          const uint8_t* src1 = smem + C::OFF_DS + (2 * (first ^ 1) + grp) * C::PANEL;
+          if (p.kv_group > 1) {
+            // grouped-query path: the query heads of a group add into their shared head's gradient
+            const int kvh = w.h / p.kv_group;
+            tma_reduce_add_4d(m, src0, 32 * first, w.blk * BLK, kvh, w.b);
+            bulk_commit_group();
+            tma_reduce_add_4d(m, src1, 32 * (first ^ 1), w.blk * BLK, kvh, w.b);
+            bulk_commit_group();
+          } else {
+            tma_store_4d(m, src0, 32 * first, w.blk * BLK, w.h, w.b);
+            bulk_commit_group();
+            tma_store_4d(m, src1, 32 * (first ^ 1), w.blk * BLK, w.h, w.b);
+            bulk_commit_group();
+          }
         }
         store_pending = 2;
       }

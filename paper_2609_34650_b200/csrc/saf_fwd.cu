@@ -164,7 +164,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             mbar_expect_tx(k_full + s, C::TILE_BYTES);
             for (int pn = 0; pn < C::NPANEL; ++pn)
               tma_load_4d(smem + C::OFF_K + s * C::TILE_BYTES + pn * C::PANEL_BYTES, &mk, k_full + s, pn * 64,
-                          j * BLK, w.h, w.b);
+                          j * BLK, w.h / p.kv_group, w.b);
             ++nk;
           }
           const int s = nv % C::NS;
@@ -173,7 +173,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           mbar_expect_tx(v_full + s, C::TILE_BYTES);
           for (int pn = 0; pn < C::NPANEL; ++pn)
             tma_load_4d(smem + C::OFF_V + s * C::TILE_BYTES + pn * C::PANEL_BYTES, &mv, v_full + s, pn * 64,
-                        j * BLK, w.h, w.b);
+                        j * BLK, w.h / p.kv_group, w.b);
           ++nv;
         }
       }

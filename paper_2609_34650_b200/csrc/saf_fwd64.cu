@@ -199,14 +199,14 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             ok = mbar_wait(k_empty + s, ((nk / C::NS) & 1) ^ 1, wc, F_K_EMPTY);
             if (!ok) break;
             mbar_expect_tx(k_full + s, C::TILE_BYTES);
-            tma_load_4d(smem + C::OFF_K + s * C::TILE_BYTES, &mk, k_full + s, 0, j * BLK, w.h, w.b);
+            tma_load_4d(smem + C::OFF_K + s * C::TILE_BYTES, &mk, k_full + s, 0, j * BLK, w.h / p.kv_group, w.b);
             ++nk;
           }
           const int s = nv % C::NS;
           ok = mbar_wait(v_empty + s, ((nv / C::NS) & 1) ^ 1, wc, F_V_EMPTY);
           if (!ok) break;
           mbar_expect_tx(v_full + s, C::TILE_BYTES);
-          tma_load_4d(smem + C::OFF_V + s * C::TILE_BYTES, &mv, v_full + s, 0, j * BLK, w.h, w.b);
+          tma_load_4d(smem + C::OFF_V + s * C::TILE_BYTES, &mv, v_full + s, 0, j * BLK, w.h / p.kv_group, w.b);
           ++nv;
         }
       }

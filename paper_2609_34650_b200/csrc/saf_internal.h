@@ -14,6 +14,7 @@ struct WorkItem { int32_t b, h, blk, kind; };
 
 struct FwdParams {
   int B, H, T, Tp;
+  int kv_group;                     // query heads per shared key/value head (>= 1)
   float scale_log2;                 // softmax_scale * log2(e)
   const float* alpha;               // [H][Tp]
   const float* rho;                 // [H][Tp]
@@ -40,6 +41,7 @@ struct FwdParams {
 
 struct BwdParams {
   int B, H, T, Tp;
+  int kv_group;                     // as in FwdParams; > 1: dK / dV are reduce-added instead of stored
   float scale, scale_log2;
   const float* alpha;
   const float* rho;
@@ -75,7 +77,7 @@ cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const fl
                                   void* band_b, cudaStream_t st);
 cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, float extra, int Tp,
                               const int* hlist, const int* pat_ok, int* ovf, int call_id, void* dst, int B, int Hf,
-                              int T, int D, cudaStream_t st);
+                              int T, int D, int src_group, cudaStream_t st);   // src head = h / src_group
 // powers of two that put the fp16 operands of the tensor-core frozen form into fp16's range
 constexpr float HK_BAND_SCALE = 16384.0f;        // bands hold 2^14 r
 constexpr float HK_A_SCALE = 2048.0f;            // the forward stages 2^11 a V
@@ -100,8 +102,8 @@ struct PrepFrozen {
 };
 cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* o_strides,
                             const uint8_t* mask_dev, void* q_ext, void* do_ext, float inv_scale, float* dQacc,
-                            void* dK, int grad_f32, const PrepFrozen& fz, int B, int H, int T, int D,
-                            cudaStream_t st);
+                            void* dK, void* dV, int grad_f32, int kv_group, const PrepFrozen& fz, int B, int H, int T,
+                            int D, cudaStream_t st);   // kv_group > 1: zeroes all of dK and dV (fp32) instead
 // dQ (grad dtype) = scale-free copy/convert of dQacc (fp32) for the bf16-gradient case.
 cudaError_t launch_bwd_finalize(const float* dQacc, void* dQ, size_t n, cudaStream_t st);
 // head dimension 64 (saf_fwd64.cu); launch_fwd dispatches to it

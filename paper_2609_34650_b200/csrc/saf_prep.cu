@@ -164,7 +164,7 @@ __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16
                                                              int Tp, const int* __restrict__ hlist,
                                                              const int* __restrict__ pat_ok, int* __restrict__ ovf,
                                                              int call_id, __half* __restrict__ dst, int B, int Hf,
-                                                             int T) {
+                                                             int T, int src_group) {
   constexpr int TPR = D / 8;
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
   const long long rowid = gid / TPR;               // over [B][Hf][T]: frozen heads only
@@ -176,7 +176,8 @@ __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16
   const int h = hlist[ord];
   if (!pat_ok[h]) return;
   const float f = vec[static_cast<size_t>(h) * Tp + t] * extra;
-  const uint4 v4 = *reinterpret_cast<const uint4*>(src + b * s0 + h * s1 + static_cast<int64_t>(t) * s2 + part * 8);
+  const uint4 v4 =
+      *reinterpret_cast<const uint4*>(src + b * s0 + (h / src_group) * s1 + static_cast<int64_t>(t) * s2 + part * 8);
   const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&v4);
   __half2 o[4];
   bool bad = false;
@@ -193,17 +194,17 @@ __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16
 
 cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, float extra, int Tp,
                               const int* hlist, const int* pat_ok, int* ovf, int call_id, void* dst, int B, int Hf,
-                              int T, int D, cudaStream_t st) {
+                              int T, int D, int src_group, cudaStream_t st) {
   const long long nthreads = static_cast<long long>(B) * Hf * T * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
   if (D == 64)
     saf_scale_rows_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
                                                     strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
-                                                    static_cast<__half*>(dst), B, Hf, T);
+                                                    static_cast<__half*>(dst), B, Hf, T, src_group);
   else
     saf_scale_rows_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
                                                      strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
-                                                     static_cast<__half*>(dst), B, Hf, T);
+                                                     static_cast<__half*>(dst), B, Hf, T, src_group);
   return cudaGetLastError();
 }
 
@@ -235,8 +236,9 @@ __global__ void __launch_bounds__(256) saf_bwd_prep_kernel(const __nv_bfloat16* 
                                                            int64_t os2, const uint8_t* __restrict__ mask,
                                                            uint8_t* __restrict__ q_ext, uint8_t* __restrict__ do_ext,
                                                            float inv_scale, float* __restrict__ dQacc,
-                                                           void* __restrict__ dK, int grad_f32, const PrepFrozen fz,
-                                                           int B, int H, int T) {
+                                                           void* __restrict__ dK, void* __restrict__ dV,
+                                                           int grad_f32, int kv_group, const PrepFrozen fz, int B,
+                                                           int H, int T) {
   constexpr int TPR = D / 8;                       // threads per row
   const int Tpad = (T + 127) / 128 * 128;
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
@@ -259,8 +261,18 @@ __global__ void __launch_bounds__(256) saf_bwd_prep_kernel(const __nv_bfloat16* 
     float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
     *reinterpret_cast<float4*>(dQacc + grow) = z;
     *reinterpret_cast<float4*>(dQacc + grow + 4) = z;
+    if (kv_group > 1 && h % kv_group == 0) {
+      // grouped-query path: the shared heads' gradients are accumulated by reduce-adds of the main kernel
+      const size_t krow = ((static_cast<size_t>(b) * (H / kv_group) + h / kv_group) * T + t) * D + part * 8;
+      *reinterpret_cast<float4*>(static_cast<float*>(dK) + krow) = z;
+      *reinterpret_cast<float4*>(static_cast<float*>(dK) + krow + 4) = z;
+      *reinterpret_cast<float4*>(static_cast<float*>(dV) + krow) = z;
+      *reinterpret_cast<float4*>(static_cast<float*>(dV) + krow + 4) = z;
+    }
     if (frozen) {
-      if (grad_f32) {
+      if (kv_group > 1) {
+        // nothing to zero per frozen head
+      } else if (grad_f32) {
         *reinterpret_cast<float4*>(static_cast<float*>(dK) + grow) = z;
         *reinterpret_cast<float4*>(static_cast<float*>(dK) + grow + 4) = z;
       } else {
@@ -321,8 +333,8 @@ __global__ void __launch_bounds__(256) saf_bwd_prep_kernel(const __nv_bfloat16* 
 }
 
 cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* os, const uint8_t* mask_dev,
-                            void* q_ext, void* do_ext, float inv_scale, float* dQacc, void* dK, int grad_f32,
-                            const PrepFrozen& fz, int B, int H, int T, int D, cudaStream_t st) {
+                            void* q_ext, void* do_ext, float inv_scale, float* dQacc, void* dK, void* dV, int grad_f32,
+                            int kv_group, const PrepFrozen& fz, int B, int H, int T, int D, cudaStream_t st) {
   const int Tpad = (T + 127) / 128 * 128;
   const long long nthreads = static_cast<long long>(B) * H * Tpad * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
@@ -330,12 +342,12 @@ cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, con
     saf_bwd_prep_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
                                                   static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2],
                                                   mask_dev, static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext),
-                                                  inv_scale, dQacc, dK, grad_f32, fz, B, H, T);
+                                                  inv_scale, dQacc, dK, dV, grad_f32, kv_group, fz, B, H, T);
   else
     saf_bwd_prep_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
                                                    static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2],
                                                    mask_dev, static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext),
-                                                   inv_scale, dQacc, dK, grad_f32, fz, B, H, T);
+                                                   inv_scale, dQacc, dK, dV, grad_f32, kv_group, fz, B, H, T);
   return cudaGetLastError();
 }
 

@@ -48,8 +48,10 @@ class Layer:
         self.O = torch.full_like(self.Q, float("nan"))
         self.LSE = torch.full((wl.B, wl.H, wl.T), float("nan"), device=dev)
         gd = torch.float32 if grad_dtype == saf.SAF_F32 else torch.bfloat16
-        self.grads = [torch.full(self.Q.shape, float("nan"), device=dev, dtype=gd) for _ in range(3)] if backward else None
-        self.prob = saf.make_problem(self.Q, wl.stored_len, softmax_scale=softmax_scale, grad_dtype=grad_dtype)
+        self.grads = [torch.full(t.shape, float("nan"), device=dev, dtype=gd)
+                      for t in (self.Q, self.K, self.V)] if backward else None
+        self.prob = saf.make_problem(self.Q, wl.stored_len, softmax_scale=softmax_scale, grad_dtype=grad_dtype,
+                                     k_like=self.K, v_like=self.V, kv_group=wl.kv_group)
         self.mask = inp.mask
 
     def run(self, backward=True, prepare=True):

@@ -260,6 +260,83 @@ def test_invalid_arguments_are_rejected():
     assert e.value.code == 1
 
 
+# --------------------------------------------------------------------------- grouped-query path
+def _check_gqa_layer(L, backward):
+    """Whole layer against the dense oracle: K, V (and dK, dV) have H / kv_group heads."""
+    inp, wl = L.inp, L.inp.wl
+    q, k, v, do = f64(inp)
+    O, LSE = L.host(L.O), L.host(L.LSE)
+    eO, eL = orc.hybrid_attn_fwd(q, k, v, inp.mask, inp.alpha.astype(np.float64), inp.rho.astype(np.float64))
+    for b in range(wl.B):
+        for h in range(wl.H):
+            assert_close(O[b, h], eO[b, h], f"O[{b},{h}]")
+            if inp.mask[h]:
+                assert not LSE[b, h].any()
+            else:
+                assert np.abs(LSE[b, h] - eL[b, h]).max() < 1e-4
+    if not backward:
+        return
+    dQ, dK, dV = (L.host(g) for g in L.grads)
+    eQ, eK, eV = orc.hybrid_attn_bwd(q, k, v, do, inp.mask, inp.alpha.astype(np.float64), inp.rho.astype(np.float64))
+    assert dK.shape == eK.shape and dV.shape == eV.shape
+    for b in range(wl.B):
+        for h in range(wl.H):
+            if inp.mask[h]:
+                assert not dQ[b, h].any(), "dQ of a frozen head must be exactly zero"
+            else:
+                assert_close(dQ[b, h], eQ[b, h], f"dQ[{b},{h}]")
+        for hk in range(wl.H // wl.kv_group):
+            assert_close(dK[b, hk], eK[b, hk], f"dK[{b},kv {hk}]")
+            # a shared head's dV sums kv_group heads: the absolute bound scales with the number of terms
+            assert_close(dV[b, hk], eV[b, hk], f"dV[{b},kv {hk}]", max_abs=MAX_ABS * np.sqrt(wl.kv_group))
+
+
+@pytest.mark.parametrize("H,g,frozen,T", [(8, 4, (1, 6), 300), (4, 2, (), 257), (6, 3, (0, 1, 2), 200),
+                                          (4, 4, (0, 1, 2, 3), 129), (4, 1, (2,), 130)])
+def test_gqa_shared_kv_heads_forward_backward(H, g, frozen, T):
+    """Query head h reads key/value head h // g; the shared heads' gradients sum over their query heads; a group
+    may be all ordinary, mixed or all frozen (then its dK is exactly zero)."""
+    wl = si.Workload("gqa", 2, H, T, 64, frozen, -0.05, seed=40 + H + g, kv_group=g)
+    L = Layer(si.generate(wl)).run()
+    _check_gqa_layer(L, True)
+    if g > 1 and len(frozen) == H:
+        assert not L.host(L.grads[1]).any()
+
+
+def test_gqa_head_dim_128_forward():
+    wl = si.Workload("gqa128", 1, 8, 384, 128, (2, 3), -0.02, seed=44, kv_group=4, backward=False)
+    L = Layer(si.generate(wl), backward=False).run(backward=False)
+    _check_gqa_layer(L, False)
+
+
+def test_gqa_qwen_like_geometry_sampled():
+    """32 query heads on 8 shared key/value heads, D = 128, forward only (the long-context geometry)."""
+    wl = si.Workload("gqa-qwen", 1, 32, 2048, 128, tuple(range(0, 32, 4)), -0.002, alpha0_spike=4.0, seed=45,
+                     kv_group=4, backward=False)
+    inp = si.generate(wl)
+    L = Layer(inp, backward=False).run(backward=False)
+    q, k, v, _ = f64(inp)
+    O = L.host(L.O)
+    for h in (0, 5, 31):
+        fr = bool(inp.mask[h])
+        eO, _ = orc.head_fwd_panels(fr, q[0, h], k[0, h // 4], v[0, h // 4], inp.alpha[h], inp.rho[h],
+                                    1.0 / np.sqrt(wl.D), 1024, None)
+        assert_close(O[0, h], eO, f"O[0,{h}] frozen={fr}")
+
+
+def test_gqa_backward_needs_fp32_gradients():
+    wl = si.Workload("gqa-bf16", 1, 4, 128, 64, (1,), -0.05, seed=46, kv_group=2)
+    L = Layer(si.generate(wl), grad_dtype=saf.SAF_BF16)
+    with pytest.raises(saf.SafError) as e:
+        L.run()
+    assert e.value.code == 2
+    L = Layer(si.generate(wl))
+    L.prob.kv_group = 3                        # does not divide H
+    with pytest.raises(saf.SafError) as e:
+        L.run()
+    assert e.value.code == 1
+
+
 # --------------------------------------------------------------------------- full sizes, sampled
 def test_config1_full_size_sampled_units():
     wl = si.config(1)
