@@ -19,6 +19,13 @@ serve as library steps; there is no online softmax, no key blocking, no factoris
                     dV = A^T dO, dP = dO V^T, delta_i = sum_j A_ij dP_ij, dS = A o (dP - delta),
                     dQ = scale dS K, dK = scale dS^T Q.
 
+* pattern gradients - the control in which the compact patterns stay trainable (Appendix, trainable-pattern
+                    ablation) differentiates the same definition: with the bias b_ij = alpha(j) + rho(i-j),
+                    P^ = softmax_causal(b) and L = sum(O o dO), G = dO V^T,
+                    dL/db_ij = P^_ij (G_ij - sum_k P^_ik G_ik), dL/dalpha(j) = sum_{i>=j} dL/db_ij,
+                    dL/drho(d) = sum_{i-j=d} dL/db_ij.  The paper prints no formula for it; this is the
+                    derivative of Eq. "compact-prior" written out.
+
 Parity status: every function below is pinned by tests that do not go through this file's own
 formulas (pure-Python brute force on tiny inputs, closed forms, shift invariance, the engineered
 ordinary-head equivalence, torch's fp64 scaled_dot_product_attention + autograd, finite
@@ -106,6 +113,34 @@ def frozen_head_bwd(dO, alpha, rho):
     """dV = P^T dO; a frozen head has no query/key gradients."""
     P = pattern_dense(alpha, rho, dO.shape[0])
     return P.T @ dO
+
+
+def pattern_grads_head(V, dO, alpha, rho):
+    """Gradients of L = sum(O o dO), O = P^ V, with respect to alpha[0..T) and rho[0..T) of one head
+    (V, dO: [T,D] float64).  Dense: the T x T matrices P^, G = dO V^T and dL/db are formed whole."""
+    T = V.shape[0]
+    P = pattern_dense(alpha, rho, T)
+    G = dO @ V.T
+    db = P * (G - (P * G).sum(axis=1, keepdims=True))       # softmax Jacobian applied row by row
+    dalpha = db.sum(axis=0)                                  # alpha(j) enters every row i >= j at column j
+    drho = np.array([np.trace(db, offset=-d) for d in range(T)])   # rho(d) enters the entries with i - j = d
+    return dalpha, drho
+
+
+def pattern_grads(V, dO, mask, alpha, rho):
+    """dalpha, drho [H,Tp] summed over the batch; rows of ordinary heads and entries beyond T are zero.
+    V: [B,Hkv,T,D] (head h reads V[:, h // (H/Hkv)]), dO: [B,H,T,D]."""
+    B, H, T, _ = dO.shape
+    g = H // V.shape[1]
+    Tp = alpha.shape[1]
+    dalpha, drho = np.zeros((H, Tp)), np.zeros((H, Tp))
+    for h in range(H):
+        if mask[h]:
+            for b in range(B):
+                da, dr = pattern_grads_head(V[b, h // g], dO[b, h], alpha[h], rho[h])
+                dalpha[h, :T] += da
+                drho[h, :T] += dr
+    return dalpha, drho
 
 
 # ----------------------------------------------------------------------------- the layer

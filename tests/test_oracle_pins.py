@@ -17,6 +17,9 @@ off-by-one in the relative distance or the causal boundary):
   P9  grouped-query path (Appendix E.2): shared key/value heads == the multi-head layer on K, V repeated per
       query head, with the shared heads' gradients summed over their query heads (torch autograd through
       repeat_interleave; torch's own enable_gqa route for the all-ordinary case; finite differences)
+  P10 pattern gradients (trainable-pattern control): central finite differences of sum(O o dO) through the
+      layer's own forward, torch autograd through a causal softmax of the bias matrix, and the two zero-sum
+      identities that shift invariance forces (sum_j dalpha(j) = 0, sum_d drho(d) = 0)
 """
 import math
 
@@ -405,3 +408,54 @@ def test_p9_gqa_finite_differences_of_shared_heads():
             am[idx] -= h
             fd = (loss(ap, V) - loss(am, V)) / (2 * h) if which == 0 else (loss(K, ap) - loss(K, am)) / (2 * h)
             assert abs(fd - grad[idx]) < 1e-7
+
+
+# ------------------------------------------------------------------ P10 pattern gradients
+def test_p10_pattern_grads_vs_torch_autograd():
+    B, H, T, D, Tp = 2, 4, 19, 5, 24
+    rng = np.random.default_rng(100)
+    V = rng.standard_normal((B, H // 2, T, D))             # shared value heads (group of 2)
+    dO = rng.standard_normal((B, H, T, D))
+    mask = np.array([1, 0, 1, 1], dtype=np.uint8)
+    alpha, rho = rng.standard_normal((H, Tp)), rng.standard_normal((H, Tp))
+    da, dr = orc.pattern_grads(V, dO, mask, alpha, rho)
+    ta, tr = torch.tensor(alpha, requires_grad=True), torch.tensor(rho, requires_grad=True)
+    i, j = np.indices((T, T))
+    causal = torch.tril(torch.ones(T, T, dtype=torch.bool))
+    loss = 0.0
+    for h in range(H):
+        if not mask[h]:
+            continue
+        bias = ta[h][torch.tensor(j)] + tr[h][torch.tensor(np.clip(i - j, 0, None))]
+        w = torch.softmax(bias.masked_fill(~causal, -math.inf), dim=-1)
+        for b in range(B):
+            loss = loss + ((w @ torch.tensor(V[b, h // 2])) * torch.tensor(dO[b, h])).sum()
+    loss.backward()
+    assert np.abs(da - ta.grad.numpy()).max() < 1e-11
+    assert np.abs(dr - tr.grad.numpy()).max() < 1e-11
+    assert not da[1].any() and not dr[1].any() and not da[:, T:].any() and not dr[:, T:].any()
+
+
+def test_p10_pattern_grads_finite_differences_and_zero_sums():
+    T, D = 11, 4
+    rng = np.random.default_rng(101)
+    V, dO = rng.standard_normal((T, D)), rng.standard_normal((T, D))
+    alpha, rho = rng.standard_normal(T), rng.standard_normal(T)
+    da, dr = orc.pattern_grads_head(V, dO, alpha, rho)
+
+    def loss(a, r):
+        O, _ = orc.frozen_head_fwd(V, a, r)
+        return float((O * dO).sum())
+
+    h = 1e-6
+    for k in range(T):
+        e = np.zeros(T)
+        e[k] = h
+        assert abs((loss(alpha + e, rho) - loss(alpha - e, rho)) / (2 * h) - da[k]) < 1e-7
+        assert abs((loss(alpha, rho + e) - loss(alpha, rho - e)) / (2 * h) - dr[k]) < 1e-7
+    # P^ does not change when a constant is added to all of alpha, or to all of rho (Appendix E.1)
+    assert abs(da.sum()) < 1e-12 and abs(dr.sum()) < 1e-12
+    # the last distance is reached by one entry only: (i, j) = (T-1, 0)
+    P = orc.pattern_dense(alpha, rho, T)
+    G = dO @ V.T
+    assert abs(dr[T - 1] - P[T - 1, 0] * (G[T - 1, 0] - (P[T - 1] * G[T - 1]).sum())) < 1e-13
