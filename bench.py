@@ -257,6 +257,21 @@ def run_ours(args):
     if code != saf.SAF_OK:
         raise RuntimeError(f"device status {code} detail {detail:#x}")
 
+    # optional extra outside the headline: gradients of the compact patterns (trainable-pattern control)
+    pgrad_ms = None
+    if len(wl.frozen_heads):
+        da, dr = torch.empty_like(alpha), torch.empty_like(alpha)
+        for _ in range(3):
+            ctx.saf_pattern_grad(prob, V, O, dO, mask, alpha, rho, logZ, da, dr)
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(10):
+            ctx.saf_pattern_grad(prob, V, O, dO, mask, alpha, rho, logZ, da, dr)
+        b.record()
+        torch.cuda.synchronize()
+        pgrad_ms = a.elapsed_time(b) / 10
+
     flops_local = wl.flops()
     rate, ms = sd.whole_job_rate(flops_local * 1.0, ms_local, dev)       # FLOP per step over all ranks / max ms
     value = rate / 1e12
@@ -352,7 +367,7 @@ def run_ours(args):
                    "parallelism": f"dp{world} (independent batches, no collective in the layer)"},
         "pct_of_bf16_peak": 100.0 * value / (peaks["bf16_tflops"] * world),
         "speedup_vs_0pct_frozen": speedup, "aa_control": aa_control,
-        "ms_0pct_frozen": 0.5 * (b1 + b2), "ms_fwd_only": fwd_only,
+        "ms_0pct_frozen": 0.5 * (b1 + b2), "ms_fwd_only": fwd_only, "ms_pattern_grad": pgrad_ms,
         "e2e": {"value": e2e_rate / 1e12, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
         # per step: V scaling + forward kernel, dO scaling + backward preparation + backward kernel

@@ -130,6 +130,19 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
                               const float* alpha_host, const float* rho_host, int32_t prepare, void* O_host,
                               float* LSE_host, void* dQ_host, void* dK_host, void* dV_host);
 
+/* Gradients of the compact patterns of the frozen heads, for the control in which alpha and rho stay trainable
+ * (appendix on pattern controls; the paper prints no formula, this is the derivative of Eq. "compact-prior").
+ * With b_ij = alpha(j) + rho(i-j), P^ = softmax_causal(b), O = P^ V and L = sum(O o dO):
+ *   G = dO V^T,  dL/db_ij = P^_ij (G_ij - dO_i . O_i),
+ *   dalpha_out[h][j] = sum_b sum_{i>=j} dL/db_ij,   drho_out[h][d] = sum_b sum_{i-j=d} dL/db_ij.
+ * V: bf16 [B][H/kv_group][T][D] (v_strides); O, dO: bf16 [B][H][T][D] (o_strides), O as returned by the forward;
+ * alpha, rho, logZ: device fp32 [H][Tp] (logZ as from saf_pattern_prepare); dalpha_out, drho_out: device fp32
+ * [H][Tp], fully overwritten (rows of ordinary heads and entries beyond T with zeros).  D in {64, 128}.
+ * After an update of alpha/rho the caller refreshes logZ with saf_pattern_prepare. */
+int saf_pattern_grad(saf_ctx* ctx, const saf_problem* problem, const void* V, const void* O, const void* dO,
+                     const uint8_t* frozen_mask_host, const float* alpha, const float* rho, const float* logZ,
+                     float* dalpha_out, float* drho_out, void* stream);
+
 /* Device-side status of the most recent launches on this context: SAF_OK or SAF_ERR_DEVICE_TIMEOUT.
  * Synchronises the context's device status word with the host (blocks until the stream used by the
  * last call has drained).  `detail_out` (may be NULL) receives the raw word: site and CTA that gave up. */
@@ -146,7 +159,8 @@ enum {
   SAF_KERNEL_BWD_FINALIZE = 3, /* fp32 -> bf16 conversion of dQ (bf16 gradients only) */
   SAF_KERNEL_LOGZ = 4,         /* pattern normalisers and tables (saf_pattern_prepare) */
   SAF_KERNEL_SCALE = 5,        /* per-call row scaling of the frozen heads' V (forward) / dO (backward) */
-  SAF_KERNEL_COUNT = 6
+  SAF_KERNEL_PGRAD = 6,        /* pattern-gradient kernel (saf_pattern_grad) */
+  SAF_KERNEL_COUNT = 7
 };
 int saf_set_profiling(saf_ctx* ctx, int32_t enable);
 int saf_get_kernel_time(saf_ctx* ctx, int32_t which, float* total_ms_out, int32_t* launches_out);

@@ -55,6 +55,7 @@ def load_library() -> C.CDLL:
     lib.saf_hybrid_attn_fwd.argtypes = [vp, pp, vp, vp, vp, u8p, f32p, f32p, f32p, vp, f32p, vp]
     lib.saf_hybrid_attn_bwd.argtypes = [vp, pp, vp, vp, vp, vp, vp, f32p, u8p, f32p, f32p, f32p, vp, vp, vp, vp]
     lib.saf_hybrid_attn_step_host.argtypes = [vp, pp, vp, vp, vp, vp, u8p, f32p, f32p, i32, vp, f32p, vp, vp, vp]
+    lib.saf_pattern_grad.argtypes = [vp, pp, vp, vp, vp, u8p, f32p, f32p, f32p, f32p, f32p, vp]
     lib.saf_last_device_status.argtypes = [vp, C.POINTER(C.c_int32)]
     lib.saf_set_profiling.argtypes = [vp, i32]
     lib.saf_get_kernel_time.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
@@ -63,7 +64,7 @@ def load_library() -> C.CDLL:
     lib.saf_build_worklist.argtypes = [i32, i32, i32, u8p, i32, i32, i32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     for name in ("saf_create", "saf_destroy", "saf_pattern_prepare", "saf_hybrid_attn_fwd", "saf_hybrid_attn_bwd",
                  "saf_hybrid_attn_step_host", "saf_last_device_status", "saf_build_worklist", "saf_set_profiling",
-                 "saf_get_kernel_time"):
+                 "saf_get_kernel_time", "saf_pattern_grad"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -172,6 +173,12 @@ class Context:
         _check(self._lib.saf_hybrid_attn_bwd(self._h, C.byref(prob), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO),
                                              _ptr(LSE), mp, _ptr(alpha), _ptr(rho), _ptr(logZ), _ptr(dQ), _ptr(dK),
                                              _ptr(dV), _stream()), "saf_hybrid_attn_bwd")
+
+    def saf_pattern_grad(self, prob, V, O, dO, mask, alpha, rho, logZ, dalpha, drho):
+        m, mp = _mask_ptr(mask)
+        _check(self._lib.saf_pattern_grad(self._h, C.byref(prob), _ptr(V), _ptr(O), _ptr(dO), mp, _ptr(alpha),
+                                          _ptr(rho), _ptr(logZ), _ptr(dalpha), _ptr(drho), _stream()),
+               "saf_pattern_grad")
 
     def saf_hybrid_attn_step_host(self, prob, Q, K, V, dO, mask, alpha, rho, prepare, O, LSE, dQ, dK, dV):
         """All tensor arguments are HOST tensors (torch CPU tensors, ideally pinned) or None."""

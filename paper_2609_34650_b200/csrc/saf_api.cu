@@ -65,7 +65,7 @@ struct saf_ctx {
   // tensor-core form of frozen heads: tables built by saf_pattern_prepare, scaled V / dO per call
   PatternCache pat;
   bool tensor_pattern = true;              // SAF_DISABLE_TENSOR_PATTERN=1 turns the form off
-  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, vt_buf, dot_buf, ok_fwd, ok_bwd;
+  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, vt_buf, dot_buf, ok_fwd, ok_bwd, pg_hlist, pg_delta;
   bool profiling = false;
   std::vector<TimedLaunch> timed;          // event pairs recorded since the last query
   std::vector<cudaEvent_t> event_pool;
@@ -357,7 +357,7 @@ int saf_destroy(saf_ctx* ctx) {
     cudaFree(e.offsets_dev);
   }
   DevBuf* pbufs[] = {&ctx->pat_consts, &ctx->pat_ok, &ctx->pat_avec, &ctx->pat_wvec, &ctx->pat_bandf, &ctx->pat_bandb,
-                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd};
+                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta};
   for (DevBuf* b : pbufs) release(*b);
   DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->hq, &ctx->hk, &ctx->hv,
                     &ctx->hdo, &ctx->ho, &ctx->hlse, &ctx->hdq, &ctx->hdk, &ctx->hdv, &ctx->halpha, &ctx->hrho,
@@ -751,6 +751,72 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
   if (!okc) return SAF_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return SAF_ERR_CUDA;
   return saf_last_device_status(ctx, nullptr);
+}
+
+int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const void* O, const void* dO,
+                     const uint8_t* frozen_mask_host, const float* alpha, const float* rho, const float* logZ,
+                     float* dalpha_out, float* drho_out, void* stream) {
+  if (!ctx || !dalpha_out || !drho_out) return SAF_ERR_INVALID_ARG;
+  int nf = 0;
+  int rc = validate(p, frozen_mask_host, &nf);
+  if (rc) return rc;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ctx->last_stream = st;
+  const size_t pbytes = static_cast<size_t>(p->H) * p->Tp * sizeof(float);
+  if (cudaMemsetAsync(dalpha_out, 0, pbytes, st) != cudaSuccess || cudaMemsetAsync(drho_out, 0, pbytes, st) != cudaSuccess)
+    return SAF_ERR_CUDA;
+  if (nf == 0) return SAF_OK;
+  if (!V || !O || !dO || !alpha || !rho || !logZ) return SAF_ERR_INVALID_ARG;
+  if (!aligned16(V) || !aligned16(O) || !aligned16(dO)) return SAF_ERR_INVALID_ARG;
+  if (check_strides(p->v_strides, p->D) || check_strides(p->o_strides, p->D)) return SAF_ERR_INVALID_ARG;
+  const int kvg = kv_group_of(p);
+  // ordinal -> head table of the frozen heads, and delta = rowsum(dO o O) of their rows
+  std::vector<int> hlist;
+  for (int h = 0; h < p->H; ++h)
+    if (frozen_mask_host[h]) hlist.push_back(h);
+  if ((rc = ensure(ctx->pg_hlist, static_cast<size_t>(p->H) * sizeof(int))) ||
+      (rc = ensure(ctx->pg_delta, static_cast<size_t>(p->B) * p->H * p->T * sizeof(float))))
+    return rc;
+  // (synchronous copy from pageable memory: the vector dies at the end of this call)
+  if (cudaStreamSynchronize(st) != cudaSuccess ||
+      cudaMemcpy(ctx->pg_hlist.ptr, hlist.data(), hlist.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
+    return SAF_ERR_CUDA;
+  {
+    ScopedTimer timer(ctx, SAF_KERNEL_BWD_PREP, st);
+    if (launch_rowdot(O, dO, p->o_strides, static_cast<const int*>(ctx->pg_hlist.ptr),
+                      static_cast<float*>(ctx->pg_delta.ptr), p->B, p->H, nf, p->T, p->D, st) != cudaSuccess)
+      return SAF_ERR_CUDA;
+  }
+  // work list over (batch, frozen-head ordinal, key block), all of one kind
+  const int nblk = (p->T + BLK - 1) / BLK;
+  const long long n_items = static_cast<long long>(p->B) * nf * nblk;
+  const int grid = static_cast<int>(std::min<long long>(2LL * ctx->num_sms, n_items));
+  std::vector<uint8_t> none(nf, 0);
+  const WorklistEntry* wl = nullptr;
+  rc = get_worklist(ctx, p->B, nf, p->T, none.data(), 1, grid, st, &wl);
+  if (rc) return rc;
+  CUtensorMap mv, mdo;
+  if ((rc = make_map(ctx, &mv, V, p, p->v_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg))) return rc;
+  if ((rc = make_map(ctx, &mdo, dO, p, p->o_strides))) return rc;
+  PgradParams gp;
+  gp.B = p->B; gp.H = p->H; gp.T = p->T; gp.Tp = p->Tp;
+  gp.kv_group = kvg;
+  gp.alpha = alpha; gp.rho = rho; gp.logZ = logZ;
+  gp.delta = static_cast<const float*>(ctx->pg_delta.ptr);
+  gp.hlist = static_cast<const int*>(ctx->pg_hlist.ptr);
+  gp.dalpha = dalpha_out;
+  gp.drho = drho_out;
+  gp.items = wl->items_dev;
+  gp.cta_offsets = wl->offsets_dev;
+  gp.status = ctx->status_dev;
+  gp.wait_limit_ns = ctx->wait_limit_ns;
+  {
+    ScopedTimer timer(ctx, SAF_KERNEL_PGRAD, st);
+    if (launch_pgrad(p->D, mv, mdo, gp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+  }
+  return SAF_OK;
 }
 
 int saf_last_device_status(saf_ctx* ctx, int32_t* detail_out) {

@@ -69,6 +69,27 @@ struct BwdParams {
   unsigned long long wait_limit_ns;
 };
 
+// Gradients of the compact patterns (saf_pgrad.cu).  Items carry the head's ordinal among the frozen heads.
+struct PgradParams {
+  int B, H, T, Tp;
+  int kv_group;
+  const float* alpha;               // [H][Tp]
+  const float* rho;
+  const float* logZ;
+  const float* delta;               // [B][H][T]: rowsum(dO o O), rows of frozen heads only
+  const int* hlist;                 // ordinal -> head
+  float* dalpha;                    // [H][Tp], zeroed before the launch; accumulated with atomicAdd
+  float* drho;
+  const WorkItem* items;
+  const int* cta_offsets;
+  int* status;
+  unsigned long long wait_limit_ns;
+};
+cudaError_t launch_rowdot(const void* O, const void* dO, const int64_t* o_strides, const int* hlist, float* delta,
+                          int B, int H, int Hf, int T, int D, cudaStream_t st);
+cudaError_t launch_pgrad(int D, const CUtensorMap& mv, const CUtensorMap& mdo, const PgradParams& p, int grid,
+                         cudaStream_t st);
+
 // Launchers (defined in the .cu files).  All return the launch error.
 cudaError_t launch_logz(const float* alpha, const float* rho, float* logZ, const uint8_t* mask_dev, int H,
                         int Tp, cudaStream_t st);
