@@ -77,7 +77,11 @@ struct BwdCfg {
   // per compute group: wq[128] z2s[128] rband[256] r2raw[256] red[16]
   static constexpr int TAB_FLOATS = 128 * 2 + 256 * 2 + 16;
   static constexpr int OFF_BAR = OFF_TAB + 2 * TAB_FLOATS * 4;
-  static constexpr int NBAR = 4 + 2 * NS + 2 + 2 + 4 + 2 + 1;
+  // slot k of the tensor-core frozen ring
+  __host__ __device__ static constexpr int fz_do(int k) { return (k < 2 ? OFF_DO : OFF_Q) + (k & 1) * PANEL; }
+  __host__ __device__ static constexpr int fz_band(int k) { return (k < 2 ? OFF_QX : OFF_DOX) + (k & 1) * 4096; }
+  static constexpr int NFZ = 4;                       // ring depth of the tensor-core frozen form (see the producer)
+  static constexpr int NBAR = 4 + 2 * NS + 2 + 2 + 4 + 2 + 1 + 2 * NFZ;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
   static constexpr int TMEM_COLS = 512;
   static constexpr int COL_DV = 0, COL_DK = 64, COL_S = 128, COL_DP = 256, COL_DQ = 384, COL_KT = 448, COL_VT = 480;
@@ -134,7 +138,9 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   uint64_t* acc_free = acc_full + 1;
   uint64_t* pfree = acc_free + 1;                // [2]
   uint64_t* kvt_full = pfree + 2;                // K_J / V_J have been copied into TMEM
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(kvt_full + 1);
+  uint64_t* fz_full = kvt_full + 1;              // [NFZ] band + scaled dO tile of a tensor-core frozen tile
+  uint64_t* fz_empty = fz_full + C::NFZ;         // [NFZ]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fz_empty + C::NFZ);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -157,6 +163,10 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       mbar_init(pfree + b, 1);
     }
     mbar_init(kvt_full, 16);
+    for (int k = 0; k < C::NFZ; ++k) {
+      mbar_init(fz_full + k, 1);
+      mbar_init(fz_empty + k, 1);
+    }
     mbar_init(dq_full, 1);
     mbar_init(dq_free, 4);
     mbar_init(acc_full, 1);
@@ -192,8 +202,8 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       tma_prefetch_desc(&mv);
       tma_prefetch_desc(&mdo);
       tma_prefetch_desc(&mdot);
-      uint32_t nkv = 0, nqdo = 0;
-      bool ok = true;
+      uint32_t nkv = 0, nqdo = 0, nfz = 0;
+      bool ok = true, fz_open = false;
       int tr_n = 0;
       (void)tr_n;
       // K_J / V_J of the ordinary items run one item ahead of the tile loads: K into the other K slot (free
@@ -221,19 +231,36 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         const size_t bh = static_cast<size_t>(w.b) * p.H + w.h;
         const bool fast = !ord && p.band_b != nullptr && p.fast_ok[w.h] != 0 && p.ovf[w.h] != p.call_id;
         if (fast) {
-          // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled dO tile
+          // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled dO tile.  These
+          // tiles have no compute step to hide the load latency behind, so they run a ring of their own, four
+          // deep, laid over the idle Q/dO stages and row-term images: slot k keeps its dO tile in dO stage k
+          // (k < 2) or Q stage k-2, its band in the Q (k < 2) or dO row-term image of stage k & 1.
+          if (!fz_open) {
+            // the stages' last ordinary / general tiles must have been consumed
+            for (uint32_t n = nqdo > 1 ? nqdo - 2 : 0; n < nqdo && ok; ++n)
+              ok = mbar_wait(qdo_empty + n % C::NS, (n / C::NS) & 1, wc, B_QDO_EMPTY);
+            if (!ok) break;
+            fz_open = true;
+          }
           const int fo = p.hord[w.h];
           const uint8_t* bands = static_cast<const uint8_t*>(p.band_b) + static_cast<size_t>(w.h) * p.nblkp * 4096;
           for (int I = w.blk; I < nblk; ++I) {
-            const int s = nqdo % C::NS;
-            ok = mbar_wait(qdo_empty + s, ((nqdo / C::NS) & 1) ^ 1, wc, B_QDO_EMPTY);
+            const uint32_t k = nfz % C::NFZ;
+            ok = mbar_wait(fz_empty + k, ((nfz / C::NFZ) & 1) ^ 1, wc, B_QDO_EMPTY);
             if (!ok) break;
-            mbar_expect_tx(qdo_full + s, C::PANEL + 4096);
-            bulk_load(smem + C::OFF_QX + s * 4096, bands + static_cast<size_t>(I - w.blk) * 4096, 4096, qdo_full + s);
-            tma_load_4d(smem + C::OFF_DO + s * C::PANEL, &mdot, qdo_full + s, 0, I * BLK, fo, w.b);
-            ++nqdo;
+            mbar_expect_tx(fz_full + k, C::PANEL + 4096);
+            bulk_load(smem + C::fz_band(k), bands + static_cast<size_t>(I - w.blk) * 4096, 4096, fz_full + k);
+            tma_load_4d(smem + C::fz_do(k), &mdot, fz_full + k, 0, I * BLK, fo, w.b);
+            ++nfz;
           }
           continue;
+        }
+        if (fz_open) {
+          // back to the shared stages: the frozen ring's tiles in flight must have been consumed
+          for (uint32_t n = nfz > C::NFZ ? nfz - C::NFZ : 0; n < nfz && ok; ++n)
+            ok = mbar_wait(fz_empty + n % C::NFZ, (n / C::NFZ) & 1, wc, B_QDO_EMPTY);
+          if (!ok) break;
+          fz_open = false;
         }
         for (int I = w.blk; I < nblk; ++I) {
           const int s = nqdo % C::NS;
@@ -275,7 +302,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     const uint32_t lo_k = desc_lo(d_k), hi_k = desc_hi(d_k), lo_x = desc_lo(d_x), hi_x = desc_hi(d_x);
     const uint32_t lo_m = desc_lo(d_m), hi_m = desc_hi(d_m);
     const uint32_t ones_lo = lo_x + (C::OFF_ONES >> 4);
-    uint32_t nqdo = 0, nitem = 0, ndq = 0, ntile_ord = 0, nkv = 0;
+    uint32_t nqdo = 0, nitem = 0, ndq = 0, ntile_ord = 0, nkv = 0, nfz = 0;
     uint32_t npds0 = 0, npds1 = 0;
     int tr_n = 0;
     (void)tr_n;
@@ -399,23 +426,23 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         const uint64_t d_band = umma_smem_desc(sb, 128, 128, UMMA_LAYOUT_NONE);
         const uint32_t lo_b = desc_lo(d_band), hi_b = desc_hi(d_band);
         for (int t = 0; t < ntiles; ++t) {
-          const uint32_t s = nqdo % C::NS;
-          ok = mbar_wait_warp(qdo_full + s, (nqdo / C::NS) & 1, wc, B_QDO_FULL);
+          const uint32_t k = nfz % C::NFZ;
+          ok = mbar_wait_warp(fz_full + k, (nfz / C::NFZ) & 1, wc, B_QDO_FULL);
           if (!ok) break;
-          ++nqdo;
+          ++nfz;
           if (t == 0) {
             ok = mbar_wait_warp(acc_free, (nitem & 1) ^ 1, wc, B_ACC_FREE);
             if (!ok) break;
           }
           tc_fence_after();
-          const uint32_t band_lo = lo_b + ((C::OFF_QX + s * 4096) >> 4);
-          const uint32_t do_lo = lo_m + ((C::OFF_DO + s * C::PANEL) >> 4);
+          const uint32_t band_lo = lo_b + (static_cast<uint32_t>(C::fz_band(k)) >> 4);
+          const uint32_t do_lo = lo_m + (static_cast<uint32_t>(C::fz_do(k)) >> 4);
           const uint32_t acc0 = t > 0 ? 1u : 0u;
           if (leader) {
 #pragma unroll
             for (int kc = 0; kc < 8; ++kc)
               umma_ss2(tmem + C::COL_DV, band_lo + 16 * kc, hi_b, do_lo + 128 * kc, hi_m, id_hk, kc > 0 ? 1u : acc0);
-            umma_commit(qdo_empty + s);
+            umma_commit(fz_empty + k);
           }
           __syncwarp();
         }
