@@ -71,6 +71,9 @@ struct saf_ctx {
   std::vector<cudaEvent_t> event_pool;
   // staging for the host-buffer entry point
   DevBuf hq, hk, hv, hdo, ho, hlse, hdq, hdk, hdv, halpha, hrho, hlogz;
+  // host-buffer step: compute stream, copy stream and the events that order them
+  cudaStream_t hs_main = nullptr, hs_copy = nullptr;
+  cudaEvent_t hs_qkv = nullptr, hs_do = nullptr, hs_fwd = nullptr, hs_out = nullptr;
 };
 
 namespace {
@@ -364,6 +367,10 @@ int saf_destroy(saf_ctx* ctx) {
                     &ctx->hlogz};
   for (DevBuf* b : bufs) release(*b);
   if (ctx->status_dev) cudaFree(ctx->status_dev);
+  if (ctx->hs_main) cudaStreamDestroy(ctx->hs_main);
+  if (ctx->hs_copy) cudaStreamDestroy(ctx->hs_copy);
+  for (cudaEvent_t e : {ctx->hs_qkv, ctx->hs_do, ctx->hs_fwd, ctx->hs_out})
+    if (e) cudaEventDestroy(e);
   for (TimedLaunch& t : ctx->timed) {
     cudaEventDestroy(t.beg);
     cudaEventDestroy(t.end);
@@ -710,7 +717,16 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
   if (bwd && ((rc = ensure(ctx->hdo, tb)) || (rc = ensure(ctx->hdq, gb)) || (rc = ensure(ctx->hdk, gb)) ||
               (rc = ensure(ctx->hdv, gb))))
     return rc;
-  cudaStream_t st = nullptr;
+  // Two streams: the copy stream brings dO in while the forward runs and takes O / LSE out while the
+  // backward runs; everything else is on the compute stream.
+  if (!ctx->hs_main) {
+    if (cudaStreamCreateWithFlags(&ctx->hs_main, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&ctx->hs_copy, cudaStreamNonBlocking) != cudaSuccess)
+      return SAF_ERR_CUDA;
+    for (cudaEvent_t* e : {&ctx->hs_qkv, &ctx->hs_do, &ctx->hs_fwd, &ctx->hs_out})
+      if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return SAF_ERR_CUDA;
+  }
+  cudaStream_t st = ctx->hs_main, sc = ctx->hs_copy;
   saf_problem q = *p;
   const int64_t s2 = p->D, s1 = static_cast<int64_t>(p->T) * p->D, s0 = s1 * p->H;
   int64_t* sets[4] = {q.q_strides, q.k_strides, q.v_strides, q.o_strides};
@@ -722,10 +738,16 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
     okc &= cudaMemcpyAsync(ctx->hk.ptr, K_host, tkv, cudaMemcpyHostToDevice, st) == cudaSuccess;
   }
   okc &= cudaMemcpyAsync(ctx->hv.ptr, V_host, tkv, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (bwd) okc &= cudaMemcpyAsync(ctx->hdo.ptr, dO_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (nf > 0 && prepare) {
     okc &= cudaMemcpyAsync(ctx->halpha.ptr, alpha_host, pb, cudaMemcpyHostToDevice, st) == cudaSuccess;
     okc &= cudaMemcpyAsync(ctx->hrho.ptr, rho_host, pb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  if (bwd) {
+    // dO follows Q, K, V on the link, on the copy stream, so that the forward does not wait for it
+    okc &= cudaEventRecord(ctx->hs_qkv, st) == cudaSuccess;
+    okc &= cudaStreamWaitEvent(sc, ctx->hs_qkv, 0) == cudaSuccess;
+    okc &= cudaMemcpyAsync(ctx->hdo.ptr, dO_host, tb, cudaMemcpyHostToDevice, sc) == cudaSuccess;
+    okc &= cudaEventRecord(ctx->hs_do, sc) == cudaSuccess;
   }
   if (!okc) return SAF_ERR_CUDA;
   const float* a = static_cast<const float*>(ctx->halpha.ptr);
@@ -735,21 +757,27 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
   rc = saf_hybrid_attn_fwd(ctx, &q, ctx->hq.ptr, ctx->hk.ptr, ctx->hv.ptr, frozen_mask_host, a, r, z, ctx->ho.ptr,
                            static_cast<float*>(ctx->hlse.ptr), st);
   if (rc) return rc;
+  // O and LSE leave on the copy stream as soon as the forward is done
+  okc &= cudaEventRecord(ctx->hs_fwd, st) == cudaSuccess;
+  okc &= cudaStreamWaitEvent(sc, ctx->hs_fwd, 0) == cudaSuccess;
+  if (O_host) okc &= cudaMemcpyAsync(O_host, ctx->ho.ptr, tb, cudaMemcpyDeviceToHost, sc) == cudaSuccess;
+  if (LSE_host) okc &= cudaMemcpyAsync(LSE_host, ctx->hlse.ptr, lb, cudaMemcpyDeviceToHost, sc) == cudaSuccess;
+  okc &= cudaEventRecord(ctx->hs_out, sc) == cudaSuccess;
+  if (!okc) return SAF_ERR_CUDA;
   if (bwd) {
+    if (cudaStreamWaitEvent(st, ctx->hs_do, 0) != cudaSuccess) return SAF_ERR_CUDA;
     rc = saf_hybrid_attn_bwd(ctx, &q, ctx->hq.ptr, ctx->hk.ptr, ctx->hv.ptr, ctx->ho.ptr, ctx->hdo.ptr,
                              static_cast<const float*>(ctx->hlse.ptr), frozen_mask_host, a, r, z, ctx->hdq.ptr,
                              ctx->hdk.ptr, ctx->hdv.ptr, st);
     if (rc) return rc;
   }
-  if (O_host) okc &= cudaMemcpyAsync(O_host, ctx->ho.ptr, tb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (LSE_host) okc &= cudaMemcpyAsync(LSE_host, ctx->hlse.ptr, lb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   if (bwd) {
     if (dQ_host) okc &= cudaMemcpyAsync(dQ_host, ctx->hdq.ptr, gb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     if (dK_host) okc &= cudaMemcpyAsync(dK_host, ctx->hdk.ptr, gkv, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     if (dV_host) okc &= cudaMemcpyAsync(dV_host, ctx->hdv.ptr, gkv, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   }
   if (!okc) return SAF_ERR_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return SAF_ERR_CUDA;
+  if (cudaStreamSynchronize(sc) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return SAF_ERR_CUDA;
   return saf_last_device_status(ctx, nullptr);
 }
 
