@@ -51,9 +51,9 @@ struct FwdCfg {
   static constexpr int TMEM_COLS = 256;
   static constexpr int COL_S = 0, COL_P = 0, COL_O = 128;
   static constexpr int NTHREADS = 320;
-  // D = 64: a thread keeps its 64 scores in registers between the max and the exp pass;
-  // D = 128: the wider O row costs registers, so the scores are read from TMEM twice instead.
-  static constexpr bool SCORES_IN_REGS = (D == 64);
+  // A thread keeps its 64 scores in registers between the max and the exp pass (reading them from TMEM
+  // twice instead measured almost twice as slow at D = 128).
+  static constexpr bool SCORES_IN_REGS = true;
 };
 
 enum FwdSite { SITE_Q_EMPTY = 1, SITE_K_EMPTY, SITE_V_EMPTY, SITE_Q_FULL, SITE_K_FULL, SITE_P_FULL, SITE_V_FULL,
