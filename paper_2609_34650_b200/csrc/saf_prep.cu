@@ -230,7 +230,7 @@ __device__ __forceinline__ uint4 split3_bf16(float x) {
 //   frozen head  : dK row = 0 (no key gradient; Sec. 3.3); with the tensor-core form, the row w(i) dO in fp16
 // Image layout per 128-row block (4 KB): byte (n/8)*256 + (k/8)*128 + (n%8)*16 + (k%8)*2 for row n, column k < 16.
 template <int D>
-__global__ void __launch_bounds__(256) saf_bwd_prep_kernel(const __nv_bfloat16* __restrict__ O,
+__global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat16* __restrict__ O,
                                                            const __nv_bfloat16* __restrict__ dO,
                                                            const float* __restrict__ LSE, int64_t os0, int64_t os1,
                                                            int64_t os2, const uint8_t* __restrict__ mask,
