@@ -81,7 +81,7 @@ struct BwdCfg {
   __host__ __device__ static constexpr int fz_do(int k) { return (k < 2 ? OFF_DO : OFF_Q) + (k & 1) * PANEL; }
   __host__ __device__ static constexpr int fz_band(int k) { return (k < 2 ? OFF_QX : OFF_DOX) + (k & 1) * 4096; }
   static constexpr int NFZ = 4;                       // ring depth of the tensor-core frozen form (see the producer)
-  static constexpr int NBAR = 4 + 2 * NS + 2 + 2 + 4 + 2 + 1 + 2 * NFZ;
+  static constexpr int NBAR = 4 + 2 * NS + 2 + 2 + 4 + 2 + 1 + 2 * NFZ + 2;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
   static constexpr int TMEM_COLS = 512;
   static constexpr int COL_DV = 0, COL_DK = 64, COL_S = 128, COL_DP = 256, COL_DQ = 384, COL_KT = 448, COL_VT = 480;
@@ -140,7 +140,8 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   uint64_t* kvt_full = pfree + 2;                // K_J / V_J have been copied into TMEM
   uint64_t* fz_full = kvt_full + 1;              // [NFZ] band + scaled dO tile of a tensor-core frozen tile
   uint64_t* fz_empty = fz_full + C::NFZ;         // [NFZ]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fz_empty + C::NFZ);
+  uint64_t* s_full = fz_empty + C::NFZ;          // [2] S'^T of buffer b is complete (dP'^T follows: sdp_full)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -159,6 +160,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(sdp_full + b, 1);
+      mbar_init(s_full + b, 1);
       mbar_init(pds_full + b, 8);                // one arrival per warp of the group
       mbar_init(pfree + b, 1);
     }
@@ -337,6 +339,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             for (int kc = 0; kc < 4; ++kc)
               umma_ts2(t_s, tmem + C::COL_KT + 8 * kc, q_lo + 2 * kc, hi_k, id_s, kc > 0);
             umma_ss2(t_s, ones_lo, hi_x, qx_lo, hi_x, id_s, 1);
+            umma_commit(s_full + b);                     // the exponentials start while dP'^T is computed
 #pragma unroll
             for (int kc = 0; kc < 4; ++kc)
               umma_ts2(t_dp, tmem + C::COL_VT + 8 * kc, do_lo + 2 * kc, hi_k, id_s, kc > 0);
@@ -629,38 +632,49 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         for (int t = 0; t < ntiles; ++t) {
           // this group's half tile of tile t: queries 64*grp .. 64*grp+63; this warp's 32 of them
           TR(4 + warp, 11);
-          if (!mbar_wait_warp(sdp_full + grp, nsdp & 1, wc, B_SDP_FULL)) ok = false;
-          ++nsdp;
+          if (!mbar_wait_warp(s_full + grp, nsdp & 1, wc, B_SDP_FULL)) ok = false;
           tc_fence_after();
-          if (t <= 1) staging_free(1 - t);
           TR(4 + warp, 12);
           const uint32_t t_s = tmem + lane_base + C::COL_S + 64 * grp;
           const uint32_t t_dp = tmem + lane_base + C::COL_DP + 64 * grp;
           const uint32_t rowaddr =
               smem_u32(smem + C::OFF_DS + ((ntile_ord + t) & 1) * 2 * C::PANEL + grp * C::PANEL) + rowl * 128;
           const bool diag = (t == 0);
+          // P^T of this warp's 32 query columns from S'^T alone; dP'^T is still on the tensor core
+          uint32_t rs[32];
+          tmem_ld32(t_s + 32 * sub, rs);
+          tmem_wait_ld();
+          {
+            uint32_t pk[16];
 #pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            const int c0 = 32 * sub + 16 * hh;             // first of this pass's 16 query columns
-            uint32_t rs[16], rd[16];
-            tmem_ld16(t_s + c0, rs);
-            tmem_ld16(t_dp + c0, rd);
-            tmem_wait_ld();
-            uint32_t pk[8], dk[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
+            for (int e = 0; e < 16; ++e) {
               float p0 = ex2_approx(__uint_as_float(rs[2 * e]) * c);
               float p1 = ex2_approx(__uint_as_float(rs[2 * e + 1]) * c);
               if (diag) {                                  // causal: query index >= key index
-                const int qa = 64 * grp + c0 + 2 * e;
+                const int qa = 64 * grp + 32 * sub + 2 * e;
                 if (qa < rowl) p0 = 0.0f;
                 if (qa + 1 < rowl) p1 = 0.0f;
               }
+              rs[2 * e] = __float_as_uint(p0);
+              rs[2 * e + 1] = __float_as_uint(p1);
               pk[e] = pack_bf16x2(p0, p1);
-              dk[e] = pack_bf16x2(p0 * __uint_as_float(rd[2 * e]), p1 * __uint_as_float(rd[2 * e + 1]));
             }
             // bf16 pairs re-use columns this warp has already consumed
-            tmem_st8(t_s + 32 * sub + 8 * hh, pk);
+            tmem_st16(t_s + 32 * sub, pk);
+          }
+          if (!mbar_wait_warp(sdp_full + grp, nsdp & 1, wc, B_SDP_FULL)) ok = false;
+          ++nsdp;
+          tc_fence_after();
+          if (t <= 1) staging_free(1 - t);
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            uint32_t rd[16], dk[8];
+            tmem_ld16(t_dp + 32 * sub + 16 * hh, rd);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              dk[e] = pack_bf16x2(__uint_as_float(rs[16 * hh + 2 * e]) * __uint_as_float(rd[2 * e]),
+                                  __uint_as_float(rs[16 * hh + 2 * e + 1]) * __uint_as_float(rd[2 * e + 1]));
             tmem_st8(t_dp + 32 * sub + 8 * hh, dk);
             // dS^T row (this key) -> smem panel of this half tile, 128-byte swizzle (chunk ^= row & 7)
 #pragma unroll
