@@ -141,7 +141,7 @@ int validate(const saf_problem* p, const uint8_t* mask, int* n_frozen) {
   if (!p || !mask) return SAF_ERR_INVALID_ARG;
   if (p->B < 1 || p->H < 1 || p->T < 1 || p->Tp < 1) return SAF_ERR_INVALID_ARG;
   if (p->T > p->Tp) return SAF_ERR_INVALID_ARG;
-  if (p->D != 64 && p->D != 128) return SAF_ERR_UNSUPPORTED;
+  if (p->D != 64 && p->D != 96 && p->D != 128) return SAF_ERR_UNSUPPORTED;   // 96: forward only
   if (p->grad_dtype != SAF_F32 && p->grad_dtype != SAF_BF16) return SAF_ERR_UNSUPPORTED;
   if (p->kv_group < 0 || (p->kv_group > 1 && p->H % p->kv_group != 0)) return SAF_ERR_INVALID_ARG;
   int nf = 0;
@@ -524,6 +524,7 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   }
   fp.B = p->B; fp.H = p->H; fp.T = p->T; fp.Tp = p->Tp;
   fp.kv_group = kvg;
+  fp.d_real = p->D;
   const float scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   fp.scale_log2 = scale * 1.4426950408889634f;
   fp.alpha = alpha; fp.rho = rho; fp.logZ = logZ;
@@ -535,7 +536,8 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   fp.status = ctx->status_dev;
   fp.wait_limit_ns = ctx->wait_limit_ns;
   ScopedTimer timer(ctx, SAF_KERNEL_FWD, st);
-  if (launch_fwd(p->D, mq, mk, mv, mvt, fp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+  // head dimension 96 runs on the 128-wide kernel: TMA zero-fills features 96..127 of every operand tile
+  if (launch_fwd(p->D == 96 ? 128 : p->D, mq, mk, mv, mvt, fp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
   return SAF_OK;
 }
 
@@ -788,6 +790,7 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
   int nf = 0;
   int rc = validate(p, frozen_mask_host, &nf);
   if (rc) return rc;
+  if (p->D == 96) return SAF_ERR_UNSUPPORTED;
   DeviceGuard g(ctx->device);
   if (!g.ok) return SAF_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

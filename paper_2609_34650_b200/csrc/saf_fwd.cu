@@ -557,7 +557,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             o.y = pack_bf16x2(__uint_as_float(r[8 * g + 2]) * inv_l, __uint_as_float(r[8 * g + 3]) * inv_l);
             o.z = pack_bf16x2(__uint_as_float(r[8 * g + 4]) * inv_l, __uint_as_float(r[8 * g + 5]) * inv_l);
             o.w = pack_bf16x2(__uint_as_float(r[8 * g + 6]) * inv_l, __uint_as_float(r[8 * g + 7]) * inv_l);
-            *reinterpret_cast<uint4*>(orow + 32 * cc + 8 * g) = o;
+            if ((D / 2) * hh + 32 * cc + 8 * g < p.d_real) *reinterpret_cast<uint4*>(orow + 32 * cc + 8 * g) = o;
           }
         }
       }

@@ -15,6 +15,7 @@ struct WorkItem { int32_t b, h, blk, kind; };
 struct FwdParams {
   int B, H, T, Tp;
   int kv_group;                     // query heads per shared key/value head (>= 1)
+  int d_real;                       // head dimension of the tensors (96 runs on the 128-wide kernel, zero-padded by TMA)
   float scale_log2;                 // softmax_scale * log2(e)
   const float* alpha;               // [H][Tp]
   const float* rho;                 // [H][Tp]

@@ -197,7 +197,11 @@ cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const flo
                               int T, int D, int src_group, cudaStream_t st) {
   const long long nthreads = static_cast<long long>(B) * Hf * T * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
-  if (D == 64)
+  if (D == 96)
+    saf_scale_rows_kernel<96><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
+                                                    strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
+                                                    static_cast<__half*>(dst), B, Hf, T, src_group);
+  else if (D == 64)
     saf_scale_rows_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
                                                     strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
                                                     static_cast<__half*>(dst), B, Hf, T, src_group);

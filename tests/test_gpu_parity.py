@@ -77,6 +77,14 @@ def test_head_dim_128_forward():
     check_units(L, all_units(wl), backward=False)
 
 
+@pytest.mark.parametrize("T,frozen,g", [(300, (1, 2), 1), (129, (), 1), (384, (0, 1, 2, 3), 2)])
+def test_head_dim_96_forward(T, frozen, g):
+    """The paper's 1B model uses 16 heads of dimension 96: forward on the 128-wide kernel with TMA zero padding."""
+    wl = si.Workload("d96", 2, 4, T, 96, frozen, -0.03, seed=96 + T, kv_group=g, backward=False)
+    L = Layer(si.generate(wl), backward=False).run(backward=False)
+    _check_gqa_layer(L, False)
+
+
 def test_backward_head_dim_128_is_reported_unsupported():
     wl = si.Workload("d128b", 1, 2, 128, 128, (), -0.01, seed=5)
     L = Layer(si.generate(wl))
@@ -249,7 +257,7 @@ def test_invalid_arguments_are_rejected():
         L.run()
     assert e.value.code == 1
     L = Layer(inp)
-    L.prob.D = 96
+    L.prob.D = 80                              # supported: 64, 96 (forward), 128 (forward)
     with pytest.raises(saf.SafError) as e:
         L.run()
     assert e.value.code == 2
