@@ -54,8 +54,8 @@ typedef struct {
   int32_t grad_dtype;          /* dtype of dQ/dK/dV: SAF_F32 or SAF_BF16 */
   int32_t kv_group;            /* grouped-query path (Appendix E.2): query heads per shared key/value head;
                                   K, V, dK, dV then have H / kv_group heads and query head h reads head
-                                  h / kv_group.  0 or 1 = multi-head attention.  The backward with
-                                  kv_group > 1 needs grad_dtype = SAF_F32 (SAF_ERR_UNSUPPORTED otherwise). */
+                                  h / kv_group.  0 or 1 = multi-head attention.  (Shared heads' gradients are
+                                  accumulated in fp32; with bf16 gradients in a context-owned workspace.) */
   int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3]; /* elements: batch, head, seq */
 } saf_problem;                 /* dO uses o_strides; O is bf16; LSE [B][H][T], dQ [B][H][T][D] and dK, dV
                                   [B][H/kv_group][T][D] are contiguous */

@@ -61,7 +61,7 @@ struct saf_ctx {
   int frozen_weight_bwd_pct = 25;          // ... and backward
   int call_counter = 0;                    // ids of the calls that stage fp16 operands (overflow marks)
   std::vector<WorklistEntry> worklists;
-  DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf;
+  DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf, dkacc_buf, dvacc_buf;
   // tensor-core form of frozen heads: tables built by saf_pattern_prepare, scaled V / dO per call
   PatternCache pat;
   bool tensor_pattern = true;              // SAF_DISABLE_TENSOR_PATTERN=1 turns the form off
@@ -362,7 +362,7 @@ int saf_destroy(saf_ctx* ctx) {
   DevBuf* pbufs[] = {&ctx->pat_consts, &ctx->pat_ok, &ctx->pat_avec, &ctx->pat_wvec, &ctx->pat_bandf, &ctx->pat_bandb,
                      &ctx->pat_hord, &ctx->pat_hlist, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta};
   for (DevBuf* b : pbufs) release(*b);
-  DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->hq, &ctx->hk, &ctx->hv,
+  DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->dkacc_buf, &ctx->dvacc_buf, &ctx->hq, &ctx->hk, &ctx->hv,
                     &ctx->hdo, &ctx->ho, &ctx->hlse, &ctx->hdq, &ctx->hdk, &ctx->hdv, &ctx->halpha, &ctx->hrho,
                     &ctx->hlogz};
   for (DevBuf* b : bufs) release(*b);
@@ -586,13 +586,25 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   const float scale_v = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   const int grad_f32 = p->grad_dtype == SAF_F32;
   const int kvg = kv_group_of(p);
-  if (kvg > 1 && !grad_f32) return SAF_ERR_UNSUPPORTED;   // shared heads' gradients are accumulated in fp32
   float* dqacc = static_cast<float*>(dQ);
   if (!grad_f32) {
     rc = ensure(ctx->dqacc_buf, nelem * sizeof(float));
     if (rc) return rc;
     dqacc = static_cast<float*>(ctx->dqacc_buf.ptr);
   }
+  // Shared key/value heads accumulate their gradients in fp32 (reduce-adds); with bf16 gradients that happens in
+  // a workspace that is converted at the end, and the kernels see fp32 targets.
+  const bool kv_acc = kvg > 1 && !grad_f32;
+  const size_t nkv = nelem / kvg;
+  void* dK_k = dK;
+  void* dV_k = dV;
+  if (kv_acc) {
+    if ((rc = ensure(ctx->dkacc_buf, nkv * sizeof(float))) || (rc = ensure(ctx->dvacc_buf, nkv * sizeof(float))))
+      return rc;
+    dK_k = ctx->dkacc_buf.ptr;
+    dV_k = ctx->dvacc_buf.ptr;
+  }
+  const int kern_f32 = (grad_f32 || kv_acc) ? 1 : 0;
   // tensor-core form of the frozen heads: the preparation kernel also stages w(i) dO in fp16
   const bool tensor_form = nf > 0 && pattern_matches(ctx, p, frozen_mask_host, alpha, rho, logZ);
   PrepFrozen fz{};
@@ -612,7 +624,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_PREP, st);
     if (launch_bwd_prep(O, dO, LSE, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr), q_ext, do_ext,
-                        1.0f / scale_v, dqacc, dK, dV, grad_f32, kvg, fz, p->B, p->H, p->T, p->D, st) != cudaSuccess)
+                        1.0f / scale_v, dqacc, dK_k, dV_k, kern_f32, kvg, fz, p->B, p->H, p->T, p->D, st) != cudaSuccess)
       return SAF_ERR_CUDA;
   }
 
@@ -651,7 +663,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     // dK, dV: [B][H/kv_group][T][64]
     dims[2] = static_cast<cuuint64_t>(p->H / kvg);
     gs[2] = static_cast<cuuint64_t>(p->T) * 64 * 4 * (p->H / kvg);
-    if (grad_f32 && (!enc(&mdk, dK) || !enc(&mdv, dV))) return SAF_ERR_CUDA;
+    if (kern_f32 && (!enc(&mdk, dK_k) || !enc(&mdv, dV_k))) return SAF_ERR_CUDA;
   }
   BwdParams bp;
   CUtensorMap mdot = mdo;
@@ -674,8 +686,8 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   bp.q_ext = q_ext;
   bp.do_ext = do_ext;
   bp.nblk = nblk;
-  bp.dK = dK; bp.dV = dV;
-  bp.grad_f32 = grad_f32;
+  bp.dK = dK_k; bp.dV = dV_k;
+  bp.grad_f32 = kern_f32;
   bp.items = wl->items_dev;
   bp.cta_offsets = wl->offsets_dev;
   bp.status = ctx->status_dev;
@@ -687,6 +699,9 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   if (!grad_f32) {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_FINALIZE, st);
     if (launch_bwd_finalize(dqacc, dQ, nelem, st) != cudaSuccess) return SAF_ERR_CUDA;
+    if (kv_acc && (launch_bwd_finalize(static_cast<const float*>(dK_k), dK, nkv, st) != cudaSuccess ||
+                   launch_bwd_finalize(static_cast<const float*>(dV_k), dV, nkv, st) != cudaSuccess))
+      return SAF_ERR_CUDA;
   }
   return SAF_OK;
 }
