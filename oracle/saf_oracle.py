@@ -148,9 +148,14 @@ def hybrid_attn_fwd(Q, K, V, mask, alpha, rho, scale=None):
     """Q: [B,H,T,D], K,V: [B,Hkv,T,D] float64 with Hkv dividing H (grouped-query path, Appendix E.2: query head h
     reads the shared key/value head h // (H/Hkv); Hkv = H is ordinary multi-head attention);
     mask: [H] (nonzero = frozen); alpha,rho: [H,Tp].
+    Packed layout (Appendix E.2: replaced heads have no query/key slot on the multi-head path): when Q has fewer
+    heads than the mask, Q and K hold the ordinary heads only, in head order.
     Returns O [B,H,T,D] and LSE [B,H,T] (0 for frozen heads, which have no softmax)."""
-    B, H, T, D = Q.shape
-    g = H // K.shape[1]
+    B, _, T, D = V.shape
+    H = len(mask)
+    packed = Q is not None and Q.shape[1] != H
+    slot = np.cumsum(np.asarray(mask) == 0) - 1            # ordinal of head h among the ordinary heads
+    g = 1 if packed else H // V.shape[1]
     scale = 1.0 / np.sqrt(D) if scale is None else scale
     O = np.zeros((B, H, T, D))
     LSE = np.zeros((B, H, T))
@@ -160,8 +165,9 @@ def hybrid_attn_fwd(Q, K, V, mask, alpha, rho, scale=None):
             for b in range(B):
                 O[b, h] = P @ V[b, h // g]
         else:
+            hq, hk = (slot[h], slot[h]) if packed else (h, h // g)
             for b in range(B):
-                O[b, h], LSE[b, h], _ = ordinary_head_fwd(Q[b, h], K[b, h // g], V[b, h // g], scale)
+                O[b, h], LSE[b, h], _ = ordinary_head_fwd(Q[b, hq], K[b, hk], V[b, h // g], scale)
     return O, LSE
 
 
@@ -169,12 +175,15 @@ def hybrid_attn_bwd(Q, K, V, dO, mask, alpha, rho, scale=None):
     """Gradients of sum(O o dO) w.r.t. Q, K, V.  Frozen heads: dQ = dK = 0, dV = P^T dO.  With shared
     key/value heads (K, V: [B,Hkv,T,D]) the gradient of a shared head is the sum over the query heads that
     read it."""
-    B, H, T, D = Q.shape
-    Hkv = K.shape[1]
+    B, _, T, D = dO.shape
+    H = len(mask)
+    packed = Q is not None and Q.shape[1] != H       # Q, K, dQ, dK hold the ordinary heads only
+    slot = np.cumsum(np.asarray(mask) == 0) - 1
+    Hkv = V.shape[1]
     g = H // Hkv
     scale = 1.0 / np.sqrt(D) if scale is None else scale
-    dQ = np.zeros((B, H, T, D))
-    dK = np.zeros((B, Hkv, T, D))
+    dQ = np.zeros(Q.shape if packed else (B, H, T, D))
+    dK = np.zeros(K.shape if packed else (B, Hkv, T, D))
     dV = np.zeros((B, Hkv, T, D))
     for h in range(H):
         if mask[h]:
@@ -183,9 +192,10 @@ def hybrid_attn_bwd(Q, K, V, dO, mask, alpha, rho, scale=None):
                 dV[b, h // g] += P.T @ dO[b, h]
         else:
             for b in range(B):
-                dq, dk, dv = ordinary_head_bwd(Q[b, h], K[b, h // g], V[b, h // g], dO[b, h], scale)
-                dQ[b, h] = dq
-                dK[b, h // g] += dk
+                hq, hk = (slot[h], slot[h]) if packed else (h, h // g)
+                dq, dk, dv = ordinary_head_bwd(Q[b, hq], K[b, hk], V[b, h // g], dO[b, h], scale)
+                dQ[b, hq] = dq
+                dK[b, hk] += dk
                 dV[b, h // g] += dv
     return dQ, dK, dV
 

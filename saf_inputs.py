@@ -55,6 +55,7 @@ class Workload:
     backward: bool = True
     seed: int = 0
     kv_group: int = 1             # grouped-query attention: query heads per shared key/value head
+    packed_qk: bool = False       # Q and K carry only the ordinary heads, in head order (multi-head only)
 
     @property
     def stored_len(self) -> int:
@@ -126,8 +127,9 @@ def generate(wl: Workload) -> Inputs:
     rng = np.random.default_rng(wl.seed)
     shape = (wl.B, wl.H, wl.T, wl.D)
     kv_shape = (wl.B, wl.H // wl.kv_group, wl.T, wl.D)
-    q = _normal_bf16(rng, shape)
-    k = _normal_bf16(rng, kv_shape)
+    qk_shape = (wl.B, wl.H - len(wl.frozen_heads), wl.T, wl.D)
+    q = _normal_bf16(rng, qk_shape if wl.packed_qk else shape)
+    k = _normal_bf16(rng, qk_shape if wl.packed_qk else kv_shape)
     v = _normal_bf16(rng, kv_shape)
     do = _normal_bf16(rng, shape)
     tp = wl.stored_len

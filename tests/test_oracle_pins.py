@@ -17,6 +17,8 @@ off-by-one in the relative distance or the causal boundary):
   P9  grouped-query path (Appendix E.2): shared key/value heads == the multi-head layer on K, V repeated per
       query head, with the shared heads' gradients summed over their query heads (torch autograd through
       repeat_interleave; torch's own enable_gqa route for the all-ordinary case; finite differences)
+  P11 packed Q/K layout (Appendix E.2: replaced heads have no query/key slot): equals the full layout with the
+      ordinary heads scattered back, whatever sits in the frozen heads' slots; torch SDPA per ordinary head
   P10 pattern gradients (trainable-pattern control): central finite differences of sum(O o dO) through the
       layer's own forward, torch autograd through a causal softmax of the bias matrix, and the two zero-sum
       identities that shift invariance forces (sum_j dalpha(j) = 0, sum_d drho(d) = 0)
@@ -459,3 +461,33 @@ def test_p10_pattern_grads_finite_differences_and_zero_sums():
     P = orc.pattern_dense(alpha, rho, T)
     G = dO @ V.T
     assert abs(dr[T - 1] - P[T - 1, 0] * (G[T - 1, 0] - (P[T - 1] * G[T - 1]).sum())) < 1e-13
+
+
+# ------------------------------------------------------------------ P11 packed Q/K layout
+def test_p11_packed_qk_equals_full_layout_and_sdpa():
+    B, H, T, D = 2, 5, 17, 6
+    rng = np.random.default_rng(110)
+    mask = np.array([0, 1, 0, 1, 0], dtype=np.uint8)
+    ordinary = [h for h in range(H) if not mask[h]]
+    Qp, Kp = rng.standard_normal((B, 3, T, D)), rng.standard_normal((B, 3, T, D))
+    V, dO = rng.standard_normal((B, H, T, D)), rng.standard_normal((B, H, T, D))
+    alpha, rho = rng.standard_normal((H, T)), rng.standard_normal((H, T))
+    O, LSE = orc.hybrid_attn_fwd(Qp, Kp, V, mask, alpha, rho)
+    dQ, dK, dV = orc.hybrid_attn_bwd(Qp, Kp, V, dO, mask, alpha, rho)
+    assert dQ.shape == Qp.shape and dK.shape == Kp.shape and dV.shape == V.shape
+    # full layout with poisoned frozen slots
+    Qf, Kf = np.full((B, H, T, D), np.nan), np.full((B, H, T, D), np.nan)
+    Qf[:, ordinary], Kf[:, ordinary] = Qp, Kp
+    Of, LSEf = orc.hybrid_attn_fwd(Qf, Kf, V, mask, alpha, rho)
+    dQf, dKf, dVf = orc.hybrid_attn_bwd(Qf, Kf, V, dO, mask, alpha, rho)
+    assert np.array_equal(O, Of) and np.array_equal(LSE, LSEf) and np.array_equal(dV, dVf)
+    assert np.array_equal(dQ, dQf[:, ordinary]) and np.array_equal(dK, dKf[:, ordinary])
+    # torch, ordinary head by ordinary head: slot s of the packed tensors belongs to head ordinary[s]
+    for s_, h in enumerate(ordinary):
+        tq, tk, tv = (torch.tensor(x, requires_grad=True) for x in (Qp[:, s_], Kp[:, s_], V[:, h]))
+        to = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True)
+        to.backward(torch.tensor(dO[:, h]))
+        assert np.abs(O[:, h] - to.detach().numpy()).max() < 1e-12
+        assert np.abs(dQ[:, s_] - tq.grad.numpy()).max() < 1e-11
+        assert np.abs(dK[:, s_] - tk.grad.numpy()).max() < 1e-11
+        assert np.abs(dV[:, h] - tv.grad.numpy()).max() < 1e-11
