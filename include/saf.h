@@ -56,9 +56,13 @@ typedef struct {
                                   K, V, dK, dV then have H / kv_group heads and query head h reads head
                                   h / kv_group.  0 or 1 = multi-head attention.  (Shared heads' gradients are
                                   accumulated in fp32; with bf16 gradients in a context-owned workspace.) */
+  int32_t packed_qk;           /* nonzero: Q, K, dQ, dK carry only the ordinary heads, in head order (Appendix E.2:
+                                  replaced heads have no query/key slot on the multi-head path); needs
+                                  kv_group <= 1.  Not available through saf_hybrid_attn_step_host. */
+  int32_t reserved;
   int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3]; /* elements: batch, head, seq */
 } saf_problem;                 /* dO uses o_strides; O is bf16; LSE [B][H][T], dQ [B][H][T][D] and dK, dV
-                                  [B][H/kv_group][T][D] are contiguous */
+                                  [B][H/kv_group][T][D] are contiguous (packed_qk: dQ, dK [B][Ho][T][D]) */
 
 /* Library version (major*100 + minor). */
 int saf_version(void);

@@ -23,6 +23,7 @@ SAF_KERNEL_FWD, SAF_KERNEL_BWD, SAF_KERNEL_BWD_PREP, SAF_KERNEL_BWD_FINALIZE, SA
 class SafProblem(C.Structure):
     _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("T", C.c_int32), ("D", C.c_int32), ("Tp", C.c_int32),
                 ("softmax_scale", C.c_float), ("grad_dtype", C.c_int32), ("kv_group", C.c_int32),
+                ("packed_qk", C.c_int32), ("reserved", C.c_int32),
                 ("q_strides", C.c_int64 * 3), ("k_strides", C.c_int64 * 3), ("v_strides", C.c_int64 * 3),
                 ("o_strides", C.c_int64 * 3)]
 
@@ -119,15 +120,17 @@ def saf_pattern_logz_static(device, mask, alpha, rho, logZ_out):
 
 
 def make_problem(q_like, Tp, softmax_scale=0.0, grad_dtype=SAF_F32, k_like=None, v_like=None, o_like=None,
-                 kv_group=1):
+                 kv_group=1, packed_qk=False, H=None):
     """saf_problem from [B,H,T,D] torch tensors (any strides with a unit feature stride); with kv_group > 1
     k_like / v_like are the [B,H/kv_group,T,D] shared key/value tensors."""
-    B, H, T, D = q_like.shape
+    B, Hq, T, D = q_like.shape
+    H = Hq if H is None else H              # packed_qk: q_like has only the ordinary heads, pass H
     p = SafProblem()
     p.B, p.H, p.T, p.D, p.Tp = B, H, T, D, Tp
     p.softmax_scale = softmax_scale
     p.grad_dtype = grad_dtype
     p.kv_group = kv_group
+    p.packed_qk = int(packed_qk)
     for name, t in (("q_strides", q_like), ("k_strides", k_like if k_like is not None else q_like),
                     ("v_strides", v_like if v_like is not None else q_like),
                     ("o_strides", o_like if o_like is not None else q_like)):

@@ -61,7 +61,7 @@ struct saf_ctx {
   int frozen_weight_bwd_pct = 25;          // ... and backward
   int call_counter = 0;                    // ids of the calls that stage fp16 operands (overflow marks)
   std::vector<WorklistEntry> worklists;
-  DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf, dkacc_buf, dvacc_buf;
+  DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf, dkacc_buf, dvacc_buf, qslot_buf;
   // tensor-core form of frozen heads: tables built by saf_pattern_prepare, scaled V / dO per call
   PatternCache pat;
   bool tensor_pattern = true;              // SAF_DISABLE_TENSOR_PATTERN=1 turns the form off
@@ -144,6 +144,7 @@ int validate(const saf_problem* p, const uint8_t* mask, int* n_frozen) {
   if (p->D != 64 && p->D != 96 && p->D != 128) return SAF_ERR_UNSUPPORTED;   // 96: forward only
   if (p->grad_dtype != SAF_F32 && p->grad_dtype != SAF_BF16) return SAF_ERR_UNSUPPORTED;
   if (p->kv_group < 0 || (p->kv_group > 1 && p->H % p->kv_group != 0)) return SAF_ERR_INVALID_ARG;
+  if (p->packed_qk && p->kv_group > 1) return SAF_ERR_INVALID_ARG;
   int nf = 0;
   for (int h = 0; h < p->H; ++h) nf += mask[h] ? 1 : 0;
   *n_frozen = nf;
@@ -151,6 +152,21 @@ int validate(const saf_problem* p, const uint8_t* mask, int* n_frozen) {
 }
 
 inline int kv_group_of(const saf_problem* p) { return p->kv_group > 1 ? p->kv_group : 1; }
+
+// Packed Q/K layout: device table head -> slot among the ordinary heads (-1 for frozen heads).
+int upload_qslot(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st, const int** out) {
+  int rc = ensure(ctx->qslot_buf, static_cast<size_t>(std::max(H, 64)) * sizeof(int));
+  if (rc) return rc;
+  std::vector<int> slot(H);
+  int n = 0;
+  for (int h = 0; h < H; ++h) slot[h] = mask[h] ? -1 : n++;
+  // pageable source: the copy is staged before the call returns
+  if (cudaMemcpyAsync(ctx->qslot_buf.ptr, slot.data(), static_cast<size_t>(H) * sizeof(int), cudaMemcpyHostToDevice,
+                      st) != cudaSuccess)
+    return SAF_ERR_CUDA;
+  *out = static_cast<const int*>(ctx->qslot_buf.ptr);
+  return SAF_OK;
+}
 
 int upload_mask(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st) {
   int rc = ensure(ctx->mask_buf, std::max(H, 256));
@@ -362,7 +378,7 @@ int saf_destroy(saf_ctx* ctx) {
   DevBuf* pbufs[] = {&ctx->pat_consts, &ctx->pat_ok, &ctx->pat_avec, &ctx->pat_wvec, &ctx->pat_bandf, &ctx->pat_bandb,
                      &ctx->pat_hord, &ctx->pat_hlist, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta};
   for (DevBuf* b : pbufs) release(*b);
-  DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->dkacc_buf, &ctx->dvacc_buf, &ctx->hq, &ctx->hk, &ctx->hv,
+  DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->dkacc_buf, &ctx->dvacc_buf, &ctx->qslot_buf, &ctx->hq, &ctx->hk, &ctx->hv,
                     &ctx->hdo, &ctx->ho, &ctx->hlse, &ctx->hdq, &ctx->hdk, &ctx->hdv, &ctx->halpha, &ctx->hrho,
                     &ctx->hlogz};
   for (DevBuf* b : bufs) release(*b);
@@ -488,9 +504,9 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   rc = make_map(ctx, &mv, V, p, p->v_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg);
   if (rc) return rc;
   if (no > 0) {
-    rc = make_map(ctx, &mq, Q, p, p->q_strides);
+    rc = make_map(ctx, &mq, Q, p, p->q_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->packed_qk ? no : p->H);
     if (rc) return rc;
-    rc = make_map(ctx, &mk, K, p, p->k_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg);
+    rc = make_map(ctx, &mk, K, p, p->k_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->packed_qk ? no : p->H / kvg);
     if (rc) return rc;
   } else {
     mq = mv;
@@ -525,6 +541,8 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   fp.B = p->B; fp.H = p->H; fp.T = p->T; fp.Tp = p->Tp;
   fp.kv_group = kvg;
   fp.d_real = p->D;
+  fp.qslot = nullptr;
+  if (p->packed_qk && no > 0 && (rc = upload_qslot(ctx, frozen_mask_host, p->H, st, &fp.qslot))) return rc;
   const float scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   fp.scale_log2 = scale * 1.4426950408889634f;
   fp.alpha = alpha; fp.rho = rho; fp.logZ = logZ;
@@ -551,7 +569,8 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   if (rc) return rc;
   if (p->D != 64) return SAF_ERR_UNSUPPORTED;
   const int no = p->H - nf;
-  if (!dO || !dQ || !dK || !dV) return SAF_ERR_INVALID_ARG;
+  const bool no_qk_out = p->packed_qk && no == 0;        // packed layout of a frozen-only layer: no dQ / dK at all
+  if (!dO || !dV || (!no_qk_out && (!dQ || !dK))) return SAF_ERR_INVALID_ARG;
   if (no > 0 && (!Q || !K || !V || !O || !LSE)) return SAF_ERR_INVALID_ARG;
   if (nf > 0 && (!alpha || !rho)) return SAF_ERR_INVALID_ARG;
   if (!aligned16(dO) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV)) return SAF_ERR_INVALID_ARG;
@@ -577,7 +596,8 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   if (rc) return rc;
 
   const int nblk = (p->T + BLK - 1) / BLK;
-  const size_t nelem = static_cast<size_t>(p->B) * p->H * p->T * p->D;
+  const int nqh = p->packed_qk ? no : p->H;                  // heads of Q, K, dQ (and of dK when packed)
+  const size_t nelem = static_cast<size_t>(p->B) * nqh * p->T * p->D;
   const size_t ext_bytes = static_cast<size_t>(p->B) * p->H * nblk * 4096;   // one 4 KB image per 128-row block
   rc = ensure(ctx->delta_buf, 2 * ext_bytes);                 // q_ext images followed by do_ext images
   if (rc) return rc;
@@ -587,15 +607,15 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   const int grad_f32 = p->grad_dtype == SAF_F32;
   const int kvg = kv_group_of(p);
   float* dqacc = static_cast<float*>(dQ);
-  if (!grad_f32) {
-    rc = ensure(ctx->dqacc_buf, nelem * sizeof(float));
+  if (!grad_f32 || no_qk_out) {
+    rc = ensure(ctx->dqacc_buf, std::max<size_t>(nelem, 64) * sizeof(float));
     if (rc) return rc;
     dqacc = static_cast<float*>(ctx->dqacc_buf.ptr);
   }
   // Shared key/value heads accumulate their gradients in fp32 (reduce-adds); with bf16 gradients that happens in
   // a workspace that is converted at the end, and the kernels see fp32 targets.
   const bool kv_acc = kvg > 1 && !grad_f32;
-  const size_t nkv = nelem / kvg;
+  const size_t nkv = static_cast<size_t>(p->B) * (p->H / kvg) * p->T * p->D;
   void* dK_k = dK;
   void* dV_k = dV;
   if (kv_acc) {
@@ -605,6 +625,8 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     dV_k = ctx->dvacc_buf.ptr;
   }
   const int kern_f32 = (grad_f32 || kv_acc) ? 1 : 0;
+  const int* qslot = nullptr;
+  if (p->packed_qk && (rc = upload_qslot(ctx, frozen_mask_host, p->H, st, &qslot))) return rc;
   // tensor-core form of the frozen heads: the preparation kernel also stages w(i) dO in fp16
   const bool tensor_form = nf > 0 && pattern_matches(ctx, p, frozen_mask_host, alpha, rho, logZ);
   PrepFrozen fz{};
@@ -624,7 +646,8 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_PREP, st);
     if (launch_bwd_prep(O, dO, LSE, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr), q_ext, do_ext,
-                        1.0f / scale_v, dqacc, dK_k, dV_k, kern_f32, kvg, fz, p->B, p->H, p->T, p->D, st) != cudaSuccess)
+                        1.0f / scale_v, dqacc, dK_k, dV_k, kern_f32, kvg, qslot, no, fz, p->B, p->H, p->T, p->D, st) !=
+        cudaSuccess)
       return SAF_ERR_CUDA;
   }
 
@@ -638,8 +661,9 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   rc = make_map(ctx, &mdo, dO, p, p->o_strides);
   if (rc) return rc;
   if (no > 0) {
-    if ((rc = make_map(ctx, &mq, Q, p, p->q_strides))) return rc;
-    if ((rc = make_map(ctx, &mk, K, p, p->k_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg))) return rc;
+    if ((rc = make_map(ctx, &mq, Q, p, p->q_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, nqh))) return rc;
+    if ((rc = make_map(ctx, &mk, K, p, p->k_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->packed_qk ? no : p->H / kvg)))
+      return rc;
     if ((rc = make_map(ctx, &mv, V, p, p->v_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg))) return rc;
   } else {
     mq = mdo; mk = mdo; mv = mdo;
@@ -648,8 +672,11 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   // (dK and dV get maps of the same shape for the tiled stores of the fp32 epilogue)
   CUtensorMap mdq, mdk, mdv;
   {
-    cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(p->T), static_cast<cuuint64_t>(p->H), static_cast<cuuint64_t>(p->B)};
-    cuuint64_t gs[3] = {64 * 4, static_cast<cuuint64_t>(p->T) * 64 * 4, static_cast<cuuint64_t>(p->T) * 64 * 4 * p->H};
+    // dQ: [B][H][T][64], or [B][Ho][T][64] in the packed layout
+    cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(p->T), static_cast<cuuint64_t>(std::max(nqh, 1)),
+                          static_cast<cuuint64_t>(p->B)};
+    cuuint64_t gs[3] = {64 * 4, static_cast<cuuint64_t>(p->T) * 64 * 4,
+                        static_cast<cuuint64_t>(p->T) * 64 * 4 * std::max(nqh, 1)};
     cuuint32_t box[4] = {32, BLK, 1, 1};
     cuuint32_t es[4] = {1, 1, 1, 1};
     auto enc = [&](CUtensorMap* m, void* base) {
@@ -660,10 +687,11 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     if (!enc(&mdq, dqacc)) return SAF_ERR_CUDA;
     mdk = mdq;
     mdv = mdq;
-    // dK, dV: [B][H/kv_group][T][64]
+    // dK: like dQ when packed, else [B][H/kv_group][T][64]; dV: [B][H/kv_group][T][64]
+    if (kern_f32 && p->packed_qk && nqh > 0 && !enc(&mdk, dK_k)) return SAF_ERR_CUDA;
     dims[2] = static_cast<cuuint64_t>(p->H / kvg);
     gs[2] = static_cast<cuuint64_t>(p->T) * 64 * 4 * (p->H / kvg);
-    if (kern_f32 && (!enc(&mdk, dK_k) || !enc(&mdv, dV_k))) return SAF_ERR_CUDA;
+    if (kern_f32 && ((!p->packed_qk && !enc(&mdk, dK_k)) || !enc(&mdv, dV_k))) return SAF_ERR_CUDA;
   }
   BwdParams bp;
   CUtensorMap mdot = mdo;
@@ -680,6 +708,8 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   }
   bp.B = p->B; bp.H = p->H; bp.T = p->T; bp.Tp = p->Tp;
   bp.kv_group = kvg;
+  bp.qslot = qslot;
+  bp.n_ord = no;
   bp.scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   bp.scale_log2 = bp.scale * 1.4426950408889634f;
   bp.alpha = alpha; bp.rho = rho; bp.logZ = logZ;
@@ -698,7 +728,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   }
   if (!grad_f32) {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_FINALIZE, st);
-    if (launch_bwd_finalize(dqacc, dQ, nelem, st) != cudaSuccess) return SAF_ERR_CUDA;
+    if (nelem > 0 && launch_bwd_finalize(dqacc, dQ, nelem, st) != cudaSuccess) return SAF_ERR_CUDA;
     if (kv_acc && (launch_bwd_finalize(static_cast<const float*>(dK_k), dK, nkv, st) != cudaSuccess ||
                    launch_bwd_finalize(static_cast<const float*>(dV_k), dV, nkv, st) != cudaSuccess))
       return SAF_ERR_CUDA;
@@ -716,6 +746,7 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
   if (rc) return rc;
   const int no = p->H - nf;
   if (!V_host || (no > 0 && (!Q_host || !K_host)) || (nf > 0 && (!alpha_host || !rho_host))) return SAF_ERR_INVALID_ARG;
+  if (p->packed_qk) return SAF_ERR_UNSUPPORTED;
   DeviceGuard g(ctx->device);
   if (!g.ok) return SAF_ERR_CUDA;
   const int kvg = kv_group_of(p);

@@ -222,7 +222,8 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         if (!ok) return;
         TR(2, 31);
         mbar_expect_tx(kv_full + ks, 2 * C::PANEL);
-        tma_load_4d(smem + C::OFF_K + ks * C::PANEL, &mk, kv_full + ks, 0, w2.blk * BLK, w2.h / p.kv_group, w2.b);
+        tma_load_4d(smem + C::OFF_K + ks * C::PANEL, &mk, kv_full + ks, 0, w2.blk * BLK,
+                    p.qslot ? p.qslot[w2.h] : w2.h / p.kv_group, w2.b);
         tma_load_4d(smem + C::OFF_V, &mv, kv_full + ks, 0, w2.blk * BLK, w2.h / p.kv_group, w2.b);
         ++nkv;
       };
@@ -231,6 +232,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         const WorkItem w = p.items[it];
         const bool ord = w.kind == KIND_ORDINARY;
         const size_t bh = static_cast<size_t>(w.b) * p.H + w.h;
+        const int qh = (ord && p.qslot) ? p.qslot[w.h] : w.h;     // head index in the Q tensor
         const bool fast = !ord && p.band_b != nullptr && p.fast_ok[w.h] != 0 && p.ovf[w.h] != p.call_id;
         if (fast) {
           // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled dO tile.  These
@@ -271,7 +273,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           TR(2, I == w.blk ? 33 : 32);
           mbar_expect_tx(qdo_full + s, ord ? 2 * C::PANEL + 8192 : C::PANEL);
           if (ord) {
-            tma_load_4d(smem + C::OFF_Q + s * C::PANEL, &mq, qdo_full + s, 0, I * BLK, w.h, w.b);
+            tma_load_4d(smem + C::OFF_Q + s * C::PANEL, &mq, qdo_full + s, 0, I * BLK, qh, w.b);
             const size_t img = (bh * nblk + I) * 4096;
             bulk_load(smem + C::OFF_QX + s * 4096, static_cast<const uint8_t*>(p.q_ext) + img, 4096, qdo_full + s);
             bulk_load(smem + C::OFF_DOX + s * 4096, static_cast<const uint8_t*>(p.do_ext) + img, 4096, qdo_full + s);
@@ -498,6 +500,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     for (int it = it_begin; it < it_end; ++it) {
       const WorkItem w = p.items[it];
       if (w.kind != KIND_ORDINARY) continue;
+      const int qh = p.qslot ? p.qslot[w.h] : w.h;       // head index in the dQ accumulator
       bool leave = false;
       for (int I = w.blk; I < nblk; ++I) {
         // the previous tile's reduce has finished reading the staging buffer (thread 512 waits for it
@@ -527,7 +530,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         fence_proxy_async_smem();
         named_bar_sync(3, 128);
         if (tid == 512 && ok) {
-          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 0, I * BLK, w.h, w.b);
+          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 0, I * BLK, qh, w.b);
           bulk_commit_group();
           bulk_wait_group_read0();
         }
@@ -543,7 +546,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         fence_proxy_async_smem();
         named_bar_sync(3, 128);
         if (tid == 512 && ok) {
-          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 32, I * BLK, w.h, w.b);
+          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 32, I * BLK, qh, w.b);
           bulk_commit_group();
           bulk_wait_group_read0();
         }
@@ -804,7 +807,8 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         const uint32_t col = grp == 0 ? C::COL_DV : C::COL_DK;
         const float mul = grp == 0 ? dv_mul : p.scale;
         void* base = grp == 0 ? p.dV : p.dK;
-        const size_t off = (bh * p.T + key) * 64;
+        const size_t bho = (grp == 1 && p.qslot) ? static_cast<size_t>(w.b) * p.n_ord + p.qslot[w.h] : bh;
+        const size_t off = (bho * p.T + key) * 64;
         {
           const int cc = sub;                             // this warp's 32 feature columns
           uint32_t r[32];
@@ -862,9 +866,11 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             tma_reduce_add_4d(m, src1, 32 * (first ^ 1), w.blk * BLK, kvh, w.b);
             bulk_commit_group();
           } else {
-            tma_store_4d(m, src0, 32 * first, w.blk * BLK, w.h, w.b);
+            // (packed layout: dK has the ordinary heads only)
+            const int oh = (grp == 1 && p.qslot) ? p.qslot[w.h] : w.h;
+            tma_store_4d(m, src0, 32 * first, w.blk * BLK, oh, w.b);
             bulk_commit_group();
-            tma_store_4d(m, src1, 32 * (first ^ 1), w.blk * BLK, w.h, w.b);
+            tma_store_4d(m, src1, 32 * (first ^ 1), w.blk * BLK, oh, w.b);
             bulk_commit_group();
           }
         }

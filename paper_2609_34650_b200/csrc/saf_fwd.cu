@@ -153,7 +153,8 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           if (!ok) break;
           mbar_expect_tx(q_full, C::TILE_BYTES);
           for (int pn = 0; pn < C::NPANEL; ++pn)
-            tma_load_4d(smem + C::OFF_Q + pn * C::PANEL_BYTES, &mq, q_full, pn * 64, w.blk * BLK, w.h, w.b);
+            tma_load_4d(smem + C::OFF_Q + pn * C::PANEL_BYTES, &mq, q_full, pn * 64, w.blk * BLK,
+                        p.qslot ? p.qslot[w.h] : w.h, w.b);
           ++nq;
         }
         for (int j = 0; j < ntiles && ok; ++j) {
@@ -164,7 +165,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             mbar_expect_tx(k_full + s, C::TILE_BYTES);
             for (int pn = 0; pn < C::NPANEL; ++pn)
               tma_load_4d(smem + C::OFF_K + s * C::TILE_BYTES + pn * C::PANEL_BYTES, &mk, k_full + s, pn * 64,
-                          j * BLK, w.h / p.kv_group, w.b);
+                          j * BLK, p.qslot ? p.qslot[w.h] : w.h / p.kv_group, w.b);
             ++nk;
           }
           const int s = nv % C::NS;

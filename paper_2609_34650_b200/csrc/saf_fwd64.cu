@@ -186,11 +186,12 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           continue;
         }
         const bool ord = w.kind == KIND_ORDINARY;
+        const int kh = !ord ? 0 : (p.qslot ? p.qslot[w.h] : w.h / p.kv_group);   // head index in the K tensor
         if (ord) {
           ok = mbar_wait(q_empty, (nq & 1) ^ 1, wc, F_Q_EMPTY);
           if (!ok) break;
           mbar_expect_tx(q_full, C::TILE_BYTES);
-          tma_load_4d(smem + C::OFF_Q, &mq, q_full, 0, w.blk * BLK, w.h, w.b);
+          tma_load_4d(smem + C::OFF_Q, &mq, q_full, 0, w.blk * BLK, p.qslot ? p.qslot[w.h] : w.h, w.b);
           ++nq;
         }
         for (int j = 0; j < ntiles && ok; ++j) {
@@ -199,7 +200,7 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             ok = mbar_wait(k_empty + s, ((nk / C::NS) & 1) ^ 1, wc, F_K_EMPTY);
             if (!ok) break;
             mbar_expect_tx(k_full + s, C::TILE_BYTES);
-            tma_load_4d(smem + C::OFF_K + s * C::TILE_BYTES, &mk, k_full + s, 0, j * BLK, w.h / p.kv_group, w.b);
+            tma_load_4d(smem + C::OFF_K + s * C::TILE_BYTES, &mk, k_full + s, 0, j * BLK, kh, w.b);
             ++nk;
           }
           const int s = nv % C::NS;

@@ -16,6 +16,7 @@ struct FwdParams {
   int B, H, T, Tp;
   int kv_group;                     // query heads per shared key/value head (>= 1)
   int d_real;                       // head dimension of the tensors (96 runs on the 128-wide kernel, zero-padded by TMA)
+  const int* qslot;                 // packed Q/K layout: head -> slot among the ordinary heads (NULL: slot = head)
   float scale_log2;                 // softmax_scale * log2(e)
   const float* alpha;               // [H][Tp]
   const float* rho;                 // [H][Tp]
@@ -43,6 +44,8 @@ struct FwdParams {
 struct BwdParams {
   int B, H, T, Tp;
   int kv_group;                     // as in FwdParams; > 1: dK / dV are reduce-added instead of stored
+  const int* qslot;                 // packed layout of Q, K, dQ, dK (see FwdParams)
+  int n_ord;                        // number of ordinary heads (head count of the packed tensors)
   float scale, scale_log2;
   const float* alpha;
   const float* rho;
@@ -124,8 +127,8 @@ struct PrepFrozen {
 };
 cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* o_strides,
                             const uint8_t* mask_dev, void* q_ext, void* do_ext, float inv_scale, float* dQacc,
-                            void* dK, void* dV, int grad_f32, int kv_group, const PrepFrozen& fz, int B, int H, int T,
-                            int D, cudaStream_t st);   // kv_group > 1: zeroes all of dK and dV (fp32) instead
+                            void* dK, void* dV, int grad_f32, int kv_group, const int* qslot, int n_ord,
+                            const PrepFrozen& fz, int B, int H, int T, int D, cudaStream_t st);   // kv_group > 1: zeroes all of dK and dV (fp32) instead
 // dQ (grad dtype) = scale-free copy/convert of dQacc (fp32) for the bf16-gradient case.
 cudaError_t launch_bwd_finalize(const float* dQacc, void* dQ, size_t n, cudaStream_t st);
 // head dimension 64 (saf_fwd64.cu); launch_fwd dispatches to it

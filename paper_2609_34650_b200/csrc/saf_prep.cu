@@ -241,8 +241,9 @@ __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat1
                                                            uint8_t* __restrict__ q_ext, uint8_t* __restrict__ do_ext,
                                                            float inv_scale, float* __restrict__ dQacc,
                                                            void* __restrict__ dK, void* __restrict__ dV,
-                                                           int grad_f32, int kv_group, const PrepFrozen fz, int B,
-                                                           int H, int T) {
+                                                           int grad_f32, int kv_group,
+                                                           const int* __restrict__ qslot, int n_ord,
+                                                           const PrepFrozen fz, int B, int H, int T) {
   constexpr int TPR = D / 8;                       // threads per row
   const int Tpad = (T + 127) / 128 * 128;
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
@@ -263,8 +264,15 @@ __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat1
   if (valid) {
     const size_t grow = ((static_cast<size_t>(b) * H + h) * T + t) * D + part * 8;
     float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-    *reinterpret_cast<float4*>(dQacc + grow) = z;
-    *reinterpret_cast<float4*>(dQacc + grow + 4) = z;
+    if (qslot == nullptr) {
+      *reinterpret_cast<float4*>(dQacc + grow) = z;
+      *reinterpret_cast<float4*>(dQacc + grow + 4) = z;
+    } else if (!frozen) {
+      // packed layout: dQ has the ordinary heads only
+      const size_t prow = ((static_cast<size_t>(b) * n_ord + qslot[h]) * T + t) * D + part * 8;
+      *reinterpret_cast<float4*>(dQacc + prow) = z;
+      *reinterpret_cast<float4*>(dQacc + prow + 4) = z;
+    }
     if (kv_group > 1 && h % kv_group == 0) {
       // grouped-query path: the shared heads' gradients are accumulated by reduce-adds of the main kernel
       const size_t krow = ((static_cast<size_t>(b) * (H / kv_group) + h / kv_group) * T + t) * D + part * 8;
@@ -274,8 +282,8 @@ __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat1
       *reinterpret_cast<float4*>(static_cast<float*>(dV) + krow + 4) = z;
     }
     if (frozen) {
-      if (kv_group > 1) {
-        // nothing to zero per frozen head
+      if (kv_group > 1 || qslot != nullptr) {
+        // nothing to zero per frozen head (shared heads are zeroed above; the packed dK has no such row)
       } else if (grad_f32) {
         *reinterpret_cast<float4*>(static_cast<float*>(dK) + grow) = z;
         *reinterpret_cast<float4*>(static_cast<float*>(dK) + grow + 4) = z;
@@ -338,7 +346,8 @@ __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat1
 
 cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* os, const uint8_t* mask_dev,
                             void* q_ext, void* do_ext, float inv_scale, float* dQacc, void* dK, void* dV, int grad_f32,
-                            int kv_group, const PrepFrozen& fz, int B, int H, int T, int D, cudaStream_t st) {
+                            int kv_group, const int* qslot, int n_ord, const PrepFrozen& fz, int B, int H, int T, int D,
+                            cudaStream_t st) {
   const int Tpad = (T + 127) / 128 * 128;
   const long long nthreads = static_cast<long long>(B) * H * Tpad * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
@@ -346,12 +355,12 @@ cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, con
     saf_bwd_prep_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
                                                   static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2],
                                                   mask_dev, static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext),
-                                                  inv_scale, dQacc, dK, dV, grad_f32, kv_group, fz, B, H, T);
+                                                  inv_scale, dQacc, dK, dV, grad_f32, kv_group, qslot, n_ord, fz, B, H, T);
   else
     saf_bwd_prep_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
                                                    static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2],
                                                    mask_dev, static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext),
-                                                   inv_scale, dQacc, dK, dV, grad_f32, kv_group, fz, B, H, T);
+                                                   inv_scale, dQacc, dK, dV, grad_f32, kv_group, qslot, n_ord, fz, B, H, T);
   return cudaGetLastError();
 }
 

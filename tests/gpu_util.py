@@ -45,13 +45,14 @@ class Layer:
         self.alpha = torch.from_numpy(inp.alpha).to(dev)
         self.rho = torch.from_numpy(inp.rho).to(dev)
         self.logZ = torch.zeros_like(self.alpha)
-        self.O = torch.full_like(self.Q, float("nan"))
+        self.O = torch.full_like(self.dO, float("nan"))
         self.LSE = torch.full((wl.B, wl.H, wl.T), float("nan"), device=dev)
         gd = torch.float32 if grad_dtype == saf.SAF_F32 else torch.bfloat16
         self.grads = [torch.full(t.shape, float("nan"), device=dev, dtype=gd)
                       for t in (self.Q, self.K, self.V)] if backward else None
         self.prob = saf.make_problem(self.Q, wl.stored_len, softmax_scale=softmax_scale, grad_dtype=grad_dtype,
-                                     k_like=self.K, v_like=self.V, kv_group=wl.kv_group)
+                                     k_like=self.K, v_like=self.V, o_like=self.O, kv_group=wl.kv_group,
+                                     packed_qk=wl.packed_qk, H=wl.H)
         self.mask = inp.mask
 
     def run(self, backward=True, prepare=True):

@@ -349,6 +349,59 @@ def test_gqa_bf16_gradients_and_bad_group():
     assert e.value.code == 1
 
 
+# --------------------------------------------------------------------------- packed Q/K layout
+def _check_packed_layer(L, backward):
+    inp, wl = L.inp, L.inp.wl
+    q, k, v, do = f64(inp)
+    al, rh = inp.alpha.astype(np.float64), inp.rho.astype(np.float64)
+    O, LSE = L.host(L.O), L.host(L.LSE)
+    eO, eL = orc.hybrid_attn_fwd(q, k, v, inp.mask, al, rh)
+    for b in range(wl.B):
+        for h in range(wl.H):
+            assert_close(O[b, h], eO[b, h], f"O[{b},{h}]")
+            if inp.mask[h]:
+                assert not LSE[b, h].any()
+            else:
+                assert np.abs(LSE[b, h] - eL[b, h]).max() < 1e-4
+    if not backward:
+        return
+    dQ, dK, dV = (L.host(g) for g in L.grads)
+    eQ, eK, eV = orc.hybrid_attn_bwd(q, k, v, do, inp.mask, al, rh)
+    assert dQ.shape == eQ.shape and dK.shape == eK.shape and dV.shape == eV.shape
+    for b in range(wl.B):
+        for s_ in range(dQ.shape[1]):
+            assert_close(dQ[b, s_], eQ[b, s_], f"dQ[{b},slot {s_}]")
+            assert_close(dK[b, s_], eK[b, s_], f"dK[{b},slot {s_}]")
+        for h in range(wl.H):
+            assert_close(dV[b, h], eV[b, h], f"dV[{b},{h}]")
+
+
+@pytest.mark.parametrize("H,frozen,T,gd", [(6, (1, 4), 300, "f32"), (4, (0, 3), 129, "bf16"), (3, (), 200, "f32"),
+                                           (5, (0, 1, 2, 3), 257, "f32")])
+def test_packed_qk_layout_forward_backward(H, frozen, T, gd):
+    """Q, K, dQ, dK hold only the ordinary heads (Appendix E.2: replaced heads have no query/key slot)."""
+    wl = si.Workload("packed", 2, H, T, 64, frozen, -0.05, seed=50 + H + T, packed_qk=True)
+    L = Layer(si.generate(wl), grad_dtype=saf.SAF_F32 if gd == "f32" else saf.SAF_BF16).run()
+    if gd == "f32":
+        _check_packed_layer(L, True)
+    else:
+        L32 = Layer(L.inp).run()
+        for g32, g16 in zip(L32.grads, L.grads):
+            a, b = L32.host(g32), L.host(g16)
+            assert a.shape == b.shape and np.abs(a - b).max() <= 2.0 ** -8 * max(np.abs(a).max(), 1.0) + 1e-6
+
+
+def test_packed_qk_layout_head_dim_128_forward_and_errors():
+    wl = si.Workload("packed128", 1, 6, 384, 128, (1, 2, 5), -0.02, seed=57, packed_qk=True, backward=False)
+    L = Layer(si.generate(wl), backward=False).run(backward=False)
+    _check_packed_layer(L, False)
+    L = Layer(si.generate(si.Workload("packed-bad", 1, 4, 128, 64, (1,), -0.05, seed=58, packed_qk=True)))
+    L.prob.kv_group = 2                        # the packed layout is a multi-head layout
+    with pytest.raises(saf.SafError) as e:
+        L.run()
+    assert e.value.code == 1
+
+
 # --------------------------------------------------------------------------- full sizes, sampled
 def test_config1_full_size_sampled_units():
     wl = si.config(1)

@@ -38,8 +38,8 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_problem_struct_layout_matches_header(lib):
     # 8 x 4-byte fields then 4 x 3 x int64
-    assert ctypes.sizeof(lib.SafProblem) == 8 * 4 + 12 * 8
-    assert lib.SafProblem.q_strides.offset == 32
+    assert ctypes.sizeof(lib.SafProblem) == 10 * 4 + 12 * 8
+    assert lib.SafProblem.q_strides.offset == 40
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure mode")
