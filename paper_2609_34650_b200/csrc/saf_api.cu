@@ -101,12 +101,12 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // [B][H][T][D] bf16 tensor with element strides (batch, head, seq); box = 64 features x 128 rows,
 // 128-byte swizzle; rows beyond T read as zero.
 int make_map(saf_ctx* ctx, CUtensorMap* out, const void* base, const saf_problem* p, const int64_t* strides,
-             CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, int heads = 0) {
+             CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, int heads = 0, int box_rows = BLK) {
   cuuint64_t dims[4] = {static_cast<cuuint64_t>(p->D), static_cast<cuuint64_t>(p->T),
                         static_cast<cuuint64_t>(heads > 0 ? heads : p->H), static_cast<cuuint64_t>(p->B)};
   cuuint64_t gs[3] = {static_cast<cuuint64_t>(strides[2]) * 2, static_cast<cuuint64_t>(strides[1]) * 2,
                       static_cast<cuuint64_t>(strides[0]) * 2};
-  cuuint32_t box[4] = {64, BLK, 1, 1};
+  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(box_rows), 1, 1};
   cuuint32_t es[4] = {1, 1, 1, 1};
   CUresult r = ctx->encode(out, dtype, 4, const_cast<void*>(base), dims, gs, box, es,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -123,11 +123,12 @@ bool pattern_matches(const saf_ctx* ctx, const saf_problem* p, const uint8_t* ma
 }
 
 // map of a contiguous [B][Hn][T][D] fp16 workspace
-int make_map_contig(saf_ctx* ctx, CUtensorMap* out, const void* base, const saf_problem* p, int Hn) {
+int make_map_contig(saf_ctx* ctx, CUtensorMap* out, const void* base, const saf_problem* p, int Hn,
+                    int box_rows = BLK) {
   saf_problem q = *p;
   q.H = Hn;
   const int64_t st[3] = {static_cast<int64_t>(Hn) * p->T * p->D, static_cast<int64_t>(p->T) * p->D, p->D};
-  return make_map(ctx, out, base, &q, st, CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+  return make_map(ctx, out, base, &q, st, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 0, box_rows);
 }
 
 int check_strides(const int64_t* s, int D) {
@@ -567,7 +568,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   int nf = 0;
   int rc = validate(p, frozen_mask_host, &nf);
   if (rc) return rc;
-  if (p->D != 64) return SAF_ERR_UNSUPPORTED;
+  if (p->D != 64 && p->D != 128) return SAF_ERR_UNSUPPORTED;
   const int no = p->H - nf;
   const bool no_qk_out = p->packed_qk && no == 0;        // packed layout of a frozen-only layer: no dQ / dK at all
   if (!dO || !dV || (!no_qk_out && (!dQ || !dK))) return SAF_ERR_INVALID_ARG;
@@ -668,6 +669,66 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   } else {
     mq = mdo; mk = mdo; mv = mdo;
   }
+  if (p->D != 64) {
+    // ---- 128-wide kernel: Q / dO travel as 64-row half tiles, dK / dV leave with plain stores
+    CUtensorMap mqh = mdo, mdoh, mdoth, mdq128;
+    if ((rc = make_map(ctx, &mdoh, dO, p, p->o_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 0, 64))) return rc;
+    if (no > 0 && (rc = make_map(ctx, &mqh, Q, p, p->q_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, nqh, 64))) return rc;
+    mdoth = mdoh;
+    {
+      const cuuint64_t Dd = static_cast<cuuint64_t>(p->D), Tt = static_cast<cuuint64_t>(p->T);
+      const cuuint64_t Hq = static_cast<cuuint64_t>(std::max(nqh, 1));
+      cuuint64_t dims[4] = {Dd, Tt, Hq, static_cast<cuuint64_t>(p->B)};
+      cuuint64_t gs[3] = {Dd * 4, Tt * Dd * 4, Tt * Dd * 4 * Hq};
+      cuuint32_t box[4] = {32, BLK, 1, 1};
+      cuuint32_t es[4] = {1, 1, 1, 1};
+      if (ctx->encode(&mdq128, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, dqacc, dims, gs, box, es,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return SAF_ERR_CUDA;
+    }
+    BwdParams bp;
+    bp.band_b = nullptr; bp.avec = nullptr; bp.fast_ok = nullptr; bp.hord = nullptr; bp.ovf = nullptr; bp.call_id = 0;
+    bp.nblkp = (p->Tp + 127) / 128;
+    if (tensor_form) {
+      if ((rc = make_map_contig(ctx, &mdoth, ctx->dot_buf.ptr, p, nf, 64))) return rc;
+      bp.band_b = ctx->pat_bandb.ptr;
+      bp.avec = static_cast<const float*>(ctx->pat_avec.ptr);
+      bp.fast_ok = fz.pat_ok;
+      bp.hord = fz.hord;
+      bp.ovf = fz.ovf;
+      bp.call_id = fz.call_id;
+    }
+    bp.B = p->B; bp.H = p->H; bp.T = p->T; bp.Tp = p->Tp;
+    bp.kv_group = kvg;
+    bp.qslot = qslot;
+    bp.n_ord = no;
+    bp.d_real = p->D;
+    bp.scale = scale_v;
+    bp.scale_log2 = scale_v * 1.4426950408889634f;
+    bp.alpha = alpha; bp.rho = rho; bp.logZ = logZ;
+    bp.q_ext = q_ext;
+    bp.do_ext = do_ext;
+    bp.nblk = nblk;
+    bp.dK = dK_k; bp.dV = dV_k;
+    bp.grad_f32 = kern_f32;
+    bp.items = wl->items_dev;
+    bp.cta_offsets = wl->offsets_dev;
+    bp.status = ctx->status_dev;
+    bp.wait_limit_ns = ctx->wait_limit_ns;
+    {
+      ScopedTimer timer(ctx, SAF_KERNEL_BWD, st);
+      if (launch_bwd128(mk, mv, mqh, mdoh, mdoth, mdq128, bp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+    }
+    if (!grad_f32) {
+      ScopedTimer timer(ctx, SAF_KERNEL_BWD_FINALIZE, st);
+      if (nelem > 0 && launch_bwd_finalize(dqacc, dQ, nelem, st) != cudaSuccess) return SAF_ERR_CUDA;
+      if (kv_acc && (launch_bwd_finalize(static_cast<const float*>(dK_k), dK, nkv, st) != cudaSuccess ||
+                     launch_bwd_finalize(static_cast<const float*>(dV_k), dV, nkv, st) != cudaSuccess))
+        return SAF_ERR_CUDA;
+    }
+    return SAF_OK;
+  }
   // fp32 dQ accumulator [B][H][T][64] as a 4-D tensor for tiled reduce-adds: box = 32 floats x 128 rows
   // (dK and dV get maps of the same shape for the tiled stores of the fp32 epilogue)
   CUtensorMap mdq, mdk, mdv;
@@ -710,6 +771,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   bp.kv_group = kvg;
   bp.qslot = qslot;
   bp.n_ord = no;
+  bp.d_real = p->D;
   bp.scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
   bp.scale_log2 = bp.scale * 1.4426950408889634f;
   bp.alpha = alpha; bp.rho = rho; bp.logZ = logZ;

@@ -45,6 +45,7 @@ struct BwdParams {
   int B, H, T, Tp;
   int kv_group;                     // as in FwdParams; > 1: dK / dV are reduce-added instead of stored
   const int* qslot;                 // packed layout of Q, K, dQ, dK (see FwdParams)
+  int d_real;                       // head dimension of the tensors (128-wide kernel: 128 or 96)
   int n_ord;                        // number of ordinary heads (head count of the packed tensors)
   float scale, scale_log2;
   const float* alpha;
@@ -135,6 +136,12 @@ cudaError_t launch_bwd_finalize(const float* dQacc, void* dQ, size_t n, cudaStre
 cudaError_t launch_fwd64(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mvt,
                          const FwdParams& p, int grid, cudaStream_t st);
 int fwd64_smem_bytes();
+// head dimension 128 / 96 (saf_bwd128.cu): mqh / mdoh / mdoth are maps with 64-row boxes (half tiles), mdq the fp32 dQ
+// accumulator [B][Hq][T][D]; dK / dV are written with plain stores (reduce-adds for shared heads)
+cudaError_t launch_bwd128(const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mqh, const CUtensorMap& mdoh,
+                          const CUtensorMap& mdoth, const CUtensorMap& mdq, const BwdParams& p, int grid,
+                          cudaStream_t st);
+int bwd128_smem_bytes();
 int fwd_smem_bytes(int D);
 int bwd_smem_bytes(int D);
 
