@@ -85,12 +85,39 @@ def test_head_dim_96_forward(T, frozen, g):
     _check_gqa_layer(L, False)
 
 
-def test_backward_head_dim_128_is_reported_unsupported():
-    wl = si.Workload("d128b", 1, 2, 128, 128, (), -0.01, seed=5)
-    L = Layer(si.generate(wl))
-    with pytest.raises(saf.SafError) as e:
-        L.run()
-    assert e.value.code == 2
+@pytest.mark.parametrize("T,frozen", [(128, ()), (300, (1, 3)), (1, (0,)), (129, (0, 1, 2, 3)), (513, (2,))])
+def test_head_dim_128_forward_backward(T, frozen):
+    """The 128-wide backward kernel: ordinary heads and the tensor-core frozen form, ragged lengths."""
+    wl = si.Workload("d128fb", 2, 4, T, 128, frozen, -0.03, seed=128 + T)
+    L = Layer(si.generate(wl)).run()
+    check_units(L, all_units(wl))
+
+
+def test_head_dim_128_backward_general_frozen_form_and_bf16():
+    """Wide-range pattern (tensor-core form refused): P^^T half tiles with one exponential per element."""
+    wl = si.Workload("d128wide", 1, 3, 300, 128, (0, 2), -0.4, seed=131)
+    inp = si.generate(wl)
+    inp.alpha[0] *= 8.0
+    inp.do[:] = si.f32_to_bf16_bits(si.bf16_bits_to_f32(inp.do) / 16.0)
+    L = Layer(inp).run()
+    check_units(L, all_units(wl))
+    L16 = Layer(inp, grad_dtype=saf.SAF_BF16).run()
+    for g32, g16 in zip(L.grads, L16.grads):
+        a, b = L.host(g32), L.host(g16)
+        assert np.abs(a - b).max() <= 2.0 ** -8 * max(np.abs(a).max(), 1.0) + 1e-6
+
+
+def test_head_dim_128_backward_shared_and_packed_heads():
+    wl = si.Workload("d128gqa", 2, 8, 260, 128, (1, 6), -0.03, seed=132, kv_group=4)
+    _check_gqa_layer(Layer(si.generate(wl)).run(), True)
+    wl = si.Workload("d128packed", 2, 5, 200, 128, (0, 3), -0.03, seed=133, packed_qk=True)
+    _check_packed_layer(Layer(si.generate(wl)).run(), True)
+
+
+def test_head_dim_128_backward_many_items_per_cta():
+    wl = si.Workload("d128mix", 4, 6, 1100, 128, (0, 3, 4), -0.02, seed=134)
+    L = Layer(si.generate(wl)).run()
+    check_units(L, [(0, 0), (3, 5), (1, 3), (2, 1), (3, 4), (0, 2)])
 
 
 def test_multi_tile_scheduler_mix():
