@@ -48,7 +48,7 @@ enum { SAF_BF16 = 0, SAF_F32 = 1 };
 
 typedef struct {
   int32_t B, H, T, D;          /* square causal attention: T queries and T keys; D in {64, 96, 128}
-                                  (forward; the backward supports 64, the pattern gradients 64 and 128) */
+                                  (forward and backward; the pattern gradients 64 and 128) */
   int32_t Tp;                  /* stored pattern length (row length of alpha/rho/logZ); T <= Tp */
   float softmax_scale;         /* <= 0 selects 1/sqrt(D) (Appendix A) */
   int32_t grad_dtype;          /* dtype of dQ/dK/dV: SAF_F32 or SAF_BF16 */

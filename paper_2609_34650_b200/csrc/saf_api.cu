@@ -568,7 +568,6 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   int nf = 0;
   int rc = validate(p, frozen_mask_host, &nf);
   if (rc) return rc;
-  if (p->D != 64 && p->D != 128) return SAF_ERR_UNSUPPORTED;
   const int no = p->H - nf;
   const bool no_qk_out = p->packed_qk && no == 0;        // packed layout of a frozen-only layer: no dQ / dK at all
   if (!dO || !dV || (!no_qk_out && (!dQ || !dK))) return SAF_ERR_INVALID_ARG;

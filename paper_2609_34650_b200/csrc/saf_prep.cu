@@ -233,7 +233,8 @@ __device__ __forceinline__ uint4 split3_bf16(float x) {
 //   every head   : dQacc row = 0 (it is accumulated by reduce-adds of the main kernel)
 //   frozen head  : dK row = 0 (no key gradient; Sec. 3.3); with the tensor-core form, the row w(i) dO in fp16
 // Image layout per 128-row block (4 KB): byte (n/8)*256 + (k/8)*128 + (n%8)*16 + (k%8)*2 for row n, column k < 16.
-template <int D>
+// (TPR threads per row: D / 8, or 16 with four idle ones at D = 96 so that a row stays inside a warp)
+template <int D, int TPR>
 __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat16* __restrict__ O,
                                                            const __nv_bfloat16* __restrict__ dO,
                                                            const float* __restrict__ LSE, int64_t os0, int64_t os1,
@@ -244,7 +245,6 @@ __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat1
                                                            int grad_f32, int kv_group,
                                                            const int* __restrict__ qslot, int n_ord,
                                                            const PrepFrozen fz, int B, int H, int T) {
-  constexpr int TPR = D / 8;                       // threads per row
   const int Tpad = (T + 127) / 128 * 128;
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
   const long long rowid = gid / TPR;               // over [B][H][Tpad]
@@ -261,7 +261,7 @@ __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat1
     frozen = mask[h] != 0;
     valid = t < T;
   }
-  if (valid) {
+  if (valid && part * 8 < D) {
     const size_t grow = ((static_cast<size_t>(b) * H + h) * T + t) * D + part * 8;
     float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
     if (qslot == nullptr) {
@@ -349,18 +349,17 @@ cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, con
                             int kv_group, const int* qslot, int n_ord, const PrepFrozen& fz, int B, int H, int T, int D,
                             cudaStream_t st) {
   const int Tpad = (T + 127) / 128 * 128;
-  const long long nthreads = static_cast<long long>(B) * H * Tpad * (D / 8);
+  const int tpr = D == 96 ? 16 : D / 8;
+  const long long nthreads = static_cast<long long>(B) * H * Tpad * tpr;
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
-  if (D == 64)
-    saf_bwd_prep_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
-                                                  static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2],
-                                                  mask_dev, static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext),
-                                                  inv_scale, dQacc, dK, dV, grad_f32, kv_group, qslot, n_ord, fz, B, H, T);
-  else
-    saf_bwd_prep_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
-                                                   static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2],
-                                                   mask_dev, static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext),
-                                                   inv_scale, dQacc, dK, dV, grad_f32, kv_group, qslot, n_ord, fz, B, H, T);
+#define SAF_PREP_ARGS                                                                                              \
+  static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2], mask_dev, \
+      static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext), inv_scale, dQacc, dK, dV, grad_f32, kv_group,   \
+      qslot, n_ord, fz, B, H, T
+  if (D == 64) saf_bwd_prep_kernel<64, 8><<<grid, 256, 0, st>>>(SAF_PREP_ARGS);
+  else if (D == 96) saf_bwd_prep_kernel<96, 16><<<grid, 256, 0, st>>>(SAF_PREP_ARGS);
+  else saf_bwd_prep_kernel<128, 16><<<grid, 256, 0, st>>>(SAF_PREP_ARGS);
+#undef SAF_PREP_ARGS
   return cudaGetLastError();
 }
 

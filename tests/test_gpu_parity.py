@@ -85,6 +85,13 @@ def test_head_dim_96_forward(T, frozen, g):
     _check_gqa_layer(L, False)
 
 
+@pytest.mark.parametrize("T,frozen,g", [(300, (1, 2), 1), (130, (), 1), (260, (0, 3), 2)])
+def test_head_dim_96_forward_backward(T, frozen, g):
+    """Head dimension 96 (the paper's 1B model) through the 128-wide kernels, gradients with row length 96."""
+    wl = si.Workload("d96fb", 2, 4, T, 96, frozen, -0.03, seed=196 + T, kv_group=g)
+    _check_gqa_layer(Layer(si.generate(wl)).run(), True)
+
+
 @pytest.mark.parametrize("T,frozen", [(128, ()), (300, (1, 3)), (1, (0,)), (129, (0, 1, 2, 3)), (513, (2,))])
 def test_head_dim_128_forward_backward(T, frozen):
     """The 128-wide backward kernel: ordinary heads and the tensor-core frozen form, ragged lengths."""
