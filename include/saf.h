@@ -48,7 +48,7 @@ enum { SAF_BF16 = 0, SAF_F32 = 1 };
 
 typedef struct {
   int32_t B, H, T, D;          /* square causal attention: T queries and T keys; D in {64, 96, 128}
-                                  (forward and backward; the pattern gradients 64 and 128) */
+                                  (96 runs on the 128-wide kernels) */
   int32_t Tp;                  /* stored pattern length (row length of alpha/rho/logZ); T <= Tp */
   float softmax_scale;         /* <= 0 selects 1/sqrt(D) (Appendix A) */
   int32_t grad_dtype;          /* dtype of dQ/dK/dV: SAF_F32 or SAF_BF16 */
@@ -142,7 +142,7 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
  *   dalpha_out[h][j] = sum_b sum_{i>=j} dL/db_ij,   drho_out[h][d] = sum_b sum_{i-j=d} dL/db_ij.
  * V: bf16 [B][H/kv_group][T][D] (v_strides); O, dO: bf16 [B][H][T][D] (o_strides), O as returned by the forward;
  * alpha, rho, logZ: device fp32 [H][Tp] (logZ as from saf_pattern_prepare); dalpha_out, drho_out: device fp32
- * [H][Tp], fully overwritten (rows of ordinary heads and entries beyond T with zeros).  D in {64, 128}.
+ * [H][Tp], fully overwritten (rows of ordinary heads and entries beyond T with zeros).
  * After an update of alpha/rho the caller refreshes logZ with saf_pattern_prepare. */
 int saf_pattern_grad(saf_ctx* ctx, const saf_problem* problem, const void* V, const void* O, const void* dO,
                      const uint8_t* frozen_mask_host, const float* alpha, const float* rho, const float* logZ,

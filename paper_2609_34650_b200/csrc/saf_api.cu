@@ -897,7 +897,6 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
   int nf = 0;
   int rc = validate(p, frozen_mask_host, &nf);
   if (rc) return rc;
-  if (p->D == 96) return SAF_ERR_UNSUPPORTED;
   DeviceGuard g(ctx->device);
   if (!g.ok) return SAF_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -952,7 +951,8 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
   gp.wait_limit_ns = ctx->wait_limit_ns;
   {
     ScopedTimer timer(ctx, SAF_KERNEL_PGRAD, st);
-    if (launch_pgrad(p->D, mv, mdo, gp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+    // (head dimension 96 runs on the 128-wide kernel: TMA zero-fills features 96..127)
+    if (launch_pgrad(p->D == 96 ? 128 : p->D, mv, mdo, gp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
   }
   return SAF_OK;
 }

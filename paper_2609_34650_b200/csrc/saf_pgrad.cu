@@ -264,13 +264,13 @@ saf_pgrad_kernel(const __grid_constant__ CUtensorMap mv, const __grid_constant__
   if (warp == 9) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
-// delta[b][h][t] = sum_c dO[b][h][t][c] * O[b][h][t][c] for the frozen heads (hlist), one warp per row.
-template <int D>
+// delta[b][h][t] = sum_c dO[b][h][t][c] * O[b][h][t][c] for the frozen heads (hlist); TPR threads per row, eight
+// features each (16 threads with four idle ones at D = 96, so that a row stays inside a warp).
+template <int D, int TPR>
 __global__ void __launch_bounds__(256) saf_rowdot_kernel(const __nv_bfloat16* __restrict__ O,
                                                          const __nv_bfloat16* __restrict__ dO, int64_t s0, int64_t s1,
                                                          int64_t s2, const int* __restrict__ hlist,
                                                          float* __restrict__ delta, int B, int H, int Hf, int T) {
-  constexpr int TPR = D / 8;                       // threads per row, eight features each
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
   const long long rowid = gid / TPR;               // over [B][Hf][T]
   const int part = static_cast<int>(gid % TPR);
@@ -281,6 +281,8 @@ __global__ void __launch_bounds__(256) saf_rowdot_kernel(const __nv_bfloat16* __
     t = static_cast<int>(rowid % T);
     h = hlist[(rowid / T) % Hf];
     b = static_cast<int>(rowid / (static_cast<long long>(T) * Hf));
+  }
+  if (inrange && part * 8 < D) {
     const int64_t off = b * s0 + h * s1 + static_cast<int64_t>(t) * s2 + part * 8;
     const uint4 o4 = *reinterpret_cast<const uint4*>(O + off);
     const uint4 d4 = *reinterpret_cast<const uint4*>(dO + off);
@@ -300,16 +302,15 @@ __global__ void __launch_bounds__(256) saf_rowdot_kernel(const __nv_bfloat16* __
 
 cudaError_t launch_rowdot(const void* O, const void* dO, const int64_t* os, const int* hlist, float* delta, int B, int H,
                           int Hf, int T, int D, cudaStream_t st) {
-  const long long nthreads = static_cast<long long>(B) * Hf * T * (D / 8);
+  const int tpr = D == 96 ? 16 : D / 8;
+  const long long nthreads = static_cast<long long>(B) * Hf * T * tpr;
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
-  if (D == 64)
-    saf_rowdot_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
-                                                static_cast<const __nv_bfloat16*>(dO), os[0], os[1], os[2], hlist, delta,
-                                                B, H, Hf, T);
-  else
-    saf_rowdot_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(O),
-                                                 static_cast<const __nv_bfloat16*>(dO), os[0], os[1], os[2], hlist,
-                                                 delta, B, H, Hf, T);
+#define SAF_ROWDOT_ARGS \
+  static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), os[0], os[1], os[2], hlist, delta, B, H, Hf, T
+  if (D == 64) saf_rowdot_kernel<64, 8><<<grid, 256, 0, st>>>(SAF_ROWDOT_ARGS);
+  else if (D == 96) saf_rowdot_kernel<96, 16><<<grid, 256, 0, st>>>(SAF_ROWDOT_ARGS);
+  else saf_rowdot_kernel<128, 16><<<grid, 256, 0, st>>>(SAF_ROWDOT_ARGS);
+#undef SAF_ROWDOT_ARGS
   return cudaGetLastError();
 }
 

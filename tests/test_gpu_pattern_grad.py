@@ -64,6 +64,12 @@ def test_pattern_grads_head_dim_128_and_shared_value_heads():
     _check(L)
 
 
+def test_pattern_grads_head_dim_96():
+    wl = si.Workload("pg96", 2, 4, 300, 96, (0, 3), -0.03, seed=74, backward=False)
+    L = Layer(si.generate(wl), backward=False).run(backward=False)
+    _check(L)
+
+
 def test_pattern_grads_many_items_per_cta():
     """8 x 6 frozen heads x 9 key blocks = 432 items on 296 CTAs, ragged last block."""
     wl = si.Workload("pgmix", 8, 8, 1100, 64, (0, 2, 3, 5, 6, 7), -0.01, seed=73)
