@@ -341,11 +341,12 @@ def run_ours(args):
     prep_ms = k_prep[0] / max(k_prep[1], 1)
     achieved = bwd_flops / (bwd_ms * 1e-3) / 1e12
     traffic = None
+    bwd_name = "saf_bwd_kernel" if wl.D == 64 else "saf_bwd128_kernel"
     tpath = os.path.join(ROOT, "profiles", "roofline_traffic.json")
     if os.path.exists(tpath):
         with open(tpath) as f:
-            traffic = json.load(f).get(f"saf_bwd_kernel@{wl.name}")
-    roofline = {"bound": "tensor", "kernel": "saf_bwd_kernel", "achieved": achieved, "peak": peaks["bf16_tflops"],
+            traffic = json.load(f).get(f"{bwd_name}@{wl.name}")
+    roofline = {"bound": "tensor", "kernel": bwd_name, "achieved": achieved, "peak": peaks["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": traffic,
                 "peak_source": f"{peaks['source']} bf16 burst (MEASURED_PEAKS.json)" if peaks["source"] == "measured"
                 else "fallback 1590 TFLOP/s",
@@ -362,7 +363,7 @@ def run_ours(args):
         "config": {"workload": wl.name, "B_per_gpu": wl.B, "H": wl.H, "Hf": len(wl.frozen_heads), "T": wl.T, "D": wl.D,
                    "grad_dtype": "f32", "frozen_fraction": len(wl.frozen_heads) / wl.H,
                    "flops_per_step_per_gpu": flops_local,
-                   "l2": "inputs+outputs per step (0.55 GB) exceed the 126 MB L2; no explicit flush",
+                   "l2": f"inputs+outputs per step ({(4 * 2 + 3 * 4) * nel / 1e9:.2f} GB) exceed the 126 MB L2; no explicit flush",
                    "pattern_prepare": "once before the timed steps (static per layer)", "pattern_prepare_ms": prepare_ms,
                    "parallelism": f"dp{world} (independent batches, no collective in the layer)"},
         "pct_of_bf16_peak": 100.0 * value / (peaks["bf16_tflops"] * world),
@@ -387,7 +388,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3])
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 5, 6])
     ap.add_argument("--ref-budget", type=float, default=12.0, help="seconds of CPU-oracle work per sample")
     args = ap.parse_args()
     if args.impl == "reference":

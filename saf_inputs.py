@@ -85,7 +85,9 @@ def sweep_frozen_heads(H: int, n_frozen: int, seed: int = 0) -> tuple:
 
 def config(k: int, n_frozen: int | None = None, seed: int = 0) -> Workload:
     """The five benchmark/test configurations (k = 0..4).  `n_frozen` overrides the frozen count
-    (config 3 is config 1's shape with n_frozen in {0,3,6,9,12})."""
+    (config 3 is config 1's shape with n_frozen in {0,3,6,9,12}).  k = 5, 6 are two extra shapes for the wider
+    head dimensions: config 1's layer at head dimension 128, and the layer of the paper's 1B model (16 heads of
+    dimension 96, batch 2 per rank, 8K context)."""
     if k == 0:
         nf = 1 if n_frozen is None else n_frozen
         return Workload("tiny", 1, 4, 256, 64, sweep_frozen_heads(4, nf, seed), -0.05, seed=seed)
@@ -100,6 +102,12 @@ def config(k: int, n_frozen: int | None = None, seed: int = 0) -> Workload:
         nf = 8 if n_frozen is None else n_frozen
         return Workload("prefill-32k-d128", 1, 32, 32768, 128, sweep_frozen_heads(32, nf, seed),
                         -0.002, alpha0_spike=4.0, backward=False, seed=seed)
+    if k == 5:
+        nf = 3 if n_frozen is None else n_frozen
+        return Workload("124m-4k-d128", 8, 12, 4096, 128, sweep_frozen_heads(12, nf, seed), -0.05, seed=seed)
+    if k == 6:
+        nf = 4 if n_frozen is None else n_frozen
+        return Workload("1b-paper-8k-d96", 2, 16, 8192, 96, sweep_frozen_heads(16, nf, seed), -0.01, seed=seed)
     raise ValueError(f"unknown config {k}")
 
 
