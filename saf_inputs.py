@@ -151,3 +151,32 @@ def generate(wl: Workload) -> Inputs:
         alpha[h] = a.astype(np.float32)
         rho[h] = (wl.rho_slope * d + 0.1 * noise).astype(np.float32)
     return Inputs(wl, q, k, v, do, alpha, rho, wl.mask)
+
+
+# --------------------------------------------------------------------------- inputs of the compact-pattern fitter
+def mean_attention_maps(Hf: int, T: int, seed: int = 0, upper_fill: float = 0.0, pmax: float = 3.0) -> np.ndarray:
+    """Synthetic stand-ins for calibration-time mean attention maps, float32 [Hf, T, T].
+
+    Row i holds positive weights over keys j <= i that sum to one: a power-law decay in the distance i-j (exponent
+    drawn per head from U(1,pmax), so far entries fall below the fitter's 1e-9 floor), a per-head weight on key 0
+    (U(0,0.5), attention-sink-like), a per-key factor and element-wise log-normal noise (sigma 0.3), then scaled so
+    that the row sums to one.  Entries above the diagonal are `upper_fill` (a consumer must ignore them).
+    Draw order per head: exponent, sink weight, key factors [T], noise [T,T].
+    """
+    rng = np.random.default_rng(seed)
+    out = np.empty((Hf, T, T), dtype=np.float32)
+    i = np.arange(T)[:, None]
+    j = np.arange(T)[None, :]
+    causal = j <= i
+    dist = np.where(causal, i - j, 0).astype(np.float64)
+    for h in range(Hf):
+        p = rng.uniform(1.0, pmax)
+        sink = rng.uniform(0.0, 0.5)
+        keyf = np.exp(0.5 * rng.standard_normal(T))
+        noise = np.exp(0.3 * rng.standard_normal((T, T), dtype=np.float32).astype(np.float64))
+        w = (1.0 + dist) ** (-p) * keyf[None, :] * noise
+        w = np.where(causal, w, 0.0)
+        w = w / w.sum(axis=1, keepdims=True) * (1.0 - sink)
+        w[:, 0] += sink
+        out[h] = np.where(causal, w, upper_fill).astype(np.float32)
+    return out
