@@ -168,6 +168,81 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------- GPU arm
+# --------------------------------------------------------------------------- the one-time fitter (extra leg)
+def fit_leg(ctx, saf, wl, peaks, dev, steps=400):
+    """Times the compact-pattern fitter on the heads one intervention of this model shape would fit: target marginals
+    of synthetic mean attention maps, then `steps` Adam steps for all heads at once, then the oracle on a bounded
+    sample of the same work.  Returns the dict reported under "fit"."""
+    import torch
+    from oracle import saf_fit_oracle as fo
+
+    T = wl.T
+    if T > 16384 or not len(wl.frozen_heads):
+        return None
+    Hf = max(1, min(12 * len(wl.frozen_heads), int(3.2e9 // (4 * T * T))))
+    base = si.mean_attention_maps(min(3, Hf), T, seed=wl.seed + 77)
+    A = torch.from_numpy(base).to(dev)
+    A = A[torch.arange(Hf, device=dev) % A.shape[0]].contiguous()
+    ea = torch.empty(Hf, T, dtype=torch.float64, device=dev)
+    er = torch.empty_like(ea)
+    pl = torch.empty(Hf, dtype=torch.float64, device=dev)
+    fa, fr, fz = (torch.empty(Hf, T, device=dev) for _ in range(3))
+    loss = torch.empty(Hf, dtype=torch.float64, device=dev)
+    kl = torch.empty_like(loss)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    for _ in range(3):
+        ctx.saf_fit_marginals(Hf, T, A, 1e-9, ea, er, pl)
+    a, b = ev(), ev()
+    a.record()
+    for _ in range(5):
+        ctx.saf_fit_marginals(Hf, T, A, 1e-9, ea, er, pl)
+    b.record()
+    torch.cuda.synchronize()
+    marg_ms = a.elapsed_time(b) / 5
+    ctx.saf_fit_compact(Hf, T, ea, er, pl, 20, 0.05, fa, fr, fz, T, loss, kl)       # warm-up
+    a, b = ev(), ev()
+    a.record()
+    ctx.saf_fit_compact(Hf, T, ea, er, pl, steps, 0.05, fa, fr, fz, T, loss, kl)
+    b.record()
+    torch.cuda.synchronize()
+    fit_ms = a.elapsed_time(b)
+    code, detail = ctx.saf_last_device_status()
+    if code != saf.SAF_OK:
+        raise RuntimeError(f"fitter: device status {code} detail {detail:#x}")
+    pairs = T * (T + 1) // 2
+    # special-function-unit bound: 16 exp2 per clock per SM, 148 SMs, at the maximum SM clock
+    mufu_peak = 16 * 148 * 1.965e9
+    exps_min = 2 * pairs * Hf * steps            # one exponential per causal pair for the normalisers, one for the marginals
+    exps_run = 3 * pairs * Hf * steps            # the marginal pass evaluates each pair twice (once per marginal)
+    marg_bytes = 4 * pairs * Hf
+    # the oracle on a bounded sample: one head, a few Adam steps at this T (dense fp64)
+    t0 = time.perf_counter()
+    P0 = fo.target_from_mean_attention(base[0])
+    oea, oer, _ = fo.marginals(P0)
+    t1 = time.perf_counter()
+    osteps = 2
+    fo.fit_compact(oea, oer, steps=osteps)
+    t2 = time.perf_counter()
+    kl_h = kl.cpu().numpy()
+    return {
+        "heads": Hf, "T": T, "adam_steps": steps, "fit_ms": fit_ms, "marginals_ms": marg_ms,
+        "kappa_min_max": [float(kl_h.min()), float(kl_h.max())], "accepted": int((kl_h <= 0.2).sum()),
+        "roofline_fit": {"bound": "alu", "kernel": "saf_fit_pass_kernel", "unit": "Gexp2/s",
+                         "achieved": exps_min / (fit_ms * 1e-3) / 1e9, "executed": exps_run / (fit_ms * 1e-3) / 1e9,
+                         "peak": mufu_peak / 1e9, "frac": exps_min / (fit_ms * 1e-3) / mufu_peak,
+                         "peak_source": "16 exp2/clk/SM x 148 SMs x 1.965 GHz"},
+        "roofline_marginals": {"bound": "hbm", "kernel": "saf_fit_marginals_kernel", "unit": "GB/s",
+                               "achieved": marg_bytes / (marg_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                               "frac": marg_bytes / (marg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "cpu_oracle": {"marginals_s_per_head": t1 - t0, "fit_s_per_head_per_step": (t2 - t1) / osteps,
+                       "fit_s_extrapolated": (t2 - t1) / osteps * steps * Hf,
+                       "sample": f"1 of {Hf} heads, {osteps} of {steps} Adam steps, dense fp64 numpy"},
+    }
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -355,6 +430,7 @@ def run_ours(args):
                                                       "frac": fwd_flops / (fwd_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]},
                                   "saf_bwd_prep_kernel": {"launch_ms": prep_ms}}}
 
+    fit = None if args.no_fit else fit_leg(ctx, saf, wl, peaks, dev)
     cpu_v, cpu_desc, cpu_threads, _ = oracle_sample(si.config(args.config), budget_s=args.ref_budget)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -375,6 +451,7 @@ def run_ours(args):
         "gpu_launches": (4 if len(wl.frozen_heads) else 3) * args.steps,
         "clocks": clocks,
         "roofline": roofline,
+        "fit": fit,
         "cpu_baseline": {"value": cpu_v, "unit": UNIT, "cores": cpu_threads, "kind": "oracle", "sample": cpu_desc},
     }
     print(json.dumps(line), flush=True)
@@ -389,6 +466,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 5, 6])
+    ap.add_argument("--no-fit", action="store_true", help="skip the extra leg that times the one-time fitter")
     ap.add_argument("--ref-budget", type=float, default=12.0, help="seconds of CPU-oracle work per sample")
     args = ap.parse_args()
     if args.impl == "reference":

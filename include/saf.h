@@ -148,6 +148,38 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* problem, const void* V, co
                      const uint8_t* frozen_mask_host, const float* alpha, const float* rho, const float* logZ,
                      float* dalpha_out, float* drho_out, void* stream);
 
+/* Compact-pattern fitter, step 1: sufficient statistics of the target (Sec. 3.2 "Fitting", text below
+ * Eq. "fit-objective"; Algorithm 1, fitting loop).  For each of `Hf` heads the causal entries (j <= i) of the mean
+ * attention map are floored at `floor_value` (the paper uses 1e-9) and every row is scaled to sum to one; of that
+ * target P the call returns eta_abs(j) = sum_{i>=j} P(i,j), eta_rel(d) = sum_{i-j=d} P(i,j) and sum_{ij} P log P
+ * (natural log), which is what the acceptance test needs besides the two marginals.
+ *   mean_attn   : device float32 [Hf, T, T] row-major (row = query); entries above the diagonal are never read.
+ *                 Read once; not modified.
+ *   eta_abs_out, eta_rel_out : device float64 [Hf, T]; plogp_out : device float64 [Hf].  Overwritten.
+ * T <= 16384 (SAF_ERR_UNSUPPORTED beyond); Hf = 0 is a no-op; Hf <= 65535.  Asynchronous on `stream`.  The sums are
+ * accumulated with floating-point atomics: results agree from run to run to rounding, not bit for bit. */
+int saf_fit_marginals(saf_ctx* ctx, int32_t Hf, int32_t T, const float* mean_attn, float floor_value,
+                      double* eta_abs_out, double* eta_rel_out, double* plogp_out, void* stream);
+
+/* Compact-pattern fitter, step 2: Fit and acceptance statistic (Eq. "fit-objective"; appendix "Selection, fitting,
+ * and installation": alpha = 0, rho(d) = log max(eta_rel(d)/(T-d), 1e-9), then `steps` Adam steps (beta1 0.9,
+ * beta2 0.999, eps 1e-8, bias-corrected) at learning rate `lr` on
+ * L = (1/T)[sum_i log Z(i) - sum_j eta_abs(j) alpha(j) - sum_d eta_rel(d) rho(d)]; the paper uses 400 steps at 0.05).
+ * All heads are fitted together; nothing of size T x T is allocated (state: 68 bytes per head and position, held by
+ * the context and reused).  Exponentials are fp32, the sums that feed Adam and Adam itself fp64.
+ *   eta_abs, eta_rel : device float64 [Hf, T] (from saf_fit_marginals, or accumulated by the caller)
+ *   plogp            : device float64 [Hf] or NULL if kl_out is NULL
+ *   alpha_out, rho_out, logZ_out : device float32, row h at offset h*out_stride (out_stride >= T elements): the
+ *                      fitted parameters and log Z(i) of Eq. "compact-prior", as saf_attn_fwd takes them
+ *   loss_out         : device float64 [Hf] or NULL: L at the fitted parameters
+ *   kl_out           : device float64 [Hf] or NULL: kappa = mean row KL(P || P^) = L + plogp/T; the paper accepts a
+ *                      head when kappa <= 0.2 nats (the caller compares)
+ * steps = 0 returns the starting point.  T <= 16384 (SAF_ERR_UNSUPPORTED beyond).  Asynchronous on `stream`
+ * (2*steps + 3 kernel launches). */
+int saf_fit_compact(saf_ctx* ctx, int32_t Hf, int32_t T, const double* eta_abs, const double* eta_rel,
+                    const double* plogp, int32_t steps, double lr, float* alpha_out, float* rho_out, float* logZ_out,
+                    int64_t out_stride, double* loss_out, double* kl_out, void* stream);
+
 /* Device-side status of the most recent launches on this context: SAF_OK or SAF_ERR_DEVICE_TIMEOUT.
  * Synchronises the context's device status word with the host (blocks until the stream used by the
  * last call has drained).  `detail_out` (may be NULL) receives the raw word: site and CTA that gave up. */
@@ -165,7 +197,9 @@ enum {
   SAF_KERNEL_LOGZ = 4,         /* pattern normalisers and tables (saf_pattern_prepare) */
   SAF_KERNEL_SCALE = 5,        /* per-call row scaling of the frozen heads' V (forward) / dO (backward) */
   SAF_KERNEL_PGRAD = 6,        /* pattern-gradient kernel (saf_pattern_grad) */
-  SAF_KERNEL_COUNT = 7
+  SAF_KERNEL_FIT = 7,          /* all launches of one saf_fit_compact call, as one interval */
+  SAF_KERNEL_FIT_MARGINALS = 8,/* target marginals (saf_fit_marginals) */
+  SAF_KERNEL_COUNT = 9
 };
 int saf_set_profiling(saf_ctx* ctx, int32_t enable);
 int saf_get_kernel_time(saf_ctx* ctx, int32_t which, float* total_ms_out, int32_t* launches_out);

@@ -18,6 +18,7 @@ SAF_OK = 0
 SAF_ERR_INVALID_ARG, SAF_ERR_UNSUPPORTED, SAF_ERR_CUDA, SAF_ERR_DEVICE_TIMEOUT, SAF_ERR_ARCH, SAF_ERR_NOMEM = range(1, 7)
 SAF_BF16, SAF_F32 = 0, 1
 SAF_KERNEL_FWD, SAF_KERNEL_BWD, SAF_KERNEL_BWD_PREP, SAF_KERNEL_BWD_FINALIZE, SAF_KERNEL_LOGZ, SAF_KERNEL_SCALE = range(6)
+SAF_KERNEL_PGRAD, SAF_KERNEL_FIT, SAF_KERNEL_FIT_MARGINALS = 6, 7, 8
 
 
 class SafProblem(C.Structure):
@@ -57,6 +58,8 @@ def load_library() -> C.CDLL:
     lib.saf_hybrid_attn_bwd.argtypes = [vp, pp, vp, vp, vp, vp, vp, f32p, u8p, f32p, f32p, f32p, vp, vp, vp, vp]
     lib.saf_hybrid_attn_step_host.argtypes = [vp, pp, vp, vp, vp, vp, u8p, f32p, f32p, i32, vp, f32p, vp, vp, vp]
     lib.saf_pattern_grad.argtypes = [vp, pp, vp, vp, vp, u8p, f32p, f32p, f32p, f32p, f32p, vp]
+    lib.saf_fit_marginals.argtypes = [vp, i32, i32, vp, C.c_float, vp, vp, vp, vp]
+    lib.saf_fit_compact.argtypes = [vp, i32, i32, vp, vp, vp, i32, C.c_double, vp, vp, vp, C.c_int64, vp, vp, vp]
     lib.saf_last_device_status.argtypes = [vp, C.POINTER(C.c_int32)]
     lib.saf_set_profiling.argtypes = [vp, i32]
     lib.saf_get_kernel_time.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
@@ -65,7 +68,7 @@ def load_library() -> C.CDLL:
     lib.saf_build_worklist.argtypes = [i32, i32, i32, u8p, i32, i32, i32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     for name in ("saf_create", "saf_destroy", "saf_pattern_prepare", "saf_hybrid_attn_fwd", "saf_hybrid_attn_bwd",
                  "saf_hybrid_attn_step_host", "saf_last_device_status", "saf_build_worklist", "saf_set_profiling",
-                 "saf_get_kernel_time", "saf_pattern_grad"):
+                 "saf_get_kernel_time", "saf_pattern_grad", "saf_fit_marginals", "saf_fit_compact"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -182,6 +185,15 @@ class Context:
         _check(self._lib.saf_pattern_grad(self._h, C.byref(prob), _ptr(V), _ptr(O), _ptr(dO), mp, _ptr(alpha),
                                           _ptr(rho), _ptr(logZ), _ptr(dalpha), _ptr(drho), _stream()),
                "saf_pattern_grad")
+
+    def saf_fit_marginals(self, Hf, T, mean_attn, floor_value, eta_abs, eta_rel, plogp):
+        _check(self._lib.saf_fit_marginals(self._h, int(Hf), int(T), _ptr(mean_attn), float(floor_value), _ptr(eta_abs),
+                                           _ptr(eta_rel), _ptr(plogp), _stream()), "saf_fit_marginals")
+
+    def saf_fit_compact(self, Hf, T, eta_abs, eta_rel, plogp, steps, lr, alpha, rho, logZ, out_stride, loss, kl):
+        _check(self._lib.saf_fit_compact(self._h, int(Hf), int(T), _ptr(eta_abs), _ptr(eta_rel), _ptr(plogp),
+                                         int(steps), float(lr), _ptr(alpha), _ptr(rho), _ptr(logZ), int(out_stride),
+                                         _ptr(loss), _ptr(kl), _stream()), "saf_fit_compact")
 
     def saf_hybrid_attn_step_host(self, prob, Q, K, V, dO, mask, alpha, rho, prepare, O, LSE, dQ, dK, dV):
         """All tensor arguments are HOST tensors (torch CPU tensors, ideally pinned) or None."""

@@ -65,7 +65,7 @@ struct saf_ctx {
   // tensor-core form of frozen heads: tables built by saf_pattern_prepare, scaled V / dO per call
   PatternCache pat;
   bool tensor_pattern = true;              // SAF_DISABLE_TENSOR_PATTERN=1 turns the form off
-  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, vt_buf, dot_buf, ok_fwd, ok_bwd, pg_hlist, pg_delta;
+  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, vt_buf, dot_buf, ok_fwd, ok_bwd, pg_hlist, pg_delta, fit_buf;
   bool profiling = false;
   std::vector<TimedLaunch> timed;          // event pairs recorded since the last query
   std::vector<cudaEvent_t> event_pool;
@@ -377,7 +377,7 @@ int saf_destroy(saf_ctx* ctx) {
     cudaFree(e.offsets_dev);
   }
   DevBuf* pbufs[] = {&ctx->pat_consts, &ctx->pat_ok, &ctx->pat_avec, &ctx->pat_wvec, &ctx->pat_bandf, &ctx->pat_bandb,
-                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta};
+                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta, &ctx->fit_buf};
   for (DevBuf* b : pbufs) release(*b);
   DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->dkacc_buf, &ctx->dvacc_buf, &ctx->qslot_buf, &ctx->hq, &ctx->hk, &ctx->hv,
                     &ctx->hdo, &ctx->ho, &ctx->hlse, &ctx->hdq, &ctx->hdk, &ctx->hdv, &ctx->halpha, &ctx->hrho,
@@ -954,6 +954,59 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
     // (head dimension 96 runs on the 128-wide kernel: TMA zero-fills features 96..127)
     if (launch_pgrad(p->D == 96 ? 128 : p->D, mv, mdo, gp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
   }
+  return SAF_OK;
+}
+
+int saf_fit_marginals(saf_ctx* ctx, int32_t Hf, int32_t T, const float* mean_attn, float floor_value,
+                      double* eta_abs_out, double* eta_rel_out, double* plogp_out, void* stream) {
+  if (!ctx || !eta_abs_out || !eta_rel_out || !plogp_out) return SAF_ERR_INVALID_ARG;
+  if (Hf < 0 || T < 1 || !(floor_value > 0.0f)) return SAF_ERR_INVALID_ARG;
+  if (T > fit_max_T()) return SAF_ERR_UNSUPPORTED;
+  if (Hf == 0) return SAF_OK;
+  if (!mean_attn || Hf > 65535) return SAF_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ctx->last_stream = st;
+  const size_t vb = static_cast<size_t>(Hf) * T * sizeof(double);
+  if (cudaMemsetAsync(eta_abs_out, 0, vb, st) != cudaSuccess || cudaMemsetAsync(eta_rel_out, 0, vb, st) != cudaSuccess ||
+      cudaMemsetAsync(plogp_out, 0, static_cast<size_t>(Hf) * sizeof(double), st) != cudaSuccess)
+    return SAF_ERR_CUDA;
+  ScopedTimer timer(ctx, SAF_KERNEL_FIT_MARGINALS, st);
+  if (launch_fit_marginals(mean_attn, floor_value, eta_abs_out, eta_rel_out, plogp_out, Hf, T, ctx->num_sms, st) !=
+      cudaSuccess)
+    return SAF_ERR_CUDA;
+  return SAF_OK;
+}
+
+int saf_fit_compact(saf_ctx* ctx, int32_t Hf, int32_t T, const double* eta_abs, const double* eta_rel,
+                    const double* plogp, int32_t steps, double lr, float* alpha_out, float* rho_out, float* logZ_out,
+                    int64_t out_stride, double* loss_out, double* kl_out, void* stream) {
+  if (!ctx || Hf < 0 || T < 1 || steps < 0 || !(lr > 0.0) || out_stride < T) return SAF_ERR_INVALID_ARG;
+  if (T > fit_max_T()) return SAF_ERR_UNSUPPORTED;
+  if (Hf == 0) return SAF_OK;
+  if (!eta_abs || !eta_rel || !alpha_out || !rho_out || !logZ_out || Hf > 65535) return SAF_ERR_INVALID_ARG;
+  if (kl_out && !plogp) return SAF_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ctx->last_stream = st;
+  // state: 6 fp64 and 5 fp32 arrays of [Hf, T]
+  const size_t n = static_cast<size_t>(Hf) * T;
+  int rc = ensure(ctx->fit_buf, n * (6 * sizeof(double) + 5 * sizeof(float)));
+  if (rc) return rc;
+  FitState s;
+  s.T = T;
+  s.lr = lr;
+  s.eta_abs = eta_abs;
+  s.eta_rel = eta_rel;
+  double* d = static_cast<double*>(ctx->fit_buf.ptr);
+  s.alpha = d; s.rho = d + n; s.m_a = d + 2 * n; s.v_a = d + 3 * n; s.m_r = d + 4 * n; s.v_r = d + 5 * n;
+  float* f = reinterpret_cast<float*>(d + 6 * n);
+  s.a2[0] = f; s.a2[1] = f + n; s.r2[0] = f + 2 * n; s.r2[1] = f + 3 * n; s.nz2 = f + 4 * n;
+  ScopedTimer timer(ctx, SAF_KERNEL_FIT, st);
+  if (launch_fit(s, Hf, steps, plogp, alpha_out, rho_out, logZ_out, out_stride, loss_out, kl_out, st) != cudaSuccess)
+    return SAF_ERR_CUDA;
   return SAF_OK;
 }
 

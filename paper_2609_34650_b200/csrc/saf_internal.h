@@ -145,4 +145,21 @@ int bwd128_smem_bytes();
 int fwd_smem_bytes(int D);
 int bwd_smem_bytes(int D);
 
+// compact-pattern fitter (saf_fit.cu): per-head state of Fit, all arrays [Hf, T]
+struct FitState {
+  int T;
+  double lr;
+  const double* eta_abs;
+  const double* eta_rel;
+  double* alpha; double* rho;          // fp64 parameters
+  double* m_a; double* v_a; double* m_r; double* v_r;   // Adam moments
+  float* a2[2]; float* r2[2];          // log2e-scaled fp32 copies, double-buffered over the steps
+  float* nz2;                          // -log2 Z(i) of the current parameters
+};
+int fit_max_T();
+cudaError_t launch_fit_marginals(const float* Abar, float floor_v, double* eta_abs, double* eta_rel, double* plogp,
+                                 int Hf, int T, int num_sms, cudaStream_t st);
+cudaError_t launch_fit(const FitState& s, int Hf, int steps, const double* plogp, float* alpha_out, float* rho_out,
+                       float* logZ_out, long long out_stride, double* loss_out, double* kl_out, cudaStream_t st);
+
 }  // namespace saf
