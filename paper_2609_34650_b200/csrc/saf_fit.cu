@@ -32,7 +32,6 @@ constexpr double LOG2E_D = 1.4426950408889634074;
 constexpr double LN2_D = 0.6931471805599453094;
 constexpr int XB = 32;             // x values per CTA of the pass kernel (one per lane)
 constexpr int PASS_WARPS = 8;      // warps of a pass CTA; they split the y range in chunks of 32
-constexpr int MARG_THREADS = 512;
 
 __device__ __forceinline__ float ex2f(float x) {
   float y;
@@ -47,72 +46,97 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // ------------------------------------------------------------------------------------------------ target marginals
-// One CTA walks rows blockIdx.x, blockIdx.x + gridDim.x, ... of head blockIdx.y.  Thread t owns the columns
-// t, t + 512, ...: their column sums stay in registers over all rows of the CTA; the diagonal sums live in shared
-// memory (for a given row every thread touches different distances, rows are separated by the CTA barrier of the
-// row-sum reduction).  The next row is loaded before the current one is reduced (where the registers allow it).
-template <int NCH, bool PREF>
-__global__ void __launch_bounds__(MARG_THREADS)
+// One CTA of NT threads walks rows blockIdx.x, blockIdx.x + gridDim.x, ... of head blockIdx.y.  Thread t owns the
+// columns t, t + NT, ...: their column sums stay in registers over all rows of the CTA; the diagonal sums live in
+// shared memory (for a given row every thread touches different distances, rows are separated by the CTA barrier of
+// the row-sum reduction).  256 threads with up to 32 columns each measured fastest (loading the next row ahead of
+// the reduction costs registers, hence resident CTAs, and measured slower).
+// Row pieces specialised on the number KK of column chunks that reach the diagonal, so that the chunks above it
+// cost nothing and the loads of a row still issue back to back.
+template <int NT, int KK>
+__device__ __forceinline__ void marg_load(const float* __restrict__ r, int row, int tid, float floor_v, float* dst) {
+#pragma unroll
+  for (int k = 0; k < KK; ++k) {
+    const int j = tid + k * NT;
+    dst[k] = (j <= row) ? fmaxf(__ldg(r + j), floor_v) : 0.0f;
+  }
+}
+template <int KK>
+__device__ __forceinline__ float marg_sum(const float* cur) {
+  float s = 0.0f;
+#pragma unroll
+  for (int k = 0; k < KK; ++k) s += cur[k];
+  return s;
+}
+template <int NT, int KK>
+__device__ __forceinline__ void marg_consume(const float* cur, float inv, float* col, float* dg, float& ent, int i,
+                                             int tid) {
+#pragma unroll
+  for (int k = 0; k < KK; ++k) {
+    if (tid + k * NT <= i) {
+      const float p = cur[k] * inv;
+      col[k] += p;
+      dg[-k * NT] += p;
+      ent = fmaf(p, __log2f(p), ent);
+    }
+  }
+}
+// (quarters of the NCH chunks: case q serves rows whose last chunk index is below (q+1) NCH/4; one case per chunk
+// count measured slower: more registers, fewer resident CTAs)
+#define SAF_MARG_DISPATCH(q, CALL)                         \
+  switch (q) {                                             \
+    case 0: { constexpr int KK = G; CALL; } break;         \
+    case 1: { constexpr int KK = 2 * G; CALL; } break;     \
+    case 2: { constexpr int KK = 3 * G; CALL; } break;     \
+    default: { constexpr int KK = NCH; CALL; } break;      \
+  }
+
+template <int NT, int NCH>
+__global__ void __launch_bounds__(NT)
 saf_fit_marginals_kernel(const float* __restrict__ Abar, float floor_v, double* __restrict__ eta_abs,
                          double* __restrict__ eta_rel, double* __restrict__ plogp, int T) {
   extern __shared__ float sm_f[];
   float* diag = sm_f;                          // [T]
-  __shared__ float red[2][MARG_THREADS / 32];
-  __shared__ double redd[MARG_THREADS / 32];
+  constexpr int NW = NT / 32;
+  constexpr int G = (NCH >= 4) ? NCH / 4 : NCH;
+  __shared__ float red[2][NW];
+  __shared__ double redd[NW];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int h = blockIdx.y;
   const float* A = Abar + static_cast<size_t>(h) * T * T;
-  for (int d = tid; d < T; d += MARG_THREADS) diag[d] = 0.0f;
+  for (int d = tid; d < T; d += NT) diag[d] = 0.0f;
   float col[NCH];
 #pragma unroll
   for (int k = 0; k < NCH; ++k) col[k] = 0.0f;
   float ent = 0.0f;                            // sum p log2 p of this thread (scaled to nats at the end)
   double ent_d = 0.0;
-  float cur[NCH], nxt[PREF ? NCH : 1];
+  float cur[NCH];
   int i = blockIdx.x;
-  auto load_row = [&](int row, float* dst) {
-    const float* r = A + static_cast<size_t>(row) * T;
-#pragma unroll
-    for (int k = 0; k < NCH; ++k) {
-      const int j = tid + k * MARG_THREADS;
-      dst[k] = (j <= row) ? fmaxf(__ldg(r + j), floor_v) : 0.0f;
-    }
-  };
-  if (i < T) load_row(i, cur);
+  if (i < T) {
+    SAF_MARG_DISPATCH((i / NT) / G, (marg_load<NT, KK>(A + static_cast<size_t>(i) * T, i, tid, floor_v, cur)));
+  }
   __syncthreads();
-  int par = 0;
-  for (; i < T; i += gridDim.x, par ^= 1) {
-    const int inext = i + gridDim.x;
-    if (PREF && inext < T) load_row(inext, nxt);
+  int par = 0, nrow = 0;
+  for (; i < T; i += gridDim.x, par ^= 1, ++nrow) {
+    const int q = (i / NT) / G;
     float s = 0.0f;
-#pragma unroll
-    for (int k = 0; k < NCH; ++k) s += cur[k];
+    SAF_MARG_DISPATCH(q, (s = marg_sum<KK>(cur)));
     s = warp_sum(s);
     if (lane == 0) red[par][warp] = s;
     __syncthreads();                           // also: the previous row's diagonal updates are complete
     float tot = 0.0f;
 #pragma unroll
-    for (int w = 0; w < MARG_THREADS / 32; ++w) tot += red[par][w];
+    for (int w = 0; w < NW; ++w) tot += red[par][w];
     const float inv = 1.0f / tot;
-#pragma unroll
-    for (int k = 0; k < NCH; ++k) {
-      const int j = tid + k * MARG_THREADS;
-      if (j <= i) {
-        const float p = cur[k] * inv;
-        col[k] += p;
-        diag[i - j] += p;
-        ent = fmaf(p, __log2f(p), ent);
-      }
-    }
-    if ((i / gridDim.x & 63) == 63) {          // keep the fp32 partial short
+    float* dg = diag + (i - tid);
+    SAF_MARG_DISPATCH(q, (marg_consume<NT, KK>(cur, inv, col, dg, ent, i, tid)));
+    if ((nrow & 63) == 63) {                   // keep the fp32 partial short
       ent_d += static_cast<double>(ent);
       ent = 0.0f;
     }
-    if (PREF) {
-#pragma unroll
-      for (int k = 0; k < NCH; ++k) cur[k] = nxt[k];
-    } else if (inext < T) {
-      load_row(inext, cur);
+    const int inext = i + gridDim.x;
+    if (inext < T) {
+      SAF_MARG_DISPATCH((inext / NT) / G, (marg_load<NT, KK>(A + static_cast<size_t>(inext) * T, inext, tid, floor_v, cur)));
     }
   }
   ent_d += static_cast<double>(ent);
@@ -121,10 +145,10 @@ saf_fit_marginals_kernel(const float* __restrict__ Abar, float floor_v, double* 
   double* er = eta_rel + static_cast<size_t>(h) * T;
 #pragma unroll
   for (int k = 0; k < NCH; ++k) {
-    const int j = tid + k * MARG_THREADS;
+    const int j = tid + k * NT;
     if (j < T && col[k] != 0.0f) atomicAdd(ea + j, static_cast<double>(col[k]));
   }
-  for (int d = tid; d < T; d += MARG_THREADS)
+  for (int d = tid; d < T; d += NT)
     if (diag[d] != 0.0f) atomicAdd(er + d, static_cast<double>(diag[d]));
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ent_d += __shfl_xor_sync(0xffffffffu, ent_d, o);
@@ -132,10 +156,11 @@ saf_fit_marginals_kernel(const float* __restrict__ Abar, float floor_v, double* 
   __syncthreads();
   if (tid == 0) {
     double t = 0.0;
-    for (int w = 0; w < MARG_THREADS / 32; ++w) t += redd[w];
+    for (int w = 0; w < NW; ++w) t += redd[w];
     atomicAdd(plogp + h, t * LN2_D);
   }
 }
+#undef SAF_MARG_DISPATCH
 
 // ------------------------------------------------------------------------------------------------ Fit: start
 // One CTA per head: alpha = 0, rho(d) = log max(eta_rel(d)/(T-d), 1e-9), Adam moments zero, and the first
@@ -291,27 +316,28 @@ int fit_max_T() { return 16384; }
 
 cudaError_t launch_fit_marginals(const float* Abar, float floor_v, double* eta_abs, double* eta_rel, double* plogp,
                                  int Hf, int T, int num_sms, cudaStream_t st) {
-  // rows per CTA: enough CTAs to fill the device three deep, but at least 32 rows each so that the final
-  // flush (2T atomics per CTA) stays small beside the rows read
-  int nb = (3 * num_sms + Hf - 1) / Hf;
-  nb = std::max(1, std::min(nb, (T + 31) / 32));
-  const dim3 grid(nb, Hf);
+  // CTAs per head: one resident wave over all heads, but at least 32 rows each so that the final flush
+  // (2T atomics per CTA) stays small beside the rows read
   const size_t smem = static_cast<size_t>(T) * sizeof(float);
-  const int nch = (T + MARG_THREADS - 1) / MARG_THREADS;
-#define SAF_MARG(N)                                                                                              \
+#define SAF_MARG(NT, N)                                                                                          \
   do {                                                                                                           \
-    auto kern = saf_fit_marginals_kernel<N, (N <= 8)>;                                                           \
+    auto kern = saf_fit_marginals_kernel<NT, N>;                                                                 \
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,                      \
                                          static_cast<int>(smem));                                                \
     if (e != cudaSuccess) return e;                                                                              \
-    kern<<<grid, MARG_THREADS, smem, st>>>(Abar, floor_v, eta_abs, eta_rel, plogp, T);                           \
+    int occ = 1;                                                                                                 \
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, NT, smem);                                     \
+    if (e != cudaSuccess) return e;                                                                              \
+    int nb = (std::max(occ, 1) * num_sms) / Hf;             /* one resident wave over all heads */               \
+    nb = std::max(1, std::min(nb, (T + 31) / 32));                                                               \
+    kern<<<dim3(nb, Hf), NT, smem, st>>>(Abar, floor_v, eta_abs, eta_rel, plogp, T);                             \
   } while (0)
-  if (nch <= 1) SAF_MARG(1);
-  else if (nch <= 2) SAF_MARG(2);
-  else if (nch <= 4) SAF_MARG(4);
-  else if (nch <= 8) SAF_MARG(8);
-  else if (nch <= 16) SAF_MARG(16);
-  else if (nch <= 32) SAF_MARG(32);
+  if (T <= 128 * 2) SAF_MARG(128, 2);
+  else if (T <= 256 * 4) SAF_MARG(256, 4);
+  else if (T <= 256 * 8) SAF_MARG(256, 8);
+  else if (T <= 256 * 16) SAF_MARG(256, 16);
+  else if (T <= 256 * 32) SAF_MARG(256, 32);
+  else if (T <= 512 * 32) SAF_MARG(512, 32);
   else return cudaErrorInvalidValue;
 #undef SAF_MARG
   return cudaGetLastError();
