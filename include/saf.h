@@ -180,6 +180,34 @@ int saf_fit_compact(saf_ctx* ctx, int32_t Hf, int32_t T, const double* eta_abs, 
                     const double* plogp, int32_t steps, double lr, float* alpha_out, float* rho_out, float* logZ_out,
                     int64_t out_stride, double* loss_out, double* kl_out, void* stream);
 
+/* Calibration statistics of one layer, streaming part (Sec. 3.1 "Calibration and head selection";
+ * Eq. "variance-score", Eq. "forward-kl-score").  For the `problem->B` calibration sequences of this call and every
+ * head, the attention maps A^(n) = softmax_causal(Q K^T scale) are formed tile by tile (never stored) and added up:
+ *   mean_sum[h][i][j] (+)= sum_n A^(n)(i,j)       device float32 [H, T, T] row-major, 16-byte aligned
+ *   sumsq[h]          (+)= sum_n ||A^(n)||_F^2     device float64 [H]
+ *   sum_plogp[h]      (+)= sum_n sum_{ij} A^(n) log A^(n)   device float64 [H]  (natural log, 0 log 0 = 0)
+ * `accumulate` = 0 overwrites (first call of a layer), non-zero adds to what earlier calls left, so N sequences may
+ * arrive in any number of calls.  Of mean_sum only the 128 x 128 tiles that meet the causal triangle are touched
+ * (inside them entries above the diagonal get zeros); the tiles strictly above it are never read or written.
+ *   Q, K    : device bf16 with problem's q_strides / k_strides; all heads are ordinary here (calibration precedes
+ *             replacement); kv_group as in the attention calls; packed_qk must be 0; Tp and the other strides are
+ *             ignored.  D in {64, 96, 128}.
+ *   LSE     : device float32 [B][H][T]: the row normalisers that saf_hybrid_attn_fwd returned for the same Q, K
+ *             (natural-log sum of exp of the scaled causal scores).
+ * Asynchronous on `stream`. */
+int saf_calib_accumulate(saf_ctx* ctx, const saf_problem* problem, const void* Q, const void* K, const float* LSE,
+                         float* mean_sum, double* sumsq, double* sum_plogp, int32_t accumulate, void* stream);
+
+/* Calibration statistics, final part: with `n_total` sequences accumulated, scales the causal part of `mean_inout`
+ * by 1/n_total in place (the empirical mean A^, the "post-softmax mean" pattern and the input of saf_fit_marginals)
+ * and returns per head
+ *   s_var_out[h] = (sumsq[h] - N ||A^||_F^2) / ((N-1) T^2)            = Eq. "variance-score"
+ *   s_kl_out[h]  = (sum_plogp[h] - N sum A^ log A^) / (N T)           = Eq. "forward-kl-score"
+ * (device float64 [H]; either may be NULL; both are clamped at zero against rounding).  s_var needs n_total >= 2
+ * (SAF_ERR_INVALID_ARG otherwise).  Asynchronous on `stream`. */
+int saf_calib_finalize(saf_ctx* ctx, int32_t H, int32_t T, int64_t n_total, float* mean_inout, const double* sumsq,
+                       const double* sum_plogp, double* s_var_out, double* s_kl_out, void* stream);
+
 /* Device-side status of the most recent launches on this context: SAF_OK or SAF_ERR_DEVICE_TIMEOUT.
  * Synchronises the context's device status word with the host (blocks until the stream used by the
  * last call has drained).  `detail_out` (may be NULL) receives the raw word: site and CTA that gave up. */
@@ -199,7 +227,9 @@ enum {
   SAF_KERNEL_PGRAD = 6,        /* pattern-gradient kernel (saf_pattern_grad) */
   SAF_KERNEL_FIT = 7,          /* all launches of one saf_fit_compact call, as one interval */
   SAF_KERNEL_FIT_MARGINALS = 8,/* target marginals (saf_fit_marginals) */
-  SAF_KERNEL_COUNT = 9
+  SAF_KERNEL_CALIB = 9,        /* calibration statistics kernel (saf_calib_accumulate) */
+  SAF_KERNEL_CALIB_FINALIZE = 10, /* mean and scores (saf_calib_finalize) */
+  SAF_KERNEL_COUNT = 11
 };
 int saf_set_profiling(saf_ctx* ctx, int32_t enable);
 int saf_get_kernel_time(saf_ctx* ctx, int32_t which, float* total_ms_out, int32_t* launches_out);

@@ -18,7 +18,7 @@ SAF_OK = 0
 SAF_ERR_INVALID_ARG, SAF_ERR_UNSUPPORTED, SAF_ERR_CUDA, SAF_ERR_DEVICE_TIMEOUT, SAF_ERR_ARCH, SAF_ERR_NOMEM = range(1, 7)
 SAF_BF16, SAF_F32 = 0, 1
 SAF_KERNEL_FWD, SAF_KERNEL_BWD, SAF_KERNEL_BWD_PREP, SAF_KERNEL_BWD_FINALIZE, SAF_KERNEL_LOGZ, SAF_KERNEL_SCALE = range(6)
-SAF_KERNEL_PGRAD, SAF_KERNEL_FIT, SAF_KERNEL_FIT_MARGINALS = 6, 7, 8
+SAF_KERNEL_PGRAD, SAF_KERNEL_FIT, SAF_KERNEL_FIT_MARGINALS, SAF_KERNEL_CALIB, SAF_KERNEL_CALIB_FINALIZE = 6, 7, 8, 9, 10
 
 
 class SafProblem(C.Structure):
@@ -60,6 +60,8 @@ def load_library() -> C.CDLL:
     lib.saf_pattern_grad.argtypes = [vp, pp, vp, vp, vp, u8p, f32p, f32p, f32p, f32p, f32p, vp]
     lib.saf_fit_marginals.argtypes = [vp, i32, i32, vp, C.c_float, vp, vp, vp, vp]
     lib.saf_fit_compact.argtypes = [vp, i32, i32, vp, vp, vp, i32, C.c_double, vp, vp, vp, C.c_int64, vp, vp, vp]
+    lib.saf_calib_accumulate.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, i32, vp]
+    lib.saf_calib_finalize.argtypes = [vp, i32, i32, C.c_int64, vp, vp, vp, vp, vp, vp]
     lib.saf_last_device_status.argtypes = [vp, C.POINTER(C.c_int32)]
     lib.saf_set_profiling.argtypes = [vp, i32]
     lib.saf_get_kernel_time.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
@@ -68,7 +70,7 @@ def load_library() -> C.CDLL:
     lib.saf_build_worklist.argtypes = [i32, i32, i32, u8p, i32, i32, i32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     for name in ("saf_create", "saf_destroy", "saf_pattern_prepare", "saf_hybrid_attn_fwd", "saf_hybrid_attn_bwd",
                  "saf_hybrid_attn_step_host", "saf_last_device_status", "saf_build_worklist", "saf_set_profiling",
-                 "saf_get_kernel_time", "saf_pattern_grad", "saf_fit_marginals", "saf_fit_compact"):
+                 "saf_get_kernel_time", "saf_pattern_grad", "saf_fit_marginals", "saf_fit_compact", "saf_calib_accumulate", "saf_calib_finalize"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -194,6 +196,15 @@ class Context:
         _check(self._lib.saf_fit_compact(self._h, int(Hf), int(T), _ptr(eta_abs), _ptr(eta_rel), _ptr(plogp),
                                          int(steps), float(lr), _ptr(alpha), _ptr(rho), _ptr(logZ), int(out_stride),
                                          _ptr(loss), _ptr(kl), _stream()), "saf_fit_compact")
+
+    def saf_calib_accumulate(self, prob, Q, K, LSE, mean_sum, sumsq, sum_plogp, accumulate):
+        _check(self._lib.saf_calib_accumulate(self._h, C.byref(prob), _ptr(Q), _ptr(K), _ptr(LSE), _ptr(mean_sum),
+                                              _ptr(sumsq), _ptr(sum_plogp), int(bool(accumulate)), _stream()),
+               "saf_calib_accumulate")
+
+    def saf_calib_finalize(self, H, T, n_total, mean, sumsq, sum_plogp, s_var, s_kl):
+        _check(self._lib.saf_calib_finalize(self._h, int(H), int(T), int(n_total), _ptr(mean), _ptr(sumsq),
+                                            _ptr(sum_plogp), _ptr(s_var), _ptr(s_kl), _stream()), "saf_calib_finalize")
 
     def saf_hybrid_attn_step_host(self, prob, Q, K, V, dO, mask, alpha, rho, prepare, O, LSE, dQ, dK, dV):
         """All tensor arguments are HOST tensors (torch CPU tensors, ideally pinned) or None."""

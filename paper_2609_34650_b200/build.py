@@ -8,7 +8,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsaf_b200.so")
-SOURCES = ["saf_api.cu", "saf_prep.cu", "saf_fwd.cu", "saf_fwd64.cu", "saf_bwd.cu", "saf_bwd128.cu", "saf_pgrad.cu", "saf_fit.cu"]
+SOURCES = ["saf_api.cu", "saf_prep.cu", "saf_fwd.cu", "saf_fwd64.cu", "saf_bwd.cu", "saf_bwd128.cu", "saf_pgrad.cu", "saf_fit.cu", "saf_calib.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math", "-Xptxas", "-v"]
 

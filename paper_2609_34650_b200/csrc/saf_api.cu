@@ -65,7 +65,7 @@ struct saf_ctx {
   // tensor-core form of frozen heads: tables built by saf_pattern_prepare, scaled V / dO per call
   PatternCache pat;
   bool tensor_pattern = true;              // SAF_DISABLE_TENSOR_PATTERN=1 turns the form off
-  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, vt_buf, dot_buf, ok_fwd, ok_bwd, pg_hlist, pg_delta, fit_buf;
+  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, vt_buf, dot_buf, ok_fwd, ok_bwd, pg_hlist, pg_delta, fit_buf, calib_tmp;
   bool profiling = false;
   std::vector<TimedLaunch> timed;          // event pairs recorded since the last query
   std::vector<cudaEvent_t> event_pool;
@@ -377,7 +377,7 @@ int saf_destroy(saf_ctx* ctx) {
     cudaFree(e.offsets_dev);
   }
   DevBuf* pbufs[] = {&ctx->pat_consts, &ctx->pat_ok, &ctx->pat_avec, &ctx->pat_wvec, &ctx->pat_bandf, &ctx->pat_bandb,
-                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta, &ctx->fit_buf};
+                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta, &ctx->fit_buf, &ctx->calib_tmp};
   for (DevBuf* b : pbufs) release(*b);
   DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->dkacc_buf, &ctx->dvacc_buf, &ctx->qslot_buf, &ctx->hq, &ctx->hk, &ctx->hv,
                     &ctx->hdo, &ctx->ho, &ctx->hlse, &ctx->hdq, &ctx->hdk, &ctx->hdv, &ctx->halpha, &ctx->hrho,
@@ -1006,6 +1006,69 @@ int saf_fit_compact(saf_ctx* ctx, int32_t Hf, int32_t T, const double* eta_abs, 
   s.a2[0] = f; s.a2[1] = f + n; s.r2[0] = f + 2 * n; s.r2[1] = f + 3 * n; s.nz2 = f + 4 * n;
   ScopedTimer timer(ctx, SAF_KERNEL_FIT, st);
   if (launch_fit(s, Hf, steps, plogp, alpha_out, rho_out, logZ_out, out_stride, loss_out, kl_out, st) != cudaSuccess)
+    return SAF_ERR_CUDA;
+  return SAF_OK;
+}
+
+int saf_calib_accumulate(saf_ctx* ctx, const saf_problem* p, const void* Q, const void* K, const float* LSE,
+                         float* mean_sum, double* sumsq, double* sum_plogp, int32_t accumulate, void* stream) {
+  if (!ctx || !p || !mean_sum || !sumsq || !sum_plogp) return SAF_ERR_INVALID_ARG;
+  if (p->B < 1 || p->H < 1 || p->T < 1) return SAF_ERR_INVALID_ARG;
+  if (p->D != 64 && p->D != 96 && p->D != 128) return SAF_ERR_UNSUPPORTED;
+  if (p->kv_group < 0 || (p->kv_group > 1 && p->H % p->kv_group != 0) || p->packed_qk) return SAF_ERR_INVALID_ARG;
+  if (!Q || !K || !LSE || !aligned16(Q) || !aligned16(K) || !aligned16(mean_sum)) return SAF_ERR_INVALID_ARG;
+  if (check_strides(p->q_strides, p->D) || check_strides(p->k_strides, p->D)) return SAF_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ctx->last_stream = st;
+  const int kvg = kv_group_of(p);
+  if (!accumulate) {
+    const size_t hb = static_cast<size_t>(p->H) * sizeof(double);
+    if (cudaMemsetAsync(sumsq, 0, hb, st) != cudaSuccess || cudaMemsetAsync(sum_plogp, 0, hb, st) != cudaSuccess)
+      return SAF_ERR_CUDA;
+  }
+  CUtensorMap mq, mk;
+  int rc;
+  if ((rc = make_map(ctx, &mq, Q, p, p->q_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H))) return rc;
+  if ((rc = make_map(ctx, &mk, K, p, p->k_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg))) return rc;
+  const int nblk = (p->T + BLK - 1) / BLK;
+  CalibParams cp;
+  cp.B = p->B; cp.H = p->H; cp.T = p->T;
+  cp.kv_group = kvg;
+  const float scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
+  cp.scale_log2e = scale * 1.4426950408889634f;
+  cp.LSE = LSE;
+  cp.mean_sum = mean_sum;
+  cp.sumsq = sumsq;
+  cp.sum_plogp = sum_plogp;
+  cp.accumulate = accumulate ? 1 : 0;
+  cp.npairs = nblk * (nblk + 1) / 2;
+  const long long n_items = static_cast<long long>(p->H) * cp.npairs;
+  if (n_items > 0x7fffffffLL) return SAF_ERR_INVALID_ARG;
+  cp.n_items = static_cast<int>(n_items);
+  cp.status = ctx->status_dev;
+  cp.wait_limit_ns = ctx->wait_limit_ns;
+  const int grid = static_cast<int>(std::min<long long>(ctx->num_sms, n_items));
+  ScopedTimer timer(ctx, SAF_KERNEL_CALIB, st);
+  // (head dimension 96 runs on the 128-wide kernel: TMA zero-fills features 96..127)
+  if (launch_calib(p->D == 64 ? 64 : 128, mq, mk, cp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+  return SAF_OK;
+}
+
+int saf_calib_finalize(saf_ctx* ctx, int32_t H, int32_t T, int64_t n_total, float* mean_inout, const double* sumsq,
+                       const double* sum_plogp, double* s_var_out, double* s_kl_out, void* stream) {
+  if (!ctx || H < 1 || T < 1 || n_total < 1 || !mean_inout || !sumsq || !sum_plogp) return SAF_ERR_INVALID_ARG;
+  if (s_var_out && n_total < 2) return SAF_ERR_INVALID_ARG;   // the sample variance needs two sequences
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SAF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ctx->last_stream = st;
+  int rc = ensure(ctx->calib_tmp, static_cast<size_t>(H) * 2 * sizeof(double));
+  if (rc) return rc;
+  ScopedTimer timer(ctx, SAF_KERNEL_CALIB_FINALIZE, st);
+  if (launch_calib_finalize(mean_inout, sumsq, sum_plogp, static_cast<double*>(ctx->calib_tmp.ptr), H, T,
+                            static_cast<double>(n_total), s_var_out, s_kl_out, ctx->num_sms, st) != cudaSuccess)
     return SAF_ERR_CUDA;
   return SAF_OK;
 }

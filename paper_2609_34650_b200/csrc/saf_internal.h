@@ -162,4 +162,23 @@ cudaError_t launch_fit_marginals(const float* Abar, float floor_v, double* eta_a
 cudaError_t launch_fit(const FitState& s, int Hf, int steps, const double* plogp, float* alpha_out, float* rho_out,
                        float* logZ_out, long long out_stride, double* loss_out, double* kl_out, cudaStream_t st);
 
+// calibration statistics (saf_calib.cu)
+struct CalibParams {
+  int B, H, T;                      // B = sequences of this call
+  int kv_group;
+  float scale_log2e;                // softmax scale x log2(e)
+  const float* LSE;                 // [B][H][T], natural-log normalisers from the attention forward
+  float* mean_sum;                  // [H][T][T]: sum over sequences of the attention maps (causal tiles only)
+  double* sumsq;                    // [H] += sum_n ||A_n||_F^2
+  double* sum_plogp;                // [H] += sum_n sum A_n log A_n
+  int accumulate;                   // 0: overwrite mean_sum tiles, 1: add to them
+  int n_items, npairs;              // items = H x npairs, npairs = nblk (nblk+1)/2
+  int* status;
+  unsigned long long wait_limit_ns;
+};
+cudaError_t launch_calib(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CalibParams& p, int grid,
+                         cudaStream_t st);
+cudaError_t launch_calib_finalize(float* mean, const double* sumsq, const double* sum_plogp, double* tmp, int H, int T,
+                                  double n_total, double* s_var, double* s_kl, int num_sms, cudaStream_t st);
+
 }  // namespace saf
