@@ -1032,8 +1032,23 @@ int saf_calib_accumulate(saf_ctx* ctx, const saf_problem* p, const void* Q, cons
   int rc;
   if ((rc = make_map(ctx, &mq, Q, p, p->q_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H))) return rc;
   if ((rc = make_map(ctx, &mk, K, p, p->k_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg))) return rc;
+  // the dense accumulator as a [1][H][T][T] fp32 tensor, boxes of 128 rows x 32 columns (128-byte rows, swizzled)
+  CUtensorMap mm = mq;
+  const bool use_tma = (p->T % 4) == 0;
+  if (use_tma) {
+    const cuuint64_t Tt = static_cast<cuuint64_t>(p->T);
+    cuuint64_t dims[4] = {Tt, Tt, static_cast<cuuint64_t>(p->H), 1};
+    cuuint64_t gs[3] = {Tt * 4, Tt * Tt * 4, Tt * Tt * 4 * static_cast<cuuint64_t>(p->H)};
+    cuuint32_t box[4] = {32, BLK, 1, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    if (ctx->encode(&mm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, mean_sum, dims, gs, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return SAF_ERR_CUDA;
+  }
   const int nblk = (p->T + BLK - 1) / BLK;
   CalibParams cp;
+  cp.use_tma = use_tma ? 1 : 0;
   cp.B = p->B; cp.H = p->H; cp.T = p->T;
   cp.kv_group = kvg;
   const float scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->D));
@@ -1052,7 +1067,7 @@ int saf_calib_accumulate(saf_ctx* ctx, const saf_problem* p, const void* Q, cons
   const int grid = static_cast<int>(std::min<long long>(ctx->num_sms, n_items));
   ScopedTimer timer(ctx, SAF_KERNEL_CALIB, st);
   // (head dimension 96 runs on the 128-wide kernel: TMA zero-fills features 96..127)
-  if (launch_calib(p->D == 64 ? 64 : 128, mq, mk, cp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+  if (launch_calib(p->D == 64 ? 64 : 128, mq, mk, mm, cp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
   return SAF_OK;
 }
 

@@ -14,7 +14,10 @@
 // over the N sequences: S = Q_I K_J^T on the tensor core (tcgen05, both operands K-major in 128B-swizzled smem via
 // TMA, accumulator double-buffered in TMEM), then per element in registers p = exp2(s c - lse'), acc += p,
 // sq += p^2, ent += p log2 p; the 128 x 128 fp32 accumulator tile lives in the registers of the 16 compute warps
-// (thread = query row x 32 keys) and is written (or added) to the dense accumulator once per item.
+// (thread = query row x 32 keys) and leaves once per item through shared memory as four TMA stores into the dense
+// accumulator, which drain while the next item computes; in the calls that add to earlier ones the old tile is
+// fetched by TMA into the same boxes during the item and summed there (TMA reduce-adds measured 1.2 TB/s, half of
+// what the plain load + store path reaches).
 // CTA = 576 threads: warps 0-15 compute (TMEM lane = query row; warp >> 2 picks the 32-key column group), warp 16
 // TMA producer, warp 17 tcgen05 issuer and TMEM owner.  Every wait is bounded.
 #include <cuda_bf16.h>
@@ -34,16 +37,45 @@ struct CalCfg {
   static constexpr int NPANEL = D / 64;                 // 64-column bf16 panels: 128-byte rows
   static constexpr int PANEL_BYTES = 128 * 64 * 2;
   static constexpr int TILE_BYTES = NPANEL * PANEL_BYTES;
-  static constexpr int NS = 2;                          // (Q, K) ring depth
+  static constexpr int NS = (D == 64) ? 4 : 2;          // (Q, K) ring depth (shared memory allows no more at 128)
   static constexpr int STAGE_BYTES = 2 * TILE_BYTES;    // Q tile then K tile
-  static constexpr int OFF_BAR = NS * STAGE_BYTES;
-  static constexpr int NBAR = 2 * NS + 4;
+  static constexpr int OFF_OUT = NS * STAGE_BYTES;      // 4 boxes of 128 rows x 32 fp32 (128-byte rows, swizzled): 64 KB
+  static constexpr int OUT_BOX_BYTES = 128 * 128;
+  static constexpr int OFF_BAR = OFF_OUT + 4 * OUT_BOX_BYTES;
+  static constexpr int NBAR = 2 * NS + 5;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
   static constexpr int TMEM_COLS = 256;                 // two score buffers of 128 fp32 columns
   static constexpr int NTHREADS = 576;
 };
 
-enum CalSite { C_QK_EMPTY = 71, C_QK_FULL, C_S_FREE, C_S_FULL };
+enum CalSite { C_QK_EMPTY = 71, C_QK_FULL, C_S_FREE, C_S_FULL, C_OLD_FULL };
+
+__device__ __forceinline__ void ld_shared_v4f(uint32_t addr, float& a, float& b, float& c, float& d) {
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(a), "=f"(b), "=f"(c), "=f"(d) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void st_shared_v4w(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// packed pairs of fp32 (one instruction per two elements on the FMA pipes)
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 
 // item index -> (h, I, J) with J <= I; pairs are numbered row by row: q = I (I+1)/2 + J
 __device__ __forceinline__ void decode_item(int idx, int npairs, int& h, int& I, int& J) {
@@ -58,9 +90,10 @@ __device__ __forceinline__ void decode_item(int idx, int npairs, int& h, int& I,
 
 }  // namespace
 
-template <int D>
+template <int D, bool ACC>
 __global__ void __launch_bounds__(576, 1)
-saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk, const CalibParams p) {
+saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
+                 const __grid_constant__ CUtensorMap mm, const CalibParams p) {
   using C = CalCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -69,7 +102,8 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   uint64_t* qk_empty = bars + C::NS;             // [NS]
   uint64_t* s_full = qk_empty + C::NS;           // [2] score buffer b holds a finished tile
   uint64_t* s_free = s_full + 2;                 // [2] the compute warps have read buffer b (16 warp arrivals)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_free + 2);
+  uint64_t* old_full = s_free + 2;               // the item's old accumulator tile has landed in the output boxes
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(old_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -85,6 +119,7 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       mbar_init(s_full + b, 1);
       mbar_init(s_free + b, 16);
     }
+    mbar_init(old_full, 1);
     mbar_fence_init();
   }
   if (warp == 17) {
@@ -156,9 +191,9 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const int rowl = q4 * 32 + lane;                   // query row within the block = TMEM lane
     const uint32_t lane_base = static_cast<uint32_t>(q4 * 32) << 16;
     const float c2 = p.scale_log2e;
-    uint32_t nl = 0;
+    uint32_t nl = 0, nit = 0;
     bool ok = true;
-    for (int idx = blockIdx.x; idx < p.n_items; idx += gridDim.x) {
+    for (int idx = blockIdx.x; idx < p.n_items; idx += gridDim.x, ++nit) {
       int h, I, J;
       decode_item(idx, p.npairs, h, I, J);
       const int qi = I * BLK + rowl;
@@ -166,53 +201,116 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       const bool diag = (I == J) || (J * BLK + BLK > p.T);   // tiles that need the per-element mask
       const float* lse_h = p.LSE + static_cast<size_t>(h) * p.T + qi;
       const size_t lse_step = static_cast<size_t>(p.H) * p.T;
-      float acc[32];
+      if (ACC && p.use_tma) {
+        // what earlier calls left in this tile is fetched into the output boxes while the sequences are processed
+        // (the previous item's store has finished reading them first)
+        if (tid == 0) {
+          bulk_wait_group_read0();
+          mbar_expect_tx(old_full, 4 * C::OUT_BOX_BYTES);
+          for (int k = 0; k < 4; ++k)
+            tma_load_4d(smem + C::OFF_OUT + k * C::OUT_BOX_BYTES, &mm, old_full, J * BLK + 32 * k, I * BLK, h, 0);
+        }
+      }
+      uint64_t acc2[16];                               // the thread's 32 accumulators as packed pairs
 #pragma unroll
-      for (int e = 0; e < 32; ++e) acc[e] = 0.0f;
-      float sq = 0.0f, ent = 0.0f;
-      float lse_next = (qi < p.T) ? lse_h[0] * LOG2E_C : INFINITY;
+      for (int k = 0; k < 16; ++k) acc2[k] = 0ull;
+      uint64_t sq2 = 0ull, ps2 = 0ull;
+      float lsum = 0.0f;
+      // the normaliser of sequence n+1 is loaded while sequence n is processed and first touched one round later
+      // (a use right after the load would stall the warp for the whole memory latency in front of the wait below)
+      const bool row_ok = qi < p.T;
+      float lse_raw = row_ok ? __ldg(lse_h) : 0.0f;
       for (int n = 0; n < p.B; ++n, ++nl) {
-        const float lse2 = lse_next;
-        if (n + 1 < p.B) lse_next = (qi < p.T) ? lse_h[(n + 1) * lse_step] * LOG2E_C : INFINITY;
+        float lse_raw_next = 0.0f;
+        if (n + 1 < p.B && row_ok) lse_raw_next = __ldg(lse_h + (n + 1) * lse_step);
         const uint32_t gb = nl & 1;
         if (ok && !mbar_wait_warp(s_full + gb, (nl >> 1) & 1, wc, C_S_FULL)) ok = false;
         if (!ok) continue;                             // (keeps the loop counters in step; nothing is read)
+        const float lse2 = row_ok ? lse_raw * LOG2E_C : INFINITY;
+        lse_raw = lse_raw_next;
         tc_fence_after();
         uint32_t r[32];
         tmem_ld32(tmem + lane_base + 128 * gb + 32 * cq, r);
         tmem_wait_ld();
         tc_fence_before();
         warp_arrive(s_free + gb);                      // the tensor core may overwrite this buffer
+        // p log2 p = p (s c - lse'): the first part is summed per element as p s, the second needs no tile at
+        // all because a row of probabilities sums to one: the threads of key block 0, column group 0 add lse'
+        // once per row and sequence.
+        if (J == 0 && cq == 0 && row_ok) lsum += lse2;
+        const uint64_t c2p = pk2(c2, c2), nlse = pk2(-lse2, -lse2);
+        if (diag) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          float arg = fmaf(__uint_as_float(r[e]), c2, -lse2);
-          if (diag && (k0 + e > qi)) arg = -INFINITY;  // causal mask (also keys beyond T: qi < T there)
-          const float pe = ex2_approx(arg);
-          acc[e] += pe;
-          sq = fmaf(pe, pe, sq);
-          ent = fmaf(pe, fmaxf(arg, -150.0f), ent);    // p log2 p; 0 * (-inf) never formed
-        }
-      }
-      if (!ok) break;
-      // the item's tile of sum_n A^(n): written, or added to what earlier calls left
-      if (qi < p.T) {
-        float* dst = p.mean_sum + (static_cast<size_t>(h) * p.T + qi) * p.T + k0;
-        if ((p.T & 3) == 0) {
-#pragma unroll
-          for (int e4 = 0; e4 < 8; ++e4) {
-            if (k0 + 4 * e4 < p.T) {
-              float4 v = make_float4(acc[4 * e4], acc[4 * e4 + 1], acc[4 * e4 + 2], acc[4 * e4 + 3]);
-              if (p.accumulate) {
-                const float4 o = *reinterpret_cast<const float4*>(dst + 4 * e4);
-                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-              }
-              *reinterpret_cast<float4*>(dst + 4 * e4) = v;
-            }
+          for (int k = 0; k < 16; ++k) {
+            const uint64_t s2 = pk2(__uint_as_float(r[2 * k]), __uint_as_float(r[2 * k + 1]));
+            float a0, a1;
+            upk2(fma2(s2, c2p, nlse), a0, a1);
+            if (k0 + 2 * k > qi) a0 = -INFINITY;       // causal mask (also keys beyond T: qi < T there)
+            if (k0 + 2 * k + 1 > qi) a1 = -INFINITY;
+            const uint64_t p2 = pk2(ex2_approx(a0), ex2_approx(a1));
+            acc2[k] = add2(acc2[k], p2);
+            sq2 = fma2(p2, p2, sq2);
+            ps2 = fma2(p2, s2, ps2);
           }
         } else {
 #pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            const uint64_t s2 = pk2(__uint_as_float(r[2 * k]), __uint_as_float(r[2 * k + 1]));
+            float a0, a1;
+            upk2(fma2(s2, c2p, nlse), a0, a1);
+            const uint64_t p2 = pk2(ex2_approx(a0), ex2_approx(a1));
+            acc2[k] = add2(acc2[k], p2);
+            sq2 = fma2(p2, p2, sq2);
+            ps2 = fma2(p2, s2, ps2);
+          }
+        }
+      }
+      float acc[32];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) upk2(acc2[k], acc[2 * k], acc[2 * k + 1]);
+      float sq, ps;
+      {
+        float x0, x1;
+        upk2(sq2, x0, x1);
+        sq = x0 + x1;
+        upk2(ps2, x0, x1);
+        ps = x0 + x1;
+      }
+      float ent = fmaf(ps, c2, -lsum);                 // sum of p log2 p of this thread's part of the item
+      // the item's tile of sum_n A^(n): written, or added to what earlier calls left
+      if (p.use_tma) {
+        // through shared memory and one TMA store / reduce-add per 32-column box: coalesced, and it drains while
+        // the next item computes.  The previous item's boxes have been read out before they are overwritten; the
+        // warps also agree here whether a wait has been abandoned.
+        if (!ACC && tid == 0) bulk_wait_group_read0();
+        if (ACC && ok && !mbar_wait_warp(old_full, nit & 1, wc, C_OLD_FULL)) ok = false;
+        if (named_bar_or(1, 512, !ok)) break;
+        const uint32_t stage_row = smem_u32(smem + C::OFF_OUT) + cq * C::OUT_BOX_BYTES + rowl * 128;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const uint32_t chunk = static_cast<uint32_t>(g ^ (rowl & 7)) * 16;
+          float o0 = 0.0f, o1 = 0.0f, o2 = 0.0f, o3 = 0.0f;
+          if (ACC) ld_shared_v4f(stage_row + chunk, o0, o1, o2, o3);
+          st_shared_v4w(stage_row + chunk, __float_as_uint(acc[4 * g] + o0), __float_as_uint(acc[4 * g + 1] + o1),
+                        __float_as_uint(acc[4 * g + 2] + o2), __float_as_uint(acc[4 * g + 3] + o3));
+        }
+        fence_proxy_async_smem();
+        named_bar_sync(2, 512);
+        if (tid == 0) {
+          for (int k = 0; k < 4; ++k) {
+            if (J * BLK + 32 * k >= p.T) break;
+            tma_store_4d(&mm, smem + C::OFF_OUT + k * C::OUT_BOX_BYTES, J * BLK + 32 * k, I * BLK, h, 0);
+          }
+          bulk_commit_group();
+        }
+      } else {
+        // row lengths that are no multiple of four floats cannot be described to TMA: plain loads and stores
+        if (!ok) break;
+        if (qi < p.T) {
+          float* dst = p.mean_sum + (static_cast<size_t>(h) * p.T + qi) * p.T + k0;
+#pragma unroll
           for (int e = 0; e < 32; ++e)
-            if (k0 + e < p.T) dst[e] = p.accumulate ? dst[e] + acc[e] : acc[e];
+            if (k0 + e < p.T) dst[e] = ACC ? dst[e] + acc[e] : acc[e];
         }
       }
 #pragma unroll
@@ -225,6 +323,7 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         atomicAdd(p.sum_plogp + h, static_cast<double>(ent) * LN2_C);
       }
     }
+    if (tid == 0) bulk_wait_group0();                  // every store / reduce-add has landed before the kernel ends
   }
 
   // ------------------------------------------------------------------ teardown
@@ -251,11 +350,19 @@ saf_calib_mean_kernel(float* __restrict__ mean, double inv_n, double* __restrict
   for (int i = blockIdx.x; i < T; i += gridDim.x) {
     float* row = M + static_cast<size_t>(i) * T;
     float a2 = 0.0f, al = 0.0f;
-    for (int j = tid; j <= i; j += 256) {
-      const float m = row[j] * invf;
-      row[j] = m;
-      a2 = fmaf(m, m, a2);
-      if (m > 0.0f) al = fmaf(m, __log2f(m), al);
+    for (int j0 = tid; j0 <= i; j0 += 1024) {        // four independent loads in flight per thread
+      float v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = (j0 + 256 * u <= i) ? row[j0 + 256 * u] : 0.0f;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (j0 + 256 * u <= i) {
+          const float m = v[u] * invf;
+          row[j0 + 256 * u] = m;
+          a2 = fmaf(m, m, a2);
+          if (m > 0.0f) al = fmaf(m, __log2f(m), al);
+        }
+      }
     }
     s2 += static_cast<double>(a2);
     sl += static_cast<double>(al);
@@ -297,19 +404,22 @@ __global__ void saf_calib_scores_kernel(const double* __restrict__ sumsq, const 
 
 int calib_smem_bytes(int D) { return D == 64 ? CalCfg<64>::SMEM : CalCfg<128>::SMEM; }
 
-cudaError_t launch_calib(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CalibParams& p, int grid,
-                         cudaStream_t st) {
-  cudaError_t e;
-  if (D == 64) {
-    e = cudaFuncSetAttribute(saf_calib_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, CalCfg<64>::SMEM);
-    if (e != cudaSuccess) return e;
-    saf_calib_kernel<64><<<grid, CalCfg<64>::NTHREADS, CalCfg<64>::SMEM, st>>>(mq, mk, p);
-  } else {
-    e = cudaFuncSetAttribute(saf_calib_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, CalCfg<128>::SMEM);
-    if (e != cudaSuccess) return e;
-    saf_calib_kernel<128><<<grid, CalCfg<128>::NTHREADS, CalCfg<128>::SMEM, st>>>(mq, mk, p);
-  }
+template <int D, bool ACC>
+static cudaError_t launch_calib_t(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mm,
+                                  const CalibParams& p, int grid, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(saf_calib_kernel<D, ACC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       CalCfg<D>::SMEM);
+  if (e != cudaSuccess) return e;
+  saf_calib_kernel<D, ACC><<<grid, CalCfg<D>::NTHREADS, CalCfg<D>::SMEM, st>>>(mq, mk, mm, p);
   return cudaGetLastError();
+}
+
+cudaError_t launch_calib(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mm,
+                         const CalibParams& p, int grid, cudaStream_t st) {
+  if (D == 64) return p.accumulate ? launch_calib_t<64, true>(mq, mk, mm, p, grid, st)
+                                   : launch_calib_t<64, false>(mq, mk, mm, p, grid, st);
+  return p.accumulate ? launch_calib_t<128, true>(mq, mk, mm, p, grid, st)
+                      : launch_calib_t<128, false>(mq, mk, mm, p, grid, st);
 }
 
 cudaError_t launch_calib_finalize(float* mean, const double* sumsq, const double* sum_plogp, double* tmp, int H, int T,

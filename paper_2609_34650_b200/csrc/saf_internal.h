@@ -172,12 +172,13 @@ struct CalibParams {
   double* sumsq;                    // [H] += sum_n ||A_n||_F^2
   double* sum_plogp;                // [H] += sum_n sum A_n log A_n
   int accumulate;                   // 0: overwrite mean_sum tiles, 1: add to them
+  int use_tma;                      // T % 4 == 0: tiles leave by TMA; else plain loads / stores
   int n_items, npairs;              // items = H x npairs, npairs = nblk (nblk+1)/2
   int* status;
   unsigned long long wait_limit_ns;
 };
-cudaError_t launch_calib(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CalibParams& p, int grid,
-                         cudaStream_t st);
+cudaError_t launch_calib(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mm,
+                         const CalibParams& p, int grid, cudaStream_t st);
 cudaError_t launch_calib_finalize(float* mean, const double* sumsq, const double* sum_plogp, double* tmp, int H, int T,
                                   double n_total, double* s_var, double* s_kl, int num_sms, cudaStream_t st);
 

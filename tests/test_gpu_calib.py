@@ -5,7 +5,10 @@ Tolerances.  A probability is exp2(s c - lse') with s the fp32 tensor-core score
 sums: about 1e-6 relative of |s| ~ 10, i.e. 1e-5 absolute in the exponent), lse' from the forward kernel (fp32) and
 ex2.approx (2^-22): about 2e-5 relative per entry, asserted as |got - want| <= 1e-6 + 2e-4 want for the mean.  The
 scores are differences of two nearly equal fp64 sums of such terms; with synthetic inputs the difference is a
-sizeable fraction of the sums, and 1e-3 relative is asserted."""
+sizeable fraction of the sums, and 1e-3 relative is asserted.  The forward-KL score also carries an absolute error
+of about 1e-6 nats per row: p log p is summed as p s c minus the row normaliser, which assumes that the fp32
+probabilities of a row sum to one (they do to about 1e-6), so 2e-6 absolute is allowed on top (it shows only when the
+score itself is zero: a single sequence, or identical ones)."""
 import numpy as np
 import pytest
 import torch
@@ -70,7 +73,7 @@ def _check(L, mean, s_var, s_kl, heads=None):
             wv = co.variance_score(A)
             assert abs(s_var[h] - wv) <= 1e-3 * wv + 1e-12, f"s_var head {h}: {s_var[h]} vs {wv}"
         wk = co.forward_kl_score(A)
-        assert abs(s_kl[h] - wk) <= 1e-3 * wk + 1e-9, f"s_kl head {h}: {s_kl[h]} vs {wk}"
+        assert abs(s_kl[h] - wk) <= 1e-3 * wk + 2e-6, f"s_kl head {h}: {s_kl[h]} vs {wk}"
 
 
 @pytest.mark.parametrize("N,H,T,D,g", [(3, 2, 300, 64, 1), (4, 2, 129, 128, 1), (2, 2, 200, 96, 1), (3, 4, 257, 64, 2),
