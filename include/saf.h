@@ -119,7 +119,7 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
  *   dQ, dK, dV : device, contiguous [B][H][T][D], fp32 or bf16 per p->grad_dtype.
  *                Frozen heads: dV = P^^T dO, dQ and dK written with zeros.
  * dQ is accumulated with floating-point atomics across key blocks, so its low-order bits can vary
- * from run to run.  Head dimension 64 only (SAF_ERR_UNSUPPORTED otherwise). */
+ * from run to run.  Head dimensions 64, 96 and 128. */
 int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const void* K, const void* V,
                         const void* O, const void* dO, const float* LSE, const uint8_t* frozen_mask_host,
                         const float* alpha, const float* rho, const float* logZ, void* dQ, void* dK,
@@ -129,7 +129,10 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
  * saf_pattern_prepare (only when `prepare` is nonzero; otherwise the normalisers of the previous
  * call on this context are reused), the forward and - when dO_host is not NULL - the backward, and
  * copies the results back.  Tensors are contiguous [B][H][T][D] (strides in `p` are ignored);
- * alpha_host/rho_host are [H][Tp].  Any output pointer may be NULL to skip its copy.  Synchronous. */
+ * alpha_host/rho_host are [H][Tp].  Any output pointer may be NULL to skip its copy.  Synchronous.
+ * Large problems are cut into up to eight chunks of whole batch entries on three streams (inputs in, compute,
+ * results out), so that the copies of neighbouring chunks overlap the compute and each other in both directions
+ * of the link; give pinned host memory for that overlap to happen. */
 int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_host, const void* K_host,
                               const void* V_host, const void* dO_host, const uint8_t* frozen_mask_host,
                               const float* alpha_host, const float* rho_host, int32_t prepare, void* O_host,

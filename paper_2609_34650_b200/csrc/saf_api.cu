@@ -72,8 +72,9 @@ struct saf_ctx {
   // staging for the host-buffer entry point
   DevBuf hq, hk, hv, hdo, ho, hlse, hdq, hdk, hdv, halpha, hrho, hlogz;
   // host-buffer step: compute stream, copy stream and the events that order them
-  cudaStream_t hs_main = nullptr, hs_copy = nullptr;
-  cudaEvent_t hs_qkv = nullptr, hs_do = nullptr, hs_fwd = nullptr, hs_out = nullptr;
+  static constexpr int HS_CHUNKS = 8;
+  cudaStream_t hs_main = nullptr, hs_copy = nullptr, hs_outs = nullptr;
+  cudaEvent_t hs_in[HS_CHUNKS] = {}, hs_do[HS_CHUNKS] = {}, hs_fwd[HS_CHUNKS] = {}, hs_cmp[HS_CHUNKS] = {};
 };
 
 namespace {
@@ -386,7 +387,9 @@ int saf_destroy(saf_ctx* ctx) {
   if (ctx->status_dev) cudaFree(ctx->status_dev);
   if (ctx->hs_main) cudaStreamDestroy(ctx->hs_main);
   if (ctx->hs_copy) cudaStreamDestroy(ctx->hs_copy);
-  for (cudaEvent_t e : {ctx->hs_qkv, ctx->hs_do, ctx->hs_fwd, ctx->hs_out})
+  if (ctx->hs_outs) cudaStreamDestroy(ctx->hs_outs);
+  for (int c = 0; c < saf_ctx::HS_CHUNKS; ++c)
+    for (cudaEvent_t e : {ctx->hs_in[c], ctx->hs_do[c], ctx->hs_fwd[c], ctx->hs_cmp[c]})
     if (e) cudaEventDestroy(e);
   for (TimedLaunch& t : ctx->timed) {
     cudaEventDestroy(t.beg);
@@ -826,67 +829,99 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
   if (bwd && ((rc = ensure(ctx->hdo, tb)) || (rc = ensure(ctx->hdq, gb)) || (rc = ensure(ctx->hdk, gb)) ||
               (rc = ensure(ctx->hdv, gb))))
     return rc;
-  // Two streams: the copy stream brings dO in while the forward runs and takes O / LSE out while the
-  // backward runs; everything else is on the compute stream.
+  // Three streams: inputs in, compute, results out.  The batch is cut into chunks; chunk c+1 is on its way in and
+  // chunk c-1 on its way out (the link is full duplex) while chunk c computes.
   if (!ctx->hs_main) {
     if (cudaStreamCreateWithFlags(&ctx->hs_main, cudaStreamNonBlocking) != cudaSuccess ||
-        cudaStreamCreateWithFlags(&ctx->hs_copy, cudaStreamNonBlocking) != cudaSuccess)
+        cudaStreamCreateWithFlags(&ctx->hs_copy, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&ctx->hs_outs, cudaStreamNonBlocking) != cudaSuccess)
       return SAF_ERR_CUDA;
-    for (cudaEvent_t* e : {&ctx->hs_qkv, &ctx->hs_do, &ctx->hs_fwd, &ctx->hs_out})
-      if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return SAF_ERR_CUDA;
+    for (int c = 0; c < saf_ctx::HS_CHUNKS; ++c)
+      for (cudaEvent_t* e : {&ctx->hs_in[c], &ctx->hs_do[c], &ctx->hs_fwd[c], &ctx->hs_cmp[c]})
+        if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return SAF_ERR_CUDA;
   }
-  cudaStream_t st = ctx->hs_main, sc = ctx->hs_copy;
+  cudaStream_t st = ctx->hs_main, sc = ctx->hs_copy, so = ctx->hs_outs;
+  // chunks of whole batches; small problems go in one piece (a chunk should keep the link busy for a while)
+  int nchunks = 1;
+  if (tb >= (8u << 20)) nchunks = std::min<int>(saf_ctx::HS_CHUNKS, p->B);
+  const int bc_max = (p->B + nchunks - 1) / nchunks;
   saf_problem q = *p;
   const int64_t s2 = p->D, s1 = static_cast<int64_t>(p->T) * p->D, s0 = s1 * p->H;
   int64_t* sets[4] = {q.q_strides, q.k_strides, q.v_strides, q.o_strides};
   for (int64_t* s : sets) { s[0] = s0; s[1] = s1; s[2] = s2; }
   q.k_strides[0] = q.v_strides[0] = s0 / kvg;
   bool okc = true;
-  if (no > 0) {
-    okc &= cudaMemcpyAsync(ctx->hq.ptr, Q_host, tb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    okc &= cudaMemcpyAsync(ctx->hk.ptr, K_host, tkv, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  }
-  okc &= cudaMemcpyAsync(ctx->hv.ptr, V_host, tkv, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (nf > 0 && prepare) {
     okc &= cudaMemcpyAsync(ctx->halpha.ptr, alpha_host, pb, cudaMemcpyHostToDevice, st) == cudaSuccess;
     okc &= cudaMemcpyAsync(ctx->hrho.ptr, rho_host, pb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  }
-  if (bwd) {
-    // dO follows Q, K, V on the link, on the copy stream, so that the forward does not wait for it
-    okc &= cudaEventRecord(ctx->hs_qkv, st) == cudaSuccess;
-    okc &= cudaStreamWaitEvent(sc, ctx->hs_qkv, 0) == cudaSuccess;
-    okc &= cudaMemcpyAsync(ctx->hdo.ptr, dO_host, tb, cudaMemcpyHostToDevice, sc) == cudaSuccess;
-    okc &= cudaEventRecord(ctx->hs_do, sc) == cudaSuccess;
   }
   if (!okc) return SAF_ERR_CUDA;
   const float* a = static_cast<const float*>(ctx->halpha.ptr);
   const float* r = static_cast<const float*>(ctx->hrho.ptr);
   float* z = static_cast<float*>(ctx->hlogz.ptr);
   if (nf > 0 && prepare && (rc = saf_pattern_prepare(ctx, p->H, p->Tp, frozen_mask_host, a, r, z, st))) return rc;
-  rc = saf_hybrid_attn_fwd(ctx, &q, ctx->hq.ptr, ctx->hk.ptr, ctx->hv.ptr, frozen_mask_host, a, r, z, ctx->ho.ptr,
-                           static_cast<float*>(ctx->hlse.ptr), st);
-  if (rc) return rc;
-  // O and LSE leave on the copy stream as soon as the forward is done
-  okc &= cudaEventRecord(ctx->hs_fwd, st) == cudaSuccess;
-  okc &= cudaStreamWaitEvent(sc, ctx->hs_fwd, 0) == cudaSuccess;
-  if (O_host) okc &= cudaMemcpyAsync(O_host, ctx->ho.ptr, tb, cudaMemcpyDeviceToHost, sc) == cudaSuccess;
-  if (LSE_host) okc &= cudaMemcpyAsync(LSE_host, ctx->hlse.ptr, lb, cudaMemcpyDeviceToHost, sc) == cudaSuccess;
-  okc &= cudaEventRecord(ctx->hs_out, sc) == cudaSuccess;
-  if (!okc) return SAF_ERR_CUDA;
-  if (bwd) {
-    if (cudaStreamWaitEvent(st, ctx->hs_do, 0) != cudaSuccess) return SAF_ERR_CUDA;
-    rc = saf_hybrid_attn_bwd(ctx, &q, ctx->hq.ptr, ctx->hk.ptr, ctx->hv.ptr, ctx->ho.ptr, ctx->hdo.ptr,
-                             static_cast<const float*>(ctx->hlse.ptr), frozen_mask_host, a, r, z, ctx->hdq.ptr,
-                             ctx->hdk.ptr, ctx->hdv.ptr, st);
+  const size_t esz = 2, gsz = (p->grad_dtype == SAF_F32 ? 4 : 2);
+  const size_t per_b = static_cast<size_t>(p->H) * p->T * p->D;          // elements of one batch entry, H heads
+  const size_t per_b_kv = per_b / kvg;
+  const size_t per_b_lse = static_cast<size_t>(p->H) * p->T;
+  auto off = [](const void* base, size_t bytes) { return static_cast<const char*>(base) + bytes; };
+  auto offw = [](void* base, size_t bytes) { return static_cast<char*>(base) + bytes; };
+  int ci = 0;
+  for (int b0 = 0; b0 < p->B; b0 += bc_max, ++ci) {
+    const int bc = std::min(bc_max, p->B - b0);
+    q.B = bc;
+    const size_t o_q = b0 * per_b, o_kv = b0 * per_b_kv, o_l = b0 * per_b_lse;
+    // ---- in: Q, K, V, then dO
+    if (no > 0) {
+      okc &= cudaMemcpyAsync(offw(ctx->hq.ptr, o_q * esz), off(Q_host, o_q * esz), bc * per_b * esz,
+                             cudaMemcpyHostToDevice, sc) == cudaSuccess;
+      okc &= cudaMemcpyAsync(offw(ctx->hk.ptr, o_kv * esz), off(K_host, o_kv * esz), bc * per_b_kv * esz,
+                             cudaMemcpyHostToDevice, sc) == cudaSuccess;
+    }
+    okc &= cudaMemcpyAsync(offw(ctx->hv.ptr, o_kv * esz), off(V_host, o_kv * esz), bc * per_b_kv * esz,
+                           cudaMemcpyHostToDevice, sc) == cudaSuccess;
+    okc &= cudaEventRecord(ctx->hs_in[ci], sc) == cudaSuccess;
+    if (bwd) {
+      okc &= cudaMemcpyAsync(offw(ctx->hdo.ptr, o_q * esz), off(dO_host, o_q * esz), bc * per_b * esz,
+                             cudaMemcpyHostToDevice, sc) == cudaSuccess;
+      okc &= cudaEventRecord(ctx->hs_do[ci], sc) == cudaSuccess;
+    }
+    // ---- compute
+    okc &= cudaStreamWaitEvent(st, ctx->hs_in[ci], 0) == cudaSuccess;
+    if (!okc) return SAF_ERR_CUDA;
+    void* Oc = offw(ctx->ho.ptr, o_q * esz);
+    float* Lc = static_cast<float*>(ctx->hlse.ptr) + o_l;
+    rc = saf_hybrid_attn_fwd(ctx, &q, offw(ctx->hq.ptr, o_q * esz), offw(ctx->hk.ptr, o_kv * esz),
+                             offw(ctx->hv.ptr, o_kv * esz), frozen_mask_host, a, r, z, Oc, Lc, st);
     if (rc) return rc;
+    // O and LSE leave as soon as the forward of the chunk is done
+    okc &= cudaEventRecord(ctx->hs_fwd[ci], st) == cudaSuccess;
+    okc &= cudaStreamWaitEvent(so, ctx->hs_fwd[ci], 0) == cudaSuccess;
+    if (O_host) okc &= cudaMemcpyAsync(offw(O_host, o_q * esz), Oc, bc * per_b * esz, cudaMemcpyDeviceToHost, so) == cudaSuccess;
+    if (LSE_host)
+      okc &= cudaMemcpyAsync(LSE_host + o_l, Lc, bc * per_b_lse * sizeof(float), cudaMemcpyDeviceToHost, so) == cudaSuccess;
+    if (bwd) {
+      // (dO was queued behind the chunk's Q, K, V on the inbound stream)
+      okc &= cudaStreamWaitEvent(st, ctx->hs_do[ci], 0) == cudaSuccess;
+      if (!okc) return SAF_ERR_CUDA;
+      void* dQc = offw(ctx->hdq.ptr, o_q * gsz);
+      void* dKc = offw(ctx->hdk.ptr, o_kv * gsz);
+      void* dVc = offw(ctx->hdv.ptr, o_kv * gsz);
+      rc = saf_hybrid_attn_bwd(ctx, &q, offw(ctx->hq.ptr, o_q * esz), offw(ctx->hk.ptr, o_kv * esz),
+                               offw(ctx->hv.ptr, o_kv * esz), Oc, offw(ctx->hdo.ptr, o_q * esz), Lc, frozen_mask_host,
+                               a, r, z, dQc, dKc, dVc, st);
+      if (rc) return rc;
+      okc &= cudaEventRecord(ctx->hs_cmp[ci], st) == cudaSuccess;
+      okc &= cudaStreamWaitEvent(so, ctx->hs_cmp[ci], 0) == cudaSuccess;
+      if (dQ_host) okc &= cudaMemcpyAsync(offw(dQ_host, o_q * gsz), dQc, bc * per_b * gsz, cudaMemcpyDeviceToHost, so) == cudaSuccess;
+      if (dK_host) okc &= cudaMemcpyAsync(offw(dK_host, o_kv * gsz), dKc, bc * per_b_kv * gsz, cudaMemcpyDeviceToHost, so) == cudaSuccess;
+      if (dV_host) okc &= cudaMemcpyAsync(offw(dV_host, o_kv * gsz), dVc, bc * per_b_kv * gsz, cudaMemcpyDeviceToHost, so) == cudaSuccess;
+    }
+    if (!okc) return SAF_ERR_CUDA;
   }
-  if (bwd) {
-    if (dQ_host) okc &= cudaMemcpyAsync(dQ_host, ctx->hdq.ptr, gb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (dK_host) okc &= cudaMemcpyAsync(dK_host, ctx->hdk.ptr, gkv, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (dV_host) okc &= cudaMemcpyAsync(dV_host, ctx->hdv.ptr, gkv, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  }
-  if (!okc) return SAF_ERR_CUDA;
-  if (cudaStreamSynchronize(sc) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return SAF_ERR_CUDA;
+  if (cudaStreamSynchronize(sc) != cudaSuccess || cudaStreamSynchronize(so) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return SAF_ERR_CUDA;
   return saf_last_device_status(ctx, nullptr);
 }
 

@@ -283,6 +283,31 @@ def test_host_buffer_step_matches_device_path():
         assert ma < 1e-4                       # atomics order only
 
 
+@pytest.mark.parametrize("g,gd", [(1, saf.SAF_F32), (2, saf.SAF_F32), (1, saf.SAF_BF16)])
+def test_host_buffer_step_in_chunks_matches_device_path(g, gd):
+    """Large enough to be cut into chunks of whole batch entries (11 entries -> chunks of 2 and a last one of 1)."""
+    inp = si.generate(si.Workload("host-chunks", 11, 4, 2048, 64, (2,), -0.05, seed=29, kv_group=g))
+    D = Layer(inp, grad_dtype=gd).run()
+    wl = inp.wl
+    ctx = saf.Context(0)
+    pin = lambda t: t.pin_memory()
+    Q, K, V, dO = (pin(bf16_tensor(x)) for x in (inp.q, inp.k, inp.v, inp.do))
+    alpha, rho = pin(torch.from_numpy(inp.alpha)), pin(torch.from_numpy(inp.rho))
+    O = pin(torch.empty_like(Q))
+    LSE = pin(torch.empty(wl.B, wl.H, wl.T))
+    gdt = torch.float32 if gd == saf.SAF_F32 else torch.bfloat16
+    dQ, dK, dV = (pin(torch.full(t.shape, float("nan"), dtype=gdt)) for t in (Q, K, V))
+    prob = saf.make_problem(Q, wl.stored_len, grad_dtype=gd, k_like=K, v_like=V, o_like=O, kv_group=g, H=wl.H)
+    ctx.saf_hybrid_attn_step_host(prob, Q, K, V, dO, inp.mask, alpha, rho, 1, O, LSE, dQ, dK, dV)
+    assert torch.equal(O, D.O.cpu()) and torch.equal(LSE, D.LSE.cpu())
+    for got, want, exact in ((dQ, D.grads[0], False), (dK, D.grads[1], g == 1), (dV, D.grads[2], g == 1)):
+        if exact:
+            assert torch.equal(got, want.cpu())
+        else:                                  # accumulated with atomics: order only
+            ma, rl = errors(got.float().numpy().astype(np.float64), D.host(want))
+            assert ma < (1e-4 if gd == saf.SAF_F32 else 2e-2) and np.isfinite(got.float().numpy()).all()
+
+
 def test_invalid_arguments_are_rejected():
     inp = si.generate(si.Workload("bad", 1, 2, 64, 64, (1,), -0.05))
     L = Layer(inp)
