@@ -54,9 +54,6 @@ struct W128 {
 enum W128Site { W_KV_EMPTY = 81, W_H_EMPTY, W_KV_FULL, W_H_FULL, W_PDS_FULL, W_ACC_FREE, W_DQ_FREE, W_S_FULL,
                 W_SDP_FULL, W_DQ_FULL, W_ACC_FULL, W_PFREE, W_C_DONE };
 
-__device__ __forceinline__ void st_shared_v4w(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }

@@ -83,8 +83,10 @@ def test_calibration_statistics_parity(N, H, T, D, g):
     _check(L, *_run(L))
 
 
-def test_streaming_in_several_calls_equals_one_call():
-    wl = _workload(6, 2, 260, 64, seed=3)
+@pytest.mark.parametrize("T,D,g", [(260, 64, 1), (257, 64, 1), (260, 128, 2), (131, 96, 1)])
+def test_streaming_in_several_calls_equals_one_call(T, D, g):
+    """Adding calls (old tile fetched and summed) against a single call; T = 257 and 131 take the path without TMA."""
+    wl = _workload(6, 2, T, D, g, seed=3)
     L = Layer(si.generate(wl), backward=False)
     m1, v1, k1 = _run(L, splits=1)
     m3, v3, k3 = _run(L, splits=3)
