@@ -42,7 +42,7 @@ struct CalCfg {
   static constexpr int OFF_OUT = NS * STAGE_BYTES;      // 4 boxes of 128 rows x 32 fp32 (128-byte rows, swizzled): 64 KB
   static constexpr int OUT_BOX_BYTES = 128 * 128;
   static constexpr int OFF_BAR = OFF_OUT + 4 * OUT_BOX_BYTES;
-  static constexpr int NBAR = 2 * NS + 5;
+  static constexpr int NBAR = 2 * NS + 8;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
   static constexpr int TMEM_COLS = 256;                 // two score buffers of 128 fp32 columns
   static constexpr int NTHREADS = 576;
@@ -75,8 +75,8 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   uint64_t* qk_empty = bars + C::NS;             // [NS]
   uint64_t* s_full = qk_empty + C::NS;           // [2] score buffer b holds a finished tile
   uint64_t* s_free = s_full + 2;                 // [2] the compute warps have read buffer b (16 warp arrivals)
-  uint64_t* old_full = s_free + 2;               // the item's old accumulator tile has landed in the output boxes
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(old_full + 1);
+  uint64_t* old_full = s_free + 2;               // [4] the old accumulator values of output box k have landed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(old_full + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -92,7 +92,7 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       mbar_init(s_full + b, 1);
       mbar_init(s_free + b, 16);
     }
-    mbar_init(old_full, 1);
+    for (int k = 0; k < 4; ++k) mbar_init(old_full + k, 1);
     mbar_fence_init();
   }
   if (warp == 17) {
@@ -164,9 +164,9 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const int rowl = q4 * 32 + lane;                   // query row within the block = TMEM lane
     const uint32_t lane_base = static_cast<uint32_t>(q4 * 32) << 16;
     const float c2 = p.scale_log2e;
-    uint32_t nl = 0, nit = 0;
+    uint32_t nl = 0, nold = 0;
     bool ok = true;
-    for (int idx = blockIdx.x; idx < p.n_items; idx += gridDim.x, ++nit) {
+    for (int idx = blockIdx.x; idx < p.n_items; idx += gridDim.x) {
       int h, I, J;
       decode_item(idx, p.npairs, h, I, J);
       const int qi = I * BLK + rowl;
@@ -174,14 +174,18 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       const bool diag = (I == J) || (J * BLK + BLK > p.T);   // tiles that need the per-element mask
       const float* lse_h = p.LSE + static_cast<size_t>(h) * p.T + qi;
       const size_t lse_step = static_cast<size_t>(p.H) * p.T;
-      if (ACC && p.use_tma) {
-        // what earlier calls left in this tile is fetched into the output boxes while the sequences are processed
-        // (the previous item's store has finished reading them first)
-        if (tid == 0) {
-          bulk_wait_group_read0();
-          mbar_expect_tx(old_full, 4 * C::OUT_BOX_BYTES);
-          for (int k = 0; k < 4; ++k)
-            tma_load_4d(smem + C::OFF_OUT + k * C::OUT_BOX_BYTES, &mm, old_full, J * BLK + 32 * k, I * BLK, h, 0);
+      // The four 32-column groups of compute warps hand their output box over independently of one another
+      // (thread 128 cq leads group cq): a barrier over all 16 warps would put them back in lockstep at every item.
+      const bool box_ok = J * BLK + 32 * cq < p.T;     // the group's box lies inside the matrix
+      const bool lead = (tid == 128 * cq);
+      uint8_t* const box = smem + C::OFF_OUT + cq * C::OUT_BOX_BYTES;
+      if (ACC && p.use_tma && lead) {
+        // what earlier calls left in this box is fetched while the sequences are processed (the previous item's
+        // store has finished reading the box first)
+        bulk_wait_group_read0();
+        if (box_ok) {
+          mbar_expect_tx(old_full + cq, C::OUT_BOX_BYTES);
+          tma_load_4d(box, &mm, old_full + cq, J * BLK + 32 * cq, I * BLK, h, 0);
         }
       }
       uint64_t acc2[16];                               // the thread's 32 accumulators as packed pairs
@@ -252,13 +256,16 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       float ent = fmaf(ps, c2, -lsum);                 // sum of p log2 p of this thread's part of the item
       // the item's tile of sum_n A^(n): written, or added to what earlier calls left
       if (p.use_tma) {
-        // through shared memory and one TMA store / reduce-add per 32-column box: coalesced, and it drains while
-        // the next item computes.  The previous item's boxes have been read out before they are overwritten; the
-        // warps also agree here whether a wait has been abandoned.
-        if (!ACC && tid == 0) bulk_wait_group_read0();
-        if (ACC && ok && !mbar_wait_warp(old_full, nit & 1, wc, C_OLD_FULL)) ok = false;
-        if (named_bar_or(1, 512, !ok)) break;
-        const uint32_t stage_row = smem_u32(smem + C::OFF_OUT) + cq * C::OUT_BOX_BYTES + rowl * 128;
+        // through shared memory and one TMA store per 32-column box: coalesced, and it drains while the next item
+        // computes.  The previous item's box has been read out before it is overwritten; the four warps of the
+        // group also agree here whether a wait has been abandoned.
+        if (!ACC && lead) bulk_wait_group_read0();
+        if (ACC && box_ok) {
+          if (ok && !mbar_wait_warp(old_full + cq, nold & 1, wc, C_OLD_FULL)) ok = false;
+          ++nold;
+        }
+        if (named_bar_or(1 + cq, 128, !ok)) break;
+        const uint32_t stage_row = smem_u32(box) + rowl * 128;
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
           const uint32_t chunk = static_cast<uint32_t>(g ^ (rowl & 7)) * 16;
@@ -268,12 +275,9 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                         __float_as_uint(acc[4 * g + 2] + o2), __float_as_uint(acc[4 * g + 3] + o3));
         }
         fence_proxy_async_smem();
-        named_bar_sync(2, 512);
-        if (tid == 0) {
-          for (int k = 0; k < 4; ++k) {
-            if (J * BLK + 32 * k >= p.T) break;
-            tma_store_4d(&mm, smem + C::OFF_OUT + k * C::OUT_BOX_BYTES, J * BLK + 32 * k, I * BLK, h, 0);
-          }
+        named_bar_sync(5 + cq, 128);
+        if (lead && box_ok) {
+          tma_store_4d(&mm, box, J * BLK + 32 * cq, I * BLK, h, 0);
           bulk_commit_group();
         }
       } else {
@@ -296,7 +300,7 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         atomicAdd(p.sum_plogp + h, static_cast<double>(ent) * LN2_C);
       }
     }
-    if (tid == 0) bulk_wait_group0();                  // every store / reduce-add has landed before the kernel ends
+    if ((tid & 127) == 0) bulk_wait_group0();          // every store has landed before the kernel ends
   }
 
   // ------------------------------------------------------------------ teardown
