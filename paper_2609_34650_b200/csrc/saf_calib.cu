@@ -12,7 +12,7 @@
 //
 // One persistent kernel, item = (head, query block I, key block J <= I), all items cost the same.  Per item a loop
 // over the N sequences: S = Q_I K_J^T on the tensor core (tcgen05, both operands K-major in 128B-swizzled smem via
-// TMA, accumulator double-buffered in TMEM), then per element in registers p = exp2(s c - lse'), acc += p,
+// TMA, score tiles in four TMEM buffers), then per element in registers p = exp2(s c - lse'), acc += p,
 // sq += p^2, ent += p log2 p; the 128 x 128 fp32 accumulator tile lives in the registers of the 16 compute warps
 // (thread = query row x 32 keys) and leaves once per item through shared memory as four TMA stores into the dense
 // accumulator, which drain while the next item computes; in the calls that add to earlier ones the old tile is
@@ -42,9 +42,10 @@ struct CalCfg {
   static constexpr int OFF_OUT = NS * STAGE_BYTES;      // 4 boxes of 128 rows x 32 fp32 (128-byte rows, swizzled): 64 KB
   static constexpr int OUT_BOX_BYTES = 128 * 128;
   static constexpr int OFF_BAR = OFF_OUT + 4 * OUT_BOX_BYTES;
-  static constexpr int NBAR = 2 * NS + 8;
+  static constexpr int NSB = 4;                         // score buffers in TMEM (128 fp32 columns each)
+  static constexpr int NBAR = 2 * NS + 2 * NSB + 4;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
-  static constexpr int TMEM_COLS = 256;                 // two score buffers of 128 fp32 columns
+  static constexpr int TMEM_COLS = 128 * NSB;
   static constexpr int NTHREADS = 576;
 };
 
@@ -73,9 +74,9 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR);
   uint64_t* qk_full = bars;                      // [NS]
   uint64_t* qk_empty = bars + C::NS;             // [NS]
-  uint64_t* s_full = qk_empty + C::NS;           // [2] score buffer b holds a finished tile
-  uint64_t* s_free = s_full + 2;                 // [2] the compute warps have read buffer b (16 warp arrivals)
-  uint64_t* old_full = s_free + 2;               // [4] the old accumulator values of output box k have landed
+  uint64_t* s_full = qk_empty + C::NS;           // [NSB] score buffer b holds a finished tile
+  uint64_t* s_free = s_full + C::NSB;            // [NSB] the compute warps have read buffer b (16 warp arrivals)
+  uint64_t* old_full = s_free + C::NSB;               // [4] the old accumulator values of output box k have landed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(old_full + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -88,7 +89,7 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       mbar_init(qk_full + s, 1);
       mbar_init(qk_empty + s, 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < C::NSB; ++b) {
       mbar_init(s_full + b, 1);
       mbar_init(s_free + b, 16);
     }
@@ -138,10 +139,10 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     bool ok = true;
     for (int idx = blockIdx.x; idx < p.n_items && ok; idx += gridDim.x) {
       for (int n = 0; n < p.B && ok; ++n, ++nl) {
-        const uint32_t s = nl % C::NS, gb = nl & 1;
+        const uint32_t s = nl % C::NS, gb = nl % C::NSB;
         ok = mbar_wait_warp(qk_full + s, (nl / C::NS) & 1, wc, C_QK_FULL);
         if (!ok) break;
-        ok = mbar_wait_warp(s_free + gb, ((nl >> 1) & 1) ^ 1, wc, C_S_FREE);
+        ok = mbar_wait_warp(s_free + gb, ((nl / C::NSB) & 1) ^ 1, wc, C_S_FREE);
         if (!ok) break;
         tc_fence_after();
         const uint32_t q_lo = lo_k + ((s * C::STAGE_BYTES) >> 4);
@@ -200,8 +201,8 @@ saf_calib_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       for (int n = 0; n < p.B; ++n, ++nl) {
         float lse_raw_next = 0.0f;
         if (n + 1 < p.B && row_ok) lse_raw_next = __ldg(lse_h + (n + 1) * lse_step);
-        const uint32_t gb = nl & 1;
-        if (ok && !mbar_wait_warp(s_full + gb, (nl >> 1) & 1, wc, C_S_FULL)) ok = false;
+        const uint32_t gb = nl % C::NSB;
+        if (ok && !mbar_wait_warp(s_full + gb, (nl / C::NSB) & 1, wc, C_S_FULL)) ok = false;
         if (!ok) continue;                             // (keeps the loop counters in step; nothing is read)
         const float lse2 = row_ok ? lse_raw * LOG2E_C : INFINITY;
         lse_raw = lse_raw_next;
