@@ -327,26 +327,36 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         ++nkv;
         TR(3, 7);
         const int U = 2 * ntiles;
-        // score MMAs of half tile u into buffer u & 1
-        auto issue_A = [&](int u) {
+        // score MMAs of half tile u into buffer u & 1, in two parts (issuing lane only): S'^T, whose completion
+        // starts the exponentials, and dP'^T
+        auto issue_S = [&](int u) {
           const uint32_t s = (nqdo + (u >> 1)) % C::NS;
           const uint32_t b = u & 1;
           const uint32_t q_lo = lo_k + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
-          const uint32_t do_lo = lo_k + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
           const uint32_t qx_lo = lo_x + ((C::OFF_QX + s * 4096 + b * 2048) >> 4);
+          const uint32_t t_s = tmem + C::COL_S + 64 * b;
+#pragma unroll
+          for (int kc = 0; kc < 4; ++kc)
+            umma_ts2(t_s, tmem + C::COL_KT + 8 * kc, q_lo + 2 * kc, hi_k, id_s, kc > 0);
+          umma_ss2(t_s, ones_lo, hi_x, qx_lo, hi_x, id_s, 1);
+          umma_commit(s_full + b);                       // the exponentials start while dP'^T is computed
+        };
+        auto issue_dP = [&](int u) {
+          const uint32_t s = (nqdo + (u >> 1)) % C::NS;
+          const uint32_t b = u & 1;
+          const uint32_t do_lo = lo_k + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
           const uint32_t dox_lo = lo_x + ((C::OFF_DOX + s * 4096 + b * 2048) >> 4);
-          const uint32_t t_s = tmem + C::COL_S + 64 * b, t_dp = tmem + C::COL_DP + 64 * b;
+          const uint32_t t_dp = tmem + C::COL_DP + 64 * b;
+#pragma unroll
+          for (int kc = 0; kc < 4; ++kc)
+            umma_ts2(t_dp, tmem + C::COL_VT + 8 * kc, do_lo + 2 * kc, hi_k, id_s, kc > 0);
+          umma_ss2(t_dp, ones_lo, hi_x, dox_lo, hi_x, id_s, 1);
+          umma_commit(sdp_full + b);
+        };
+        auto issue_A = [&](int u) {
           if (leader) {
-#pragma unroll
-            for (int kc = 0; kc < 4; ++kc)
-              umma_ts2(t_s, tmem + C::COL_KT + 8 * kc, q_lo + 2 * kc, hi_k, id_s, kc > 0);
-            umma_ss2(t_s, ones_lo, hi_x, qx_lo, hi_x, id_s, 1);
-            umma_commit(s_full + b);                     // the exponentials start while dP'^T is computed
-#pragma unroll
-            for (int kc = 0; kc < 4; ++kc)
-              umma_ts2(t_dp, tmem + C::COL_VT + 8 * kc, do_lo + 2 * kc, hi_k, id_s, kc > 0);
-            umma_ss2(t_dp, ones_lo, hi_x, dox_lo, hi_x, id_s, 1);
-            umma_commit(sdp_full + b);
+            issue_S(u);
+            issue_dP(u);
           }
           __syncwarp();
         };
@@ -374,35 +384,36 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             ok = mbar_wait_warp(acc_free, (nitem & 1) ^ 1, wc, B_ACC_FREE);
             if (!ok) break;
           }
-          tc_fence_after();
           const uint32_t pos = nqdo + (u >> 1);
+          const bool more = u + 2 < U;
+          if (more && b == 0) {
+            // Q / dO of the next tile (its first half tile goes into this buffer below)
+            ok = mbar_wait_warp(qdo_full + (pos + 1) % C::NS, ((pos + 1) / C::NS) & 1, wc, B_QDO_FULL);
+            if (!ok) break;
+          }
+          tc_fence_after();
           const uint32_t s = pos % C::NS;
           const uint32_t q_lo = lo_m + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
           const uint32_t do_lo = lo_m + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
           const uint32_t acc0 = u > 0 ? 1u : 0u;
           const uint32_t t_p = tmem + C::COL_S + 64 * b, t_ds = tmem + C::COL_DP + 64 * b;
           if (leader) {
+            // MMAs execute in issue order: the buffer's next S'^T may overwrite P^T as soon as the dV MMAs that
+            // read it are queued, and the next dP'^T follows the dK MMAs that read dS^T.  Putting S'^T ahead of
+            // dK brings the compute warps' next exponentials forward by four MMAs.
 #pragma unroll
             for (int kc = 0; kc < 4; ++kc)
               umma_ts2(tmem + C::COL_DV, t_p + 8 * kc + (kc >= 2 ? 16 : 0), do_lo + 128 * kc, hi_m, id_acc,
                        kc > 0 ? 1u : acc0);
+            if (more) issue_S(u + 2);
 #pragma unroll
             for (int kc = 0; kc < 4; ++kc)
               umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc + (kc >= 2 ? 16 : 0), q_lo + 128 * kc, hi_m, id_acc,
                        kc > 0 ? 1u : acc0);
+            if (more) issue_dP(u + 2);
           }
           __syncwarp();
           TR(0, 6);
-          // the buffer's next score MMAs follow its gradient MMAs directly (in-order execution)
-          if (u + 2 < U) {
-            if (b == 0) {
-              ok = mbar_wait_warp(qdo_full + (pos + 1) % C::NS, ((pos + 1) / C::NS) & 1, wc, B_QDO_FULL);
-              if (!ok) break;
-              tc_fence_after();
-            }
-            issue_A(u + 2);
-            TR(3, 3);
-          }
           if (b == 1) {
             // full tile done: its Q/dO stage can be refilled, and dQ of the tile follows
             if (leader) umma_commit(qdo_empty + s);
