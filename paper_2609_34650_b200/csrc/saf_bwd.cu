@@ -326,7 +326,6 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         if (!ok) break;
         ++nkv;
         TR(3, 7);
-        const int U = 2 * ntiles;
         // score MMAs of half tile u into buffer u & 1, in two parts (issuing lane only): S'^T, whose completion
         // starts the exponentials, and dP'^T
         auto issue_S = [&](int u) {
@@ -368,70 +367,79 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         TR(3, 2);
         issue_A(1);
         TR(3, 3);
-        for (int u = 0; u < U && ok; ++u) {
-          const uint32_t b = u & 1;
-          TR(0, 4);
-          if (b == 0) {
-            ok = mbar_wait_warp(pds_full, npds0 & 1, wc, B_PDS_FULL);
-            ++npds0;
-          } else {
-            ok = mbar_wait_warp(pds_full + 1, npds1 & 1, wc, B_PDS_FULL);
-            ++npds1;
+        // Per tile: first what the compute warps wait for - for each buffer, dV of its half tile and right behind
+        // it the buffer's next S'^T (MMAs execute in issue order, so S'^T may overwrite P^T once the dV MMAs that
+        // read it are queued) - then what they need only after their exponentials: dK and the next dP'^T of both
+        // buffers (dP'^T follows the dK MMAs that read dS^T), the release of the Q/dO stage, and dQ of the tile.
+        for (int t = 0; t < ntiles && ok; ++t) {
+          const uint32_t pos = nqdo + t;
+          const uint32_t s = pos % C::NS;
+          const bool more = t + 1 < ntiles;
+          const uint32_t acc0 = t > 0 ? 1u : 0u;
+#pragma unroll
+          for (int b = 0; b < 2; ++b) {
+            TR(0, 4);
+            if (b == 0) {
+              ok = mbar_wait_warp(pds_full, npds0 & 1, wc, B_PDS_FULL);
+              ++npds0;
+            } else {
+              ok = mbar_wait_warp(pds_full + 1, npds1 & 1, wc, B_PDS_FULL);
+              ++npds1;
+            }
+            if (!ok) break;
+            TR(0, 5);
+            if (t == 0 && b == 0) {
+              ok = mbar_wait_warp(acc_free, (nitem & 1) ^ 1, wc, B_ACC_FREE);
+              if (!ok) break;
+            }
+            if (more && b == 0) {
+              // Q / dO of the next tile (its first half tile goes into this buffer below)
+              ok = mbar_wait_warp(qdo_full + (pos + 1) % C::NS, ((pos + 1) / C::NS) & 1, wc, B_QDO_FULL);
+              if (!ok) break;
+            }
+            tc_fence_after();
+            const uint32_t do_lo = lo_m + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
+            const uint32_t t_p = tmem + C::COL_S + 64 * b;
+            if (leader) {
+#pragma unroll
+              for (int kc = 0; kc < 4; ++kc)
+                umma_ts2(tmem + C::COL_DV, t_p + 8 * kc + (kc >= 2 ? 16 : 0), do_lo + 128 * kc, hi_m, id_acc,
+                         (kc > 0 || b > 0) ? 1u : acc0);
+              if (more) issue_S(2 * t + 2 + b);
+            }
+            __syncwarp();
           }
           if (!ok) break;
-          TR(0, 5);
-          if (u == 0) {
-            ok = mbar_wait_warp(acc_free, (nitem & 1) ^ 1, wc, B_ACC_FREE);
-            if (!ok) break;
-          }
-          const uint32_t pos = nqdo + (u >> 1);
-          const bool more = u + 2 < U;
-          if (more && b == 0) {
-            // Q / dO of the next tile (its first half tile goes into this buffer below)
-            ok = mbar_wait_warp(qdo_full + (pos + 1) % C::NS, ((pos + 1) / C::NS) & 1, wc, B_QDO_FULL);
-            if (!ok) break;
-          }
-          tc_fence_after();
-          const uint32_t s = pos % C::NS;
-          const uint32_t q_lo = lo_m + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
-          const uint32_t do_lo = lo_m + ((C::OFF_DO + s * C::PANEL + b * 8192) >> 4);
-          const uint32_t acc0 = u > 0 ? 1u : 0u;
-          const uint32_t t_p = tmem + C::COL_S + 64 * b, t_ds = tmem + C::COL_DP + 64 * b;
           if (leader) {
-            // MMAs execute in issue order: the buffer's next S'^T may overwrite P^T as soon as the dV MMAs that
-            // read it are queued, and the next dP'^T follows the dK MMAs that read dS^T.  Putting S'^T ahead of
-            // dK brings the compute warps' next exponentials forward by four MMAs.
 #pragma unroll
-            for (int kc = 0; kc < 4; ++kc)
-              umma_ts2(tmem + C::COL_DV, t_p + 8 * kc + (kc >= 2 ? 16 : 0), do_lo + 128 * kc, hi_m, id_acc,
-                       kc > 0 ? 1u : acc0);
-            if (more) issue_S(u + 2);
+            for (int b = 0; b < 2; ++b) {
+              const uint32_t q_lo = lo_m + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
+              const uint32_t t_ds = tmem + C::COL_DP + 64 * b;
 #pragma unroll
-            for (int kc = 0; kc < 4; ++kc)
-              umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc + (kc >= 2 ? 16 : 0), q_lo + 128 * kc, hi_m, id_acc,
-                       kc > 0 ? 1u : acc0);
-            if (more) issue_dP(u + 2);
+              for (int kc = 0; kc < 4; ++kc)
+                umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc + (kc >= 2 ? 16 : 0), q_lo + 128 * kc, hi_m, id_acc,
+                         (kc > 0 || b > 0) ? 1u : acc0);
+              if (more) issue_dP(2 * t + 2 + b);
+            }
+            // full tile done: its Q/dO stage can be refilled, and dQ of the tile follows
+            umma_commit(qdo_empty + s);
           }
           __syncwarp();
           TR(0, 6);
-          if (b == 1) {
-            // full tile done: its Q/dO stage can be refilled, and dQ of the tile follows
-            if (leader) umma_commit(qdo_empty + s);
-            ok = mbar_wait_warp(dq_free, (ndq & 1) ^ 1, wc, B_DQ_FREE);
-            if (!ok) break;
-            ++ndq;
-            tc_fence_after();
-            const uint32_t ds_lo = lo_m + ((C::OFF_DS + (ntile_ord & 1) * 2 * C::PANEL) >> 4);
-            if (leader) {
+          ok = mbar_wait_warp(dq_free, (ndq & 1) ^ 1, wc, B_DQ_FREE);
+          if (!ok) break;
+          ++ndq;
+          tc_fence_after();
+          const uint32_t ds_lo = lo_m + ((C::OFF_DS + (ntile_ord & 1) * 2 * C::PANEL) >> 4);
+          if (leader) {
 #pragma unroll
-              for (int kc = 0; kc < 8; ++kc)
-                umma_ss2(tmem + C::COL_DQ, ds_lo + 128 * kc, hi_m, km_lo + 128 * kc, hi_m, id_dq, kc > 0);
-              umma_commit(dq_full);
-            }
-            TR(0, 9);
-            ++ntile_ord;
-            __syncwarp();
+            for (int kc = 0; kc < 8; ++kc)
+              umma_ss2(tmem + C::COL_DQ, ds_lo + 128 * kc, hi_m, km_lo + 128 * kc, hi_m, id_dq, kc > 0);
+            umma_commit(dq_full);
           }
+          TR(0, 9);
+          ++ntile_ord;
+          __syncwarp();
         }
         if (!ok) break;
         nqdo += ntiles;
