@@ -65,7 +65,8 @@ def _dev(x):
 
 
 # ------------------------------------------------------------------------------------------------ marginals
-@pytest.mark.parametrize("Hf,T,seed", [(2, 300, 1), (3, 1100, 2), (1, 2500, 3), (1, 1, 4), (2, 33, 5)])
+@pytest.mark.parametrize("Hf,T,seed", [(2, 300, 1), (3, 1100, 2), (1, 2500, 3), (1, 1, 4), (2, 33, 5),
+                                       (1, 5000, 6), (1, 8200, 7)])       # (the last two: 32 columns per thread)
 def test_marginals_parity(Hf, T, seed):
     # garbage above the diagonal must be ignored; a steep decay puts entries under the 1e-9 floor
     A = si.mean_attention_maps(Hf, T, seed, upper_fill=7.0, pmax=5.0)
@@ -122,6 +123,17 @@ def test_fit_parity(T, steps, tol):
         assert abs(loss[h] - fo.fit_objective(wa, wr, ea[h], er[h])) < 1e-4
         assert abs(kl[h] - fo.fit_kl_dense(P[h], wa, wr)) < 1e-4
     _check_self_consistent(a, r, z, loss, kl, P, ea, er, pl)
+
+
+def test_fit_long_sequence_two_steps():
+    """T beyond 4096: the pass kernels stage more than 48 KB of operands per CTA."""
+    T = 5000
+    A = si.mean_attention_maps(1, T, 31)
+    P, ea, er, pl = _oracle_stats(A)
+    a, r, z, loss, kl = _gpu_fit(_ctx(), _dev(ea), _dev(er), _dev(pl), 2)
+    wa, wr, wz = fo.fit_compact(ea[0], er[0], steps=2)
+    assert np.max(np.abs(a[0] - wa)) < 2e-4 and np.max(np.abs(r[0] - wr)) < 2e-4 and np.max(np.abs(z[0] - wz)) < 1e-4
+    assert abs(kl[0] - fo.fit_kl_dense(P[0], wa, wr)) < 1e-4
 
 
 def test_fit_start_is_prescribed_point():
