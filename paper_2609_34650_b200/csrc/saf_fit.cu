@@ -32,6 +32,7 @@ constexpr double LOG2E_D = 1.4426950408889634074;
 constexpr double LN2_D = 0.6931471805599453094;
 constexpr int XB = 32;             // x values per CTA of the pass kernel (one per lane)
 constexpr int PASS_WARPS = 8;      // warps of a pass CTA; they split the y range in chunks of 32
+constexpr int YC = 4096;           // y values staged in shared memory at a time
 
 __device__ __forceinline__ float ex2f(float x) {
   float y;
@@ -195,9 +196,9 @@ saf_fit_init_kernel(FitState s) {
 // MODE 0 (pass A): x = query i, y = distance d <= i:   u = r', window = a'[i-d],  c = -z'(i)   -> z'(i) += log2 S
 // MODE 1 (pass B): blockIdx.z = 0: x = key j, y = d <= T-1-j:  u = r', window = -z'[j+d], c = a'(j) -> Adam on alpha(j)
 //                  blockIdx.z = 1: x = d,     y = j <= T-1-d:  u = a', window = -z'[d+j], c = r'(d) -> Adam on rho(d)
-// CTA = 32 consecutive x (one per lane) x 8 warps that take the 32-wide chunks of y in turn.  Both operands of the
-// CTA's y range are staged in shared memory; the window carries 32 entries of -inf on the side where the causal
-// range ends, which is the mask.
+// CTA = 32 consecutive x (one per lane) x 8 warps that take the 32-wide chunks of y in turn.  Both operands are
+// staged in shared memory, 4096 values of y at a time; window entries outside the causal range are -inf, which is the
+// mask.
 template <int MODE>
 __global__ void __launch_bounds__(PASS_WARPS * 32)
 saf_fit_pass_kernel(FitState s, int cur, double bc1, double bc2) {
@@ -213,40 +214,52 @@ saf_fit_pass_kernel(FitState s, int cur, double bc1, double bc2) {
   const int which = (MODE == 0) ? 0 : static_cast<int>(blockIdx.z);
   const int ny = (MODE == 0) ? min(T, x0 + XB) : T - x0;          // y = 0 .. ny-1 covers every lane's range
   const int nyp = (ny + 31) & ~31;
-  float* us = sm_f;                       // [nyp]
-  float* ws = sm_f + nyp;                 // [nyp + 32]
+  const int ycap = min(YC, (T + 31) & ~31);
+  float* us = sm_f;                       // [ycap]
+  float* ws = sm_f + ycap;                // [ycap + 32]
   const float* a2c = cur ? s.a2[1] : s.a2[0];
   const float* r2c = cur ? s.r2[1] : s.r2[0];
   const float* u_g = (MODE == 1 && which == 1) ? a2c + o : r2c + o;
   const float* w_g = (MODE == 0) ? a2c + o : s.nz2 + o;
-  for (int y = tid; y < nyp; y += PASS_WARPS * 32) us[y] = (y < ny) ? u_g[y] : -INFINITY;
-  if (MODE == 0) {
-    // ws[k] = a'[k - 32] for k >= 32, -inf below: lane x at distance y reads index x - y + 32
-    for (int k = tid; k < nyp + 32; k += PASS_WARPS * 32) ws[k] = (k >= 32 && k - 32 < ny) ? w_g[k - 32] : -INFINITY;
-  } else {
-    // ws[k] = -z'[x0 + k] for x0 + k < T, -inf beyond: lane x - x0 at offset y reads index (x - x0) + y
-    for (int k = tid; k < nyp + 32; k += PASS_WARPS * 32) ws[k] = (x0 + k < T) ? w_g[x0 + k] : -INFINITY;
-  }
   const int x = x0 + lane;
   float c = -INFINITY;
   if (x < T) c = (MODE == 0) ? s.nz2[o + x] : (which == 0 ? a2c[o + x] : r2c[o + x]);
-  __syncthreads();
   float acc0 = 0.0f, acc1 = 0.0f;
-  for (int y0 = warp * 32; y0 < nyp; y0 += PASS_WARPS * 32) {
-    const float4* u4 = reinterpret_cast<const float4*>(us + y0);
-    const float* wp = (MODE == 0) ? ws + (x - y0 + 32) : ws + (lane + y0);
+  // the y range in chunks of YC: shared memory per CTA stays at 33 KB whatever T is (six CTAs per SM)
+  for (int yb = 0; yb < nyp; yb += YC) {
+    const int nyc = min(YC, nyp - yb);                 // a multiple of 32
+    if (yb > 0) __syncthreads();                       // the previous chunk has been read
+    for (int y = tid; y < nyc; y += PASS_WARPS * 32) us[y] = (yb + y < ny) ? u_g[yb + y] : -INFINITY;
+    if (MODE == 0) {
+      // lane x at distance y reads a'[x - y]: the chunk's window starts at g0 = x0 - (yb + nyc - 1), and
+      // ws[k] = a'[g0 + k] (-inf below index 0); the lane's entry for y is ws[lane + (yb + nyc - 1 - y)]
+      const int g0 = x0 - (yb + nyc - 1);
+      for (int k = tid; k < nyc + 32; k += PASS_WARPS * 32) {
+        const int g = g0 + k;
+        ws[k] = (g >= 0 && g < ny) ? w_g[g] : -INFINITY;
+      }
+    } else {
+      // lane x at offset y reads -z'[x + y]: ws[k] = -z'[x0 + yb + k] (-inf beyond T); the lane's entry is
+      // ws[lane + (y - yb)]
+      for (int k = tid; k < nyc + 32; k += PASS_WARPS * 32) ws[k] = (x0 + yb + k < T) ? w_g[x0 + yb + k] : -INFINITY;
+    }
+    __syncthreads();
+    for (int y0 = warp * 32; y0 < nyc; y0 += PASS_WARPS * 32) {
+      const float4* u4 = reinterpret_cast<const float4*>(us + y0);
+      const float* wp = (MODE == 0) ? ws + (lane + nyc - 1 - y0) : ws + (lane + y0);
 #pragma unroll
-    for (int t4 = 0; t4 < 8; ++t4) {
-      const float4 u = u4[t4];
-      const int t = 4 * t4;
-      const float w0 = (MODE == 0) ? wp[-t] : wp[t];
-      const float w1 = (MODE == 0) ? wp[-t - 1] : wp[t + 1];
-      const float w2 = (MODE == 0) ? wp[-t - 2] : wp[t + 2];
-      const float w3 = (MODE == 0) ? wp[-t - 3] : wp[t + 3];
-      acc0 += ex2f((u.x + c) + w0);
-      acc1 += ex2f((u.y + c) + w1);
-      acc0 += ex2f((u.z + c) + w2);
-      acc1 += ex2f((u.w + c) + w3);
+      for (int t4 = 0; t4 < 8; ++t4) {
+        const float4 u = u4[t4];
+        const int t = 4 * t4;
+        const float w0 = (MODE == 0) ? wp[-t] : wp[t];
+        const float w1 = (MODE == 0) ? wp[-t - 1] : wp[t + 1];
+        const float w2 = (MODE == 0) ? wp[-t - 2] : wp[t + 2];
+        const float w3 = (MODE == 0) ? wp[-t - 3] : wp[t + 3];
+        acc0 += ex2f((u.x + c) + w0);
+        acc1 += ex2f((u.y + c) + w1);
+        acc0 += ex2f((u.z + c) + w2);
+        acc1 += ex2f((u.w + c) + w3);
+      }
     }
   }
   __shared__ float red[PASS_WARPS][32];
@@ -347,7 +360,7 @@ cudaError_t launch_fit(const FitState& s, int Hf, int steps, const double* plogp
                        float* logZ_out, long long out_stride, double* loss_out, double* kl_out, cudaStream_t st) {
   const int T = s.T;
   const int nxb = (T + XB - 1) / XB;
-  const size_t smem = (2 * static_cast<size_t>((T + 31) & ~31) + 32) * sizeof(float);
+  const size_t smem = (2 * static_cast<size_t>(std::min((T + 31) & ~31, YC)) + 32) * sizeof(float);
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(saf_fit_pass_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 static_cast<int>(smem))) != cudaSuccess)
