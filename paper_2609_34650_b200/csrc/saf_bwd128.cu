@@ -216,9 +216,12 @@ saf_bwd128_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant_
     const bool leader = elect_one() != 0;
     const uint32_t sb = smem_u32(smem);
     constexpr uint32_t id_s = umma_idesc_bf16(128, 64, 0, 0);      // S^T, dP^T half tiles: both operands K-major
-    constexpr uint32_t id_acc = umma_idesc_bf16(128, 128, 0, 1);   // dV, dK: A from TMEM, B MN-major
-    constexpr uint32_t id_dq = umma_idesc_bf16(128, 128, 1, 1);    // dQ: A (dS^T tile) M-major, B MN-major
-    constexpr uint32_t id_hk = umma_idesc_f16(128, 128, 0, 1);     // fp16 band x fp16 scaled dO
+    // (head dimension 96 runs here with features 96..127 zero-filled by TMA: the gradient MMAs produce only 96
+    // columns and the score MMAs skip the two empty k-steps)
+    const uint32_t id_acc = umma_idesc_bf16(128, p.d_real, 0, 1);  // dV, dK: A from TMEM, B MN-major
+    const uint32_t id_dq = umma_idesc_bf16(128, p.d_real, 1, 1);   // dQ: A (dS^T tile) M-major, B MN-major
+    const uint32_t id_hk = umma_idesc_f16(128, p.d_real, 0, 1);    // fp16 band x fp16 scaled dO
+    const int nk16 = p.d_real / 16;
     // descriptor halves for smem offset 0: 128B-swizzled K-major (k-step +32 B inside a 64-feature panel), the
     // no-swizzle K-major row-term tiles (LBO 128 B, SBO 256 B), 128B-swizzled MN-major tiles whose two 64-wide
     // halves are a half panel (Q / dO stages) or a panel (K_J, dS^T) apart, and the Hankel band
@@ -256,6 +259,7 @@ saf_bwd128_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant_
           if (leader) {
 #pragma unroll
             for (int kc = 0; kc < 8; ++kc) {
+              if (kc >= nk16) break;
               const uint32_t ok_ = ((kc >> 2) * C::PANEL + (kc & 3) * 32) >> 4;
               const uint32_t oh_ = ((kc >> 2) * C::HP + (kc & 3) * 32) >> 4;
               umma_ss2(t_s, k_lo + ok_, hi_k, q_lo + oh_, hi_k, id_s, kc > 0);
@@ -264,6 +268,7 @@ saf_bwd128_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant_
             umma_commit(s_full);                         // the exponentials start while dP'^T is computed
 #pragma unroll
             for (int kc = 0; kc < 8; ++kc) {
+              if (kc >= nk16) break;
               const uint32_t ok_ = ((kc >> 2) * C::PANEL + (kc & 3) * 32) >> 4;
               const uint32_t oh_ = ((kc >> 2) * C::HP + (kc & 3) * 32) >> 4;
               umma_ss2(t_dp, v_lo + ok_, hi_k, do_lo + oh_, hi_k, id_s, kc > 0);

@@ -185,8 +185,11 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     const bool leader = elect_one() != 0;
     const uint32_t sb = smem_u32(smem);
     constexpr uint32_t idesc_s = umma_idesc_bf16(128, 128, 0, 0);
-    constexpr uint32_t idesc_o = umma_idesc_bf16(128, D, 0, 1);
-    constexpr uint32_t idesc_hk = umma_idesc_f16(128, D, 0, 1);    // tensor-core frozen form: fp16 band x fp16 scaled V
+    // (head dimension 96 runs here with features 96..127 zero-filled by TMA: its MMAs skip the two empty k-steps of
+    // the scores and produce only 96 output columns)
+    const uint32_t idesc_o = umma_idesc_bf16(128, p.d_real, 0, 1);
+    const int nk16 = p.d_real / 16;
+    const uint32_t idesc_hk = umma_idesc_f16(128, p.d_real, 0, 1);  // tensor-core frozen form: fp16 band x fp16 scaled V
     uint32_t nq = 0, nk = 0, nv = 0, np = 0, nitem = 0;
     bool ok = true;
     // descriptor halves for smem offset 0: K-major tiles (k-step +32 B within a 64-column panel) and
@@ -249,6 +252,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           if (leader) {
 #pragma unroll
             for (int kc = 0; kc < D / 16; ++kc) {
+              if (kc >= nk16) break;
               const uint32_t off = ((kc >> 2) * C::PANEL_BYTES + (kc & 3) * 32) >> 4;
               umma_ss2(tmem + C::COL_S, q_lo + off, hi_k, k_lo + off, hi_k, idesc_s, kc > 0);
             }
