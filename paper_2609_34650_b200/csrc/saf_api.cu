@@ -816,9 +816,7 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
   const int kvg = kv_group_of(p);
   const size_t nelem = static_cast<size_t>(p->B) * p->H * p->T * p->D;
   const size_t tb = nelem * 2;
-  const size_t tkv = tb / kvg;                      // K, V: H / kv_group heads
   const size_t gb = nelem * (p->grad_dtype == SAF_F32 ? 4 : 2);
-  const size_t gkv = gb / kvg;
   const size_t pb = static_cast<size_t>(p->H) * p->Tp * sizeof(float);
   const size_t lb = static_cast<size_t>(p->B) * p->H * p->T * sizeof(float);
   const bool bwd = dO_host != nullptr;

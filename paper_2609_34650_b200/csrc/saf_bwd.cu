@@ -206,8 +206,9 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       tma_prefetch_desc(&mdot);
       uint32_t nkv = 0, nqdo = 0, nfz = 0;
       bool ok = true, fz_open = false;
+#ifdef SAF_TRACE
       int tr_n = 0;
-      (void)tr_n;
+#endif
       // K_J / V_J of the ordinary items run one item ahead of the tile loads: K into the other K slot (free
       // once the item before the current one has finished), V into the single V slot (free once the
       // current item's V has been copied to TMEM).
@@ -308,8 +309,9 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     const uint32_t ones_lo = lo_x + (C::OFF_ONES >> 4);
     uint32_t nqdo = 0, nitem = 0, ndq = 0, ntile_ord = 0, nkv = 0, nfz = 0;
     uint32_t npds0 = 0, npds1 = 0;
+#ifdef SAF_TRACE
     int tr_n = 0;
-    (void)tr_n;
+#endif
     bool ok = true;
     ItemView nxt = load_item(p, it_begin, it_end);
     for (int it = it_begin; it < it_end && ok; ++it, ++nitem) {
@@ -589,8 +591,9 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     const int bar_id = 4 + grp;                          // named barrier of this group
     uint32_t nacc = 0, ntile_ord = 0, nsdp = 0, npf = 0, nkvc = 0;
     bool ok = true;
+#ifdef SAF_TRACE
     int tr_n = 0;
-    (void)tr_n;
+#endif
     // K_J (group 0) / V_J (group 1) of the next ordinary item: this thread's half row from the swizzled
     // smem tile into TMEM as the A operand of the score MMAs (bf16 pairs, feature index = reduction index)
     // The fp32 epilogue leaves through TMA stores that read this group's dS^T panels; before the group

@@ -117,8 +117,9 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const WaitCtx wc{abort_flag, p.status, p.wait_limit_ns};
+#ifdef SAF_TRACE
   int tr_n = 0;
-  (void)tr_n;
+#endif
 
   if (tid == 0) {
     *abort_flag = 0;
