@@ -488,6 +488,13 @@ def test_config2_full_size_sampled_units():
     check_units(L, [(1, wl.frozen_heads[3]), (2, oh)], panel=1024)
 
 
+def test_long_sequence_16k_forward_backward_sampled_units():
+    """T = 16384 (the longest training context of the paper's cross-context comparison): 128 key blocks per head."""
+    wl = si.Workload("long-16k", 1, 3, 16384, 64, (1,), -0.005, seed=61)
+    L = Layer(si.generate(wl)).run()
+    check_units(L, [(0, 0), (0, 1)], panel=1024)
+
+
 def test_config4_long_prefill_sampled_row_panels():
     wl = si.config(4)
     L = Layer(si.generate(wl), backward=False).run(backward=False)
