@@ -308,6 +308,34 @@ def test_host_buffer_step_in_chunks_matches_device_path(g, gd):
             assert ma < (1e-4 if gd == saf.SAF_F32 else 2e-2) and np.isfinite(got.float().numpy()).all()
 
 
+def test_forward_backward_capture_into_a_cuda_graph():
+    """After a warm-up call (which allocates the context's workspaces and uploads the work lists) a forward +
+    backward step records into a CUDA graph, and replays reproduce the eager results bit for bit (dQ to rounding:
+    its reduce-adds arrive in varying order)."""
+    inp = si.generate(si.Workload("graph", 2, 4, 600, 64, (1,), -0.05, seed=71))
+    L = Layer(inp)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        L.run()
+        want = [t.clone() for t in (L.O, L.LSE, *L.grads)]
+        for t in (L.O, L.LSE, *L.grads):
+            t.fill_(float("nan"))
+        g = torch.cuda.CUDAGraph()
+        c = L.ctx
+        with torch.cuda.graph(g, stream=s):
+            c.saf_hybrid_attn_fwd(L.prob, L.Q, L.K, L.V, L.mask, L.alpha, L.rho, L.logZ, L.O, L.LSE)
+            c.saf_hybrid_attn_bwd(L.prob, L.Q, L.K, L.V, L.O, L.dO, L.LSE, L.mask, L.alpha, L.rho, L.logZ, *L.grads)
+        for _ in range(2):
+            g.replay()
+        torch.cuda.synchronize()
+    code, detail = L.ctx.saf_last_device_status()
+    assert code == saf.SAF_OK, f"device status {code} detail {detail:#x}"
+    got = (L.O, L.LSE, *L.grads)
+    assert torch.equal(got[0], want[0]) and torch.equal(got[1], want[1])
+    assert torch.equal(got[3], want[3]) and torch.equal(got[4], want[4])
+    assert (got[2] - want[2]).abs().max().item() < 1e-4
+
+
 def test_invalid_arguments_are_rejected():
     inp = si.generate(si.Workload("bad", 1, 2, 64, 64, (1,), -0.05))
     L = Layer(inp)
