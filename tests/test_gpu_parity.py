@@ -356,7 +356,7 @@ def test_invalid_arguments_are_rejected():
 
 
 # --------------------------------------------------------------------------- grouped-query path
-def _check_gqa_layer(L, backward):
+def _check_gqa_layer(L, backward, grad_rel_l2=REL_L2):
     """Whole layer against the dense oracle: K, V (and dK, dV) have H / kv_group heads."""
     inp, wl = L.inp, L.inp.wl
     q, k, v, do = f64(inp)
@@ -379,11 +379,12 @@ def _check_gqa_layer(L, backward):
             if inp.mask[h]:
                 assert not dQ[b, h].any(), "dQ of a frozen head must be exactly zero"
             else:
-                assert_close(dQ[b, h], eQ[b, h], f"dQ[{b},{h}]")
+                assert_close(dQ[b, h], eQ[b, h], f"dQ[{b},{h}]", rel_l2=grad_rel_l2)
         for hk in range(wl.H // wl.kv_group):
-            assert_close(dK[b, hk], eK[b, hk], f"dK[{b},kv {hk}]")
+            assert_close(dK[b, hk], eK[b, hk], f"dK[{b},kv {hk}]", rel_l2=grad_rel_l2)
             # a shared head's dV sums kv_group heads: the absolute bound scales with the number of terms
-            assert_close(dV[b, hk], eV[b, hk], f"dV[{b},kv {hk}]", max_abs=MAX_ABS * np.sqrt(wl.kv_group))
+            assert_close(dV[b, hk], eV[b, hk], f"dV[{b},kv {hk}]", max_abs=MAX_ABS * np.sqrt(wl.kv_group),
+                         rel_l2=grad_rel_l2)
 
 
 @pytest.mark.parametrize("H,g,frozen,T", [(8, 4, (1, 6), 300), (4, 2, (), 257), (6, 3, (0, 1, 2), 200),
@@ -437,7 +438,7 @@ def test_gqa_bf16_gradients_and_bad_group():
 
 
 # --------------------------------------------------------------------------- packed Q/K layout
-def _check_packed_layer(L, backward):
+def _check_packed_layer(L, backward, grad_rel_l2=REL_L2):
     inp, wl = L.inp, L.inp.wl
     q, k, v, do = f64(inp)
     al, rh = inp.alpha.astype(np.float64), inp.rho.astype(np.float64)
@@ -457,10 +458,10 @@ def _check_packed_layer(L, backward):
     assert dQ.shape == eQ.shape and dK.shape == eK.shape and dV.shape == eV.shape
     for b in range(wl.B):
         for s_ in range(dQ.shape[1]):
-            assert_close(dQ[b, s_], eQ[b, s_], f"dQ[{b},slot {s_}]")
-            assert_close(dK[b, s_], eK[b, s_], f"dK[{b},slot {s_}]")
+            assert_close(dQ[b, s_], eQ[b, s_], f"dQ[{b},slot {s_}]", rel_l2=grad_rel_l2)
+            assert_close(dK[b, s_], eK[b, s_], f"dK[{b},slot {s_}]", rel_l2=grad_rel_l2)
         for h in range(wl.H):
-            assert_close(dV[b, h], eV[b, h], f"dV[{b},{h}]")
+            assert_close(dV[b, h], eV[b, h], f"dV[{b},{h}]", rel_l2=grad_rel_l2)
 
 
 @pytest.mark.parametrize("H,frozen,T,gd", [(6, (1, 4), 300, "f32"), (4, (0, 3), 129, "bf16"), (3, (), 200, "f32"),
@@ -487,6 +488,43 @@ def test_packed_qk_layout_head_dim_128_forward_and_errors():
     with pytest.raises(saf.SafError) as e:
         L.run()
     assert e.value.code == 1
+
+
+# --------------------------------------------------------------------------- seeded random geometries
+def _random_workload(seed):
+    """A geometry drawn from the options of the layer (head size, grouping, packed layout, frozen set, lengths
+    around tile edges, stored pattern longer than the sequence, sink-like alpha, decay rate)."""
+    rng = np.random.default_rng(1000 + seed)
+    D = int(rng.choice([64, 96, 128]))
+    layout = rng.choice(["mha", "gqa", "packed"])
+    g = int(rng.choice([2, 3, 4])) if layout == "gqa" else 1
+    H = g * int(rng.integers(1, 4)) if layout == "gqa" else int(rng.integers(1, 7))
+    B = int(rng.integers(1, 4))
+    T = int(rng.choice([rng.integers(1, 130), rng.integers(130, 400), 128 * rng.integers(1, 4) + rng.choice([-1, 0, 1])]))
+    nf = int(rng.integers(0, H + 1))
+    frozen = tuple(sorted(rng.choice(H, size=nf, replace=False).tolist()))
+    Tp = T + int(rng.integers(0, 70)) if rng.random() < 0.4 else 0
+    spike = float(rng.choice([0.0, 3.0]))
+    slope = float(rng.choice([-0.3, -0.05, -0.005]))
+    return si.Workload(f"random-{seed}", B, H, max(T, 1), D, frozen, slope, Tp=Tp, alpha0_spike=spike,
+                       seed=2000 + seed, kv_group=g, packed_qk=(layout == "packed"))
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_geometries_forward_backward(seed):
+    """Combinations that no fixed case pairs up (for example 96-wide heads with shared key/value heads and a
+    stored pattern longer than the sequence), each against the dense oracle over the whole layer."""
+    wl = _random_workload(seed)
+    L = Layer(si.generate(wl)).run()
+    # The backward forms delta_i = dO_i . O_i from the bf16 O it is given.  With rows of only a few keys, dP - delta
+    # nearly cancels and that rounding of O (2^-9 relative) is not averaged out: measured at T = 3 the gradients lie
+    # within 2.5e-3 (relative L2) of the oracle's formulas evaluated with the same rounded O, but up to 1.1e-2 from
+    # the oracle's exact delta.  Sequences shorter than 8 therefore get twice the relative bound on the gradients.
+    tol = 2 * REL_L2 if wl.T < 8 else REL_L2
+    if wl.packed_qk:
+        _check_packed_layer(L, True, grad_rel_l2=tol)
+    else:
+        _check_gqa_layer(L, True, grad_rel_l2=tol)
 
 
 # --------------------------------------------------------------------------- full sizes, sampled
