@@ -1,15 +1,14 @@
 // Backward of the hybrid causal attention layer on sm_100a (head dimension 64): one persistent
 // kernel, one work item per (batch, head, 128-key block J), looping over query blocks I >= J.
 //
-// CTA = 736 threads:
+// CTA = 704 threads:
 //   warps 0-7   compute group 0: even 64-query half tiles (TMEM buffer 0); TMEM lane = key row, two warps
 //               per lane quarter, each on 32 of the half tile's 64 query columns
 //   warps 8-15  compute group 1: odd half tiles (TMEM buffer 1)
 //   warps 16-19 dQ drain: TMEM -> swizzled smem -> TMA reduce-add into the fp32 dQ accumulator
 //   warp 20     TMA producer
-//   warp 21     tcgen05 issuer of the score MMAs A(u); warp 22 issuer of the gradient MMAs B(u), C(t) and
-//               TMEM owner.  An issuing thread is stalled while its MMAs queue, so two issuers let one
-//               stream's bookkeeping (barrier waits) overlap the other stream's tensor work.
+//   warp 21     tcgen05 issuer of every MMA (A(u), B(u), C(t) below) and TMEM owner.  MMAs of one thread execute
+//               in issue order, which the schedule relies on; splitting the issue over two warps measured slower.
 // The per-tile critical path is a chain (scores -> exponentials -> gradient MMAs -> next scores on the
 // same buffer), so the exponential step is spread over as many warps as the register file allows.
 //
@@ -410,6 +409,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
               if (more) issue_S(2 * t + 2 + b);
             }
             __syncwarp();
+            TR(0, 10 + b);
           }
           if (!ok) break;
           if (leader) {
@@ -421,17 +421,23 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
               for (int kc = 0; kc < 4; ++kc)
                 umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc + (kc >= 2 ? 16 : 0), q_lo + 128 * kc, hi_m, id_acc,
                          (kc > 0 || b > 0) ? 1u : acc0);
-              if (more) issue_dP(2 * t + 2 + b);
             }
-            // full tile done: its Q/dO stage can be refilled, and dQ of the tile follows
+            // full tile done: its Q/dO stage can be refilled (ahead of the next dP'^T, which read the other stage,
+            // so that the refill starts ten MMAs earlier), and dQ of the tile follows
             umma_commit(qdo_empty + s);
+            if (more) {
+              issue_dP(2 * t + 2);
+              issue_dP(2 * t + 3);
+            }
           }
           __syncwarp();
           TR(0, 6);
           ok = mbar_wait_warp(dq_free, (ndq & 1) ^ 1, wc, B_DQ_FREE);
           if (!ok) break;
           ++ndq;
+          TR(0, 12);
           tc_fence_after();
+          TR(0, 13);
           const uint32_t ds_lo = lo_m + ((C::OFF_DS + (ntile_ord & 1) * 2 * C::PANEL) >> 4);
           if (leader) {
 #pragma unroll
@@ -442,6 +448,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           TR(0, 9);
           ++ntile_ord;
           __syncwarp();
+          TR(0, 14);
         }
         if (!ok) break;
         nqdo += ntiles;
