@@ -509,6 +509,26 @@ def run_ours(args):
                                                       "frac": fwd_flops / (fwd_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]},
                                   "saf_bwd_prep_kernel": {"launch_ms": prep_ms}}}
 
+    # context for the roofline's denominator: a library bf16 GEMM (8192^3) timed in this same process
+    live_gemm = None
+    try:
+        n = 8192
+        ga = torch.randn(n, n, device=dev, dtype=torch.bfloat16)
+        gb_ = torch.randn(n, n, device=dev, dtype=torch.bfloat16)
+        for _ in range(3):
+            torch.matmul(ga, gb_)
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(10):
+            torch.matmul(ga, gb_)
+        b.record()
+        torch.cuda.synchronize()
+        live_gemm = 2.0 * n ** 3 * 10 / (a.elapsed_time(b) * 1e-3) / 1e12
+        del ga, gb_
+    except Exception:                                                  # context only
+        live_gemm = None
+        torch.cuda.synchronize()
+
     fit = None if args.no_fit else fit_leg(ctx, saf, wl, peaks, dev)
     calib = None
     if not args.no_fit:
@@ -536,6 +556,8 @@ def run_ours(args):
         "gpu_launches": (4 if len(wl.frozen_heads) else 3) * args.steps,
         "clocks": clocks,
         "roofline": roofline,
+        "peak_context": {"library_bf16_gemm_8192_tflops_live": live_gemm,
+                         "measured_peaks_file_bf16_tflops": peaks["bf16_tflops"]},
         "fit": fit,
         "calibration": calib,
         "cpu_baseline": {"value": cpu_v, "unit": UNIT, "cores": cpu_threads, "kind": "oracle", "sample": cpu_desc},
