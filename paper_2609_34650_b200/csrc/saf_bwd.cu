@@ -460,12 +460,15 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         const uint32_t lo_b = desc_lo(d_band), hi_b = desc_hi(d_band);
         for (int t = 0; t < ntiles; ++t) {
           const uint32_t k = nfz % C::NFZ;
+          TR(0, 20);
           ok = mbar_wait_warp(fz_full + k, (nfz / C::NFZ) & 1, wc, B_QDO_FULL);
           if (!ok) break;
           ++nfz;
+          TR(0, 21);
           if (t == 0) {
             ok = mbar_wait_warp(acc_free, (nitem & 1) ^ 1, wc, B_ACC_FREE);
             if (!ok) break;
+            TR(0, 23);
           }
           tc_fence_after();
           const uint32_t band_lo = lo_b + (static_cast<uint32_t>(C::fz_band(k)) >> 4);
@@ -478,6 +481,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
             umma_commit(fz_empty + k);
           }
           __syncwarp();
+          TR(0, 22);
         }
         if (!ok) break;
       } else {
