@@ -240,8 +240,13 @@ int saf_get_kernel_time(saf_ctx* ctx, int32_t which, float* total_ms_out, int32_
 /* Head scheduler (host only, no GPU needed).  Builds the per-CTA work lists the persistent kernels
  * walk: one item per (batch, head, 128-row block); ordinary and frozen items are packed into the
  * same grid, longest-processing-time first, with a frozen tile weighted `frozen_weight_pct` percent
- * of an ordinary one.  `backward` = 0: block is a query block and costs (block+1) key tiles;
- * 1: block is a key block and costs (nblocks-block) query tiles.
+ * of an ordinary one plus a fixed cost per item (150 % of an ordinary tile forward, 100 % backward:
+ * the values the library uses for the 64-wide kernels).  `backward` = 0: block is a query block and
+ * costs (block+1) key tiles; 1: block is a key block and costs (nblocks-block) query tiles.
+ * The layer calls use measured weights per kernel family (frozen tile 30 / 20 % forward / backward at
+ * head dimension 64, 50 / 20 % at 96 and 128; item 150 / 100 % and 300 / 200 %), which the
+ * environment variables SAF_FROZEN_WEIGHT_PCT, SAF_FROZEN_WEIGHT_BWD_PCT, SAF_ITEM_OVERHEAD_PCT and
+ * SAF_ITEM_OVERHEAD_BWD_PCT (read by saf_create) override.
  *   items_out   : host int32[n_items*4] = (b, h, block, kind) with kind 0 ordinary / 1 frozen,
  *                 grouped by CTA; n_items = B*H*ceil(T/128)
  *   offsets_out : host int32[n_ctas+1], CSR offsets into items_out

@@ -21,7 +21,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 struct WorklistEntry {
-  int B, H, T, backward, grid;
+  int B, H, T, backward, grid, wide;
   std::vector<uint8_t> mask;
   WorkItem* items_dev = nullptr;
   int* offsets_dev = nullptr;
@@ -57,8 +57,13 @@ struct saf_ctx {
   cudaStream_t last_stream = nullptr;
   EncodeTiledFn encode = nullptr;
   unsigned long long wait_limit_ns = 2000000000ull;
-  int frozen_weight_pct = 30;              // cost of a frozen tile relative to an ordinary one, forward
-  int frozen_weight_bwd_pct = 25;          // ... and backward
+  // Scheduler cost model, in percent of an ordinary tile: a frozen tile (forward, backward) and the fixed cost of a
+  // work item (prologue, epilogue, pipeline refill).  0 = the measured default of the kernel family
+  // (sched_defaults); set by the SAF_FROZEN_WEIGHT_* / SAF_ITEM_OVERHEAD_* environment variables.
+  int frozen_weight_pct = 0;
+  int frozen_weight_bwd_pct = 0;
+  int item_overhead_pct = 0;
+  int item_overhead_bwd_pct = 0;
   int call_counter = 0;                    // ids of the calls that stage fp16 operands (overflow marks)
   std::vector<WorklistEntry> worklists;
   DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf, dkacc_buf, dvacc_buf, qslot_buf;
@@ -185,7 +190,7 @@ int upload_mask(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st) {
 // end, and each item goes to the CTA that becomes free first (list scheduling, which is what a dynamic
 // queue would do); only the last items are ordered longest-first so that the tail stays short.
 void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward, int n_ctas, int frozen_pct,
-                         std::vector<WorkItem>& items, std::vector<int>& offsets) {
+                         int overhead_pct, std::vector<WorkItem>& items, std::vector<int>& offsets) {
   const int nblk = (T + BLK - 1) / BLK;
   struct Cand { WorkItem w; long long cost; };
   std::vector<Cand> cand;
@@ -198,7 +203,7 @@ void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward,
         const int r = (z & 1) ? (nblk - 1 - z / 2) : (z / 2);        // rank by cost, 0 = most expensive
         const int k = backward ? r : (nblk - 1 - r);
         const long long tiles = backward ? (nblk - k) : (k + 1);
-        const long long cost = tiles * (kind == KIND_FROZEN ? frozen_pct : 100) + 20;   // + fixed per-item overhead
+        const long long cost = tiles * (kind == KIND_FROZEN ? frozen_pct : 100) + overhead_pct;   // + fixed per-item overhead
         cand.push_back({{b, h, k, kind}, cost});
       }
     }
@@ -224,10 +229,21 @@ void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward,
   offsets[n_ctas] = static_cast<int>(items.size());
 }
 
-int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int backward, int grid, cudaStream_t st,
-                 const WorklistEntry** out) {
+// Measured cost-model defaults: `wide` = the 128-wide kernels (head dimension 96 or 128), else the 64-wide ones.
+void sched_defaults(int wide, int backward, int* frozen_pct, int* overhead_pct) {
+  if (backward) {
+    *frozen_pct = 20;
+    *overhead_pct = wide ? 200 : 100;
+  } else {
+    *frozen_pct = wide ? 50 : 30;
+    *overhead_pct = wide ? 300 : 150;
+  }
+}
+
+int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int backward, int grid, int wide,
+                 cudaStream_t st, const WorklistEntry** out) {
   for (const WorklistEntry& e : ctx->worklists)
-    if (e.B == B && e.H == H && e.T == T && e.backward == backward && e.grid == grid &&
+    if (e.B == B && e.H == H && e.T == T && e.backward == backward && e.grid == grid && e.wide == wide &&
         std::memcmp(e.mask.data(), mask, H) == 0) {
       *out = &e;
       return SAF_OK;
@@ -240,10 +256,15 @@ int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int bac
   }
   std::vector<WorkItem> items;
   std::vector<int> offsets;
-  build_worklist_host(B, H, T, mask, backward, grid, backward ? ctx->frozen_weight_bwd_pct : ctx->frozen_weight_pct,
-                      items, offsets);
+  int frozen_pct, overhead_pct;
+  sched_defaults(wide, backward, &frozen_pct, &overhead_pct);
+  const int fw = backward ? ctx->frozen_weight_bwd_pct : ctx->frozen_weight_pct;
+  const int ov = backward ? ctx->item_overhead_bwd_pct : ctx->item_overhead_pct;
+  if (fw > 0) frozen_pct = fw;
+  if (ov > 0) overhead_pct = ov;
+  build_worklist_host(B, H, T, mask, backward, grid, frozen_pct, overhead_pct, items, offsets);
   WorklistEntry e;
-  e.B = B; e.H = H; e.T = T; e.backward = backward; e.grid = grid;
+  e.B = B; e.H = H; e.T = T; e.backward = backward; e.grid = grid; e.wide = wide;
   e.mask.assign(mask, mask + H);
   e.n_items = static_cast<int>(items.size());
   if (cudaMalloc(&e.items_dev, items.size() * sizeof(WorkItem)) != cudaSuccess) return SAF_ERR_NOMEM;
@@ -364,6 +385,14 @@ int saf_create(saf_ctx** out, int device) {
   if (const char* e = std::getenv("SAF_FROZEN_WEIGHT_BWD_PCT")) {
     long v = std::atol(e);
     if (v > 0 && v <= 400) ctx->frozen_weight_bwd_pct = static_cast<int>(v);
+  }
+  if (const char* e = std::getenv("SAF_ITEM_OVERHEAD_PCT")) {
+    long v = std::atol(e);
+    if (v > 0 && v <= 2000) ctx->item_overhead_pct = static_cast<int>(v);
+  }
+  if (const char* e = std::getenv("SAF_ITEM_OVERHEAD_BWD_PCT")) {
+    long v = std::atol(e);
+    if (v > 0 && v <= 2000) ctx->item_overhead_bwd_pct = static_cast<int>(v);
   }
   *out = ctx;
   return SAF_OK;
@@ -499,7 +528,7 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   const long long n_items = static_cast<long long>(p->B) * p->H * nblk;
   const int grid = static_cast<int>(std::min<long long>(2LL * ctx->num_sms, n_items));
   const WorklistEntry* wl = nullptr;
-  rc = get_worklist(ctx, p->B, p->H, p->T, frozen_mask_host, 0, grid, st, &wl);
+  rc = get_worklist(ctx, p->B, p->H, p->T, frozen_mask_host, 0, grid, p->D != 64, st, &wl);
   if (rc) return rc;
 
   CUtensorMap mq, mk, mv;
@@ -657,7 +686,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   const long long n_items = static_cast<long long>(p->B) * p->H * nblk;
   const int grid = static_cast<int>(std::min<long long>(ctx->num_sms, n_items));
   const WorklistEntry* wl = nullptr;
-  rc = get_worklist(ctx, p->B, p->H, p->T, frozen_mask_host, 1, grid, st, &wl);
+  rc = get_worklist(ctx, p->B, p->H, p->T, frozen_mask_host, 1, grid, p->D != 64, st, &wl);
   if (rc) return rc;
 
   CUtensorMap mq, mk, mv, mdo;
@@ -965,7 +994,7 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
   const int grid = static_cast<int>(std::min<long long>(2LL * ctx->num_sms, n_items));
   std::vector<uint8_t> none(nf, 0);
   const WorklistEntry* wl = nullptr;
-  rc = get_worklist(ctx, p->B, nf, p->T, none.data(), 1, grid, st, &wl);
+  rc = get_worklist(ctx, p->B, nf, p->T, none.data(), 1, grid, p->D != 64, st, &wl);
   if (rc) return rc;
   CUtensorMap mv, mdo;
   if ((rc = make_map(ctx, &mv, V, p, p->v_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg))) return rc;
@@ -1175,7 +1204,8 @@ int saf_build_worklist(int32_t B, int32_t H, int32_t T, const uint8_t* frozen_ma
     return SAF_ERR_INVALID_ARG;
   std::vector<WorkItem> items;
   std::vector<int> offsets;
-  build_worklist_host(B, H, T, frozen_mask_host, backward ? 1 : 0, n_ctas, frozen_weight_pct, items, offsets);
+  build_worklist_host(B, H, T, frozen_mask_host, backward ? 1 : 0, n_ctas, frozen_weight_pct, backward ? 100 : 150, items,
+                      offsets);
   std::memcpy(items_out, items.data(), items.size() * sizeof(WorkItem));
   std::memcpy(offsets_out, offsets.data(), offsets.size() * sizeof(int));
   return SAF_OK;
