@@ -64,6 +64,10 @@ struct saf_ctx {
   int frozen_weight_bwd_pct = 0;
   int item_overhead_pct = 0;
   int item_overhead_bwd_pct = 0;
+  // Forward grid = two CTAs per SM: the CTA that arrives second on an SM (block index >= grid / 2) runs slower
+  // than the first (measured 13 % at head dimension 64, 2 % on the 128-wide kernel; best settings 15 and 6) and gets that much less
+  // work.  -1 = the measured default; SAF_SECOND_WAVE_PCT overrides.
+  int second_wave_pct = -1;
   int call_counter = 0;                    // ids of the calls that stage fp16 operands (overflow marks)
   std::vector<WorklistEntry> worklists;
   DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf, dkacc_buf, dvacc_buf, qslot_buf;
@@ -190,7 +194,8 @@ int upload_mask(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st) {
 // end, and each item goes to the CTA that becomes free first (list scheduling, which is what a dynamic
 // queue would do); only the last items are ordered longest-first so that the tail stays short.
 void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward, int n_ctas, int frozen_pct,
-                         int overhead_pct, std::vector<WorkItem>& items, std::vector<int>& offsets) {
+                         int overhead_pct, int second_wave_pct, std::vector<WorkItem>& items,
+                         std::vector<int>& offsets) {
   const int nblk = (T + BLK - 1) / BLK;
   struct Cand { WorkItem w; long long cost; };
   std::vector<Cand> cand;
@@ -218,7 +223,9 @@ void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward,
     Load l = heap.top();
     heap.pop();
     per[l.second].push_back(c.w);
-    heap.push({l.first + c.cost, l.second});
+    // CTAs of the second half of the grid (the second CTA of each SM when the grid is two per SM) run slower
+    const long long scaled = l.second >= n_ctas / 2 ? c.cost * (100 + second_wave_pct) : c.cost * 100;
+    heap.push({l.first + scaled, l.second});
   }
   items.clear();
   offsets.assign(n_ctas + 1, 0);
@@ -262,7 +269,8 @@ int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int bac
   const int ov = backward ? ctx->item_overhead_bwd_pct : ctx->item_overhead_pct;
   if (fw > 0) frozen_pct = fw;
   if (ov > 0) overhead_pct = ov;
-  build_worklist_host(B, H, T, mask, backward, grid, frozen_pct, overhead_pct, items, offsets);
+  const int second_wave = backward ? 0 : (ctx->second_wave_pct >= 0 ? ctx->second_wave_pct : (wide ? 6 : 15));
+  build_worklist_host(B, H, T, mask, backward, grid, frozen_pct, overhead_pct, second_wave, items, offsets);
   WorklistEntry e;
   e.B = B; e.H = H; e.T = T; e.backward = backward; e.grid = grid; e.wide = wide;
   e.mask.assign(mask, mask + H);
@@ -385,6 +393,10 @@ int saf_create(saf_ctx** out, int device) {
   if (const char* e = std::getenv("SAF_FROZEN_WEIGHT_BWD_PCT")) {
     long v = std::atol(e);
     if (v > 0 && v <= 400) ctx->frozen_weight_bwd_pct = static_cast<int>(v);
+  }
+  if (const char* e = std::getenv("SAF_SECOND_WAVE_PCT")) {
+    long v = std::atol(e);
+    if (v >= 0 && v <= 100) ctx->second_wave_pct = static_cast<int>(v);
   }
   if (const char* e = std::getenv("SAF_ITEM_OVERHEAD_PCT")) {
     long v = std::atol(e);
@@ -1204,8 +1216,8 @@ int saf_build_worklist(int32_t B, int32_t H, int32_t T, const uint8_t* frozen_ma
     return SAF_ERR_INVALID_ARG;
   std::vector<WorkItem> items;
   std::vector<int> offsets;
-  build_worklist_host(B, H, T, frozen_mask_host, backward ? 1 : 0, n_ctas, frozen_weight_pct, backward ? 100 : 150, items,
-                      offsets);
+  build_worklist_host(B, H, T, frozen_mask_host, backward ? 1 : 0, n_ctas, frozen_weight_pct, backward ? 100 : 150, 0,
+                      items, offsets);
   std::memcpy(items_out, items.data(), items.size() * sizeof(WorkItem));
   std::memcpy(offsets_out, offsets.data(), offsets.size() * sizeof(int));
   return SAF_OK;

@@ -50,18 +50,10 @@ __device__ unsigned long long g_saf_trace[24][4096];
 extern "C" int saf_debug_read_trace(unsigned long long* out) {
   return static_cast<int>(cudaMemcpyFromSymbol(out, g_saf_trace, sizeof(g_saf_trace)));
 }
-__device__ unsigned long long g_saf_span[1024][2];   // per CTA: first and last instruction (globaltimer, ns)
-extern "C" int saf_debug_read_span(unsigned long long* out) {
-  return static_cast<int>(cudaMemcpyFromSymbol(out, g_saf_span, sizeof(g_saf_span)));
-}
-#define SPAN(k)                                                                    \
-  do {                                                                             \
-    if (threadIdx.x == 0) g_saf_span[blockIdx.x & 1023][k] = saf::globaltimer_ns(); \
-  } while (0)
 #else
 #define TR(role, id)
-#define SPAN(k)
 #endif
+SAF_SPAN_DEFINE(bwd)
 
 namespace saf {
 
@@ -155,7 +147,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const WaitCtx wc{abort_flag, p.status, p.wait_limit_ns};
   const int nblk = p.nblk;
-  SPAN(0);
+  SAF_SPAN(bwd, 0);
 
   if (tid == 0) {
     *abort_flag = 0;
@@ -933,7 +925,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   }
   tc_fence_before();
   __syncthreads();
-  SPAN(1);
+  SAF_SPAN(bwd, 1);
   if (warp == 21) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 

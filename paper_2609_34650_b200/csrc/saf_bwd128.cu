@@ -23,6 +23,8 @@
 #include "ptx.cuh"
 #include "saf_internal.h"
 
+SAF_SPAN_DEFINE(bwd128)
+
 namespace saf {
 
 namespace {
@@ -105,6 +107,7 @@ saf_bwd128_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant_
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const WaitCtx wc{abort_flag, p.status, p.wait_limit_ns};
+  SAF_SPAN(bwd128, 0);
   const int nblk = p.nblk;
 
   if (tid == 0) {
@@ -600,6 +603,7 @@ saf_bwd128_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant_
   }
   tc_fence_before();
   __syncthreads();
+  SAF_SPAN(bwd128, 1);
   if (warp == 21) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 

@@ -28,6 +28,8 @@
 
 #define TRF(role, id)
 
+SAF_SPAN_DEFINE(fwd128)
+
 namespace saf {
 
 constexpr float LOG2E_F = 1.4426950408889634f;
@@ -83,6 +85,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const WaitCtx wc{abort_flag, p.status, p.wait_limit_ns};
+  SAF_SPAN(fwd128, 0);
   int tr_n = 0;
   (void)tr_n;
 
@@ -582,6 +585,7 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   }
   tc_fence_before();
   __syncthreads();
+  SAF_SPAN(fwd128, 1);
   if (warp == 9) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 

@@ -45,6 +45,8 @@ extern "C" int saf_debug_read_trace_fwd(unsigned long long* out) {
 #define TRF(role, id)
 #endif
 
+SAF_SPAN_DEFINE(fwd64)
+
 namespace saf {
 
 namespace {
@@ -117,6 +119,7 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const WaitCtx wc{abort_flag, p.status, p.wait_limit_ns};
+  SAF_SPAN(fwd64, 0);
 #ifdef SAF_TRACE
   int tr_n = 0;
 #endif
@@ -665,6 +668,7 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   }
   tc_fence_before();
   __syncthreads();
+  SAF_SPAN(fwd64, 1);
   if (warp == 9) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 

@@ -183,3 +183,21 @@ cudaError_t launch_calib_finalize(float* mean, const double* sumsq, const double
                                   double n_total, double* s_var, double* s_kl, int num_sms, cudaStream_t st);
 
 }  // namespace saf
+
+// Trace builds only: per-CTA first/last time stamps (globaltimer, ns) of a kernel, read back by
+// saf_debug_read_span_<name>; regular builds compile these to nothing.
+#ifdef SAF_TRACE
+#define SAF_SPAN_DEFINE(name)                                                                   \
+  __device__ unsigned long long g_saf_span_##name[1024][2];                                     \
+  extern "C" int saf_debug_read_span_##name(unsigned long long* out) {                          \
+    return static_cast<int>(cudaMemcpyFromSymbol(out, g_saf_span_##name, sizeof(g_saf_span_##name))); \
+  }
+#define SAF_SPAN(name, k)                                                                       \
+  do {                                                                                          \
+    if (threadIdx.x == 0) g_saf_span_##name[blockIdx.x & 1023][k] = saf::globaltimer_ns();      \
+  } while (0)
+#else
+#define SAF_SPAN_DEFINE(name)
+#define SAF_SPAN(name, k)
+#endif
+
