@@ -600,7 +600,11 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   fp.wait_limit_ns = ctx->wait_limit_ns;
   ScopedTimer timer(ctx, SAF_KERNEL_FWD, st);
   // head dimension 96 runs on the 128-wide kernel: TMA zero-fills features 96..127 of every operand tile
-  if (launch_fwd(p->D == 96 ? 128 : p->D, mq, mk, mv, mvt, fp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
+  // O leaves the D = 64 kernel as whole tiles by TMA stores (rows beyond T are clipped by the map)
+  CUtensorMap mo;
+  rc = make_map(ctx, &mo, O, p, p->o_strides);
+  if (rc) return rc;
+  if (launch_fwd(p->D == 96 ? 128 : p->D, mq, mk, mv, mvt, mo, fp, grid, st) != cudaSuccess) return SAF_ERR_CUDA;
   return SAF_OK;
 }
 

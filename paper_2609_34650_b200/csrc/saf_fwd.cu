@@ -592,10 +592,10 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
 int fwd_smem_bytes(int D) { return D == 64 ? fwd64_smem_bytes() : FwdCfg<128>::SMEM; }
 
 cudaError_t launch_fwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const CUtensorMap& mvt, const FwdParams& p, int grid, cudaStream_t st) {
+                       const CUtensorMap& mvt, const CUtensorMap& mo, const FwdParams& p, int grid, cudaStream_t st) {
   cudaError_t e;
   if (D == 64) {
-    return launch_fwd64(mq, mk, mv, mvt, p, grid, st);   // head dimension 64 has its own kernel
+    return launch_fwd64(mq, mk, mv, mvt, mo, p, grid, st);   // head dimension 64 has its own kernel
   } else {
     e = cudaFuncSetAttribute(saf_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128>::SMEM);
     if (e != cudaSuccess) return e;

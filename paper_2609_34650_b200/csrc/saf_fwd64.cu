@@ -61,7 +61,8 @@ struct Fwd64Cfg {
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = TILE_BYTES;
   static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
-  static constexpr int OFF_TAB = OFF_V + NS * TILE_BYTES;
+  static constexpr int OFF_OST = OFF_V + NS * TILE_BYTES;   // O tile staged for its TMA store (128-byte swizzle)
+  static constexpr int OFF_TAB = OFF_OST + TILE_BYTES;
   // floats: aJ[128] rband[256] a2raw[128] r2raw[256] red[32] ml[2][2][128]
   static constexpr int TAB_FLOATS = 128 + 256 + 128 + 256 + 32 + 512;
   static constexpr int OFF_BAR = OFF_TAB + TAB_FLOATS * 4;
@@ -97,7 +98,8 @@ __device__ __forceinline__ ItemView64 load_item64(const FwdParams& p, int it, in
 
 __global__ void __launch_bounds__(320, 2)
 saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
-                 const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mvt, const FwdParams p) {
+                 const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mvt,
+                 const __grid_constant__ CUtensorMap mo, const FwdParams p) {
   using C = Fwd64Cfg;
   constexpr int D = 64;
   extern __shared__ uint8_t smem_raw[];
@@ -426,6 +428,7 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       float f0 = 1.0f, f1 = 1.0f, inv_l = 1.0f, lse = 0.0f;
       bool use1 = true;
       if (named_bar_or(5, 256, !ok)) break;
+      if (q4 == 0) TRF(trr, 19);
       if (fast) {
         // tensor-core form: nothing to do per tile; lane m holds query 127-m, scaled by w(i) below
         row = w.blk * BLK + 127 - rowl;
@@ -621,9 +624,15 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         ++npv;
       }
       tc_fence_after();
-      __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + w.b * p.o_strides[0] + w.h * p.o_strides[1] +
-                            static_cast<int64_t>(row) * p.o_strides[2] + 32 * g;
+      if (q4 == 0) TRF(trr, 17);
+      // The O tile goes through a swizzled staging tile and leaves by one TMA store: a row per thread written
+      // straight to global memory touches 32 lines per store instruction and kept the load/store unit busy for
+      // ~1800 clk per item.  The staging tile is free once the previous item's store has read it.
+      if (tid == 0) bulk_wait_group_read0();
+      named_bar_sync(7, 256);
       {
+        const int rl = row - w.blk * BLK;                 // row within the tile (reversed in the tensor-core form)
+        const uint32_t strow = smem_u32(smem + C::OFF_OST) + static_cast<uint32_t>(rl) * 128;
         const float s0 = f0 * inv_l, s1 = f1 * inv_l;
 #pragma unroll
         for (int hc = 0; hc < 2; ++hc) {
@@ -635,31 +644,34 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             tc_fence_before();
             warp_arrive(o_free);                          // the accumulators may be overwritten
           }
-          if (row < p.T && ok) {
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              float v[8];
+          for (int q = 0; q < 2; ++q) {
+            float v[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                v[e] = __uint_as_float(ra[8 * q + e]) * s0;
-                if (use1) v[e] = fmaf(__uint_as_float(rb2[8 * q + e]), s1, v[e]);
-              }
-              uint4 o;
-              o.x = pack_bf16x2(v[0], v[1]);
-              o.y = pack_bf16x2(v[2], v[3]);
-              o.z = pack_bf16x2(v[4], v[5]);
-              o.w = pack_bf16x2(v[6], v[7]);
-              *reinterpret_cast<uint4*>(orow + 16 * hc + 8 * q) = o;
+            for (int e = 0; e < 8; ++e) {
+              v[e] = __uint_as_float(ra[8 * q + e]) * s0;
+              if (use1) v[e] = fmaf(__uint_as_float(rb2[8 * q + e]), s1, v[e]);
             }
+            const uint32_t chunk = static_cast<uint32_t>((4 * g + 2 * hc + q) ^ (rl & 7));
+            st_shared_v4w(strow + chunk * 16, pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+                          pack_bf16x2(v[6], v[7]));
           }
         }
       }
+      fence_proxy_async_smem();
+      const bool all_ok = !named_bar_or(8, 256, !ok);
+      if (tid == 0 && all_ok) {
+        tma_store_4d(&mo, smem + C::OFF_OST, 0, w.blk * BLK, w.h, w.b);
+        bulk_commit_group();
+      }
       if (p.LSE != nullptr && g == 0 && row < p.T && ok)
         p.LSE[(static_cast<size_t>(w.b) * p.H + w.h) * p.T + row] = lse;
+      if (q4 == 0) TRF(trr, 18);
     }
   }
 
   // ------------------------------------------------------------------ teardown
+  if (tid == 0) bulk_wait_group0();               // the last O tile has left the staging tile
   __syncwarp();
   if (*abort_flag) {
     // A wait gave up: let copies and MMAs that are still in flight land before the CTA's
@@ -675,11 +687,11 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 int fwd64_smem_bytes() { return Fwd64Cfg::SMEM; }
 
 cudaError_t launch_fwd64(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mvt,
-                         const FwdParams& p, int grid, cudaStream_t st) {
+                         const CUtensorMap& mo, const FwdParams& p, int grid, cudaStream_t st) {
   cudaError_t e =
       cudaFuncSetAttribute(saf_fwd64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Fwd64Cfg::SMEM);
   if (e != cudaSuccess) return e;
-  saf_fwd64_kernel<<<grid, Fwd64Cfg::NTHREADS, Fwd64Cfg::SMEM, st>>>(mq, mk, mv, mvt, p);
+  saf_fwd64_kernel<<<grid, Fwd64Cfg::NTHREADS, Fwd64Cfg::SMEM, st>>>(mq, mk, mv, mvt, mo, p);
   return cudaGetLastError();
 }
 

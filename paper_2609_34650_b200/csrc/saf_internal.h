@@ -109,7 +109,7 @@ constexpr float HK_BAND_SCALE = 16384.0f;        // bands hold 2^14 r
 constexpr float HK_A_SCALE = 2048.0f;            // the forward stages 2^11 a V
 // mvt: map of the a-scaled V of the frozen heads [B][Hf][T][D] (any valid map when band_f is NULL)
 cudaError_t launch_fwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const CUtensorMap& mvt, const FwdParams& p, int grid, cudaStream_t st);
+                       const CUtensorMap& mvt, const CUtensorMap& mo, const FwdParams& p, int grid, cudaStream_t st);
 // mdot: map of the w-scaled dO of the frozen heads [B][Hf][T][D] (any valid map when band_b is NULL);
 // mdk / mdv: fp32 maps of dK / dV shaped like mdq (only used when grad_f32 is set)
 cudaError_t launch_bwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
@@ -134,7 +134,7 @@ cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, con
 cudaError_t launch_bwd_finalize(const float* dQacc, void* dQ, size_t n, cudaStream_t st);
 // head dimension 64 (saf_fwd64.cu); launch_fwd dispatches to it
 cudaError_t launch_fwd64(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mvt,
-                         const FwdParams& p, int grid, cudaStream_t st);
+                         const CUtensorMap& mo, const FwdParams& p, int grid, cudaStream_t st);
 int fwd64_smem_bytes();
 // head dimension 128 / 96 (saf_bwd128.cu): mqh / mdoh / mdoth are maps with 64-row boxes (half tiles), mdq the fp32 dQ
 // accumulator [B][Hq][T][D]; dK / dV are written with plain stores (reduce-adds for shared heads)
