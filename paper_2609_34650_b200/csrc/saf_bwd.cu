@@ -648,8 +648,8 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     ItemView nxt = load_item(p, it_begin, it_end);
     for (int it = it_begin; it < it_end; ++it) {
       const WorkItem w = nxt.w;
-      const bool fast = nxt.fast;
-      nxt = load_item(p, it + 1, it_end);
+      const bool fast = nxt.fast;                        // (the next item is fetched below, under the wait for the
+                                                         // item's last MMAs, where its load latency costs nothing)
       const bool ord = w.kind == KIND_ORDINARY;
       const int ntiles = nblk - w.blk;
       int key = w.blk * BLK + rowl;
@@ -834,6 +834,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         }
       }
       // ---------------- epilogue: dV (group 0) and dK (group 1) of this key block
+      nxt = load_item(p, it + 1, it_end);
       if (!mbar_wait_warp(acc_full, nacc & 1, wc, B_ACC_FULL)) ok = false;
       ++nacc;
       tc_fence_after();

@@ -438,8 +438,7 @@ saf_bwd128_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant_
     ItemW nxt = load_item_w(p, it_begin, it_end);
     for (int it = it_begin; it < it_end; ++it) {
       const WorkItem w = nxt.w;
-      const bool fast = nxt.fast;
-      nxt = load_item_w(p, it + 1, it_end);
+      const bool fast = nxt.fast;                        // (the next item is fetched under the epilogue's wait)
       const bool ord = w.kind == KIND_ORDINARY;
       const int U = 2 * (nblk - w.blk);
       int key = w.blk * BLK + rowl;
@@ -550,6 +549,7 @@ saf_bwd128_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant_
         ++npf;
       }
       // ---------------- epilogue: this warp's 32 feature columns of dV and (ordinary items) dK
+      nxt = load_item_w(p, it + 1, it_end);              // its load latency passes under the wait for the last MMAs
       if (!mbar_wait_warp(acc_full, nacc & 1, wc, W_ACC_FULL)) ok = false;
       ++nacc;
       tc_fence_after();

@@ -242,9 +242,11 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     for (int it = it_begin; it < it_end && ok; ++it, ++nitem) {
       const WorkItem w = nxt.w;
       const bool fast = nxt.fast;
-      nxt = load_item64(p, it + 1, it_end);
       const int ntiles = w.blk + 1;
       const bool ord = w.kind == KIND_ORDINARY;
+      // The next record's load latency must not delay the item's first score MMAs: ordinary items fetch it once
+      // those are queued.
+      if (!ord) nxt = load_item64(p, it + 1, it_end);
       if (fast) {
         for (int j = 0; j < ntiles && ok; ++j) {
           const uint32_t sk = nk % C::NS, sv = nv % C::NS;
@@ -313,6 +315,7 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           if (leader) umma_commit(k_empty + s);
           __syncwarp();
         }
+        nxt = load_item64(p, it + 1, it_end);
         for (int j = 0; j < ntiles && ok; ++j) {
           const uint32_t sv = nv % C::NS;
           const bool more = j + 1 < ntiles;
@@ -420,8 +423,7 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     ItemView64 nxt = load_item64(p, it_begin, it_end);
     for (int it = it_begin; it < it_end; ++it) {
       const WorkItem w = nxt.w;
-      const bool fast = nxt.fast;
-      nxt = load_item64(p, it + 1, it_end);
+      const bool fast = nxt.fast;                        // (the next item is fetched under the epilogue's wait)
       const int ntiles = w.blk + 1;
       int row = w.blk * BLK + rowl;
       // epilogue weights of the two accumulators and the common row factor
@@ -617,6 +619,7 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (leave) break;
       }
       // ---------------- epilogue: wait for the last P V of both groups, merge, scale, store 32 columns each
+      nxt = load_item64(p, it + 1, it_end);              // its load latency passes under the wait for the last MMAs
       {
         const uint32_t par = npv & 1;
         if (!mbar_wait_warp(pv_done, par, wc, F_PV_DONE)) ok = false;
