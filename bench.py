@@ -431,15 +431,19 @@ def run_ours(args):
     value = rate / 1e12
 
     # ---- speedup vs the same library with zero frozen heads: interleaved A B B A, plus an A/A control
-    reps = max(3, args.steps // 4)
-    a1 = timed(mask, reps)
-    b1 = timed(mask0, reps)
-    b2 = timed(mask0, reps)
-    a2 = timed(mask, reps)
-    c1 = timed(mask, reps)
-    c2 = timed(mask, reps)
-    speedup = (b1 + b2) / (a1 + a2)
-    aa_control = c1 / c2
+    # (a comparison whose A/A control is off by more than 2 % is discarded and taken again, at most three times)
+    reps = max(5, args.steps)
+    for aa_attempt in range(1, 4):
+        a1 = timed(mask, reps)
+        b1 = timed(mask0, reps)
+        b2 = timed(mask0, reps)
+        a2 = timed(mask, reps)
+        c1 = timed(mask, reps)
+        c2 = timed(mask, reps)
+        speedup = (b1 + b2) / (a1 + a2)
+        aa_control = c1 / c2
+        if world > 1 or abs(aa_control - 1.0) <= 0.02:     # (ranks must take the same number of timed runs)
+            break
     # the sampler ran through the K timed steps and the interleaved repeats of the same step
     clocks = sampler.stop() if rank == 0 else None
     fwd_only = None
@@ -547,7 +551,7 @@ def run_ours(args):
                    "pattern_prepare": "once before the timed steps (static per layer)", "pattern_prepare_ms": prepare_ms,
                    "parallelism": f"dp{world} (independent batches, no collective in the layer)"},
         "pct_of_bf16_peak": 100.0 * value / (peaks["bf16_tflops"] * world),
-        "speedup_vs_0pct_frozen": speedup, "aa_control": aa_control,
+        "speedup_vs_0pct_frozen": speedup, "aa_control": aa_control, "aa_attempts": aa_attempt,
         "ms_0pct_frozen": 0.5 * (b1 + b2), "ms_fwd_only": fwd_only, "ms_pattern_grad": pgrad_ms,
         "ms_per_step_cuda_graph": graph_ms,
         "e2e": {"value": e2e_rate / 1e12, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
