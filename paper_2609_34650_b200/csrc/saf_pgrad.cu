@@ -230,7 +230,7 @@ saf_pgrad_kernel(const __grid_constant__ CUtensorMap mv, const __grid_constant__
               const float pij = ex2_approx(a2 + rb[e] - zz[k]);
               const float db = pij * (__uint_as_float(r[e]) - dd[k]);
               dacc += db;
-              const float got = __shfl_sync(0xffffffffu, db, (lane + e) & 31);
+              const float got = __shfl_sync(0xffffffffu, db, lane + e);      // (the source lane is taken modulo 32)
               if (lane + e < 32) dg[cc][0] += got;
               else dg[cc][1] += got;
             }
