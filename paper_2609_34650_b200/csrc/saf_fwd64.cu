@@ -429,6 +429,7 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       // epilogue weights of the two accumulators and the common row factor
       float f0 = 1.0f, f1 = 1.0f, inv_l = 1.0f, lse = 0.0f;
       bool use1 = true;
+      if (tid == 0) bulk_wait_group_read0();             // the previous item's O tile has left the staging tile
       if (named_bar_or(5, 256, !ok)) break;
       if (q4 == 0) TRF(trr, 19);
       if (fast) {
@@ -630,9 +631,8 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       if (q4 == 0) TRF(trr, 17);
       // The O tile goes through a swizzled staging tile and leaves by one TMA store: a row per thread written
       // straight to global memory touches 32 lines per store instruction and kept the load/store unit busy for
-      // ~1800 clk per item.  The staging tile is free once the previous item's store has read it.
-      if (tid == 0) bulk_wait_group_read0();
-      named_bar_sync(7, 256);
+      // ~1800 clk per item.  The staging tile is free once the previous item's store has read it, which the
+      // agreement barrier at the top of the item has made known to all compute warps.
       {
         const int rl = row - w.blk * BLK;                 // row within the tile (reversed in the tensor-core form)
         const uint32_t strow = smem_u32(smem + C::OFF_OST) + static_cast<uint32_t>(rl) * 128;
