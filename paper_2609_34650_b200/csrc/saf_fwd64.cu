@@ -66,7 +66,13 @@ struct Fwd64Cfg {
   // floats: aJ[128] rband[256] a2raw[128] r2raw[256] red[32] ml[2][2][128]
   static constexpr int TAB_FLOATS = 128 + 256 + 128 + 256 + 32 + 512;
   static constexpr int OFF_BAR = OFF_TAB + TAB_FLOATS * 4;
-  static constexpr int NBAR = 2 + 4 * NS + 2 + 2 + 2 + 1;
+  // Ring of the tensor-core frozen form, three deep (its tiles have no compute step to hide the load latency
+  // behind): slot k keeps its scaled V tile in V stage k (k < 2) or in the Q tile (k = 2) and its 4 KB band in the
+  // K ring's area.
+  static constexpr int NFZ = 3;
+  __host__ __device__ static constexpr int fz_v(int k) { return k < 2 ? OFF_V + k * TILE_BYTES : OFF_Q; }
+  __host__ __device__ static constexpr int fz_band(int k) { return OFF_K + k * 4096; }
+  static constexpr int NBAR = 2 + 4 * NS + 2 + 2 + 2 + 1 + 2 * NFZ;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;   // + slack for 1024-byte alignment
   static constexpr int TMEM_COLS = 256;
   static constexpr int COL_S = 0, COL_O = 128;          // + 64 g
@@ -115,7 +121,9 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   uint64_t* p_full = s_full + 2;                 // [2] group g has written its P pairs (4 warp arrivals)
   uint64_t* pv_done = p_full + 2;                // [2] P V MMAs of group g have completed (see the issuer)
   uint64_t* o_free = pv_done + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_free + 1);
+  uint64_t* fz_full = o_free + 1;                // [NFZ] band + scaled V tile of a tensor-core frozen tile
+  uint64_t* fz_empty = fz_full + C::NFZ;         // [NFZ]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fz_empty + C::NFZ);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* tab = reinterpret_cast<float*>(smem + C::OFF_TAB);
 
@@ -142,6 +150,10 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       mbar_init(pv_done + g, 1);
     }
     mbar_init(o_free, 8);
+    for (int k = 0; k < C::NFZ; ++k) {
+      mbar_init(fz_full + k, 1);
+      mbar_init(fz_empty + k, 1);
+    }
     mbar_fence_init();
   }
   if (warp == 9) {
@@ -162,8 +174,8 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       tma_prefetch_desc(&mk);
       tma_prefetch_desc(&mv);
       tma_prefetch_desc(&mvt);
-      uint32_t nq = 0, nk = 0, nv = 0;
-      bool ok = true;
+      uint32_t nq = 0, nk = 0, nv = 0, nfz = 0;
+      bool ok = true, fz_open = false;
       ItemView64 nxt = load_item64(p, it_begin, it_end);
       for (int it = it_begin; it < it_end && ok; ++it) {
         const WorkItem w = nxt.w;
@@ -171,25 +183,37 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         nxt = load_item64(p, it + 1, it_end);
         const int ntiles = w.blk + 1;
         if (fast) {
-          // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled V tile
+          // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled V tile, in a ring of
+          // their own laid over the K and V stages and the Q tile
+          if (!fz_open) {
+            // the last tiles that went through those stages must have been consumed
+            for (uint32_t n = nk > C::NS ? nk - C::NS : 0; n < nk && ok; ++n)
+              ok = mbar_wait(k_empty + n % C::NS, (n / C::NS) & 1, wc, F_K_EMPTY);
+            for (uint32_t n = nv > C::NS ? nv - C::NS : 0; n < nv && ok; ++n)
+              ok = mbar_wait(v_empty + n % C::NS, (n / C::NS) & 1, wc, F_V_EMPTY);
+            if (ok && nq > 0) ok = mbar_wait(q_empty, (nq - 1) & 1, wc, F_Q_EMPTY);
+            if (!ok) break;
+            fz_open = true;
+          }
           const int ord = p.hord[w.h];
           const uint8_t* bands = static_cast<const uint8_t*>(p.band_f) + static_cast<size_t>(w.h) * p.nblkp * 4096;
           for (int j = 0; j < ntiles; ++j) {
-            const int sk = nk % C::NS;
-            ok = mbar_wait(k_empty + sk, ((nk / C::NS) & 1) ^ 1, wc, F_K_EMPTY);
+            const uint32_t k = nfz % C::NFZ;
+            ok = mbar_wait(fz_empty + k, ((nfz / C::NFZ) & 1) ^ 1, wc, F_V_EMPTY);
             if (!ok) break;
-            mbar_expect_tx(k_full + sk, 4096);
-            bulk_load(smem + C::OFF_K + sk * C::TILE_BYTES, bands + static_cast<size_t>(w.blk - j) * 4096, 4096,
-                      k_full + sk);
-            ++nk;
-            const int sv = nv % C::NS;
-            ok = mbar_wait(v_empty + sv, ((nv / C::NS) & 1) ^ 1, wc, F_V_EMPTY);
-            if (!ok) break;
-            mbar_expect_tx(v_full + sv, C::TILE_BYTES);
-            tma_load_4d(smem + C::OFF_V + sv * C::TILE_BYTES, &mvt, v_full + sv, 0, j * BLK, ord, w.b);
-            ++nv;
+            mbar_expect_tx(fz_full + k, C::TILE_BYTES + 4096);
+            bulk_load(smem + C::fz_band(k), bands + static_cast<size_t>(w.blk - j) * 4096, 4096, fz_full + k);
+            tma_load_4d(smem + C::fz_v(k), &mvt, fz_full + k, 0, j * BLK, ord, w.b);
+            ++nfz;
           }
           continue;
+        }
+        if (fz_open) {
+          // back to the ordinary stages: the frozen ring's tiles in flight must have been consumed
+          for (uint32_t n = nfz > C::NFZ ? nfz - C::NFZ : 0; n < nfz && ok; ++n)
+            ok = mbar_wait(fz_empty + n % C::NFZ, (n / C::NFZ) & 1, wc, F_V_EMPTY);
+          if (!ok) break;
+          fz_open = false;
         }
         const bool ord = w.kind == KIND_ORDINARY;
         const int kh = !ord ? 0 : (p.qslot ? p.qslot[w.h] : w.h / p.kv_group);   // head index in the K tensor
@@ -226,7 +250,7 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     constexpr uint32_t idesc_s = umma_idesc_bf16(128, 64, 0, 0);   // S_g: 128 queries x 64 keys, both K-major
     constexpr uint32_t idesc_o = umma_idesc_bf16(128, D, 0, 1);    // O_g: A = P_g from TMEM, B = V rows MN-major
     constexpr uint32_t idesc_hk = umma_idesc_f16(128, D, 0, 1);    // tensor-core frozen form: fp16 band x fp16 scaled V
-    uint32_t nq = 0, nk = 0, nv = 0, nitem = 0;
+    uint32_t nq = 0, nk = 0, nv = 0, nitem = 0, nfz = 0;
     uint32_t np0 = 0, np1 = 0;
     bool ok = true;
     // descriptor halves for smem offset 0: K-major tiles (k-step +32 B) and the MN-major V tile (k-step
@@ -249,27 +273,23 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       if (!ord) nxt = load_item64(p, it + 1, it_end);
       if (fast) {
         for (int j = 0; j < ntiles && ok; ++j) {
-          const uint32_t sk = nk % C::NS, sv = nv % C::NS;
-          ok = mbar_wait_warp(k_full + sk, (nk / C::NS) & 1, wc, F_K_FULL);
+          const uint32_t k = nfz % C::NFZ;
+          ok = mbar_wait_warp(fz_full + k, (nfz / C::NFZ) & 1, wc, F_V_FULL);
           if (!ok) break;
-          ++nk;
-          ok = mbar_wait_warp(v_full + sv, (nv / C::NS) & 1, wc, F_V_FULL);
-          if (!ok) break;
-          ++nv;
+          ++nfz;
           if (j == 0) {
             ok = mbar_wait_warp(o_free, (nitem & 1) ^ 1, wc, F_O_FREE);
             if (!ok) break;
           }
           tc_fence_after();
-          const uint32_t band_lo = lo_b + ((C::OFF_K + sk * C::TILE_BYTES) >> 4);
-          const uint32_t v_lo = lo_m + ((C::OFF_V + sv * C::TILE_BYTES) >> 4);
+          const uint32_t band_lo = lo_b + (static_cast<uint32_t>(C::fz_band(k)) >> 4);
+          const uint32_t v_lo = lo_m + (static_cast<uint32_t>(C::fz_v(k)) >> 4);
           const uint32_t acc0 = j > 0 ? 1u : 0u;
           if (leader) {
 #pragma unroll
             for (int kc = 0; kc < 8; ++kc)
               umma_ss2(tmem + C::COL_O, band_lo + 16 * kc, hi_b, v_lo + 128 * kc, hi_m, idesc_hk, kc > 0 ? 1u : acc0);
-            umma_commit(k_empty + sk);
-            umma_commit(v_empty + sv);
+            umma_commit(fz_empty + k);
             if (j == ntiles - 1) {
               umma_commit(pv_done);
               umma_commit(pv_done + 1);
