@@ -247,7 +247,7 @@ int saf_get_kernel_time(saf_ctx* ctx, int32_t which, float* total_ms_out, int32_
  * head dimension 64, 50 / 20 % at 96 and 128; item 150 / 100 % and 300 / 200 %), which the
  * environment variables SAF_FROZEN_WEIGHT_PCT, SAF_FROZEN_WEIGHT_BWD_PCT, SAF_ITEM_OVERHEAD_PCT and
  * SAF_ITEM_OVERHEAD_BWD_PCT (read by saf_create) override.  In a forward grid (two CTAs per SM) the
- * layer calls also charge the second half of the grid 15 % (head dimension 64) or 6 % more for the
+ * layer calls also charge the second half of the grid 20 % (head dimension 64) or 6 % more for the
  * same work, since the CTA that arrives second on an SM runs slower (SAF_SECOND_WAVE_PCT).
  *   items_out   : host int32[n_items*4] = (b, h, block, kind) with kind 0 ordinary / 1 frozen,
  *                 grouped by CTA; n_items = B*H*ceil(T/128)

@@ -65,7 +65,7 @@ struct saf_ctx {
   int item_overhead_pct = 0;
   int item_overhead_bwd_pct = 0;
   // Forward grid = two CTAs per SM: the CTA that arrives second on an SM (block index >= grid / 2) runs slower
-  // than the first (measured 13 % at head dimension 64, 2 % on the 128-wide kernel; best settings 15 and 6) and gets that much less
+  // than the first (measured 13 % at head dimension 64, 2 % on the 128-wide kernel; best settings 20 and 6) and gets that much less
   // work.  -1 = the measured default; SAF_SECOND_WAVE_PCT overrides.
   int second_wave_pct = -1;
   int call_counter = 0;                    // ids of the calls that stage fp16 operands (overflow marks)
@@ -269,7 +269,7 @@ int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int bac
   const int ov = backward ? ctx->item_overhead_bwd_pct : ctx->item_overhead_pct;
   if (fw > 0) frozen_pct = fw;
   if (ov > 0) overhead_pct = ov;
-  const int second_wave = backward ? 0 : (ctx->second_wave_pct >= 0 ? ctx->second_wave_pct : (wide ? 6 : 15));
+  const int second_wave = backward ? 0 : (ctx->second_wave_pct >= 0 ? ctx->second_wave_pct : (wide ? 6 : 20));
   build_worklist_host(B, H, T, mask, backward, grid, frozen_pct, overhead_pct, second_wave, items, offsets);
   WorklistEntry e;
   e.B = B; e.H = H; e.T = T; e.backward = backward; e.grid = grid; e.wide = wide;
