@@ -134,6 +134,23 @@ def test_multi_tile_scheduler_mix():
     check_units(L, [(0, 0), (7, 5), (3, 3), (5, 1), (2, 4), (6, 2)])
 
 
+def test_item_kinds_alternate_within_a_cta():
+    """Ordinary items, frozen items in the tensor-core form and frozen items in the general form (a head whose pattern
+    leaves the factorised form's range) follow one another in the CTAs' work lists: 8 x 8 heads x 10 blocks = 640
+    forward items on 296 CTAs.  The tensor-core frozen tiles run a shared-memory ring of their own that is laid over
+    the other kinds' stages, so every change of kind is a hand-over between the rings."""
+    T = 1200
+    wl = si.Workload("kinds", 8, 8, T, 64, (0, 2, 3, 5, 6), -0.05, seed=23)
+    inp = si.generate(wl)
+    for h in (2, 5):                                     # far outside the range of the tensor-core form
+        inp.alpha[h] = (inp.alpha[h] + 25.0 * np.sin(0.37 * np.arange(T))).astype(np.float32)
+    # such patterns put a row's mass on a few keys, whose dV then sums hundreds of output gradients; dO / 16 (exact
+    # in bf16) keeps the gradients in the value range the absolute tolerance is meant for
+    inp.do[...] = si.f32_to_bf16_bits(si.bf16_bits_to_f32(inp.do) / 16.0)
+    L = Layer(inp).run()
+    check_units(L, [(0, 0), (0, 2), (1, 1), (2, 5), (3, 3), (4, 4), (5, 6), (6, 7), (7, 2), (7, 0)])
+
+
 # --------------------------------------------------------------------------- invariants on the GPU
 def test_frozen_heads_never_read_q_k_and_get_zero_grads():
     wl = si.Workload("poison", 2, 4, 300, 64, (0, 2), -0.05, seed=8)
