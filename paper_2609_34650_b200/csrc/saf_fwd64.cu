@@ -26,7 +26,10 @@
 //   O = diag(w) R (diag(a) V), R(i,j) = r(i-j).  A tile of R with reversed rows is a Hankel matrix that the
 //   tensor core reads straight from a 4 KB band table (no-swizzle descriptor, both strides 128 bytes), so
 //   a tile is one bulk copy of the band, one TMA load of the a-scaled V tile and 8 MMAs into O_0; the compute
-//   warps only scale the finished rows by w(i) (TMEM lane m holds query 127-m of the block).
+//   warps only scale the finished rows by w(i) (TMEM lane m holds query 127-m of the block).  These tiles run
+//   a ring of their own, three deep, laid over the K and V stages and the Q tile.
+// Epilogue of every item: the merged, scaled O tile is written into a swizzled staging tile and leaves by one
+//   TMA store (rows beyond T are clipped by the tensor map).
 #include <cuda_bf16.h>
 #include "ptx.cuh"
 #include "saf_internal.h"
