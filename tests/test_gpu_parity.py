@@ -325,6 +325,31 @@ def test_host_buffer_step_in_chunks_matches_device_path(g, gd):
             assert ma < (1e-4 if gd == saf.SAF_F32 else 2e-2) and np.isfinite(got.float().numpy()).all()
 
 
+@pytest.mark.parametrize("D,g", [(128, 1), (96, 2)])
+def test_host_buffer_step_wide_heads_in_chunks(D, g):
+    """The host-buffer step on the 128-wide kernels (head dimension 128, and 96 with shared key/value heads), cut
+    into chunks of whole batch entries, against the device path on the same inputs."""
+    inp = si.generate(si.Workload("host-wide", 9, 4, 1024, D, (1, 3), -0.05, seed=33, kv_group=g))
+    Dv = Layer(inp).run()
+    wl = inp.wl
+    ctx = saf.Context(0)
+    pin = lambda t: t.pin_memory()
+    Q, K, V, dO = (pin(bf16_tensor(x)) for x in (inp.q, inp.k, inp.v, inp.do))
+    alpha, rho = pin(torch.from_numpy(inp.alpha)), pin(torch.from_numpy(inp.rho))
+    O = pin(torch.empty_like(Q))
+    LSE = pin(torch.empty(wl.B, wl.H, wl.T))
+    dQ, dK, dV = (pin(torch.full(t.shape, float("nan"), dtype=torch.float32)) for t in (Q, K, V))
+    prob = saf.make_problem(Q, wl.stored_len, k_like=K, v_like=V, o_like=O, kv_group=g, H=wl.H)
+    ctx.saf_hybrid_attn_step_host(prob, Q, K, V, dO, inp.mask, alpha, rho, 1, O, LSE, dQ, dK, dV)
+    assert torch.equal(O, Dv.O.cpu()) and torch.equal(LSE, Dv.LSE.cpu())
+    for got, want, exact in ((dQ, Dv.grads[0], False), (dK, Dv.grads[1], g == 1), (dV, Dv.grads[2], g == 1)):
+        if exact:
+            assert torch.equal(got, want.cpu())
+        else:                                  # accumulated with reduce-adds: order only
+            ma, rl = errors(got.numpy().astype(np.float64), Dv.host(want))
+            assert ma < 1e-4 and np.isfinite(got.numpy()).all()
+
+
 def test_forward_backward_capture_into_a_cuda_graph():
     """After a warm-up call (which allocates the context's workspaces and uploads the work lists) a forward +
     backward step records into a CUDA graph, and replays reproduce the eager results bit for bit (dQ to rounding:
