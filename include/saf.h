@@ -15,7 +15,8 @@
  *     The library never frees or reallocates caller memory.
  *   - Q, K, V, O, dO are bf16 tensors indexed [b][h][t][c] through element strides (c has stride 1);
  *     base addresses and strides must be multiples of 8 elements (16 bytes).
- *   - frozen_mask_host is a host array uint8[H]; nonzero = frozen head.  It is read during the call.
+ *   - frozen_mask_host is a host array uint8[H]; nonzero = frozen head.  It is read (copied) before the call
+ *     returns, whatever kind of host memory it lives in.
  *   - alpha, rho, logZ are fp32 [H][Tp] row-major device arrays; rows of ordinary heads are ignored.
  *     They may be NULL when no head is frozen.  Q/K/LSE rows of frozen heads are never read.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream).
@@ -77,7 +78,14 @@ int saf_destroy(saf_ctx* ctx);
  * (alpha, rho, log Z) per replaced head):
  *   logZ_dev_out[h][i] = log sum_{k<=i} exp(alpha[h][k] + rho[h][i-k]),  i in [0,Tp), frozen h only.
  * Row i uses alpha[0..i] and rho[0..i] only, so the result serves every T <= Tp.  alpha_dev, rho_dev,
- * logZ_dev_out: device fp32 [H][Tp].  Call again whenever alpha or rho change. */
+ * logZ_dev_out: device fp32 [H][Tp].  Call again whenever alpha or rho change.
+ * frozen_mask_host (here and in every other entry point) is read before the call returns; the caller may change
+ * or free it afterwards.
+ * The call also builds the context's tables for the tensor-core form of the frozen heads and remembers the three
+ * device pointers and their contents.  A later layer call uses the tables only for heads whose alpha, rho and logZ
+ * still hold exactly those bits; a head whose vectors were rewritten in place since (by the caller, by
+ * saf_fit_compact, by saf_pattern_logz_static) is computed from the vectors it is given, in the slower general form,
+ * until saf_pattern_prepare is called again. */
 int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* frozen_mask_host,
                         const float* alpha_dev, const float* rho_dev, float* logZ_dev_out, void* stream);
 
@@ -93,7 +101,9 @@ int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* froz
  *   - No context.  `device` is the CUDA device to run on.  Other arguments as saf_pattern_prepare.
  *   - H must not exceed SAF_STATIC_MAX_HEADS; a larger H returns SAF_ERR_INVALID_ARG and launches nothing.
  *   - The call makes no cudaMalloc / cudaFree and uses no allocating library routine.  It only computes
- *     logZ; the tensor-core pattern tables of saf_pattern_prepare are not built.
+ *     logZ; the tensor-core pattern tables of saf_pattern_prepare are not built, and tables a context built
+ *     earlier from the same buffers are not refreshed: layer calls on that context notice the changed contents
+ *     and take the general form for those heads until saf_pattern_prepare runs again.
  *   - The first call on a device resolves the array's device address (one cudaGetSymbolAddress, cached per
  *     device).  Make that first call during set-up, before any stream capture is begun.
  *   - The array (SAF_STATIC_MAX_HEADS bytes per GPU, held until the process exits) is shared by every

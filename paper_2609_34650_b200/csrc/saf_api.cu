@@ -23,6 +23,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct WorklistEntry {
   int B, H, T, backward, grid, wide;
   std::vector<uint8_t> mask;
+  std::vector<WorkItem> items_host;       // kept alive: the upload is asynchronous on the caller's stream
+  std::vector<int> offsets_host;
   WorkItem* items_dev = nullptr;
   int* offsets_dev = nullptr;
   int n_items = 0;
@@ -71,10 +73,15 @@ struct saf_ctx {
   int call_counter = 0;                    // ids of the calls that stage fp16 operands (overflow marks)
   std::vector<WorklistEntry> worklists;
   DevBuf mask_buf, logz_buf, delta_buf, dqacc_buf, dkacc_buf, dvacc_buf, qslot_buf;
+  // what mask_buf / qslot_buf currently hold (host copies) and the stream that wrote them
+  std::vector<uint8_t> mask_host, mask_staging, qslot_mask_host;
+  std::vector<int> qslot_host;
+  cudaStream_t mask_stream = nullptr, qslot_stream = nullptr;
   // tensor-core form of frozen heads: tables built by saf_pattern_prepare, scaled V / dO per call
   PatternCache pat;
   bool tensor_pattern = true;              // SAF_DISABLE_TENSOR_PATTERN=1 turns the form off
-  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, vt_buf, dot_buf, ok_fwd, ok_bwd, pg_hlist, pg_delta, fit_buf, calib_tmp;
+  bool selftest_drop_load = false;         // SAF_SELFTEST_DROP_LOAD=1: see FwdParams::selftest_drop_load
+  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, pat_snap, vt_buf, dot_buf, ok_fwd, ok_bwd, pg_hlist, pg_delta, fit_buf, calib_tmp;
   bool profiling = false;
   std::vector<TimedLaunch> timed;          // event pairs recorded since the last query
   std::vector<cudaEvent_t> event_pool;
@@ -132,6 +139,11 @@ bool pattern_matches(const saf_ctx* ctx, const saf_problem* p, const uint8_t* ma
          c.Tp == p->Tp && std::memcmp(c.mask.data(), mask, p->H) == 0;
 }
 
+PatternCheck pattern_check(const saf_ctx* ctx, const float* alpha, const float* rho, const float* logZ) {
+  return PatternCheck{alpha, rho, logZ, static_cast<const uint32_t*>(ctx->pat_snap.ptr),
+                      static_cast<size_t>(ctx->pat.H) * ctx->pat.Tp};
+}
+
 // map of a contiguous [B][Hn][T][D] fp16 workspace
 int make_map_contig(saf_ctx* ctx, CUtensorMap* out, const void* base, const saf_problem* p, int Hn,
                     int box_rows = BLK) {
@@ -164,26 +176,45 @@ int validate(const saf_problem* p, const uint8_t* mask, int* n_frozen) {
 
 inline int kv_group_of(const saf_problem* p) { return p->kv_group > 1 ? p->kv_group : 1; }
 
-// Packed Q/K layout: device table head -> slot among the ordinary heads (-1 for frozen heads).
+// Packed Q/K layout: device table head -> slot among the ordinary heads (-1 for frozen heads).  The table is
+// uploaded only when the mask differs from the one it was built from (a layer's mask is static), from a vector
+// owned by the context, so the caller's array is read before the call returns whatever memory it lives in.
 int upload_qslot(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st, const int** out) {
+  const void* before = ctx->qslot_buf.ptr;
   int rc = ensure(ctx->qslot_buf, static_cast<size_t>(std::max(H, 64)) * sizeof(int));
   if (rc) return rc;
-  std::vector<int> slot(H);
-  int n = 0;
-  for (int h = 0; h < H; ++h) slot[h] = mask[h] ? -1 : n++;
-  // pageable source: the copy is staged before the call returns
-  if (cudaMemcpyAsync(ctx->qslot_buf.ptr, slot.data(), static_cast<size_t>(H) * sizeof(int), cudaMemcpyHostToDevice,
-                      st) != cudaSuccess)
-    return SAF_ERR_CUDA;
+  if (ctx->qslot_buf.ptr != before) ctx->qslot_mask_host.clear();
   *out = static_cast<const int*>(ctx->qslot_buf.ptr);
+  if (ctx->qslot_mask_host.size() == static_cast<size_t>(H) && ctx->qslot_stream == st &&
+      std::memcmp(ctx->qslot_mask_host.data(), mask, H) == 0)
+    return SAF_OK;
+  ctx->qslot_host.resize(H);
+  int n = 0;
+  for (int h = 0; h < H; ++h) ctx->qslot_host[h] = mask[h] ? -1 : n++;
+  ctx->qslot_mask_host.clear();
+  if (cudaMemcpyAsync(ctx->qslot_buf.ptr, ctx->qslot_host.data(), static_cast<size_t>(H) * sizeof(int),
+                      cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return SAF_ERR_CUDA;
+  ctx->qslot_mask_host.assign(mask, mask + H);
+  ctx->qslot_stream = st;
   return SAF_OK;
 }
 
+// Device copy of the frozen-head mask, uploaded only when it changes (see upload_qslot).
 int upload_mask(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st) {
+  const void* before = ctx->mask_buf.ptr;
   int rc = ensure(ctx->mask_buf, std::max(H, 256));
   if (rc) return rc;
-  // pageable source: the copy is staged before the call returns, so the caller's array may change
-  if (cudaMemcpyAsync(ctx->mask_buf.ptr, mask, H, cudaMemcpyHostToDevice, st) != cudaSuccess) return SAF_ERR_CUDA;
+  if (ctx->mask_buf.ptr != before) ctx->mask_host.clear();
+  if (ctx->mask_host.size() == static_cast<size_t>(H) && ctx->mask_stream == st &&
+      std::memcmp(ctx->mask_host.data(), mask, H) == 0)
+    return SAF_OK;
+  ctx->mask_staging.assign(mask, mask + H);
+  ctx->mask_host.clear();
+  if (cudaMemcpyAsync(ctx->mask_buf.ptr, ctx->mask_staging.data(), H, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return SAF_ERR_CUDA;
+  ctx->mask_host.assign(mask, mask + H);
+  ctx->mask_stream = st;
   return SAF_OK;
 }
 
@@ -280,9 +311,14 @@ int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int bac
     cudaFree(e.items_dev);
     return SAF_ERR_NOMEM;
   }
-  // synchronous copies from pageable memory: the vectors die at the end of this scope
-  if (cudaMemcpy(e.items_dev, items.data(), items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMemcpy(e.offsets_dev, offsets.data(), offsets.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) {
+  // uploaded on the stream the kernel will run on (a non-blocking stream does not order with the legacy stream);
+  // the source vectors live as long as the entry
+  e.items_host = std::move(items);
+  e.offsets_host = std::move(offsets);
+  if (cudaMemcpyAsync(e.items_dev, e.items_host.data(), e.items_host.size() * sizeof(WorkItem), cudaMemcpyHostToDevice,
+                      st) != cudaSuccess ||
+      cudaMemcpyAsync(e.offsets_dev, e.offsets_host.data(), e.offsets_host.size() * sizeof(int),
+                      cudaMemcpyHostToDevice, st) != cudaSuccess) {
     cudaFree(e.items_dev);
     cudaFree(e.offsets_dev);
     return SAF_ERR_CUDA;
@@ -386,6 +422,7 @@ int saf_create(saf_ctx** out, int device) {
     if (v > 0) ctx->wait_limit_ns = static_cast<unsigned long long>(v) * 1000000ull;
   }
   if (const char* e = std::getenv("SAF_DISABLE_TENSOR_PATTERN")) ctx->tensor_pattern = std::atoi(e) == 0;
+  if (const char* e = std::getenv("SAF_SELFTEST_DROP_LOAD")) ctx->selftest_drop_load = std::atoi(e) == 1;
   if (const char* e = std::getenv("SAF_FROZEN_WEIGHT_PCT")) {
     long v = std::atol(e);
     if (v > 0 && v <= 400) ctx->frozen_weight_pct = static_cast<int>(v);
@@ -419,7 +456,7 @@ int saf_destroy(saf_ctx* ctx) {
     cudaFree(e.offsets_dev);
   }
   DevBuf* pbufs[] = {&ctx->pat_consts, &ctx->pat_ok, &ctx->pat_avec, &ctx->pat_wvec, &ctx->pat_bandf, &ctx->pat_bandb,
-                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta, &ctx->fit_buf, &ctx->calib_tmp};
+                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->pat_snap, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta, &ctx->fit_buf, &ctx->calib_tmp};
   for (DevBuf* b : pbufs) release(*b);
   DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->dkacc_buf, &ctx->dvacc_buf, &ctx->qslot_buf, &ctx->hq, &ctx->hk, &ctx->hv,
                     &ctx->hdo, &ctx->ho, &ctx->hlse, &ctx->hdq, &ctx->hdk, &ctx->hdv, &ctx->halpha, &ctx->hrho,
@@ -470,7 +507,7 @@ int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* froz
       (rc = ensure(ctx->pat_ok, static_cast<size_t>(H) * sizeof(int))) || (rc = ensure(ctx->pat_avec, vecb)) ||
       (rc = ensure(ctx->pat_wvec, vecb)) || (rc = ensure(ctx->pat_bandf, bandb)) ||
       (rc = ensure(ctx->pat_bandb, bandb)) || (rc = ensure(ctx->pat_hord, static_cast<size_t>(H) * sizeof(int))) ||
-      (rc = ensure(ctx->pat_hlist, static_cast<size_t>(H) * sizeof(int))) ||
+      (rc = ensure(ctx->pat_hlist, static_cast<size_t>(H) * sizeof(int))) || (rc = ensure(ctx->pat_snap, 3 * vecb)) ||
       (rc = ensure(ctx->ok_fwd, static_cast<size_t>(H) * sizeof(int))) ||
       (rc = ensure(ctx->ok_bwd, static_cast<size_t>(H) * sizeof(int))))
     return rc;
@@ -496,6 +533,16 @@ int saf_pattern_prepare(saf_ctx* ctx, int32_t H, int32_t Tp, const uint8_t* froz
                               static_cast<float*>(ctx->pat_consts.ptr), static_cast<int*>(ctx->pat_ok.ptr),
                               static_cast<float*>(ctx->pat_avec.ptr), static_cast<float*>(ctx->pat_wvec.ptr),
                               ctx->pat_bandf.ptr, ctx->pat_bandb.ptr, st) != cudaSuccess)
+      return SAF_ERR_CUDA;
+  }
+  // Snapshot of the three vectors: the tables are matched to a later call by these pointers, and the staging kernels
+  // compare the bits, so a head whose vectors were rewritten in place since (by the caller, by the fitter, by the
+  // allocation-free normaliser entry point) falls back to the general form instead of using stale tables.
+  {
+    uint8_t* snap = static_cast<uint8_t*>(ctx->pat_snap.ptr);
+    if (cudaMemcpyAsync(snap, alpha_dev, vecb, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(snap + vecb, rho_dev, vecb, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(snap + 2 * vecb, logZ_dev_out, vecb, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return SAF_ERR_CUDA;
   }
   ctx->pat.valid = true;
@@ -572,7 +619,7 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
       if (launch_scale_rows(V, p->v_strides, static_cast<const float*>(ctx->pat_avec.ptr), HK_A_SCALE, p->Tp,
                             static_cast<const int*>(ctx->pat_hlist.ptr), static_cast<const int*>(ctx->pat_ok.ptr),
                             static_cast<int*>(ctx->ok_fwd.ptr), fp.call_id, ctx->vt_buf.ptr, p->B, nf, p->T, p->D,
-                            kvg, st) != cudaSuccess)
+                            kvg, pattern_check(ctx, alpha, rho, logZ), st) != cudaSuccess)
         return SAF_ERR_CUDA;
     }
     rc = make_map_contig(ctx, &mvt, ctx->vt_buf.ptr, p, nf);
@@ -598,6 +645,8 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   fp.cta_offsets = wl->offsets_dev;
   fp.status = ctx->status_dev;
   fp.wait_limit_ns = ctx->wait_limit_ns;
+  fp.selftest_drop_load =
+      (ctx->selftest_drop_load && grid <= 16 && ctx->wait_limit_ns <= 50000000ull && p->D == 64) ? 1 : 0;
   ScopedTimer timer(ctx, SAF_KERNEL_FWD, st);
   // head dimension 96 runs on the 128-wide kernel: TMA zero-fills features 96..127 of every operand tile
   // O leaves the D = 64 kernel as whole tiles by TMA stores (rows beyond T are clipped by the map)
@@ -689,6 +738,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
     fz.dot_dst = ctx->dot_buf.ptr;
     fz.Hf = nf;
     fz.Tp = p->Tp;
+    fz.chk = pattern_check(ctx, alpha, rho, logZ);
   }
   // O is only read for ordinary heads; a frozen-only layer may pass O = NULL
   {

@@ -179,6 +179,7 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       tma_prefetch_desc(&mvt);
       uint32_t nq = 0, nk = 0, nv = 0, nfz = 0;
       bool ok = true, fz_open = false;
+      bool drop_load = p.selftest_drop_load != 0;        // self-test of the give-up path: see FwdParams
       ItemView64 nxt = load_item64(p, it_begin, it_end);
       for (int it = it_begin; it < it_end && ok; ++it) {
         const WorkItem w = nxt.w;
@@ -232,8 +233,11 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             const int s = nk % C::NS;
             ok = mbar_wait(k_empty + s, ((nk / C::NS) & 1) ^ 1, wc, F_K_EMPTY);
             if (!ok) break;
-            mbar_expect_tx(k_full + s, C::TILE_BYTES);
-            tma_load_4d(smem + C::OFF_K + s * C::TILE_BYTES, &mk, k_full + s, 0, j * BLK, kh, w.b);
+            if (!drop_load) {
+              mbar_expect_tx(k_full + s, C::TILE_BYTES);
+              tma_load_4d(smem + C::OFF_K + s * C::TILE_BYTES, &mk, k_full + s, 0, j * BLK, kh, w.b);
+            }
+            drop_load = false;
             ++nk;
           }
           const int s = nv % C::NS;

@@ -39,6 +39,10 @@ struct FwdParams {
   const int* cta_offsets;           // [grid+1]
   int* status;                      // device status word
   unsigned long long wait_limit_ns;
+  // Self-test of the give-up path (0 in normal use): the producer of the D = 64 forward leaves out the load of the
+  // first key tile of its first ordinary item, so that the waits for it run out.  Set by saf_create from
+  // SAF_SELFTEST_DROP_LOAD, and only for grids of at most 16 CTAs with a wait limit of at most 50 ms.
+  int selftest_drop_load;
 };
 
 struct BwdParams {
@@ -95,6 +99,15 @@ cudaError_t launch_rowdot(const void* O, const void* dO, const int64_t* o_stride
 cudaError_t launch_pgrad(int D, const CUtensorMap& mv, const CUtensorMap& mdo, const PgradParams& p, int grid,
                          cudaStream_t st);
 
+// The vectors a call passes against the bits the pattern tables were built from (snapshot: alpha, rho, logZ,
+// each [H][Tp] as raw 32-bit words, one after the other).
+struct PatternCheck {
+  const float* alpha;
+  const float* rho;
+  const float* logZ;
+  const uint32_t* snap;
+  size_t vec_elems;                 // H * Tp
+};
 // Launchers (defined in the .cu files).  All return the launch error.
 cudaError_t launch_logz(const float* alpha, const float* rho, float* logZ, const uint8_t* mask_dev, int H,
                         int Tp, cudaStream_t st);
@@ -103,7 +116,7 @@ cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const fl
                                   void* band_b, cudaStream_t st);
 cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, float extra, int Tp,
                               const int* hlist, const int* pat_ok, int* ovf, int call_id, void* dst, int B, int Hf,
-                              int T, int D, int src_group, cudaStream_t st);   // src head = h / src_group
+                              int T, int D, int src_group, const PatternCheck& chk, cudaStream_t st);   // src head = h / src_group
 // powers of two that put the fp16 operands of the tensor-core frozen form into fp16's range
 constexpr float HK_BAND_SCALE = 16384.0f;        // bands hold 2^14 r
 constexpr float HK_A_SCALE = 2048.0f;            // the forward stages 2^11 a V
@@ -125,6 +138,7 @@ struct PrepFrozen {
   int call_id;
   void* dot_dst;                    // fp16 [B][Hf][T][D], or NULL
   int Hf, Tp;
+  PatternCheck chk;
 };
 cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* o_strides,
                             const uint8_t* mask_dev, void* q_ext, void* do_ext, float inv_scale, float* dQacc,

@@ -2,6 +2,7 @@
 // pass and the fp32 -> bf16 conversion of the accumulated query gradient.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <cstring>
 #include <mutex>
 
 #include "../../include/saf.h"
@@ -157,14 +158,22 @@ cudaError_t launch_pattern_tables(const float* alpha, const float* rho, const fl
 // dst[b][ord][t][:] = fp16(extra * vec[h][t] * src[b][h][t][:]), h = hlist[ord], for the frozen heads whose tensor-core form is
 // enabled (V scaled by a, or dO scaled by w).  Eight features per thread.  A product that leaves fp16's range
 // marks the head (ovf[h] = call_id), which sends it down the general path in the kernel that follows; the
-// mark of an earlier call has another id and needs no reset.
+// mark of an earlier call has another id and needs no reset.  The same mark is raised when alpha, rho or logZ of the
+// head no longer hold the bits the tables were built from (another call may have rewritten the vectors in place):
+// the threads of batch entry 0 compare their row's three values with the snapshot taken at preparation.
+__device__ __forceinline__ bool pattern_row_changed(const PatternCheck& c, size_t i) {
+  const size_t n = c.vec_elems;
+  return __float_as_uint(c.alpha[i]) != c.snap[i] || __float_as_uint(c.rho[i]) != c.snap[n + i] ||
+         __float_as_uint(c.logZ[i]) != c.snap[2 * n + i];
+}
+
 template <int D>
 __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16* __restrict__ src, int64_t s0, int64_t s1,
                                                              int64_t s2, const float* __restrict__ vec, float extra,
                                                              int Tp, const int* __restrict__ hlist,
                                                              const int* __restrict__ pat_ok, int* __restrict__ ovf,
                                                              int call_id, __half* __restrict__ dst, int B, int Hf,
-                                                             int T, int src_group) {
+                                                             int T, int src_group, const PatternCheck chk) {
   constexpr int TPR = D / 8;
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
   const long long rowid = gid / TPR;               // over [B][Hf][T]: frozen heads only
@@ -188,27 +197,28 @@ __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16
     bad |= !(fabsf(y0) <= 65504.0f) || !(fabsf(y1) <= 65504.0f);     // also catches NaN
     o[e] = __floats2half2_rn(y0, y1);
   }
+  if (b == 0 && part == 0) bad |= pattern_row_changed(chk, static_cast<size_t>(h) * Tp + t);
   if (bad) ovf[h] = call_id;
   *reinterpret_cast<uint4*>(dst + (static_cast<size_t>(rowid)) * D + part * 8) = *reinterpret_cast<uint4*>(o);
 }
 
 cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const float* vec, float extra, int Tp,
                               const int* hlist, const int* pat_ok, int* ovf, int call_id, void* dst, int B, int Hf,
-                              int T, int D, int src_group, cudaStream_t st) {
+                              int T, int D, int src_group, const PatternCheck& chk, cudaStream_t st) {
   const long long nthreads = static_cast<long long>(B) * Hf * T * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
   if (D == 96)
     saf_scale_rows_kernel<96><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
                                                     strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
-                                                    static_cast<__half*>(dst), B, Hf, T, src_group);
+                                                    static_cast<__half*>(dst), B, Hf, T, src_group, chk);
   else if (D == 64)
     saf_scale_rows_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
                                                     strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
-                                                    static_cast<__half*>(dst), B, Hf, T, src_group);
+                                                    static_cast<__half*>(dst), B, Hf, T, src_group, chk);
   else
     saf_scale_rows_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
                                                      strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
-                                                     static_cast<__half*>(dst), B, Hf, T, src_group);
+                                                     static_cast<__half*>(dst), B, Hf, T, src_group, chk);
   return cudaGetLastError();
 }
 
@@ -304,6 +314,7 @@ __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat1
           bad |= !(fabsf(y0) <= 65504.0f) || !(fabsf(y1) <= 65504.0f);     // also catches NaN
           o[e] = __floats2half2_rn(y0, y1);
         }
+        if (b == 0 && part == 0) bad |= pattern_row_changed(fz.chk, static_cast<size_t>(h) * fz.Tp + t);
         if (bad) fz.ovf[h] = fz.call_id;
         const size_t drow = (static_cast<size_t>(b) * fz.Hf + fz.hord[h]) * T + t;
         *reinterpret_cast<uint4*>(static_cast<__half*>(fz.dot_dst) + drow * D + part * 8) =
@@ -400,6 +411,9 @@ static __device__ __align__(256) uint8_t g_static_mask_scratch[SAF_STATIC_MAX_HE
 constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 uint8_t* g_static_mask_ptr[kMaxDevices] = {};   // device address of the array, per device, resolved once
+// The caller's mask is copied here first (under the mutex) and uploaded from here: the upload then never reads the
+// caller's array after the call has returned, whatever kind of host memory that array lives in.
+uint8_t g_static_mask_host[SAF_STATIC_MAX_HEADS];
 
 }  // namespace
 
@@ -436,7 +450,10 @@ extern "C" int saf_pattern_logz_static(int32_t device, int32_t H, int32_t Tp, co
   if (rc == SAF_OK) {
     // The array keeps whatever the previous call left; the first H bytes are all this call reads,
     // and they are overwritten here.
-    if (cudaMemcpyAsync(scratch, frozen_mask_host, static_cast<size_t>(H), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    std::memcpy(g_static_mask_host, frozen_mask_host, static_cast<size_t>(H));
+    // (pageable source: the runtime stages the bytes before this call returns)
+    if (cudaMemcpyAsync(scratch, g_static_mask_host, static_cast<size_t>(H), cudaMemcpyHostToDevice, st) != cudaSuccess)
       rc = SAF_ERR_CUDA;
   }
   if (rc == SAF_OK && saf::launch_logz(alpha_dev, rho_dev, logZ_dev_out, scratch, H, Tp, st) != cudaSuccess)

@@ -8,7 +8,7 @@ import paper_2609_34650_b200 as saf
 import saf_inputs as si
 from oracle import saf_oracle as orc
 
-from gpu_util import Layer, assert_close, errors, f64, bf16_tensor, MAX_ABS, REL_L2
+from gpu_util import Layer, assert_close, errors, f64, bf16_tensor, bf16_half_ulp, MAX_ABS, REL_L2
 
 pytestmark = pytest.mark.gpu
 
@@ -21,11 +21,12 @@ def check_units(L: Layer, units, backward=True, rows=None, panel=512):
     O, LSE = L.host(L.O), L.host(L.LSE)
     G = [L.host(g) for g in L.grads] if backward else None
     worst = {}
+    deg = wl.T <= 2                                      # one or two tokens: see assert_close
     for b, h in units:
         fr = bool(inp.mask[h])
         eO, eL = orc.head_fwd_panels(fr, q[b, h], k[b, h], v[b, h], inp.alpha[h], inp.rho[h], scale, panel, rows)
         sl = rows or slice(0, wl.T)
-        worst[("O", fr)] = assert_close(O[b, h][sl], eO, f"O[{b},{h}] frozen={fr}")
+        worst[("O", fr)] = assert_close(O[b, h][sl], eO, f"O[{b},{h}] frozen={fr}", degenerate=deg)
         if fr:
             assert not LSE[b, h].any(), "LSE slot of a frozen head must be zero"
         else:
@@ -36,8 +37,80 @@ def check_units(L: Layer, units, backward=True, rows=None, panel=512):
                 if fr and name != "dV":
                     assert not g[b, h].any(), f"{name}[{b},{h}] of a frozen head must be exactly zero"
                 else:
-                    assert_close(g[b, h], ee, f"{name}[{b},{h}] frozen={fr}")
+                    assert_close(g[b, h], ee, f"{name}[{b},{h}] frozen={fr}", degenerate=deg)
     return worst
+
+
+def sampled_units(wl, n, seed, backward=True):
+    """Units for the full-size comparisons: `n` (b,h) pairs from a seeded draw that holds at least one frozen and
+    one ordinary head where the workload has them, plus the unit of the last work item of the last CTA of the
+    scheduler's list (the tail of the persistent grid)."""
+    rng = np.random.default_rng(seed)
+    fz = [h for h in range(wl.H) if wl.mask[h]]
+    od = [h for h in range(wl.H) if not wl.mask[h]]
+    units = []
+    if fz:
+        units.append((int(rng.integers(wl.B)), int(rng.choice(fz))))
+    if od:
+        units.append((int(rng.integers(wl.B)), int(rng.choice(od))))
+    while len(units) < n:
+        u = (int(rng.integers(wl.B)), int(rng.integers(wl.H)))
+        if u not in units:
+            units.append(u)
+    n_ctas = torch.cuda.get_device_properties(0).multi_processor_count
+    items, offsets = saf.saf_build_worklist(wl.B, wl.H, wl.T, wl.mask, backward, n_ctas)
+    last = items[offsets[-1] - 1]
+    tail = (int(last[0]), int(last[1]))
+    if tail not in units:
+        units.append(tail)
+    return units
+
+
+def grads_with_rounded_output(inp):
+    """The backward's formulas (Sec. 3.3 / Appendix E.2) with delta_i = dO_i . O_i taken from the bf16-rounded O,
+    as the layer is handed it, instead of the exact sum_j A_ij dP_ij: a test-side restatement built from the
+    oracle's forward (no value comes from the GPU).  Same layouts as oracle.hybrid_attn_bwd."""
+    wl = inp.wl
+    q, k, v, do = f64(inp)
+    mask = inp.mask
+    H, T, D = wl.H, wl.T, wl.D
+    packed = wl.packed_qk
+    slot = np.cumsum(np.asarray(mask) == 0) - 1
+    g = wl.kv_group
+    scale = 1.0 / np.sqrt(D)
+    dQ, dK, dV = np.zeros(q.shape), np.zeros(k.shape), np.zeros(v.shape)
+    for h in range(H):
+        for b in range(wl.B):
+            if mask[h]:
+                dV[b, h // g] += orc.frozen_head_bwd(do[b, h], inp.alpha[h], inp.rho[h])
+                continue
+            hq, hk = (slot[h], slot[h]) if packed else (h, h // g)
+            O, _, A = orc.ordinary_head_fwd(q[b, hq], k[b, hk], v[b, h // g], scale)
+            O_r = si.bf16_bits_to_f64(si.f32_to_bf16_bits(O.astype(np.float32)))
+            dP = do[b, h] @ v[b, h // g].T
+            dS = A * (dP - (do[b, h] * O_r).sum(axis=1, keepdims=True))
+            dQ[b, hq] = scale * (dS @ k[b, hk])
+            dK[b, hk] += scale * (dS.T @ q[b, hq])
+            dV[b, h // g] += A.T @ do[b, h]
+    return dQ, dK, dV
+
+
+def check_bf16_grads_against_oracle(L16):
+    """bf16 gradients against the fp64 oracle: the result is rounded once more, so the absolute bound grows by half
+    a bf16 unit in the last place at the tensor's largest magnitude; the relative L2 bound is unchanged."""
+    inp, wl = L16.inp, L16.inp.wl
+    q, k, v, do = f64(inp)
+    want = orc.hybrid_attn_bwd(q, k, v, do, inp.mask, inp.alpha.astype(np.float64), inp.rho.astype(np.float64))
+    for name, got, ee in zip(("dQ", "dK", "dV"), (L16.host(g) for g in L16.grads), want):
+        assert got.shape == ee.shape, name
+        shared = wl.kv_group if name == "dV" else 1
+        for b in range(ee.shape[0]):
+            for h in range(ee.shape[1]):
+                if not ee[b, h].any():
+                    assert not got[b, h].any(), f"{name}[{b},{h}] must be exactly zero"
+                    continue
+                bound = MAX_ABS * np.sqrt(shared) + bf16_half_ulp(np.abs(ee[b, h]).max())
+                assert_close(got[b, h], ee[b, h], f"bf16 {name}[{b},{h}]", max_abs=bound, degenerate=wl.T <= 2)
 
 
 def all_units(wl):
@@ -135,6 +208,7 @@ def test_head_dim_128_backward_general_frozen_form_and_bf16():
     for g32, g16 in zip(L.grads, L16.grads):
         a, b = L.host(g32), L.host(g16)
         assert np.abs(a - b).max() <= 2.0 ** -8 * max(np.abs(a).max(), 1.0) + 1e-6
+    check_bf16_grads_against_oracle(L16)
 
 
 def test_head_dim_128_backward_shared_and_packed_heads():
@@ -289,6 +363,7 @@ def test_bf16_gradients():
     for g16, g32 in zip(L.grads, ref.grads):
         ma, rl = errors(L.host(g16), L.host(g32))
         assert ma <= 3.2e-2 and rl <= 5e-3
+    check_bf16_grads_against_oracle(L)
 
 
 def test_forward_is_deterministic_and_internal_prepare_matches():
@@ -409,7 +484,7 @@ def test_invalid_arguments_are_rejected():
         L.run()
     assert e.value.code == 1
     L = Layer(inp)
-    L.prob.D = 80                              # supported: 64, 96 (forward), 128 (forward)
+    L.prob.D = 80                              # supported: 64, 96, 128
     with pytest.raises(saf.SafError) as e:
         L.run()
     assert e.value.code == 2
@@ -421,15 +496,16 @@ def test_invalid_arguments_are_rejected():
 
 
 # --------------------------------------------------------------------------- grouped-query path
-def _check_gqa_layer(L, backward, grad_rel_l2=REL_L2):
+def _check_gqa_layer(L, backward, grad_rel_l2=REL_L2, expected_grads=None):
     """Whole layer against the dense oracle: K, V (and dK, dV) have H / kv_group heads."""
     inp, wl = L.inp, L.inp.wl
+    deg = wl.T <= 2
     q, k, v, do = f64(inp)
     O, LSE = L.host(L.O), L.host(L.LSE)
     eO, eL = orc.hybrid_attn_fwd(q, k, v, inp.mask, inp.alpha.astype(np.float64), inp.rho.astype(np.float64))
     for b in range(wl.B):
         for h in range(wl.H):
-            assert_close(O[b, h], eO[b, h], f"O[{b},{h}]")
+            assert_close(O[b, h], eO[b, h], f"O[{b},{h}]", degenerate=deg)
             if inp.mask[h]:
                 assert not LSE[b, h].any()
             else:
@@ -437,19 +513,20 @@ def _check_gqa_layer(L, backward, grad_rel_l2=REL_L2):
     if not backward:
         return
     dQ, dK, dV = (L.host(g) for g in L.grads)
-    eQ, eK, eV = orc.hybrid_attn_bwd(q, k, v, do, inp.mask, inp.alpha.astype(np.float64), inp.rho.astype(np.float64))
+    eQ, eK, eV = expected_grads or orc.hybrid_attn_bwd(q, k, v, do, inp.mask, inp.alpha.astype(np.float64),
+                                                       inp.rho.astype(np.float64))
     assert dK.shape == eK.shape and dV.shape == eV.shape
     for b in range(wl.B):
         for h in range(wl.H):
             if inp.mask[h]:
                 assert not dQ[b, h].any(), "dQ of a frozen head must be exactly zero"
             else:
-                assert_close(dQ[b, h], eQ[b, h], f"dQ[{b},{h}]", rel_l2=grad_rel_l2)
+                assert_close(dQ[b, h], eQ[b, h], f"dQ[{b},{h}]", rel_l2=grad_rel_l2, degenerate=deg)
         for hk in range(wl.H // wl.kv_group):
-            assert_close(dK[b, hk], eK[b, hk], f"dK[{b},kv {hk}]", rel_l2=grad_rel_l2)
+            assert_close(dK[b, hk], eK[b, hk], f"dK[{b},kv {hk}]", rel_l2=grad_rel_l2, degenerate=deg)
             # a shared head's dV sums kv_group heads: the absolute bound scales with the number of terms
             assert_close(dV[b, hk], eV[b, hk], f"dV[{b},kv {hk}]", max_abs=MAX_ABS * np.sqrt(wl.kv_group),
-                         rel_l2=grad_rel_l2)
+                         rel_l2=grad_rel_l2, degenerate=deg)
 
 
 @pytest.mark.parametrize("H,g,frozen,T", [(8, 4, (1, 6), 300), (4, 2, (), 257), (6, 3, (0, 1, 2), 200),
@@ -495,6 +572,7 @@ def test_gqa_bf16_gradients_and_bad_group():
         a, b = L32.host(g32), L16.host(g16)
         assert a.shape == b.shape
         assert np.abs(a - b).max() <= 2.0 ** -8 * max(np.abs(a).max(), 1.0) + 1e-6, name   # one bf16 rounding
+    check_bf16_grads_against_oracle(L16)
     L = Layer(inp)
     L.prob.kv_group = 3                        # does not divide H
     with pytest.raises(saf.SafError) as e:
@@ -503,15 +581,16 @@ def test_gqa_bf16_gradients_and_bad_group():
 
 
 # --------------------------------------------------------------------------- packed Q/K layout
-def _check_packed_layer(L, backward, grad_rel_l2=REL_L2):
+def _check_packed_layer(L, backward, grad_rel_l2=REL_L2, expected_grads=None):
     inp, wl = L.inp, L.inp.wl
+    deg = wl.T <= 2
     q, k, v, do = f64(inp)
     al, rh = inp.alpha.astype(np.float64), inp.rho.astype(np.float64)
     O, LSE = L.host(L.O), L.host(L.LSE)
     eO, eL = orc.hybrid_attn_fwd(q, k, v, inp.mask, al, rh)
     for b in range(wl.B):
         for h in range(wl.H):
-            assert_close(O[b, h], eO[b, h], f"O[{b},{h}]")
+            assert_close(O[b, h], eO[b, h], f"O[{b},{h}]", degenerate=deg)
             if inp.mask[h]:
                 assert not LSE[b, h].any()
             else:
@@ -519,14 +598,14 @@ def _check_packed_layer(L, backward, grad_rel_l2=REL_L2):
     if not backward:
         return
     dQ, dK, dV = (L.host(g) for g in L.grads)
-    eQ, eK, eV = orc.hybrid_attn_bwd(q, k, v, do, inp.mask, al, rh)
+    eQ, eK, eV = expected_grads or orc.hybrid_attn_bwd(q, k, v, do, inp.mask, al, rh)
     assert dQ.shape == eQ.shape and dK.shape == eK.shape and dV.shape == eV.shape
     for b in range(wl.B):
         for s_ in range(dQ.shape[1]):
-            assert_close(dQ[b, s_], eQ[b, s_], f"dQ[{b},slot {s_}]", rel_l2=grad_rel_l2)
-            assert_close(dK[b, s_], eK[b, s_], f"dK[{b},slot {s_}]", rel_l2=grad_rel_l2)
+            assert_close(dQ[b, s_], eQ[b, s_], f"dQ[{b},slot {s_}]", rel_l2=grad_rel_l2, degenerate=deg)
+            assert_close(dK[b, s_], eK[b, s_], f"dK[{b},slot {s_}]", rel_l2=grad_rel_l2, degenerate=deg)
         for h in range(wl.H):
-            assert_close(dV[b, h], eV[b, h], f"dV[{b},{h}]", rel_l2=grad_rel_l2)
+            assert_close(dV[b, h], eV[b, h], f"dV[{b},{h}]", rel_l2=grad_rel_l2, degenerate=deg)
 
 
 @pytest.mark.parametrize("H,frozen,T,gd", [(6, (1, 4), 300, "f32"), (4, (0, 3), 129, "bf16"), (3, (), 200, "f32"),
@@ -542,6 +621,7 @@ def test_packed_qk_layout_forward_backward(H, frozen, T, gd):
         for g32, g16 in zip(L32.grads, L.grads):
             a, b = L32.host(g32), L.host(g16)
             assert a.shape == b.shape and np.abs(a - b).max() <= 2.0 ** -8 * max(np.abs(a).max(), 1.0) + 1e-6
+        check_bf16_grads_against_oracle(L)
 
 
 def test_packed_qk_layout_head_dim_128_forward_and_errors():
@@ -585,38 +665,33 @@ def test_random_geometries_forward_backward(seed):
     # nearly cancels and that rounding of O (2^-9 relative) is not averaged out: measured at T = 3 the gradients lie
     # within 2.5e-3 (relative L2) of the oracle's formulas evaluated with the same rounded O, but up to 1.1e-2 from
     # the oracle's exact delta.  Sequences shorter than 8 therefore get twice the relative bound on the gradients.
+    # That the doubled bound is needed only for this reason is asserted, not assumed: against the same formulas with
+    # delta from the rounded O the stated bound holds at every length.
     tol = 2 * REL_L2 if wl.T < 8 else REL_L2
-    if wl.packed_qk:
-        _check_packed_layer(L, True, grad_rel_l2=tol)
-    else:
-        _check_gqa_layer(L, True, grad_rel_l2=tol)
+    check = _check_packed_layer if wl.packed_qk else _check_gqa_layer
+    check(L, True, grad_rel_l2=tol)
+    if wl.T < 8:
+        check(L, True, grad_rel_l2=REL_L2, expected_grads=grads_with_rounded_output(L.inp))
 
 
 # --------------------------------------------------------------------------- full sizes, sampled
 def test_config1_full_size_sampled_units():
     wl = si.config(1)
     L = Layer(si.generate(wl)).run()
-    fh, oh = wl.frozen_heads[0], [h for h in range(wl.H) if h not in wl.frozen_heads][0]
-    check_units(L, [(0, fh), (wl.B - 1, oh), (3, wl.frozen_heads[-1])], panel=1024)
+    check_units(L, sampled_units(wl, 4, seed=101), panel=1024)
 
 
 @pytest.mark.parametrize("nf", [0, 6, 9, 12])
 def test_config3_sweep_full_size_sampled_units(nf):
     wl = si.config(3, nf)
     L = Layer(si.generate(wl)).run()
-    units = []
-    if nf > 0:
-        units.append((nf % wl.B, wl.frozen_heads[nf // 2]))
-    if nf < wl.H:
-        units.append(((nf + 1) % wl.B, [h for h in range(wl.H) if h not in wl.frozen_heads][0]))
-    check_units(L, units, panel=1024)
+    check_units(L, sampled_units(wl, 2, seed=300 + nf), panel=1024)
 
 
 def test_config2_full_size_sampled_units():
     wl = si.config(2)
     L = Layer(si.generate(wl)).run()
-    oh = [h for h in range(wl.H) if h not in wl.frozen_heads][-1]
-    check_units(L, [(1, wl.frozen_heads[3]), (2, oh)], panel=1024)
+    check_units(L, sampled_units(wl, 2, seed=102), panel=1024)
 
 
 def test_long_sequence_16k_forward_backward_sampled_units():
