@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the hybrid causal attention layer (forward + backward) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 1|2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 1|2|4|5|6]
 
 One step = one pass of the whole hot path over one synthetic batch: forward kernel, backward
 preparation (delta, zero-fill) and backward kernel, for the GPT-2-124M-shaped layer
@@ -14,6 +14,13 @@ Prints ONE JSON line (rank 0).  `value` is TFLOP/s on the layer's algorithmic FL
 metric through the host-buffer entry point with every input copied to the device and every output
 copied back inside the timed region.  `--impl reference` times the fp64 CPU oracle on a bounded
 sample of the same workload.
+
+The K-step region is timed `--repeats` times (default 5) and `ms_per_step` is the median region; the per-kernel
+CUDA-event pairs that give the roofline's kernel duration cost a few microseconds per launch, so they are recorded
+in one further K-step region of the same steps (`ms_per_step_with_kernel_events`), not in the headline regions.
+`--config 4` is the forward-only long-prefill workload.  On config 1 the line carries `sweep`: the same step at 0,
+25, 50, 75 and 100 % frozen heads.  With `--gpus N`, N > 1, and no torchrun environment, bench.py starts the N
+ranks itself (one process per GPU, rendezvous on 127.0.0.1).
 """
 from __future__ import annotations
 
@@ -315,19 +322,21 @@ def run_ours(args):
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
 
     wl = si.config(args.config, seed=sd.rank_seed(0, rank))
+    bwd = wl.backward
     inp = si.generate(wl)
 
     def t16(bits):
         return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
 
     hostQ, hostK, hostV, hostdO = (t16(x).pin_memory() for x in (inp.q, inp.k, inp.v, inp.do))
-    Q, K, V, dO = (x.to(dev) for x in (hostQ, hostK, hostV, hostdO))
+    Q, K, V = (x.to(dev) for x in (hostQ, hostK, hostV))
+    dO = hostdO.to(dev) if bwd else None
     alpha_h, rho_h = torch.from_numpy(inp.alpha).pin_memory(), torch.from_numpy(inp.rho).pin_memory()
     alpha, rho = alpha_h.to(dev), rho_h.to(dev)
     logZ = torch.zeros_like(alpha)
     O = torch.empty_like(Q)
     LSE = torch.empty(wl.B, wl.H, wl.T, device=dev)
-    dQ, dK, dV = (torch.empty(Q.shape, device=dev, dtype=torch.float32) for _ in range(3))
+    dQ, dK, dV = (torch.empty(Q.shape, device=dev, dtype=torch.float32) for _ in range(3)) if bwd else (None,) * 3
     ctx = saf.Context(local_rank)
     prob = saf.make_problem(Q, wl.stored_len)
     mask = inp.mask
@@ -346,21 +355,22 @@ def run_ours(args):
     torch.cuda.synchronize()
     prepare_ms = e0.elapsed_time(e1)
 
-    def step(m):
-        ctx.saf_hybrid_attn_fwd(prob, Q, K, V, m, alpha, rho, logZ, O, LSE)
-        ctx.saf_hybrid_attn_bwd(prob, Q, K, V, O, dO, LSE, m, alpha, rho, logZ, dQ, dK, dV)
+    def step(m, c=ctx, al=alpha, rh=rho, lz=logZ):
+        c.saf_hybrid_attn_fwd(prob, Q, K, V, m, al, rh, lz, O, LSE)
+        if bwd:
+            c.saf_hybrid_attn_bwd(prob, Q, K, V, O, dO, LSE, m, al, rh, lz, dQ, dK, dV)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(m, steps):
+    def timed(m, steps, **kw):
         barrier()
         a, b = ev(), ev()
         a.record()
         for _ in range(steps):
-            step(m)
+            step(m, **kw)
         b.record()
         barrier()
         return a.elapsed_time(b) / steps
@@ -370,19 +380,29 @@ def run_ours(args):
         step(mask0)
     torch.cuda.synchronize()
 
-    # ---- headline: exactly K timed steps, clocks sampled during the region, per-kernel events on
+    # ---- headline: the K-step region, timed `repeats` times; clocks sampled while the regions run
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
+    flops_local = wl.flops()
+    regions = []
+    for _ in range(max(args.repeats, 1)):
+        # an idle gap first: every region is then a burst measurement like a single K-step run (and like the burst
+        # peak the roofline divides by); without it the later regions run into the board's power cap (~10 % slower)
+        time.sleep(args.region_gap)
+        regions.append(sd.max_over_ranks(timed(mask, args.steps), dev))       # slowest rank of each region
+    time.sleep(args.region_gap)
+    ms = float(np.median(regions))
+    value = sd.sum_over_ranks(flops_local, dev) / (ms * 1e-3) / 1e12
+
+    # ---- one more K-step region with an event pair around every kernel (the roofline's kernel durations)
     ctx.saf_set_profiling(True)
-    ctx.saf_get_kernel_time(saf.SAF_KERNEL_FWD)
-    ctx.saf_get_kernel_time(saf.SAF_KERNEL_BWD)
-    ctx.saf_get_kernel_time(saf.SAF_KERNEL_BWD_PREP)
-    ms_local = timed(mask, args.steps)
-    k_fwd = ctx.saf_get_kernel_time(saf.SAF_KERNEL_FWD)
-    k_bwd = ctx.saf_get_kernel_time(saf.SAF_KERNEL_BWD)
-    k_prep = ctx.saf_get_kernel_time(saf.SAF_KERNEL_BWD_PREP)
+    kinds = (saf.SAF_KERNEL_FWD, saf.SAF_KERNEL_BWD, saf.SAF_KERNEL_BWD_PREP, saf.SAF_KERNEL_SCALE)
+    for k in kinds:
+        ctx.saf_get_kernel_time(k)
+    ms_events = sd.max_over_ranks(timed(mask, args.steps), dev)
+    k_fwd, k_bwd, k_prep, k_scale = (ctx.saf_get_kernel_time(k) for k in kinds)
     ctx.saf_set_profiling(False)
     code, detail = ctx.saf_last_device_status()
     if code != saf.SAF_OK:
@@ -390,7 +410,7 @@ def run_ours(args):
 
     # optional extra outside the headline: gradients of the compact patterns (trainable-pattern control)
     pgrad_ms = None
-    if len(wl.frozen_heads):
+    if bwd and len(wl.frozen_heads):
         da, dr = torch.empty_like(alpha), torch.empty_like(alpha)
         for _ in range(3):
             ctx.saf_pattern_grad(prob, V, O, dO, mask, alpha, rho, logZ, da, dr)
@@ -403,7 +423,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         pgrad_ms = a.elapsed_time(b) / 10
 
-    # extra: the same step recorded into a CUDA graph and replayed (no launch gaps from the host side)
+    # extra: the same step recorded into a CUDA graph and replayed
     graph_ms = None
     try:
         gs = torch.cuda.Stream()
@@ -426,14 +446,10 @@ def run_ours(args):
         graph_ms = None
         torch.cuda.synchronize()
 
-    flops_local = wl.flops()
-    rate, ms = sd.whole_job_rate(flops_local * 1.0, ms_local, dev)       # FLOP per step over all ranks / max ms
-    value = rate / 1e12
-
-    # ---- speedup vs the same library with zero frozen heads: interleaved A B B A, plus an A/A control
-    # (a comparison whose A/A control is off by more than 2 % is discarded and taken again, at most three times)
+    # ---- speedup vs the same library with zero frozen heads: interleaved A B B A, plus an A/A control that must
+    # read 1.00 within 1 % or the comparison is discarded and taken again (the paper's rule; at most five times)
     reps = max(5, args.steps)
-    for aa_attempt in range(1, 4):
+    for aa_attempt in range(1, 6):
         a1 = timed(mask, reps)
         b1 = timed(mask0, reps)
         b2 = timed(mask0, reps)
@@ -442,12 +458,42 @@ def run_ours(args):
         c2 = timed(mask, reps)
         speedup = (b1 + b2) / (a1 + a2)
         aa_control = c1 / c2
-        if world > 1 or abs(aa_control - 1.0) <= 0.02:     # (ranks must take the same number of timed runs)
+        if world > 1 or abs(aa_control - 1.0) <= 0.01:     # (ranks must take the same number of timed runs)
             break
-    # the sampler ran through the K timed steps and the interleaved repeats of the same step
+    aa_ok = abs(aa_control - 1.0) <= 0.01
+
+    # ---- frozen-rate sweep at this shape (config 1 only): nested frozen sets of one seeded permutation
+    sweep = None
+    if args.config == 1 and world == 1:
+        sweep = []
+        ctx_s = saf.Context(local_rank)
+        full = si.generate(si.Workload("sweep-patterns", 1, wl.H, 8, wl.D, tuple(range(wl.H)), wl.rho_slope,
+                                       Tp=wl.stored_len, seed=wl.seed + 1))
+        al_s, rh_s = torch.from_numpy(full.alpha).to(dev), torch.from_numpy(full.rho).to(dev)
+        lz_s = torch.zeros_like(al_s)
+        for nf in (0, 3, 6, 9, 12):
+            wls = si.config(3, nf)
+            m = wls.mask
+            ctx_s.saf_pattern_prepare(m, al_s, rh_s, lz_s)
+            kw = dict(c=ctx_s, al=al_s, rh=rh_s, lz=lz_s)
+            for _ in range(3):
+                step(m, **kw)
+            t = float(np.median([timed(m, reps, **kw) for _ in range(3)]))
+            tf = wls.flops() / (t * 1e-3) / 1e12
+            sweep.append({"frozen_heads": nf, "frozen_fraction": nf / wl.H, "ms_per_step": t, "tflops": tf})
+        code, detail = ctx_s.saf_last_device_status()
+        if code != saf.SAF_OK:
+            raise RuntimeError(f"sweep: device status {code} detail {detail:#x}")
+        t0 = sweep[0]["ms_per_step"]
+        for r in sweep:
+            r["speedup_vs_0pct_frozen"] = t0 / r["ms_per_step"]
+        ctx_s.close()
+        step(mask)                                           # leave the outputs consistent with `mask`
+
+    # the sampler ran through the timed regions and the interleaved repeats of the same step
     clocks = sampler.stop() if rank == 0 else None
     fwd_only = None
-    if True:
+    if bwd:
         barrier()
         a, b = ev(), ev()
         a.record()
@@ -461,19 +507,33 @@ def run_ours(args):
     # ---- end to end through host buffers (pinned): inputs copied in, every output copied back
     hO = torch.empty_like(hostQ).pin_memory()
     hLSE = torch.empty(wl.B, wl.H, wl.T).pin_memory()
-    hdQ, hdK, hdV = (torch.empty(Q.shape, dtype=torch.float32).pin_memory() for _ in range(3))
-    ctx2 = saf.Context(local_rank)
-    probh = saf.make_problem(hostQ, wl.stored_len)
+    nel = wl.B * wl.H * wl.T * wl.D
+    if bwd:
+        hdQ, hdK, hdV = (torch.empty(Q.shape, dtype=torch.float32).pin_memory() for _ in range(3))
+        ctx2 = saf.Context(local_rank)
+        probh = saf.make_problem(hostQ, wl.stored_len)
 
-    def step_host(prepare):
-        ctx2.saf_hybrid_attn_step_host(probh, hostQ, hostK, hostV, hostdO, mask, alpha_h, rho_h, prepare, hO, hLSE,
-                                       hdQ, hdK, hdV)
+        def step_host(prepare):
+            ctx2.saf_hybrid_attn_step_host(probh, hostQ, hostK, hostV, hostdO, mask, alpha_h, rho_h, prepare, hO,
+                                           hLSE, hdQ, hdK, hdV)
+        h2d = 4 * nel * 2
+        d2h = nel * 2 + wl.B * wl.H * wl.T * 4 + 3 * nel * 4
+    else:
+        # forward-only workload: the device entry point between pinned-memory copies of Q, K, V in and O, LSE out
+        def step_host(prepare):
+            Q.copy_(hostQ, non_blocking=True)
+            K.copy_(hostK, non_blocking=True)
+            V.copy_(hostV, non_blocking=True)
+            ctx.saf_hybrid_attn_fwd(prob, Q, K, V, mask, alpha, rho, logZ, O, LSE)
+            hO.copy_(O, non_blocking=True)
+            hLSE.copy_(LSE, non_blocking=True)
+        h2d = 3 * nel * 2
+        d2h = nel * 2 + wl.B * wl.H * wl.T * 4
 
     step_host(1)
     step_host(0)
     e2e_steps = max(2, min(args.steps, 5))
     barrier()
-    t0 = time.perf_counter()
     a, b = ev(), ev()
     a.record()
     for _ in range(e2e_steps):
@@ -482,9 +542,6 @@ def run_ours(args):
     barrier()
     e2e_ms_local = a.elapsed_time(b) / e2e_steps
     e2e_rate, e2e_ms = sd.whole_job_rate(flops_local, e2e_ms_local, dev)
-    nel = wl.B * wl.H * wl.T * wl.D
-    h2d = 4 * nel * 2
-    d2h = nel * 2 + wl.B * wl.H * wl.T * 4 + 3 * nel * 4
 
     if rank != 0:
         if world > 1:
@@ -492,26 +549,37 @@ def run_ours(args):
         return
 
     peaks = measured_peaks()
-    bwd_flops = wl.B * wl.D * wl.T * (wl.T + 1) * (5 * (wl.H - len(wl.frozen_heads)) + len(wl.frozen_heads))
+    hf = len(wl.frozen_heads)
     fwd_flops = wl.flops(backward=False)
-    bwd_ms = k_bwd[0] / max(k_bwd[1], 1)
     fwd_ms = k_fwd[0] / max(k_fwd[1], 1)
-    prep_ms = k_prep[0] / max(k_prep[1], 1)
-    achieved = bwd_flops / (bwd_ms * 1e-3) / 1e12
+    fwd_name = "saf_fwd64_kernel" if wl.D == 64 else "saf_fwd_kernel<128>"
+    fwd_entry = {"launch_ms": fwd_ms, "achieved": fwd_flops / (fwd_ms * 1e-3) / 1e12,
+                 "frac": fwd_flops / (fwd_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+    others = {}
+    if k_scale[1]:
+        others["saf_scale_rows_kernel"] = {"launch_ms": k_scale[0] / k_scale[1]}
+    if bwd:
+        dom_name = "saf_bwd_kernel" if wl.D == 64 else "saf_bwd128_kernel"
+        dom_flops = wl.B * wl.D * wl.T * (wl.T + 1) * (5 * (wl.H - hf) + hf)
+        dom_ms = k_bwd[0] / max(k_bwd[1], 1)
+        others[fwd_name] = fwd_entry
+        others["saf_bwd_prep_kernel"] = {"launch_ms": k_prep[0] / max(k_prep[1], 1)}
+    else:
+        dom_name, dom_flops, dom_ms = fwd_name, fwd_flops, fwd_ms
+    kernel_sum_ms = (k_fwd[0] + k_bwd[0] + k_prep[0] + k_scale[0]) / max(k_fwd[1], 1)
+    achieved = dom_flops / (dom_ms * 1e-3) / 1e12
     traffic = None
-    bwd_name = "saf_bwd_kernel" if wl.D == 64 else "saf_bwd128_kernel"
     tpath = os.path.join(ROOT, "profiles", "roofline_traffic.json")
     if os.path.exists(tpath):
         with open(tpath) as f:
-            traffic = json.load(f).get(f"{bwd_name}@{wl.name}")
-    roofline = {"bound": "tensor", "kernel": bwd_name, "achieved": achieved, "peak": peaks["bf16_tflops"],
+            traffic = json.load(f).get(f"{dom_name}@{wl.name}")
+    roofline = {"bound": "tensor", "kernel": dom_name, "achieved": achieved, "peak": peaks["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": traffic,
                 "peak_source": f"{peaks['source']} bf16 burst (MEASURED_PEAKS.json)" if peaks["source"] == "measured"
                 else "fallback 1590 TFLOP/s",
-                "launch_ms": bwd_ms, "flops_per_launch": bwd_flops,
-                "other_kernels": {"saf_fwd64_kernel" if wl.D == 64 else "saf_fwd_kernel<128>": {"launch_ms": fwd_ms, "achieved": fwd_flops / (fwd_ms * 1e-3) / 1e12,
-                                                      "frac": fwd_flops / (fwd_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]},
-                                  "saf_bwd_prep_kernel": {"launch_ms": prep_ms}}}
+                "launch_ms": dom_ms, "flops_per_launch": dom_flops,
+                "timed_in": "a K-step region of the same steps with an event pair around every kernel",
+                "kernel_sum_ms_per_step": kernel_sum_ms, "other_kernels": others}
 
     # context for the roofline's denominator: a library bf16 GEMM (8192^3) timed in this same process
     live_gemm = None
@@ -533,31 +601,42 @@ def run_ours(args):
         live_gemm = None
         torch.cuda.synchronize()
 
-    fit = None if args.no_fit else fit_leg(ctx, saf, wl, peaks, dev)
+    fit = None if (args.no_fit or not bwd) else fit_leg(ctx, saf, wl, peaks, dev)
     calib = None
-    if not args.no_fit:
+    if not args.no_fit and bwd:
         # normalisers of the all-ordinary layer (calibration precedes replacement)
         ctx.saf_hybrid_attn_fwd(prob, Q, K, V, mask0, alpha, rho, logZ, O, LSE)
         calib = calib_leg(ctx, saf, wl, prob, Q, K, LSE, peaks, dev)
     cpu_v, cpu_desc, cpu_threads, _ = oracle_sample(si.config(args.config), budget_s=args.ref_budget)
+    # forward kernel, the V staging kernel of the frozen heads, backward preparation and backward kernel
+    launches_per_step = 1 + (1 if hf else 0) + (2 if bwd else 0)
+    tensors_gb = ((4 * 2 + 3 * 4) if bwd else 4 * 2) * nel / 1e9
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl.name, "B_per_gpu": wl.B, "H": wl.H, "Hf": len(wl.frozen_heads), "T": wl.T, "D": wl.D,
-                   "grad_dtype": "f32", "frozen_fraction": len(wl.frozen_heads) / wl.H,
+        "metric": METRIC if bwd else "hybrid_attn_fwd_tflops", "value": value, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "B_per_gpu": wl.B, "B": wl.B, "H": wl.H, "Hf": hf, "T": wl.T, "D": wl.D,
+                   "pass": "fwd+bwd" if bwd else "fwd only",
+                   "grad_dtype": "f32", "frozen_fraction": hf / wl.H,
                    "flops_per_step_per_gpu": flops_local,
-                   "l2": f"inputs+outputs per step ({(4 * 2 + 3 * 4) * nel / 1e9:.2f} GB) exceed the 126 MB L2; no explicit flush",
+                   "l2": f"inputs+outputs per step ({tensors_gb:.2f} GB) exceed the 126 MB L2; no explicit flush",
                    "pattern_prepare": "once before the timed steps (static per layer)", "pattern_prepare_ms": prepare_ms,
+                   "timed_regions": len(regions), "ms_per_step_regions": regions,
+                   "region_gap_s": args.region_gap,
                    "parallelism": f"dp{world} (independent batches, no collective in the layer)"},
         "pct_of_bf16_peak": 100.0 * value / (peaks["bf16_tflops"] * world),
+        "ms_per_step_with_kernel_events": ms_events,
         "speedup_vs_0pct_frozen": speedup, "aa_control": aa_control, "aa_attempts": aa_attempt,
+        "aa_within_1pct": aa_ok,
         "ms_0pct_frozen": 0.5 * (b1 + b2), "ms_fwd_only": fwd_only, "ms_pattern_grad": pgrad_ms,
         "ms_per_step_cuda_graph": graph_ms,
+        "sweep": sweep,
         "e2e": {"value": e2e_rate / 1e12, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
-        # per step: V scaling + forward kernel, dO scaling + backward preparation + backward kernel
-        "gpu_launches": (4 if len(wl.frozen_heads) else 3) * args.steps,
+        # per step: V scaling + forward kernel, backward preparation (which also stages w dO) + backward kernel;
+        # counted over the timed regions that give ms_per_step
+        "gpu_launches": launches_per_step * args.steps * len(regions),
+        "gpu_launches_per_step": launches_per_step,
         "clocks": clocks,
         "roofline": roofline,
         "peak_context": {"library_bf16_gemm_8192_tflops_live": live_gemm,
@@ -571,17 +650,59 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def launch_ranks(args, argv):
+    """`--gpus N` without a torchrun environment: start the N ranks here, one process per GPU, with the
+    environment torchrun would give them (rendezvous on 127.0.0.1), and pass rank 0's JSON line through."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(args.gpus):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(args.gpus),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__), *argv], env=env,
+                                      stdout=subprocess.PIPE if r == 0 else subprocess.DEVNULL, text=True))
+    out, _ = procs[0].communicate()
+    rcs = [procs[0].returncode] + [p.wait() for p in procs[1:]]
+    sys.stdout.write(out)
+    sys.stdout.flush()
+    if any(rcs):
+        raise SystemExit(f"ranks exited with {rcs}")
+
+
+def launcher_selftest(args):
+    """What the ranks of `--gpus N` do around the timed steps, without a GPU: rendezvous (gloo), reduce a timing
+    (max) and a unit count (sum), rank 0 prints one line.  Run by the CPU tests through the launcher above."""
+    import torch.distributed as dist
+    from paper_2609_34650_b200 import dist as sd
+    rank, _, world = sd.env_world()
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rate, ms = sd.whole_job_rate(100.0 * (rank + 1), 1.0 + rank)
+    dist.barrier()
+    if rank == 0:
+        print(json.dumps({"launcher_selftest": True, "n_gpus": world, "units_per_s": rate, "ms": ms}), flush=True)
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--repeats", type=int, default=5, help="how many times the K-step region is timed (median reported)")
+    ap.add_argument("--region-gap", type=float, default=0.3, help="idle seconds before each timed region")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 5, 6])
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 4, 5, 6])
     ap.add_argument("--no-fit", action="store_true", help="skip the extra legs that time the one-time fitter and the calibration statistics")
     ap.add_argument("--ref-budget", type=float, default=12.0, help="seconds of CPU-oracle work per sample")
+    ap.add_argument("--launcher-selftest", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.impl == "ours" and args.gpus > 1 and "RANK" not in os.environ:
+        launch_ranks(args, sys.argv[1:])
+    elif args.launcher_selftest:
+        launcher_selftest(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

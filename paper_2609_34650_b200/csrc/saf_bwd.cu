@@ -195,6 +195,9 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // the prologue above overlapped the previous kernel's tail; global memory is touched only from here on
+  pdl_launch_dependents();
+  pdl_wait();
   const int it_begin = p.cta_offsets[blockIdx.x], it_end = p.cta_offsets[blockIdx.x + 1];
 
   if (warp == 20) {
@@ -938,8 +941,8 @@ cudaError_t launch_bwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, cons
   if (D != 64) return cudaErrorNotSupported;
   cudaError_t e = cudaFuncSetAttribute(saf_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg::SMEM);
   if (e != cudaSuccess) return e;
-  saf_bwd_kernel<<<grid, BwdCfg::NTHREADS, BwdCfg::SMEM, st>>>(mq, mk, mv, mdo, mdq, mdot, mdk, mdv, p);
-  return cudaGetLastError();
+  return launch_pdl(PDL_BWD, saf_bwd_kernel, dim3(grid), dim3(BwdCfg::NTHREADS), BwdCfg::SMEM, st, mq, mk, mv, mdo,
+                    mdq, mdot, mdk, mdv, p);
 }
 
 }  // namespace saf

@@ -148,6 +148,9 @@ saf_bwd128_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // the prologue above overlapped the previous kernel's tail; global memory is touched only from here on
+  pdl_launch_dependents();
+  pdl_wait();
   const int it_begin = p.cta_offsets[blockIdx.x], it_end = p.cta_offsets[blockIdx.x + 1];
 
   if (warp == 20) {
@@ -615,8 +618,7 @@ cudaError_t launch_bwd128(const CUtensorMap& mk, const CUtensorMap& mv, const CU
   cudaError_t e =
       cudaFuncSetAttribute(saf_bwd128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, W128::SMEM);
   if (e != cudaSuccess) return e;
-  saf_bwd128_kernel<<<grid, W128::NTHREADS, W128::SMEM, st>>>(mk, mv, mqh, mdoh, mdoth, mdq, p);
-  return cudaGetLastError();
+  return launch_pdl(PDL_BWD, saf_bwd128_kernel, dim3(grid), dim3(W128::NTHREADS), W128::SMEM, st, mk, mv, mqh, mdoh, mdoth, mdq, p);
 }
 
 }  // namespace saf

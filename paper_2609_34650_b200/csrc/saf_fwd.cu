@@ -113,6 +113,9 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // the prologue above overlapped the previous kernel's tail; global memory is touched only from here on
+  pdl_launch_dependents();
+  pdl_wait();
 
   const int it_begin = p.cta_offsets[blockIdx.x], it_end = p.cta_offsets[blockIdx.x + 1];
 
@@ -599,9 +602,8 @@ cudaError_t launch_fwd(int D, const CUtensorMap& mq, const CUtensorMap& mk, cons
   } else {
     e = cudaFuncSetAttribute(saf_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128>::SMEM);
     if (e != cudaSuccess) return e;
-    saf_fwd_kernel<128><<<grid, 320, FwdCfg<128>::SMEM, st>>>(mq, mk, mv, mvt, p);
+    return launch_pdl(PDL_FWD, saf_fwd_kernel<128>, dim3(grid), dim3(320), FwdCfg<128>::SMEM, st, mq, mk, mv, mvt, p);
   }
-  return cudaGetLastError();
 }
 
 }  // namespace saf

@@ -167,6 +167,9 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // the prologue above overlapped the previous kernel's tail; global memory is touched only from here on
+  pdl_launch_dependents();
+  pdl_wait();
 
   const int it_begin = p.cta_offsets[blockIdx.x], it_end = p.cta_offsets[blockIdx.x + 1];
 
@@ -721,8 +724,7 @@ cudaError_t launch_fwd64(const CUtensorMap& mq, const CUtensorMap& mk, const CUt
   cudaError_t e =
       cudaFuncSetAttribute(saf_fwd64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Fwd64Cfg::SMEM);
   if (e != cudaSuccess) return e;
-  saf_fwd64_kernel<<<grid, Fwd64Cfg::NTHREADS, Fwd64Cfg::SMEM, st>>>(mq, mk, mv, mvt, mo, p);
-  return cudaGetLastError();
+  return launch_pdl(PDL_FWD, saf_fwd64_kernel, dim3(grid), dim3(Fwd64Cfg::NTHREADS), Fwd64Cfg::SMEM, st, mq, mk, mv, mvt, mo, p);
 }
 
 }  // namespace saf

@@ -6,6 +6,7 @@
 #include <mutex>
 
 #include "../../include/saf.h"
+#include "ptx.cuh"
 #include "saf_internal.h"
 
 namespace saf {
@@ -175,6 +176,8 @@ __global__ void __launch_bounds__(256) saf_scale_rows_kernel(const __nv_bfloat16
                                                              int call_id, __half* __restrict__ dst, int B, int Hf,
                                                              int T, int src_group, const PatternCheck chk) {
   constexpr int TPR = D / 8;
+  pdl_launch_dependents();
+  pdl_wait();                                      // (launched with programmatic stream serialization)
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
   const long long rowid = gid / TPR;               // over [B][Hf][T]: frozen heads only
   const int part = static_cast<int>(gid % TPR);
@@ -207,19 +210,20 @@ cudaError_t launch_scale_rows(const void* src, const int64_t* strides, const flo
                               int T, int D, int src_group, const PatternCheck& chk, cudaStream_t st) {
   const long long nthreads = static_cast<long long>(B) * Hf * T * (D / 8);
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
+  cudaError_t e;
   if (D == 96)
-    saf_scale_rows_kernel<96><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
+    e = launch_pdl(PDL_STAGE, saf_scale_rows_kernel<96>, dim3(grid), dim3(256), 0, st, static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
                                                     strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
                                                     static_cast<__half*>(dst), B, Hf, T, src_group, chk);
   else if (D == 64)
-    saf_scale_rows_kernel<64><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
+    e = launch_pdl(PDL_STAGE, saf_scale_rows_kernel<64>, dim3(grid), dim3(256), 0, st, static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
                                                     strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
                                                     static_cast<__half*>(dst), B, Hf, T, src_group, chk);
   else
-    saf_scale_rows_kernel<128><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
+    e = launch_pdl(PDL_STAGE, saf_scale_rows_kernel<128>, dim3(grid), dim3(256), 0, st, static_cast<const __nv_bfloat16*>(src), strides[0], strides[1],
                                                      strides[2], vec, extra, Tp, hlist, pat_ok, ovf, call_id,
                                                      static_cast<__half*>(dst), B, Hf, T, src_group, chk);
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // Three-way bf16 split of an fp32 value: hi + mid + lo reproduces x to ~24 bits.
@@ -256,6 +260,8 @@ __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat1
                                                            const int* __restrict__ qslot, int n_ord,
                                                            const PrepFrozen fz, int B, int H, int T) {
   const int Tpad = (T + 127) / 128 * 128;
+  pdl_launch_dependents();
+  pdl_wait();                                      // (launched with programmatic stream serialization)
   const long long gid = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
   const long long rowid = gid / TPR;               // over [B][H][Tpad]
   const int part = static_cast<int>(gid % TPR);
@@ -367,11 +373,12 @@ cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, con
   static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2], mask_dev, \
       static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext), inv_scale, dQacc, dK, dV, grad_f32, kv_group,   \
       qslot, n_ord, fz, B, H, T
-  if (D == 64) saf_bwd_prep_kernel<64, 8><<<grid, 256, 0, st>>>(SAF_PREP_ARGS);
-  else if (D == 96) saf_bwd_prep_kernel<96, 16><<<grid, 256, 0, st>>>(SAF_PREP_ARGS);
-  else saf_bwd_prep_kernel<128, 16><<<grid, 256, 0, st>>>(SAF_PREP_ARGS);
+  cudaError_t e;
+  if (D == 64) e = launch_pdl(PDL_PREP, saf_bwd_prep_kernel<64, 8>, dim3(grid), dim3(256), 0, st, SAF_PREP_ARGS);
+  else if (D == 96) e = launch_pdl(PDL_PREP, saf_bwd_prep_kernel<96, 16>, dim3(grid), dim3(256), 0, st, SAF_PREP_ARGS);
+  else e = launch_pdl(PDL_PREP, saf_bwd_prep_kernel<128, 16>, dim3(grid), dim3(256), 0, st, SAF_PREP_ARGS);
 #undef SAF_PREP_ARGS
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 __global__ void __launch_bounds__(256) saf_f32_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst,

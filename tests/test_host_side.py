@@ -158,3 +158,16 @@ def test_whole_job_rate_over_two_gloo_ranks(tmp_path):
     for r, p in enumerate(procs):
         out, _ = p.communicate(timeout=120)
         assert p.returncode == 0 and f"ok {r}" in out, out
+
+
+def test_bench_starts_its_own_ranks_when_not_under_torchrun():
+    """`bench.py --gpus 2` outside a torchrun environment must start two ranks itself and report n_gpus = 2; the
+    ranks here run the launcher's self-test (gloo rendezvous and the two reductions of the benchmark) instead of
+    GPU work."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--launcher-selftest"], env=env,
+                       stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, timeout=180)
+    assert r.returncode == 0, r.stderr
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["n_gpus"] == 2 and line["ms"] == 2.0 and abs(line["units_per_s"] - 300.0 / 2e-3) < 1e-6
