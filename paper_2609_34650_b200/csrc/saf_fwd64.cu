@@ -352,28 +352,26 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           const uint32_t sk = nk % C::NS;                 // stage of tile j+1's K (if any)
           const uint32_t acc0 = j > 0 ? 1u : 0u;
           // ---- group 0
-          ok = mbar_wait_warp(p_full, np0 & 1, wc, F_P_FULL);
-          if (!ok) break;
-          ++np0;
+          // the tiles' loads land long before P is ready: test their barriers first, so that only one test
+          // stands between "P is ready" and the MMAs that wait for it
           ok = mbar_wait_warp(v_full + sv, (nv / C::NS) & 1, wc, F_V_FULL);
           if (!ok) break;
           ++nv;
-          if (j == 0) {
-            ok = mbar_wait_warp(o_free, (nitem & 1) ^ 1, wc, F_O_FREE);
-            if (!ok) break;
-          }
-          tc_fence_after();
-          TRF(0, 1);
-          issue_pv(0, sv, acc0);
-          TRF(0, 2);
           if (more) {
             ok = mbar_wait_warp(k_full + sk, (nk / C::NS) & 1, wc, F_K_FULL);
             if (!ok) break;
             ++nk;
-            tc_fence_after();
-            issue_qk(0, sk);                              // executes after P V_0: same thread, in order
-            TRF(0, 3);
           }
+          if (j == 0) {
+            ok = mbar_wait_warp(o_free, (nitem & 1) ^ 1, wc, F_O_FREE);
+            if (!ok) break;
+          }
+          ok = mbar_wait_warp(p_full, np0 & 1, wc, F_P_FULL);
+          if (!ok) break;
+          ++np0;
+          tc_fence_after();
+          issue_pv(0, sv, acc0);
+          if (more) issue_qk(0, sk);                      // executes after P V_0: same thread, in order
           // ---- group 1
           ok = mbar_wait_warp(p_full + 1, np1 & 1, wc, F_P_FULL);
           if (!ok) break;
