@@ -27,6 +27,8 @@ struct WorklistEntry {
   std::vector<int> offsets_host;
   WorkItem* items_dev = nullptr;
   int* offsets_dev = nullptr;
+  WorkItem* order_dev = nullptr;          // the same items in queue order (kernels that take work dynamically)
+  std::vector<WorkItem> order_host;
   int n_items = 0;
 };
 
@@ -56,6 +58,7 @@ struct saf_ctx {
   int device = 0;
   int num_sms = 0;
   int* status_dev = nullptr;
+  int* queue_dev = nullptr;                // work-queue counters: {next item, CTAs done} per kernel that uses one
   cudaStream_t last_stream = nullptr;
   EncodeTiledFn encode = nullptr;
   unsigned long long wait_limit_ns = 2000000000ull;
@@ -226,7 +229,7 @@ int upload_mask(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st) {
 // queue would do); only the last items are ordered longest-first so that the tail stays short.
 void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward, int n_ctas, int frozen_pct,
                          int overhead_pct, int second_wave_pct, std::vector<WorkItem>& items,
-                         std::vector<int>& offsets) {
+                         std::vector<int>& offsets, std::vector<WorkItem>* order = nullptr) {
   const int nblk = (T + BLK - 1) / BLK;
   struct Cand { WorkItem w; long long cost; };
   std::vector<Cand> cand;
@@ -246,6 +249,11 @@ void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward,
   // the tail (about two items per CTA) longest-first
   const size_t tail = std::min(cand.size(), static_cast<size_t>(2) * n_ctas);
   std::stable_sort(cand.end() - tail, cand.end(), [](const Cand& a, const Cand& b) { return a.cost > b.cost; });
+  if (order) {
+    // the sequence itself is the work queue of the kernels that claim items at run time
+    order->clear();
+    for (const Cand& c : cand) order->push_back(c.w);
+  }
   typedef std::pair<long long, int> Load;   // (load, cta)
   std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
   for (int c = 0; c < n_ctas; ++c) heap.push({0, c});
@@ -290,6 +298,7 @@ int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int bac
     cudaStreamSynchronize(st);
     cudaFree(ctx->worklists.front().items_dev);
     cudaFree(ctx->worklists.front().offsets_dev);
+    cudaFree(ctx->worklists.front().order_dev);
     ctx->worklists.erase(ctx->worklists.begin());
   }
   std::vector<WorkItem> items;
@@ -301,14 +310,20 @@ int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int bac
   if (fw > 0) frozen_pct = fw;
   if (ov > 0) overhead_pct = ov;
   const int second_wave = backward ? 0 : (ctx->second_wave_pct >= 0 ? ctx->second_wave_pct : (wide ? 6 : 20));
-  build_worklist_host(B, H, T, mask, backward, grid, frozen_pct, overhead_pct, second_wave, items, offsets);
   WorklistEntry e;
+  build_worklist_host(B, H, T, mask, backward, grid, frozen_pct, overhead_pct, second_wave, items, offsets,
+                      &e.order_host);
   e.B = B; e.H = H; e.T = T; e.backward = backward; e.grid = grid; e.wide = wide;
   e.mask.assign(mask, mask + H);
   e.n_items = static_cast<int>(items.size());
   if (cudaMalloc(&e.items_dev, items.size() * sizeof(WorkItem)) != cudaSuccess) return SAF_ERR_NOMEM;
   if (cudaMalloc(&e.offsets_dev, offsets.size() * sizeof(int)) != cudaSuccess) {
     cudaFree(e.items_dev);
+    return SAF_ERR_NOMEM;
+  }
+  if (cudaMalloc(&e.order_dev, e.order_host.size() * sizeof(WorkItem)) != cudaSuccess) {
+    cudaFree(e.items_dev);
+    cudaFree(e.offsets_dev);
     return SAF_ERR_NOMEM;
   }
   // uploaded on the stream the kernel will run on (a non-blocking stream does not order with the legacy stream);
@@ -318,7 +333,10 @@ int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int bac
   if (cudaMemcpyAsync(e.items_dev, e.items_host.data(), e.items_host.size() * sizeof(WorkItem), cudaMemcpyHostToDevice,
                       st) != cudaSuccess ||
       cudaMemcpyAsync(e.offsets_dev, e.offsets_host.data(), e.offsets_host.size() * sizeof(int),
-                      cudaMemcpyHostToDevice, st) != cudaSuccess) {
+                      cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(e.order_dev, e.order_host.data(), e.order_host.size() * sizeof(WorkItem), cudaMemcpyHostToDevice,
+                      st) != cudaSuccess) {
+    cudaFree(e.order_dev);
     cudaFree(e.items_dev);
     cudaFree(e.offsets_dev);
     return SAF_ERR_CUDA;
@@ -413,6 +431,11 @@ int saf_create(saf_ctx** out, int device) {
     return SAF_ERR_CUDA;
   }
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (cudaMalloc(&ctx->queue_dev, 8 * sizeof(int)) != cudaSuccess ||
+      cudaMemset(ctx->queue_dev, 0, 8 * sizeof(int)) != cudaSuccess) {
+    delete ctx;
+    return SAF_ERR_NOMEM;
+  }
   if (cudaMalloc(&ctx->status_dev, sizeof(int)) != cudaSuccess || cudaMemset(ctx->status_dev, 0, sizeof(int)) != cudaSuccess) {
     delete ctx;
     return SAF_ERR_NOMEM;
@@ -454,6 +477,7 @@ int saf_destroy(saf_ctx* ctx) {
   for (WorklistEntry& e : ctx->worklists) {
     cudaFree(e.items_dev);
     cudaFree(e.offsets_dev);
+    cudaFree(e.order_dev);
   }
   DevBuf* pbufs[] = {&ctx->pat_consts, &ctx->pat_ok, &ctx->pat_avec, &ctx->pat_wvec, &ctx->pat_bandf, &ctx->pat_bandb,
                      &ctx->pat_hord, &ctx->pat_hlist, &ctx->pat_snap, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta, &ctx->fit_buf, &ctx->calib_tmp};
@@ -463,6 +487,7 @@ int saf_destroy(saf_ctx* ctx) {
                     &ctx->hlogz};
   for (DevBuf* b : bufs) release(*b);
   if (ctx->status_dev) cudaFree(ctx->status_dev);
+  if (ctx->queue_dev) cudaFree(ctx->queue_dev);
   if (ctx->hs_main) cudaStreamDestroy(ctx->hs_main);
   if (ctx->hs_copy) cudaStreamDestroy(ctx->hs_copy);
   if (ctx->hs_outs) cudaStreamDestroy(ctx->hs_outs);
@@ -643,6 +668,9 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   fp.LSE = LSE;
   fp.items = wl->items_dev;
   fp.cta_offsets = wl->offsets_dev;
+  fp.order = wl->order_dev;
+  fp.n_items = wl->n_items;
+  fp.queue = ctx->queue_dev;
   fp.status = ctx->status_dev;
   fp.wait_limit_ns = ctx->wait_limit_ns;
   fp.selftest_drop_load =

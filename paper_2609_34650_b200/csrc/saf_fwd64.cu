@@ -75,32 +75,41 @@ struct Fwd64Cfg {
   static constexpr int NFZ = 3;
   __host__ __device__ static constexpr int fz_v(int k) { return k < 2 ? OFF_V + k * TILE_BYTES : OFF_Q; }
   __host__ __device__ static constexpr int fz_band(int k) { return OFF_K + k * 4096; }
-  static constexpr int NBAR = 2 + 4 * NS + 2 + 2 + 2 + 1 + 2 * NFZ;
-  static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;   // + slack for 1024-byte alignment
+  // Work items are claimed at run time (atomic counter in global memory) by the producer thread, which hands them
+  // to the other roles through a ring of NRING records in shared memory.
+  static constexpr int NRING = 4;
+  static constexpr int NBAR = 2 + 4 * NS + 2 + 2 + 2 + 1 + 2 * NFZ + 2 * NRING;
+  static constexpr int OFF_RING = (OFF_BAR + NBAR * 8 + 16 + 15) / 16 * 16;   // int4 records (after the barriers, the TMEM slot
+                                                                // and the abort flag)
+  static constexpr int SMEM = OFF_RING + NRING * 16 + 1024;     // + slack for 1024-byte alignment
   static constexpr int TMEM_COLS = 256;
   static constexpr int COL_S = 0, COL_O = 128;          // + 64 g
   static constexpr int NTHREADS = 320;
 };
 
 enum Fwd64Site { F_Q_EMPTY = 41, F_K_EMPTY, F_V_EMPTY, F_Q_FULL, F_K_FULL, F_P_FULL, F_V_FULL, F_O_FREE, F_S_FULL,
-                 F_PV_DONE };
+                 F_PV_DONE, F_RING_EMPTY, F_RING_FULL };
 
-// Work item `it` and whether it takes the tensor-core frozen form, fetched one item ahead of its use.
+// A work item as the roles see it: the record of the scheduler's list plus whether a frozen item takes the
+// tensor-core form.  kind < 0 marks the end of the queue.
 struct ItemView64 {
   WorkItem w;
   bool fast;
 };
-__device__ __forceinline__ ItemView64 load_item64(const FwdParams& p, int it, int it_end) {
-  ItemView64 v;
-  v.w = WorkItem{0, 0, 0, KIND_ORDINARY};
-  v.fast = false;
-  if (it < it_end) {
-    const int4 raw = __ldg(reinterpret_cast<const int4*>(p.items + it));
-    v.w = WorkItem{raw.x, raw.y, raw.z, raw.w};
-    v.fast = raw.w != KIND_ORDINARY && p.band_f != nullptr && __ldg(p.fast_ok + raw.y) != 0 &&
-             __ldg(p.ovf + raw.y) != p.call_id;
-  }
-  return v;
+constexpr int RING_FAST = 1 << 8;
+constexpr int RING_END = -1;
+
+// Consumer side of the item ring (warp-uniform): wait for record n, copy it, release the slot at once (the copy is
+// all a role needs).  Returns false when the wait was abandoned.
+__device__ __forceinline__ bool ring_take(const int4* ring, uint64_t* ring_full, uint64_t* ring_empty, uint32_t n,
+                                          const WaitCtx& wc, ItemView64& v) {
+  const uint32_t slot = n % Fwd64Cfg::NRING;
+  if (!mbar_wait_warp(ring_full + slot, (n / Fwd64Cfg::NRING) & 1, wc, F_RING_FULL)) return false;
+  const int4 raw = ring[slot];
+  warp_arrive(ring_empty + slot);
+  v.w = WorkItem{raw.x, raw.y, raw.z, raw.w < 0 ? RING_END : (raw.w & 0xff)};
+  v.fast = raw.w >= 0 && (raw.w & RING_FAST) != 0;
+  return true;
 }
 
 }  // namespace
@@ -126,8 +135,11 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   uint64_t* o_free = pv_done + 2;
   uint64_t* fz_full = o_free + 1;                // [NFZ] band + scaled V tile of a tensor-core frozen tile
   uint64_t* fz_empty = fz_full + C::NFZ;         // [NFZ]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fz_empty + C::NFZ);
+  uint64_t* ring_full = fz_empty + C::NFZ;       // [NRING] record n has been published by the producer
+  uint64_t* ring_empty = ring_full + C::NRING;   // [NRING] issuer + 8 compute warps have copied it
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ring_empty + C::NRING);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int4* ring = reinterpret_cast<int4*>(smem + C::OFF_RING);
   float* tab = reinterpret_cast<float*>(smem + C::OFF_TAB);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -157,6 +169,10 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       mbar_init(fz_full + k, 1);
       mbar_init(fz_empty + k, 1);
     }
+    for (int k = 0; k < C::NRING; ++k) {
+      mbar_init(ring_full + k, 1);
+      mbar_init(ring_empty + k, 9);
+    }
     mbar_fence_init();
   }
   if (warp == 9) {
@@ -171,8 +187,6 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   pdl_launch_dependents();
   pdl_wait();
 
-  const int it_begin = p.cta_offsets[blockIdx.x], it_end = p.cta_offsets[blockIdx.x + 1];
-
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -183,11 +197,24 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       uint32_t nq = 0, nk = 0, nv = 0, nfz = 0;
       bool ok = true, fz_open = false;
       bool drop_load = p.selftest_drop_load != 0;        // self-test of the give-up path: see FwdParams
-      ItemView64 nxt = load_item64(p, it_begin, it_end);
-      for (int it = it_begin; it < it_end && ok; ++it) {
-        const WorkItem w = nxt.w;
-        const bool fast = nxt.fast;
-        nxt = load_item64(p, it + 1, it_end);
+      for (uint32_t nclaim = 0; ok; ++nclaim) {
+        // claim the next item of the queue and publish it to the other roles
+        const uint32_t slot = nclaim % C::NRING;
+        ok = mbar_wait(ring_empty + slot, ((nclaim / C::NRING) & 1) ^ 1, wc, F_RING_EMPTY);
+        if (!ok) break;
+        const int idx = atomicAdd(p.queue, 1);
+        int4 rec = make_int4(0, 0, 0, RING_END);
+        bool fast = false;
+        if (idx < p.n_items) {
+          rec = __ldg(reinterpret_cast<const int4*>(p.order + idx));
+          fast = rec.w != KIND_ORDINARY && p.band_f != nullptr && __ldg(p.fast_ok + rec.y) != 0 &&
+                 __ldg(p.ovf + rec.y) != p.call_id;
+          if (fast) rec.w |= RING_FAST;
+        }
+        ring[slot] = rec;
+        mbar_arrive(ring_full + slot);                   // (release: the record is visible to whoever sees the phase)
+        if (idx >= p.n_items) break;
+        const WorkItem w = WorkItem{rec.x, rec.y, rec.z, rec.w & 0xff};
         const int ntiles = w.blk + 1;
         if (fast) {
           // tensor-core form: per tile the Hankel band of distance block (I - J) and the scaled V tile, in a ring of
@@ -272,15 +299,14 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     // Hankel band: no-swizzle K-major, core matrices 128 bytes apart in both directions
     const uint64_t d_band = umma_smem_desc(sb, 128, 128, UMMA_LAYOUT_NONE);
     const uint32_t lo_b = desc_lo(d_band), hi_b = desc_hi(d_band);
-    ItemView64 nxt = load_item64(p, it_begin, it_end);
-    for (int it = it_begin; it < it_end && ok; ++it, ++nitem) {
-      const WorkItem w = nxt.w;
-      const bool fast = nxt.fast;
+    for (uint32_t nrec = 0; ok; ++nrec, ++nitem) {
+      ItemView64 cur;
+      ok = ring_take(ring, ring_full, ring_empty, nrec, wc, cur);
+      if (!ok || cur.w.kind == RING_END) break;
+      const WorkItem w = cur.w;
+      const bool fast = cur.fast;
       const int ntiles = w.blk + 1;
       const bool ord = w.kind == KIND_ORDINARY;
-      // The next record's load latency must not delay the item's first score MMAs: ordinary items fetch it once
-      // those are queued.
-      if (!ord) nxt = load_item64(p, it + 1, it_end);
       if (fast) {
         for (int j = 0; j < ntiles && ok; ++j) {
           const uint32_t k = nfz % C::NFZ;
@@ -345,7 +371,6 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           if (leader) umma_commit(k_empty + s);
           __syncwarp();
         }
-        nxt = load_item64(p, it + 1, it_end);
         for (int j = 0; j < ntiles && ok; ++j) {
           const uint32_t sv = nv % C::NS;
           const bool more = j + 1 < ntiles;
@@ -448,17 +473,23 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     (void)trr;
     // A compute warp whose wait was abandoned keeps walking (without storing) until the next
     // agreement barrier, where all eight leave together; none is ever left alone at a barrier.
-    ItemView64 nxt = load_item64(p, it_begin, it_end);
-    for (int it = it_begin; it < it_end; ++it) {
-      const WorkItem w = nxt.w;
-      const bool fast = nxt.fast;                        // (the next item is fetched under the epilogue's wait)
+    for (uint32_t nrec = 0;; ++nrec) {
+      ItemView64 cur;
+      if (!ring_take(ring, ring_full, ring_empty, nrec, wc, cur)) {
+        ok = false;                                      // keep walking to the agreement barrier below
+        cur.w = WorkItem{0, 0, 0, KIND_ORDINARY};
+        cur.fast = false;
+      }
+      const bool at_end = cur.w.kind == RING_END;
+      const WorkItem w = cur.w;
+      const bool fast = cur.fast;
       const int ntiles = w.blk + 1;
       int row = w.blk * BLK + rowl;
       // epilogue weights of the two accumulators and the common row factor
       float f0 = 1.0f, f1 = 1.0f, inv_l = 1.0f, lse = 0.0f;
       bool use1 = true;
       if (tid == 0) bulk_wait_group_read0();             // the previous item's O tile has left the staging tile
-      if (named_bar_or(5, 256, !ok)) break;
+      if (named_bar_or(5, 256, !ok) || at_end) break;    // (the end record reaches all eight warps alike)
       if (q4 == 0) TRF(trr, 19);
       if (fast) {
         // tensor-core form: nothing to do per tile; lane m holds query 127-m, scaled by w(i) below
@@ -648,7 +679,6 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (leave) break;
       }
       // ---------------- epilogue: wait for the last P V of both groups, merge, scale, store 32 columns each
-      nxt = load_item64(p, it + 1, it_end);              // its load latency passes under the wait for the last MMAs
       {
         const uint32_t par = npv & 1;
         if (!mbar_wait_warp(pv_done, par, wc, F_PV_DONE)) ok = false;
@@ -713,6 +743,15 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   __syncthreads();
   SAF_SPAN(fwd64, 1);
   if (warp == 9) tmem_dealloc(tmem, C::TMEM_COLS);
+  if (tid == 0) {
+    // this CTA claims nothing more; the last CTA to get here rewinds the queue for the next launch
+    __threadfence();
+    if (atomicAdd(p.queue + 1, 1) == static_cast<int>(gridDim.x) - 1) {
+      p.queue[0] = 0;
+      p.queue[1] = 0;
+      __threadfence();
+    }
+  }
 }
 
 int fwd64_smem_bytes() { return Fwd64Cfg::SMEM; }

@@ -78,6 +78,11 @@ struct FwdParams {
   int nblkp;
   const WorkItem* items;            // grouped by CTA
   const int* cta_offsets;           // [grid+1]
+  // D = 64 forward: the items in queue order, claimed at run time.  queue[0] = next unclaimed item, queue[1] = CTAs
+  // that have finished; the last CTA to finish sets both back to zero for the next launch.
+  const WorkItem* order;
+  int n_items;
+  int* queue;
   int* status;                      // device status word
   unsigned long long wait_limit_ns;
   // Self-test of the give-up path (0 in normal use): the producer of the D = 64 forward leaves out the load of the
