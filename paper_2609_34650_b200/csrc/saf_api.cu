@@ -870,9 +870,12 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
     };
+    // (the dQ boxes are 32 rows high: every drain warp reduces the rows of its own TMEM lane quarter)
+    box[1] = 32;
     if (!enc(&mdq, dqacc)) return SAF_ERR_CUDA;
-    mdk = mdq;
-    mdv = mdq;
+    box[1] = BLK;
+    if (!enc(&mdk, dqacc)) return SAF_ERR_CUDA;
+    mdv = mdk;
     // dK: like dQ when packed, else [B][H/kv_group][T][64]; dV: [B][H/kv_group][T][64]
     if (kern_f32 && p->packed_qk && nqh > 0 && !enc(&mdk, dK_k)) return SAF_ERR_CUDA;
     dims[2] = static_cast<cuuint64_t>(p->H / kvg);

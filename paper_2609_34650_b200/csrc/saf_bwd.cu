@@ -533,21 +533,27 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     const uint32_t lane_base = static_cast<uint32_t>(q4 * 32) << 16;
     uint32_t ndq = 0;
     bool ok = true;
-    const uint32_t stage_row = smem_u32(smem + C::OFF_DQ) + rowl * 128;
-    for (int it = it_begin; it < it_end; ++it) {
+    // Each drain warp moves the 32 query rows of its TMEM lane quarter on its own, through its own 4 KB of the staging
+    // area: TMEM -> registers -> [32 rows][32 floats] box (128-byte swizzle: 16-byte chunk index ^= row & 7) -> tiled
+    // TMA reduce-add, two boxes (feature halves) per tile.  A warp waits for its previous reduce-add to have read
+    // the box only when it is about to write it again, so four small reduce-adds are in flight per CTA while the
+    // warps stage the next ones (one 16 KB box per half, staged and reduced in turn by all four warps together,
+    // kept these warps busy 90 % of a tile's time: they, not the tensor pipe, set the tile period).
+    uint8_t* const my_box = smem + C::OFF_DQ + q4 * 4096;
+    const uint32_t my_row = smem_u32(my_box) + lane * 128;
+    (void)rowl;
+    for (int it = it_begin; it < it_end && ok; ++it) {
       const WorkItem w = p.items[it];
       if (w.kind != KIND_ORDINARY) continue;
       const int qh = p.qslot ? p.qslot[w.h] : w.h;       // head index in the dQ accumulator
-      bool leave = false;
       for (int I = w.blk; I < nblk; ++I) {
-        // the previous tile's reduce has finished reading the staging buffer (thread 512 waits for it
-        // before arriving here); the drain warps also agree here whether a wait has been abandoned
-        if (named_bar_or(2, 128, !ok)) {
-          leave = true;
+        TR(4 + warp, 40);
+        if (!mbar_wait_warp(dq_full, ndq & 1, wc, B_DQ_FULL)) {
+          ok = false;
           break;
         }
-        if (!mbar_wait_warp(dq_full, ndq & 1, wc, B_DQ_FULL)) ok = false;
         ++ndq;
+        TR(4 + warp, 41);
         tc_fence_after();
         uint32_t r0[32], r1[32];
         tmem_ld32(tmem + lane_base + C::COL_DQ, r0);
@@ -555,42 +561,31 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         tmem_wait_ld();
         tc_fence_before();
         warp_arrive(dq_free);                           // the tensor core may overwrite dQ
-        // fp32 rows -> one [128][32] box at a time, 128-byte swizzle (16-byte chunk index ^= row & 7)
+        const int row_first = I * BLK + 32 * q4;         // sequence position of this warp's first row
 #pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          const uint32_t chunk = static_cast<uint32_t>(g ^ (rowl & 7)) * 16;
-          st_shared_v4(stage_row + chunk, __float_as_uint(__uint_as_float(r0[4 * g]) * p.scale),
-                       __float_as_uint(__uint_as_float(r0[4 * g + 1]) * p.scale),
-                       __float_as_uint(__uint_as_float(r0[4 * g + 2]) * p.scale),
-                       __float_as_uint(__uint_as_float(r0[4 * g + 3]) * p.scale));
-        }
-        fence_proxy_async_smem();
-        named_bar_sync(3, 128);
-        if (tid == 512 && ok) {
-          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 0, I * BLK, qh, w.b);
-          bulk_commit_group();
-          bulk_wait_group_read0();
-        }
-        named_bar_sync(6, 128);                         // the first box has been read
+        for (int box = 0; box < 2; ++box) {
+          if (lane == 0) bulk_wait_group_read0();       // this warp's previous reduce-add has read the box
+          __syncwarp();
+          const uint32_t* r = box ? r1 : r0;
 #pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          const uint32_t chunk = static_cast<uint32_t>(g ^ (rowl & 7)) * 16;
-          st_shared_v4(stage_row + chunk, __float_as_uint(__uint_as_float(r1[4 * g]) * p.scale),
-                       __float_as_uint(__uint_as_float(r1[4 * g + 1]) * p.scale),
-                       __float_as_uint(__uint_as_float(r1[4 * g + 2]) * p.scale),
-                       __float_as_uint(__uint_as_float(r1[4 * g + 3]) * p.scale));
+          for (int g = 0; g < 8; ++g) {
+            const uint32_t chunk = static_cast<uint32_t>(g ^ (lane & 7)) * 16;
+            st_shared_v4(my_row + chunk, __float_as_uint(__uint_as_float(r[4 * g]) * p.scale),
+                         __float_as_uint(__uint_as_float(r[4 * g + 1]) * p.scale),
+                         __float_as_uint(__uint_as_float(r[4 * g + 2]) * p.scale),
+                         __float_as_uint(__uint_as_float(r[4 * g + 3]) * p.scale));
+          }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0 && row_first < p.T) {           // (rows beyond T inside the box are clipped by the map)
+            tma_reduce_add_4d(&mdq, my_box, 32 * box, row_first, qh, w.b);
+            bulk_commit_group();
+          }
         }
-        fence_proxy_async_smem();
-        named_bar_sync(3, 128);
-        if (tid == 512 && ok) {
-          tma_reduce_add_4d(&mdq, smem + C::OFF_DQ, 32, I * BLK, qh, w.b);
-          bulk_commit_group();
-          bulk_wait_group_read0();
-        }
+        TR(4 + warp, 42);
       }
-      if (leave) break;
     }
-    if (tid == 512) bulk_wait_group0();                 // all reduce-adds have landed before the kernel ends
+    if (lane == 0) bulk_wait_group0();                  // the reduce-adds have landed before the kernel ends
   } else {
     // ------------------------------------------------------------------ compute groups (2 x 256 threads)
     // warp = 8 grp + 4 sub + q4: two warps per TMEM lane quarter, `sub` picks the 32-column half
