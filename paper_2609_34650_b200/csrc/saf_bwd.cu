@@ -81,7 +81,7 @@ struct BwdCfg {
   __host__ __device__ static constexpr int fz_do(int k) { return (k < 2 ? OFF_DO : OFF_Q) + (k & 1) * PANEL; }
   __host__ __device__ static constexpr int fz_band(int k) { return (k < 2 ? OFF_QX : OFF_DOX) + (k & 1) * 4096; }
   static constexpr int NFZ = 4;                       // ring depth of the tensor-core frozen form (see the producer)
-  static constexpr int NBAR = 4 + 2 * NS + 2 + 2 + 4 + 2 + 1 + 2 * NFZ + 2;
+  static constexpr int NBAR = 4 + 2 * NS + 2 + 2 + 4 + 2 + 1 + 2 * NFZ + 2 + 2;
   static constexpr int SMEM = OFF_BAR + NBAR * 8 + 16 + 1024;
   static constexpr int TMEM_COLS = 512;
   static constexpr int COL_DV = 0, COL_DK = 64, COL_S = 128, COL_DP = 256, COL_DQ = 384, COL_KT = 448, COL_VT = 480;
@@ -141,7 +141,11 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
   uint64_t* fz_full = kvt_full + 1;              // [NFZ] band + scaled dO tile of a tensor-core frozen tile
   uint64_t* fz_empty = fz_full + C::NFZ;         // [NFZ]
   uint64_t* s_full = fz_empty + C::NFZ;          // [2] S'^T of buffer b is complete (dP'^T follows: sdp_full)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 2);
+  // [2] ordinary tiles: group b has written P^T / dS^T of its half tile.  The barrier of buffer 1 also counts the four
+  // drain warps, which arrive once they have read the previous tile's dQ out of TMEM: the issuer's one wait in front
+  // of a tile's second half then covers the accumulator that the tile's dQ MMAs (issued behind it) overwrite.
+  uint64_t* pds_ord = s_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pds_ord + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -164,6 +168,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
       mbar_init(s_full + b, 1);
       mbar_init(pds_full + b, 8);                // one arrival per warp of the group
       mbar_init(pfree + b, 1);
+      mbar_init(pds_ord + b, b == 0 ? 8 : 12);
     }
     mbar_init(kvt_full, 16);
     for (int k = 0; k < C::NFZ; ++k) {
@@ -385,13 +390,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
 #pragma unroll
           for (int b = 0; b < 2; ++b) {
             TR(0, 4);
-            if (b == 0) {
-              ok = mbar_wait_warp(pds_full, npds0 & 1, wc, B_PDS_FULL);
-              ++npds0;
-            } else {
-              ok = mbar_wait_warp(pds_full + 1, npds1 & 1, wc, B_PDS_FULL);
-              ++npds1;
-            }
+            ok = mbar_wait_warp(pds_ord + b, ntile_ord & 1, wc, B_PDS_FULL);
             if (!ok) break;
             TR(0, 5);
             if (t == 0 && b == 0) {
@@ -412,37 +411,27 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
                 umma_ts2(tmem + C::COL_DV, t_p + 8 * kc + (kc >= 2 ? 16 : 0), do_lo + 128 * kc, hi_m, id_acc,
                          (kc > 0 || b > 0) ? 1u : acc0);
               if (more) issue_S(2 * t + 2 + b);
-            }
-            __syncwarp();
-            TR(0, 10 + b);
-          }
-          if (!ok) break;
-          if (leader) {
-#pragma unroll
-            for (int b = 0; b < 2; ++b) {
+              // dK of this half tile and the buffer's next dP'^T follow at once (rather than after the other buffer's
+              // dV and S'^T): the second group's scores are then issued a good 700 clk after the first group's, which
+              // keeps the two groups' exponential phases apart - in phase, they halve each other's rate on the
+              // 16-per-clock special-function unit
               const uint32_t q_lo = lo_m + ((C::OFF_Q + s * C::PANEL + b * 8192) >> 4);
               const uint32_t t_ds = tmem + C::COL_DP + 64 * b;
 #pragma unroll
               for (int kc = 0; kc < 4; ++kc)
                 umma_ts2(tmem + C::COL_DK, t_ds + 8 * kc + (kc >= 2 ? 16 : 0), q_lo + 128 * kc, hi_m, id_acc,
                          (kc > 0 || b > 0) ? 1u : acc0);
+              // full tile done: its Q/dO stage can be refilled
+              if (b == 1) umma_commit(qdo_empty + s);
+              if (more) issue_dP(2 * t + 2 + b);
             }
-            // full tile done: its Q/dO stage can be refilled (ahead of the next dP'^T, which read the other stage,
-            // so that the refill starts ten MMAs earlier), and dQ of the tile follows
-            umma_commit(qdo_empty + s);
-            if (more) {
-              issue_dP(2 * t + 2);
-              issue_dP(2 * t + 3);
-            }
+            __syncwarp();
+            TR(0, 10 + b);
           }
+          if (!ok) break;
           __syncwarp();
           TR(0, 6);
-          ok = mbar_wait_warp(dq_free, (ndq & 1) ^ 1, wc, B_DQ_FREE);
-          if (!ok) break;
-          ++ndq;
-          TR(0, 12);
-          tc_fence_after();
-          TR(0, 13);
+          // (no wait for the dQ accumulator: the drain warps' arrivals were part of this tile's pds_ord[1] phase)
           const uint32_t ds_lo = lo_m + ((C::OFF_DS + (ntile_ord & 1) * 2 * C::PANEL) >> 4);
           if (leader) {
 #pragma unroll
@@ -533,6 +522,9 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     const uint32_t lane_base = static_cast<uint32_t>(q4 * 32) << 16;
     uint32_t ndq = 0;
     bool ok = true;
+#ifdef SAF_TRACE
+    int tr_n = 0;
+#endif
     // Each drain warp moves the 32 query rows of its TMEM lane quarter on its own, through its own 4 KB of the staging
     // area: TMEM -> registers -> [32 rows][32 floats] box (128-byte swizzle: 16-byte chunk index ^= row & 7) -> tiled
     // TMA reduce-add, two boxes (feature halves) per tile.  A warp waits for its previous reduce-add to have read
@@ -542,6 +534,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
     uint8_t* const my_box = smem + C::OFF_DQ + q4 * 4096;
     const uint32_t my_row = smem_u32(my_box) + lane * 128;
     (void)rowl;
+    warp_arrive(pds_ord + 1);                           // the first tile finds the dQ accumulator free
     for (int it = it_begin; it < it_end && ok; ++it) {
       const WorkItem w = p.items[it];
       if (w.kind != KIND_ORDINARY) continue;
@@ -560,7 +553,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         tmem_ld32(tmem + lane_base + C::COL_DQ + 32, r1);
         tmem_wait_ld();
         tc_fence_before();
-        warp_arrive(dq_free);                           // the tensor core may overwrite dQ
+        warp_arrive(pds_ord + 1);                       // the tensor core may overwrite dQ (counted in the next tile's phase)
         const int row_first = I * BLK + 32 * q4;         // sequence position of this warp's first row
 #pragma unroll
         for (int box = 0; box < 2; ++box) {
@@ -722,7 +715,7 @@ saf_bwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
           tmem_wait_st();
           fence_proxy_async_smem();
           tc_fence_before();
-          warp_arrive(pds_full + grp);
+          warp_arrive(pds_ord + grp);
           TR(4 + warp, 16);
         }
         ntile_ord += ntiles;
