@@ -478,7 +478,11 @@ def run_ours(args):
             kw = dict(c=ctx_s, al=al_s, rh=rh_s, lz=lz_s)
             for _ in range(3):
                 step(m, **kw)
-            t = float(np.median([timed(m, reps, **kw) for _ in range(3)]))
+            ts = []
+            for _ in range(3):
+                time.sleep(args.region_gap)                  # burst regions, as for the headline
+                ts.append(timed(m, reps, **kw))
+            t = float(np.median(ts))
             tf = wls.flops() / (t * 1e-3) / 1e12
             sweep.append({"frozen_heads": nf, "frozen_fraction": nf / wl.H, "ms_per_step": t, "tflops": tf})
         code, detail = ctx_s.saf_last_device_status()
