@@ -629,6 +629,9 @@ def run_ours(args):
                    "region_gap_s": args.region_gap,
                    "parallelism": f"dp{world} (independent batches, no collective in the layer)"},
         "pct_of_bf16_peak": 100.0 * value / (peaks["bf16_tflops"] * world),
+        # (context: the same against the sustained, power-capped peak, which long regions run into)
+        "pct_of_bf16_peak_sustained": (100.0 * value / (peaks["bf16_tflops_sustained"] * world)
+                                       if peaks.get("bf16_tflops_sustained") else None),
         "ms_per_step_with_kernel_events": ms_events,
         "speedup_vs_0pct_frozen": speedup, "aa_control": aa_control, "aa_attempts": aa_attempt,
         "aa_within_1pct": aa_ok,
