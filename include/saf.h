@@ -62,7 +62,9 @@ typedef struct {
                                   kv_group <= 1.  Not available through saf_hybrid_attn_step_host. */
   int32_t reserved;
   int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3]; /* elements: batch, head, seq */
-} saf_problem;                 /* dO uses o_strides; O is bf16; LSE [B][H][T], dQ [B][H][T][D] and dK, dV
+} saf_problem;                 /* dO uses o_strides; O is bf16 only (there is no fp32-O option: the backward's
+                                  row term sum(dO*O) is taken from the stored bf16 O, which is why the parity tests
+                                  feed the reference the same rounded O when T < 8); LSE [B][H][T], dQ [B][H][T][D] and dK, dV
                                   [B][H/kv_group][T][D] are contiguous (packed_qk: dQ, dK [B][Ho][T][D]) */
 
 /* Library version (major*100 + minor). */
@@ -183,7 +185,7 @@ int saf_fit_marginals(saf_ctx* ctx, int32_t Hf, int32_t T, const float* mean_att
  *   eta_abs, eta_rel : device float64 [Hf, T] (from saf_fit_marginals, or accumulated by the caller)
  *   plogp            : device float64 [Hf] or NULL if kl_out is NULL
  *   alpha_out, rho_out, logZ_out : device float32, row h at offset h*out_stride (out_stride >= T elements): the
- *                      fitted parameters and log Z(i) of Eq. "compact-prior", as saf_attn_fwd takes them
+ *                      fitted parameters and log Z(i) of Eq. "compact-prior", as saf_pattern_prepare takes them
  *   loss_out         : device float64 [Hf] or NULL: L at the fitted parameters
  *   kl_out           : device float64 [Hf] or NULL: kappa = mean row KL(P || P^) = L + plogp/T; the paper accepts a
  *                      head when kappa <= 0.2 nats (the caller compares)

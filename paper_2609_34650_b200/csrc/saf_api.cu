@@ -167,7 +167,7 @@ int validate(const saf_problem* p, const uint8_t* mask, int* n_frozen) {
   if (!p || !mask) return SAF_ERR_INVALID_ARG;
   if (p->B < 1 || p->H < 1 || p->T < 1 || p->Tp < 1) return SAF_ERR_INVALID_ARG;
   if (p->T > p->Tp) return SAF_ERR_INVALID_ARG;
-  if (p->D != 64 && p->D != 96 && p->D != 128) return SAF_ERR_UNSUPPORTED;   // 96: forward only
+  if (p->D != 64 && p->D != 96 && p->D != 128) return SAF_ERR_UNSUPPORTED;   // 96 runs padded on the 128-wide kernels
   if (p->grad_dtype != SAF_F32 && p->grad_dtype != SAF_BF16) return SAF_ERR_UNSUPPORTED;
   if (p->kv_group < 0 || (p->kv_group > 1 && p->H % p->kv_group != 0)) return SAF_ERR_INVALID_ARG;
   if (p->packed_qk && p->kv_group > 1) return SAF_ERR_INVALID_ARG;
