@@ -1,6 +1,7 @@
 // Host side of the C ABI: argument validation, context (workspace, cached work lists, device status
 // word), TMA tensor maps, the head scheduler and the launches.
 #include <algorithm>
+#include <array>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -84,7 +85,10 @@ struct saf_ctx {
   PatternCache pat;
   bool tensor_pattern = true;              // SAF_DISABLE_TENSOR_PATTERN=1 turns the form off
   bool selftest_drop_load = false;         // SAF_SELFTEST_DROP_LOAD=1: see FwdParams::selftest_drop_load
-  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, pat_snap, vt_buf, dot_buf, ok_fwd, ok_bwd, pg_hlist, pg_delta, fit_buf, calib_tmp;
+  DevBuf pat_consts, pat_ok, pat_avec, pat_wvec, pat_bandf, pat_bandb, pat_hord, pat_hlist, pat_snap, vt_buf, dot_buf, ok_fwd, ok_bwd, pg_hlist, pg_delta, pg_items, pg_offsets, fit_buf, calib_tmp;
+  std::vector<int> pg_hlist_host, pg_offsets_host;   // host copies of the pattern-gradient tables (upload sources)
+  std::vector<PgItem> pg_items_host;
+  std::array<int, 5> pg_key = {0, 0, 0, 0, 0};      // (B, frozen heads, T, D, grid) the work list was built for
   bool profiling = false;
   std::vector<TimedLaunch> timed;          // event pairs recorded since the last query
   std::vector<cudaEvent_t> event_pool;
@@ -480,7 +484,7 @@ int saf_destroy(saf_ctx* ctx) {
     cudaFree(e.order_dev);
   }
   DevBuf* pbufs[] = {&ctx->pat_consts, &ctx->pat_ok, &ctx->pat_avec, &ctx->pat_wvec, &ctx->pat_bandf, &ctx->pat_bandb,
-                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->pat_snap, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta, &ctx->fit_buf, &ctx->calib_tmp};
+                     &ctx->pat_hord, &ctx->pat_hlist, &ctx->pat_snap, &ctx->vt_buf, &ctx->dot_buf, &ctx->ok_fwd, &ctx->ok_bwd, &ctx->pg_hlist, &ctx->pg_delta, &ctx->pg_items, &ctx->pg_offsets, &ctx->fit_buf, &ctx->calib_tmp};
   for (DevBuf* b : pbufs) release(*b);
   DevBuf* bufs[] = {&ctx->mask_buf, &ctx->logz_buf, &ctx->delta_buf, &ctx->dqacc_buf, &ctx->dkacc_buf, &ctx->dvacc_buf, &ctx->qslot_buf, &ctx->hq, &ctx->hk, &ctx->hv,
                     &ctx->hdo, &ctx->ho, &ctx->hlse, &ctx->hdq, &ctx->hdk, &ctx->hdv, &ctx->halpha, &ctx->hrho,
@@ -1072,27 +1076,69 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
   std::vector<int> hlist;
   for (int h = 0; h < p->H; ++h)
     if (frozen_mask_host[h]) hlist.push_back(h);
+  const void* const hlist_dev_before = ctx->pg_hlist.ptr;
   if ((rc = ensure(ctx->pg_hlist, static_cast<size_t>(p->H) * sizeof(int))) ||
       (rc = ensure(ctx->pg_delta, static_cast<size_t>(p->B) * p->H * p->T * sizeof(float))))
     return rc;
-  // (synchronous copy from pageable memory: the vector dies at the end of this call)
-  if (cudaStreamSynchronize(st) != cudaSuccess ||
-      cudaMemcpy(ctx->pg_hlist.ptr, hlist.data(), hlist.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
-    return SAF_ERR_CUDA;
+  if (ctx->pg_hlist.ptr != hlist_dev_before) ctx->pg_hlist_host.clear();   // a new buffer holds nothing yet
+  // The tables are uploaded on the caller's stream from vectors the context owns, and only when they change (an
+  // earlier launch may still be reading the device copy: stream order keeps the two apart).
+  if (hlist != ctx->pg_hlist_host) {
+    ctx->pg_hlist_host = hlist;
+    if (cudaMemcpyAsync(ctx->pg_hlist.ptr, ctx->pg_hlist_host.data(), hlist.size() * sizeof(int), cudaMemcpyHostToDevice,
+                        st) != cudaSuccess)
+      return SAF_ERR_CUDA;
+  }
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_PREP, st);
     if (launch_rowdot(O, dO, p->o_strides, static_cast<const int*>(ctx->pg_hlist.ptr),
                       static_cast<float*>(ctx->pg_delta.ptr), p->B, p->H, nf, p->T, p->D, st) != cudaSuccess)
       return SAF_ERR_CUDA;
   }
-  // work list over (batch, frozen-head ordinal, key block), all of one kind
+  // Work list: (frozen-head ordinal, key block J, run of query blocks, run of batch entries), cut so that there are
+  // about four items per CTA, dealt longest first to the least loaded CTA.
   const int nblk = (p->T + BLK - 1) / BLK;
-  const long long n_items = static_cast<long long>(p->B) * nf * nblk;
-  const int grid = static_cast<int>(std::min<long long>(2LL * ctx->num_sms, n_items));
-  std::vector<uint8_t> none(nf, 0);
-  const WorklistEntry* wl = nullptr;
-  rc = get_worklist(ctx, p->B, nf, p->T, none.data(), 1, grid, p->D != 64, st, &wl);
-  if (rc) return rc;
+  const int vb = pgrad_batch_chunk(p->D);
+  const int nbc = (p->B + vb - 1) / vb;
+  const long long total_tiles = static_cast<long long>(nf) * nbc * nblk * (nblk + 1) / 2;
+  const int grid = static_cast<int>(std::min<long long>(ctx->num_sms, total_tiles));
+  const std::array<int, 5> key = {p->B, nf, p->T, p->D, grid};
+  if (key != ctx->pg_key) {
+    const int run = static_cast<int>(std::max<long long>(1, std::min<long long>(8, total_tiles / (4LL * grid))));
+    std::vector<PgItem> items;
+    for (int hf = 0; hf < nf; ++hf)
+      for (int c = 0; c < nbc; ++c)
+        for (int J = 0; J < nblk; ++J)
+          for (int I0 = J; I0 < nblk; I0 += run)
+            items.push_back(PgItem{hf, J, I0, std::min(nblk, I0 + run), c * vb, std::min(p->B, (c + 1) * vb), 0, 0});
+    // cost of an item in tile loads: its dO tiles plus the V tile
+    auto cost = [](const PgItem& w) { return (w.I1 - w.I0) + 1; };
+    std::stable_sort(items.begin(), items.end(), [&](const PgItem& a, const PgItem& b) { return cost(a) > cost(b); });
+    std::vector<std::vector<PgItem>> per_cta(grid);
+    std::priority_queue<std::pair<long long, int>, std::vector<std::pair<long long, int>>, std::greater<>> load;
+    for (int c = 0; c < grid; ++c) load.push({0, c});
+    for (const PgItem& w : items) {
+      auto [l, c] = load.top();
+      load.pop();
+      per_cta[c].push_back(w);
+      load.push({l + cost(w), c});
+    }
+    ctx->pg_items_host.clear();
+    ctx->pg_offsets_host.assign(1, 0);
+    for (int c = 0; c < grid; ++c) {
+      ctx->pg_items_host.insert(ctx->pg_items_host.end(), per_cta[c].begin(), per_cta[c].end());
+      ctx->pg_offsets_host.push_back(static_cast<int>(ctx->pg_items_host.size()));
+    }
+    if ((rc = ensure(ctx->pg_items, ctx->pg_items_host.size() * sizeof(PgItem))) ||
+        (rc = ensure(ctx->pg_offsets, ctx->pg_offsets_host.size() * sizeof(int))))
+      return rc;
+    if (cudaMemcpyAsync(ctx->pg_items.ptr, ctx->pg_items_host.data(), ctx->pg_items_host.size() * sizeof(PgItem),
+                        cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ctx->pg_offsets.ptr, ctx->pg_offsets_host.data(), ctx->pg_offsets_host.size() * sizeof(int),
+                        cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return SAF_ERR_CUDA;
+    ctx->pg_key = key;
+  }
   CUtensorMap mv, mdo;
   if ((rc = make_map(ctx, &mv, V, p, p->v_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg))) return rc;
   if ((rc = make_map(ctx, &mdo, dO, p, p->o_strides))) return rc;
@@ -1104,8 +1150,8 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
   gp.hlist = static_cast<const int*>(ctx->pg_hlist.ptr);
   gp.dalpha = dalpha_out;
   gp.drho = drho_out;
-  gp.items = wl->items_dev;
-  gp.cta_offsets = wl->offsets_dev;
+  gp.items = static_cast<const PgItem*>(ctx->pg_items.ptr);
+  gp.cta_offsets = static_cast<const int*>(ctx->pg_offsets.ptr);
   gp.status = ctx->status_dev;
   gp.wait_limit_ns = ctx->wait_limit_ns;
   {

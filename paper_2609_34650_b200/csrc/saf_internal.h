@@ -125,17 +125,24 @@ struct BwdParams {
 };
 
 // Gradients of the compact patterns (saf_pgrad.cu).  Items carry the head's ordinal among the frozen heads.
+// One unit of work of the pattern-gradient kernel: key block J of frozen head number hf (ordinal among the frozen
+// heads), query blocks I0 .. I1-1, accumulated over batch entries b0 .. b1-1 on the tensor core.
+struct PgItem {
+  int hf, J, I0, I1, b0, b1, pad0, pad1;
+};
+// Batch entries whose V tile stays in shared memory for the length of an item (the item's batch range is at most this).
+inline int pgrad_batch_chunk(int D) { return D == 64 ? 8 : 4; }
 struct PgradParams {
   int B, H, T, Tp;
   int kv_group;
   const float* alpha;               // [H][Tp]
   const float* rho;
   const float* logZ;
-  const float* delta;               // [B][H][T]: rowsum(dO o O), rows of frozen heads only
+  const float* delta;               // [batch chunks][H][T]: rowsum(dO o O) summed over a chunk, frozen heads only
   const int* hlist;                 // ordinal -> head
   float* dalpha;                    // [H][Tp], zeroed before the launch; accumulated with atomicAdd
   float* drho;
-  const WorkItem* items;
+  const PgItem* items;
   const int* cta_offsets;
   int* status;
   unsigned long long wait_limit_ns;

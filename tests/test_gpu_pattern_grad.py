@@ -70,8 +70,17 @@ def test_pattern_grads_head_dim_96():
     _check(L)
 
 
+@pytest.mark.parametrize("B,D", [(9, 64), (19, 64), (5, 128), (6, 96)])
+def test_pattern_grads_batch_larger_than_the_resident_chunk(B, D):
+    """The batch sum runs inside the contraction over at most 8 (D = 64) or 4 (wider heads) entries whose V tiles stay
+    in shared memory; larger batches are cut into several such runs, the last one shorter."""
+    wl = si.Workload("pgB", B, 2, 333, D, (1,), -0.02, seed=75 + B, backward=False)
+    L = Layer(si.generate(wl), backward=False).run(backward=False)
+    _check(L)
+
+
 def test_pattern_grads_many_items_per_cta():
-    """8 x 6 frozen heads x 9 key blocks = 432 items on 296 CTAs, ragged last block."""
+    """6 frozen heads x 9 key blocks with up to 9 query blocks each on 148 CTAs, ragged last block."""
     wl = si.Workload("pgmix", 8, 8, 1100, 64, (0, 2, 3, 5, 6, 7), -0.01, seed=73)
     L = Layer(si.generate(wl), backward=False).run(backward=False)
     _check(L)
