@@ -13,7 +13,7 @@
  * Conventions (all entry points):
  *   - "dev" pointers are device pointers owned by the caller; "host" pointers are host pointers.
  *     The library never frees or reallocates caller memory.
- *   - Q, K, V, O, dO are bf16 tensors indexed [b][h][t][c] through element strides (c has stride 1);
+ *   - Q, K, V, dO and (unless saf_problem.o_dtype says fp32) O are bf16 tensors indexed [b][h][t][c] through element strides (c has stride 1);
  *     base addresses and strides must be multiples of 8 elements (16 bytes).
  *   - frozen_mask_host is a host array uint8[H]; nonzero = frozen head.  It is read (copied) before the call
  *     returns, whatever kind of host memory it lives in.
@@ -60,11 +60,13 @@ typedef struct {
   int32_t packed_qk;           /* nonzero: Q, K, dQ, dK carry only the ordinary heads, in head order (Appendix E.2:
                                   replaced heads have no query/key slot on the multi-head path); needs
                                   kv_group <= 1.  Not available through saf_hybrid_attn_step_host. */
-  int32_t reserved;
+  int32_t o_dtype;             /* dtype of O: SAF_BF16 (0, the default) or SAF_F32.  dO stays bf16 and uses the same
+                                  element strides.  SAF_F32 is not available through saf_hybrid_attn_step_host. */
   int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3]; /* elements: batch, head, seq */
-} saf_problem;                 /* dO uses o_strides; O is bf16 only (there is no fp32-O option: the backward's
-                                  row term sum(dO*O) is taken from the stored bf16 O, which is why the parity tests
-                                  feed the reference the same rounded O when T < 8); LSE [B][H][T], dQ [B][H][T][D] and dK, dV
+} saf_problem;                 /* dO uses o_strides (elements; o_strides must be multiples of 8 in both cases);
+                                  with bf16 O the backward's row term sum(dO*O) is taken from the rounded O (the
+                                  parity tests feed the reference the same rounded O when T < 8), with fp32 O from
+                                  the unrounded one; LSE [B][H][T], dQ [B][H][T][D] and dK, dV
                                   [B][H/kv_group][T][D] are contiguous (packed_qk: dQ, dK [B][Ho][T][D]) */
 
 /* Library version (major*100 + minor). */
@@ -119,7 +121,7 @@ int saf_pattern_logz_static(int32_t device, int32_t H, int32_t Tp, const uint8_t
  *   Q, K, V : device bf16, strided as in `p`.
  *   logZ    : device fp32 [H][Tp] from saf_pattern_prepare, or NULL to have it computed into
  *             context-owned memory on every call (slower).
- *   O       : device bf16, strided by p->o_strides, every head in its original slot.
+ *   O       : device bf16 (fp32 with p->o_dtype = SAF_F32), strided by p->o_strides, every head in its original slot.
  *   LSE     : device fp32 [B][H][T]; natural-log sum of exp of the scaled causal scores for ordinary
  *             heads, 0 for frozen heads (they have no softmax).  May be NULL if every head is frozen. */
 int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const void* K, const void* V,
@@ -155,7 +157,8 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
  * With b_ij = alpha(j) + rho(i-j), P^ = softmax_causal(b), O = P^ V and L = sum(O o dO):
  *   G = dO V^T,  dL/db_ij = P^_ij (G_ij - dO_i . O_i),
  *   dalpha_out[h][j] = sum_b sum_{i>=j} dL/db_ij,   drho_out[h][d] = sum_b sum_{i-j=d} dL/db_ij.
- * V: bf16 [B][H/kv_group][T][D] (v_strides); O, dO: bf16 [B][H][T][D] (o_strides), O as returned by the forward;
+ * V: bf16 [B][H/kv_group][T][D] (v_strides); O (p->o_dtype), dO (bf16): [B][H][T][D] (o_strides), O as returned by the
+ * forward;
  * alpha, rho, logZ: device fp32 [H][Tp] (logZ as from saf_pattern_prepare); dalpha_out, drho_out: device fp32
  * [H][Tp], fully overwritten (rows of ordinary heads and entries beyond T with zeros).
  * After an update of alpha/rho the caller refreshes logZ with saf_pattern_prepare. */

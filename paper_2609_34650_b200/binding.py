@@ -24,7 +24,7 @@ SAF_KERNEL_PGRAD, SAF_KERNEL_FIT, SAF_KERNEL_FIT_MARGINALS, SAF_KERNEL_CALIB, SA
 class SafProblem(C.Structure):
     _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("T", C.c_int32), ("D", C.c_int32), ("Tp", C.c_int32),
                 ("softmax_scale", C.c_float), ("grad_dtype", C.c_int32), ("kv_group", C.c_int32),
-                ("packed_qk", C.c_int32), ("reserved", C.c_int32),
+                ("packed_qk", C.c_int32), ("o_dtype", C.c_int32),
                 ("q_strides", C.c_int64 * 3), ("k_strides", C.c_int64 * 3), ("v_strides", C.c_int64 * 3),
                 ("o_strides", C.c_int64 * 3)]
 
@@ -125,7 +125,7 @@ def saf_pattern_logz_static(device, mask, alpha, rho, logZ_out):
 
 
 def make_problem(q_like, Tp, softmax_scale=0.0, grad_dtype=SAF_F32, k_like=None, v_like=None, o_like=None,
-                 kv_group=1, packed_qk=False, H=None):
+                 kv_group=1, packed_qk=False, H=None, o_dtype=SAF_BF16):
     """saf_problem from [B,H,T,D] torch tensors (any strides with a unit feature stride); with kv_group > 1
     k_like / v_like are the [B,H/kv_group,T,D] shared key/value tensors."""
     B, Hq, T, D = q_like.shape
@@ -136,6 +136,7 @@ def make_problem(q_like, Tp, softmax_scale=0.0, grad_dtype=SAF_F32, k_like=None,
     p.grad_dtype = grad_dtype
     p.kv_group = kv_group
     p.packed_qk = int(packed_qk)
+    p.o_dtype = o_dtype
     for name, t in (("q_strides", q_like), ("k_strides", k_like if k_like is not None else q_like),
                     ("v_strides", v_like if v_like is not None else q_like),
                     ("o_strides", o_like if o_like is not None else q_like)):

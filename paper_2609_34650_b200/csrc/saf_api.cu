@@ -173,6 +173,7 @@ int validate(const saf_problem* p, const uint8_t* mask, int* n_frozen) {
   if (p->T > p->Tp) return SAF_ERR_INVALID_ARG;
   if (p->D != 64 && p->D != 96 && p->D != 128) return SAF_ERR_UNSUPPORTED;   // 96 runs padded on the 128-wide kernels
   if (p->grad_dtype != SAF_F32 && p->grad_dtype != SAF_BF16) return SAF_ERR_UNSUPPORTED;
+  if (p->o_dtype != SAF_F32 && p->o_dtype != SAF_BF16) return SAF_ERR_UNSUPPORTED;
   if (p->kv_group < 0 || (p->kv_group > 1 && p->H % p->kv_group != 0)) return SAF_ERR_INVALID_ARG;
   if (p->packed_qk && p->kv_group > 1) return SAF_ERR_INVALID_ARG;
   int nf = 0;
@@ -668,6 +669,7 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   fp.scale_log2 = scale * 1.4426950408889634f;
   fp.alpha = alpha; fp.rho = rho; fp.logZ = logZ;
   fp.O = O;
+  fp.o_f32 = p->o_dtype == SAF_F32 ? 1 : 0;
   for (int i = 0; i < 3; ++i) fp.o_strides[i] = p->o_strides[i];
   fp.LSE = LSE;
   fp.items = wl->items_dev;
@@ -681,7 +683,8 @@ int saf_hybrid_attn_fwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
       (ctx->selftest_drop_load && grid <= 16 && ctx->wait_limit_ns <= 50000000ull && p->D == 64) ? 1 : 0;
   ScopedTimer timer(ctx, SAF_KERNEL_FWD, st);
   // head dimension 96 runs on the 128-wide kernel: TMA zero-fills features 96..127 of every operand tile
-  // O leaves the D = 64 kernel as whole tiles by TMA stores (rows beyond T are clipped by the map)
+  // bf16 O leaves the D = 64 kernel as whole tiles by TMA stores (rows beyond T are clipped by the map); with fp32 O
+  // the kernel stores rows itself and never touches this map
   CUtensorMap mo;
   rc = make_map(ctx, &mo, O, p, p->o_strides);
   if (rc) return rc;
@@ -775,7 +778,7 @@ int saf_hybrid_attn_bwd(saf_ctx* ctx, const saf_problem* p, const void* Q, const
   // O is only read for ordinary heads; a frozen-only layer may pass O = NULL
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_PREP, st);
-    if (launch_bwd_prep(O, dO, LSE, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr), q_ext, do_ext,
+    if (launch_bwd_prep(O, p->o_dtype == SAF_F32, dO, LSE, p->o_strides, static_cast<const uint8_t*>(ctx->mask_buf.ptr), q_ext, do_ext,
                         1.0f / scale_v, dqacc, dK_k, dV_k, kern_f32, kvg, qslot, no, fz, p->B, p->H, p->T, p->D, st) !=
         cudaSuccess)
       return SAF_ERR_CUDA;
@@ -939,8 +942,8 @@ int saf_hybrid_attn_step_host(saf_ctx* ctx, const saf_problem* p, const void* Q_
   int rc = validate(p, frozen_mask_host, &nf);
   if (rc) return rc;
   const int no = p->H - nf;
+  if (p->packed_qk || p->o_dtype != SAF_BF16) return SAF_ERR_UNSUPPORTED;
   if (!V_host || (no > 0 && (!Q_host || !K_host)) || (nf > 0 && (!alpha_host || !rho_host))) return SAF_ERR_INVALID_ARG;
-  if (p->packed_qk) return SAF_ERR_UNSUPPORTED;
   DeviceGuard g(ctx->device);
   if (!g.ok) return SAF_ERR_CUDA;
   const int kvg = kv_group_of(p);
@@ -1091,7 +1094,7 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
   }
   {
     ScopedTimer timer(ctx, SAF_KERNEL_BWD_PREP, st);
-    if (launch_rowdot(O, dO, p->o_strides, static_cast<const int*>(ctx->pg_hlist.ptr),
+    if (launch_rowdot(O, p->o_dtype == SAF_F32, dO, p->o_strides, static_cast<const int*>(ctx->pg_hlist.ptr),
                       static_cast<float*>(ctx->pg_delta.ptr), p->B, p->H, nf, p->T, p->D, st) != cudaSuccess)
       return SAF_ERR_CUDA;
   }

@@ -560,7 +560,16 @@ saf_fwd_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ C
         uint32_t r[32];
         tmem_ld32(t_o + 32 * cc, r);
         tmem_wait_ld();
-        if (row < p.T && ok) {
+        if (row < p.T && ok && p.o_f32) {
+          float* orow32 = static_cast<float*>(p.O) + w.b * p.o_strides[0] + w.h * p.o_strides[1] +
+                          static_cast<int64_t>(row) * p.o_strides[2] + (D / 2) * hh + 32 * cc;
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            if ((D / 2) * hh + 32 * cc + 4 * g < p.d_real)
+              *reinterpret_cast<float4*>(orow32 + 4 * g) =
+                  make_float4(__uint_as_float(r[4 * g + 0]) * inv_l, __uint_as_float(r[4 * g + 1]) * inv_l,
+                              __uint_as_float(r[4 * g + 2]) * inv_l, __uint_as_float(r[4 * g + 3]) * inv_l);
+        } else if (row < p.T && ok) {
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             uint4 o;

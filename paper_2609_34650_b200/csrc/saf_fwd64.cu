@@ -114,6 +114,7 @@ __device__ __forceinline__ bool ring_take(const int4* ring, uint64_t* ring_full,
 
 }  // namespace
 
+template <bool OF32>
 __global__ void __launch_bounds__(320, 2)
 saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                  const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mvt,
@@ -687,14 +688,11 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       }
       tc_fence_after();
       if (q4 == 0) TRF(trr, 17);
-      // The O tile goes through a swizzled staging tile and leaves by one TMA store: a row per thread written
-      // straight to global memory touches 32 lines per store instruction and kept the load/store unit busy for
-      // ~1800 clk per item.  The staging tile is free once the previous item's store has read it, which the
-      // agreement barrier at the top of the item has made known to all compute warps.
-      {
-        const int rl = row - w.blk * BLK;                 // row within the tile (reversed in the tensor-core form)
-        const uint32_t strow = smem_u32(smem + C::OFF_OST) + static_cast<uint32_t>(rl) * 128;
+      if constexpr (OF32) {
+        // fp32 output: every thread writes its 32 columns of its row straight to global memory
         const float s0 = f0 * inv_l, s1 = f1 * inv_l;
+        float* orow = static_cast<float*>(p.O) + w.b * p.o_strides[0] + w.h * p.o_strides[1] +
+                      static_cast<int64_t>(row) * p.o_strides[2] + 32 * g;
 #pragma unroll
         for (int hc = 0; hc < 2; ++hc) {
           uint32_t ra[16], rb2[16];
@@ -705,25 +703,58 @@ saf_fwd64_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             tc_fence_before();
             warp_arrive(o_free);                          // the accumulators may be overwritten
           }
+          if (row < p.T && ok) {
 #pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            float v[8];
+            for (int q = 0; q < 4; ++q) {
+              float v[4];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              v[e] = __uint_as_float(ra[8 * q + e]) * s0;
-              if (use1) v[e] = fmaf(__uint_as_float(rb2[8 * q + e]), s1, v[e]);
+              for (int e = 0; e < 4; ++e) {
+                v[e] = __uint_as_float(ra[4 * q + e]) * s0;
+                if (use1) v[e] = fmaf(__uint_as_float(rb2[4 * q + e]), s1, v[e]);
+              }
+              *reinterpret_cast<float4*>(orow + 16 * hc + 4 * q) = make_float4(v[0], v[1], v[2], v[3]);
             }
-            const uint32_t chunk = static_cast<uint32_t>((4 * g + 2 * hc + q) ^ (rl & 7));
-            st_shared_v4w(strow + chunk * 16, pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
-                          pack_bf16x2(v[6], v[7]));
           }
         }
-      }
-      fence_proxy_async_smem();
-      const bool all_ok = !named_bar_or(8, 256, !ok);
-      if (tid == 0 && all_ok) {
-        tma_store_4d(&mo, smem + C::OFF_OST, 0, w.blk * BLK, w.h, w.b);
-        bulk_commit_group();
+      } else {
+        // The O tile goes through a swizzled staging tile and leaves by one TMA store: a row per thread written
+        // straight to global memory touches 32 lines per store instruction and kept the load/store unit busy for
+        // ~1800 clk per item.  The staging tile is free once the previous item's store has read it, which the
+        // agreement barrier at the top of the item has made known to all compute warps.
+        {
+          const int rl = row - w.blk * BLK;                 // row within the tile (reversed in the tensor-core form)
+          const uint32_t strow = smem_u32(smem + C::OFF_OST) + static_cast<uint32_t>(rl) * 128;
+          const float s0 = f0 * inv_l, s1 = f1 * inv_l;
+  #pragma unroll
+          for (int hc = 0; hc < 2; ++hc) {
+            uint32_t ra[16], rb2[16];
+            tmem_ld16(tmem + lane_base + C::COL_O + 32 * g + 16 * hc, ra);
+            if (use1) tmem_ld16(tmem + lane_base + C::COL_O + 64 + 32 * g + 16 * hc, rb2);
+            tmem_wait_ld();
+            if (hc == 1) {
+              tc_fence_before();
+              warp_arrive(o_free);                          // the accumulators may be overwritten
+            }
+  #pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              float v[8];
+  #pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                v[e] = __uint_as_float(ra[8 * q + e]) * s0;
+                if (use1) v[e] = fmaf(__uint_as_float(rb2[8 * q + e]), s1, v[e]);
+              }
+              const uint32_t chunk = static_cast<uint32_t>((4 * g + 2 * hc + q) ^ (rl & 7));
+              st_shared_v4w(strow + chunk * 16, pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+                            pack_bf16x2(v[6], v[7]));
+            }
+          }
+        }
+        fence_proxy_async_smem();
+        const bool all_ok = !named_bar_or(8, 256, !ok);
+        if (tid == 0 && all_ok) {
+          tma_store_4d(&mo, smem + C::OFF_OST, 0, w.blk * BLK, w.h, w.b);
+          bulk_commit_group();
+        }
       }
       if (p.LSE != nullptr && g == 0 && row < p.T && ok)
         p.LSE[(static_cast<size_t>(w.b) * p.H + w.h) * p.T + row] = lse;
@@ -758,10 +789,17 @@ int fwd64_smem_bytes() { return Fwd64Cfg::SMEM; }
 
 cudaError_t launch_fwd64(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mvt,
                          const CUtensorMap& mo, const FwdParams& p, int grid, cudaStream_t st) {
-  cudaError_t e =
-      cudaFuncSetAttribute(saf_fwd64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Fwd64Cfg::SMEM);
+  cudaError_t e;
+  if (p.o_f32) {
+    e = cudaFuncSetAttribute(saf_fwd64_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Fwd64Cfg::SMEM);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(PDL_FWD, saf_fwd64_kernel<true>, dim3(grid), dim3(Fwd64Cfg::NTHREADS), Fwd64Cfg::SMEM, st, mq, mk, mv,
+                      mvt, mo, p);
+  }
+  e = cudaFuncSetAttribute(saf_fwd64_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Fwd64Cfg::SMEM);
   if (e != cudaSuccess) return e;
-  return launch_pdl(PDL_FWD, saf_fwd64_kernel, dim3(grid), dim3(Fwd64Cfg::NTHREADS), Fwd64Cfg::SMEM, st, mq, mk, mv, mvt, mo, p);
+  return launch_pdl(PDL_FWD, saf_fwd64_kernel<false>, dim3(grid), dim3(Fwd64Cfg::NTHREADS), Fwd64Cfg::SMEM, st, mq, mk, mv,
+                    mvt, mo, p);
 }
 
 }  // namespace saf

@@ -62,7 +62,8 @@ struct FwdParams {
   const float* alpha;               // [H][Tp]
   const float* rho;                 // [H][Tp]
   const float* logZ;                // [H][Tp]
-  void* O;                          // bf16, strided
+  void* O;                          // bf16 (fp32 if o_f32), strided
+  int o_f32;
   int64_t o_strides[3];             // elements: batch, head, seq
   float* LSE;                       // [B][H][T]
   // Tensor-core form of frozen heads (all NULL when the pattern tables are not prepared): band_f is the
@@ -147,8 +148,8 @@ struct PgradParams {
   int* status;
   unsigned long long wait_limit_ns;
 };
-cudaError_t launch_rowdot(const void* O, const void* dO, const int64_t* o_strides, const int* hlist, float* delta,
-                          int B, int H, int Hf, int T, int D, cudaStream_t st);
+cudaError_t launch_rowdot(const void* O, int o_f32, const void* dO, const int64_t* o_strides, const int* hlist,
+                          float* delta, int B, int H, int Hf, int T, int D, cudaStream_t st);
 cudaError_t launch_pgrad(int D, const CUtensorMap& mv, const CUtensorMap& mdo, const PgradParams& p, int grid,
                          cudaStream_t st);
 
@@ -193,10 +194,10 @@ struct PrepFrozen {
   int Hf, Tp;
   PatternCheck chk;
 };
-cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* o_strides,
-                            const uint8_t* mask_dev, void* q_ext, void* do_ext, float inv_scale, float* dQacc,
-                            void* dK, void* dV, int grad_f32, int kv_group, const int* qslot, int n_ord,
-                            const PrepFrozen& fz, int B, int H, int T, int D, cudaStream_t st);   // kv_group > 1: zeroes all of dK and dV (fp32) instead
+cudaError_t launch_bwd_prep(const void* O, int o_f32, const void* dO, const float* LSE, const int64_t* o_strides,
+                            const uint8_t* mask_dev, void* q_ext, void* do_ext, float inv_scale, float* dQacc, void* dK,
+                            void* dV, int grad_f32, int kv_group, const int* qslot, int n_ord, const PrepFrozen& fz, int B,
+                            int H, int T, int D, cudaStream_t st);   // kv_group > 1: zeroes all of dK and dV (fp32) instead
 // dQ (grad dtype) = scale-free copy/convert of dQacc (fp32) for the bf16-gradient case.
 cudaError_t launch_bwd_finalize(const float* dQacc, void* dQ, size_t n, cudaStream_t st);
 // head dimension 64 (saf_fwd64.cu); launch_fwd dispatches to it

@@ -300,8 +300,8 @@ saf_pgrad_kernel(const __grid_constant__ CUtensorMap mv, const __grid_constant__
 // delta[c][h][t] = sum over the batch entries b of chunk c (VB consecutive entries) of sum_f dO[b][h][t][f] O[b][h][t][f]
 // for the frozen heads (hlist); TPR threads per row, eight features each (16 threads with four idle ones at D = 96, so
 // that a row stays inside a warp).
-template <int D, int TPR>
-__global__ void __launch_bounds__(256) saf_rowdot_kernel(const __nv_bfloat16* __restrict__ O,
+template <int D, int TPR, bool OF32>
+__global__ void __launch_bounds__(256) saf_rowdot_kernel(const void* __restrict__ O,
                                                          const __nv_bfloat16* __restrict__ dO, int64_t s0, int64_t s1,
                                                          int64_t s2, const int* __restrict__ hlist,
                                                          float* __restrict__ delta, int B, int H, int Hf, int T, int VB) {
@@ -322,15 +322,27 @@ __global__ void __launch_bounds__(256) saf_rowdot_kernel(const __nv_bfloat16* __
 #pragma unroll 4
     for (int b = c * VB; b < b1; ++b) {
       const int64_t off = b * s0 + h * s1 + static_cast<int64_t>(t) * s2 + part * 8;
-      const uint4 o4 = *reinterpret_cast<const uint4*>(O + off);
       const uint4 d4 = *reinterpret_cast<const uint4*>(dO + off);
-      const __nv_bfloat162* o2 = reinterpret_cast<const __nv_bfloat162*>(&o4);
       const __nv_bfloat162* d2 = reinterpret_cast<const __nv_bfloat162*>(&d4);
+      if constexpr (OF32) {
+        const float* of = static_cast<const float*>(O) + off;
+        const float4 oa = *reinterpret_cast<const float4*>(of), ob = *reinterpret_cast<const float4*>(of + 4);
+        const float ov[8] = {oa.x, oa.y, oa.z, oa.w, ob.x, ob.y, ob.z, ob.w};
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 of = __bfloat1622float2(o2[e]), df = __bfloat1622float2(d2[e]);
-        acc = fmaf(of.x, df.x, acc);
-        acc = fmaf(of.y, df.y, acc);
+        for (int e = 0; e < 4; ++e) {
+          const float2 df = __bfloat1622float2(d2[e]);
+          acc = fmaf(ov[2 * e], df.x, acc);
+          acc = fmaf(ov[2 * e + 1], df.y, acc);
+        }
+      } else {
+        const uint4 o4 = *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(O) + off);
+        const __nv_bfloat162* o2 = reinterpret_cast<const __nv_bfloat162*>(&o4);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 of = __bfloat1622float2(o2[e]), df = __bfloat1622float2(d2[e]);
+          acc = fmaf(of.x, df.x, acc);
+          acc = fmaf(of.y, df.y, acc);
+        }
       }
     }
   }
@@ -339,18 +351,19 @@ __global__ void __launch_bounds__(256) saf_rowdot_kernel(const __nv_bfloat16* __
   if (inrange && part == 0) delta[(static_cast<size_t>(c) * H + h) * T + t] = acc;
 }
 
-cudaError_t launch_rowdot(const void* O, const void* dO, const int64_t* os, const int* hlist, float* delta, int B, int H,
-                          int Hf, int T, int D, cudaStream_t st) {
+cudaError_t launch_rowdot(const void* O, int o_f32, const void* dO, const int64_t* os, const int* hlist, float* delta,
+                          int B, int H, int Hf, int T, int D, cudaStream_t st) {
   const int tpr = D == 96 ? 16 : D / 8;
   const int vb = pgrad_batch_chunk(D);
   const long long nthreads = static_cast<long long>((B + vb - 1) / vb) * Hf * T * tpr;
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
-#define SAF_ROWDOT_ARGS \
-  static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), os[0], os[1], os[2], hlist, delta, B, H, Hf, T, vb
-  if (D == 64) saf_rowdot_kernel<64, 8><<<grid, 256, 0, st>>>(SAF_ROWDOT_ARGS);
-  else if (D == 96) saf_rowdot_kernel<96, 16><<<grid, 256, 0, st>>>(SAF_ROWDOT_ARGS);
-  else saf_rowdot_kernel<128, 16><<<grid, 256, 0, st>>>(SAF_ROWDOT_ARGS);
-#undef SAF_ROWDOT_ARGS
+#define SAF_ROWDOT(DD, TT, FF) \
+  saf_rowdot_kernel<DD, TT, FF><<<grid, 256, 0, st>>>(O, static_cast<const __nv_bfloat16*>(dO), os[0], os[1], os[2], \
+                                                      hlist, delta, B, H, Hf, T, vb)
+  if (D == 64) { if (o_f32) SAF_ROWDOT(64, 8, true); else SAF_ROWDOT(64, 8, false); }
+  else if (D == 96) { if (o_f32) SAF_ROWDOT(96, 16, true); else SAF_ROWDOT(96, 16, false); }
+  else { if (o_f32) SAF_ROWDOT(128, 16, true); else SAF_ROWDOT(128, 16, false); }
+#undef SAF_ROWDOT
   return cudaGetLastError();
 }
 

@@ -248,8 +248,9 @@ __device__ __forceinline__ uint4 split3_bf16(float x) {
 //   frozen head  : dK row = 0 (no key gradient; Sec. 3.3); with the tensor-core form, the row w(i) dO in fp16
 // Image layout per 128-row block (4 KB): byte (n/8)*256 + (k/8)*128 + (n%8)*16 + (k%8)*2 for row n, column k < 16.
 // (TPR threads per row: D / 8, or 16 with four idle ones at D = 96 so that a row stays inside a warp)
-template <int D, int TPR>
-__global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat16* __restrict__ O,
+// (OF32: O is fp32 instead of bf16, same element strides)
+template <int D, int TPR, bool OF32>
+__global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const void* __restrict__ O,
                                                            const __nv_bfloat16* __restrict__ dO,
                                                            const float* __restrict__ LSE, int64_t os0, int64_t os1,
                                                            int64_t os2, const uint8_t* __restrict__ mask,
@@ -328,15 +329,27 @@ __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat1
       }
     } else {
       const int64_t off = b * os0 + h * os1 + static_cast<int64_t>(t) * os2 + part * 8;
-      const uint4 o4 = *reinterpret_cast<const uint4*>(O + off);
       const uint4 d4 = *reinterpret_cast<const uint4*>(dO + off);
-      const __nv_bfloat162* o2 = reinterpret_cast<const __nv_bfloat162*>(&o4);
       const __nv_bfloat162* d2 = reinterpret_cast<const __nv_bfloat162*>(&d4);
+      if constexpr (OF32) {
+        const float* of = static_cast<const float*>(O) + off;
+        const float4 oa = *reinterpret_cast<const float4*>(of), ob = *reinterpret_cast<const float4*>(of + 4);
+        const float ov[8] = {oa.x, oa.y, oa.z, oa.w, ob.x, ob.y, ob.z, ob.w};
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 of = __bfloat1622float2(o2[e]), df = __bfloat1622float2(d2[e]);
-        acc = fmaf(of.x, df.x, acc);
-        acc = fmaf(of.y, df.y, acc);
+        for (int e = 0; e < 4; ++e) {
+          const float2 df = __bfloat1622float2(d2[e]);
+          acc = fmaf(ov[2 * e], df.x, acc);
+          acc = fmaf(ov[2 * e + 1], df.y, acc);
+        }
+      } else {
+        const uint4 o4 = *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(O) + off);
+        const __nv_bfloat162* o2 = reinterpret_cast<const __nv_bfloat162*>(&o4);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 of = __bfloat1622float2(o2[e]), df = __bfloat1622float2(d2[e]);
+          acc = fmaf(of.x, df.x, acc);
+          acc = fmaf(of.y, df.y, acc);
+        }
       }
     }
   }
@@ -361,22 +374,24 @@ __global__ void __launch_bounds__(256, 8) saf_bwd_prep_kernel(const __nv_bfloat1
   }
 }
 
-cudaError_t launch_bwd_prep(const void* O, const void* dO, const float* LSE, const int64_t* os, const uint8_t* mask_dev,
-                            void* q_ext, void* do_ext, float inv_scale, float* dQacc, void* dK, void* dV, int grad_f32,
-                            int kv_group, const int* qslot, int n_ord, const PrepFrozen& fz, int B, int H, int T, int D,
-                            cudaStream_t st) {
+cudaError_t launch_bwd_prep(const void* O, int o_f32, const void* dO, const float* LSE, const int64_t* os,
+                            const uint8_t* mask_dev, void* q_ext, void* do_ext, float inv_scale, float* dQacc, void* dK,
+                            void* dV, int grad_f32, int kv_group, const int* qslot, int n_ord, const PrepFrozen& fz, int B,
+                            int H, int T, int D, cudaStream_t st) {
   const int Tpad = (T + 127) / 128 * 128;
   const int tpr = D == 96 ? 16 : D / 8;
   const long long nthreads = static_cast<long long>(B) * H * Tpad * tpr;
   const unsigned grid = static_cast<unsigned>((nthreads + 255) / 256);
-#define SAF_PREP_ARGS                                                                                              \
-  static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2], mask_dev, \
-      static_cast<uint8_t*>(q_ext), static_cast<uint8_t*>(do_ext), inv_scale, dQacc, dK, dV, grad_f32, kv_group,   \
-      qslot, n_ord, fz, B, H, T
+#define SAF_PREP_ARGS                                                                                                  \
+  O, static_cast<const __nv_bfloat16*>(dO), LSE, os[0], os[1], os[2], mask_dev, static_cast<uint8_t*>(q_ext),          \
+      static_cast<uint8_t*>(do_ext), inv_scale, dQacc, dK, dV, grad_f32, kv_group, qslot, n_ord, fz, B, H, T
+#define SAF_PREP_LAUNCH(DD, TT, FF) \
+  launch_pdl(PDL_PREP, saf_bwd_prep_kernel<DD, TT, FF>, dim3(grid), dim3(256), 0, st, SAF_PREP_ARGS)
   cudaError_t e;
-  if (D == 64) e = launch_pdl(PDL_PREP, saf_bwd_prep_kernel<64, 8>, dim3(grid), dim3(256), 0, st, SAF_PREP_ARGS);
-  else if (D == 96) e = launch_pdl(PDL_PREP, saf_bwd_prep_kernel<96, 16>, dim3(grid), dim3(256), 0, st, SAF_PREP_ARGS);
-  else e = launch_pdl(PDL_PREP, saf_bwd_prep_kernel<128, 16>, dim3(grid), dim3(256), 0, st, SAF_PREP_ARGS);
+  if (D == 64) e = o_f32 ? SAF_PREP_LAUNCH(64, 8, true) : SAF_PREP_LAUNCH(64, 8, false);
+  else if (D == 96) e = o_f32 ? SAF_PREP_LAUNCH(96, 16, true) : SAF_PREP_LAUNCH(96, 16, false);
+  else e = o_f32 ? SAF_PREP_LAUNCH(128, 16, true) : SAF_PREP_LAUNCH(128, 16, false);
+#undef SAF_PREP_LAUNCH
 #undef SAF_PREP_ARGS
   return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -44,7 +44,8 @@ def bf16_half_ulp(peak: float) -> float:
 class Layer:
     """One seeded workload resident on the GPU plus its outputs."""
 
-    def __init__(self, inp: si.Inputs, grad_dtype=saf.SAF_F32, backward=True, ctx=None, softmax_scale=0.0):
+    def __init__(self, inp: si.Inputs, grad_dtype=saf.SAF_F32, backward=True, ctx=None, softmax_scale=0.0,
+                 o_f32=False):
         self.inp = inp
         wl = inp.wl
         dev = "cuda"
@@ -53,14 +54,15 @@ class Layer:
         self.alpha = torch.from_numpy(inp.alpha).to(dev)
         self.rho = torch.from_numpy(inp.rho).to(dev)
         self.logZ = torch.zeros_like(self.alpha)
-        self.O = torch.full_like(self.dO, float("nan"))
+        self.O = torch.full_like(self.dO, float("nan"), dtype=torch.float32 if o_f32 else torch.bfloat16)
         self.LSE = torch.full((wl.B, wl.H, wl.T), float("nan"), device=dev)
         gd = torch.float32 if grad_dtype == saf.SAF_F32 else torch.bfloat16
         self.grads = [torch.full(t.shape, float("nan"), device=dev, dtype=gd)
                       for t in (self.Q, self.K, self.V)] if backward else None
         self.prob = saf.make_problem(self.Q, wl.stored_len, softmax_scale=softmax_scale, grad_dtype=grad_dtype,
                                      k_like=self.K, v_like=self.V, o_like=self.O, kv_group=wl.kv_group,
-                                     packed_qk=wl.packed_qk, H=wl.H)
+                                     packed_qk=wl.packed_qk, H=wl.H,
+                                     o_dtype=saf.SAF_F32 if o_f32 else saf.SAF_BF16)
         self.mask = inp.mask
 
     def run(self, backward=True, prepare=True):
