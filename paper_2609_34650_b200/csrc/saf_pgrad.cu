@@ -12,7 +12,8 @@
 // One persistent kernel, item = (frozen head, 128-key block J, a run of query blocks I >= J, a run of batch
 // entries of at most VB); the V_J tiles of the item's batch entries stay in shared memory, per query block:
 //   Gs^T tile [128 keys x 128 queries] = sum_b V_J,b dO_I,b^T on the tensor core (tcgen05, both operands K-major in
-//   128B-swizzled smem via TMA, dO streamed through a ring, accumulator double-buffered in TMEM), then per element
+//   128B-swizzled smem via TMA, dO streamed through a ring of stages of SB batch entries each, accumulator
+//   double-buffered in TMEM), then per element
 //   in registers p = exp2(alpha'(j) + rho'(i-j) - logZ'(i)) (primes: log2e-scaled; distances < 0 and rows/keys
 //   beyond T carry -inf, which is the causal mask), db = p (Gs - Ds_i).
 //   dalpha(j): the thread that owns key row j sums its db over the whole item and adds once (atomicAdd).
@@ -27,6 +28,11 @@
 #include "ptx.cuh"
 #include "saf_internal.h"
 
+// batch entries per ring stage at D = 64 (1, 2 or 4)
+#ifndef SAF_PG_SB
+#define SAF_PG_SB 2
+#endif
+
 namespace saf {
 
 namespace {
@@ -39,10 +45,12 @@ struct PgCfg {
   static constexpr int PANEL_BYTES = 128 * 64 * 2;
   static constexpr int TILE_BYTES = NPANEL * PANEL_BYTES;
   static constexpr int VB = (D == 64) ? 8 : 4;          // resident V tiles = batch entries per item (pgrad_batch_chunk)
-  static constexpr int NS = (D == 64) ? 4 : 2;          // dO ring depth (five stages measured the same)
+  static constexpr int SB = (D == 64) ? SAF_PG_SB : 1;  // batch entries (dO tiles) per ring stage
+  static constexpr int NS = (D == 64) ? 4 / SB : 2;     // dO ring depth (five single-tile stages measured the same)
+  static constexpr int STAGE_BYTES = SB * TILE_BYTES;
   static constexpr int OFF_V = 0;
   static constexpr int OFF_DO = VB * TILE_BYTES;
-  static constexpr int OFF_TAB = OFF_DO + NS * TILE_BYTES;
+  static constexpr int OFF_TAB = OFF_DO + NS * STAGE_BYTES;
   // floats, two sets (tile parity): r2raw[256] z2s[128] dl[128]
   static constexpr int TAB_FLOATS = 2 * (256 + 128 + 128);
   static constexpr int OFF_BAR = OFF_TAB + TAB_FLOATS * 4;
@@ -120,14 +128,16 @@ saf_pgrad_kernel(const __grid_constant__ CUtensorMap mv, const __grid_constant__
                         w.J * BLK, h / p.kv_group, b);
         ++nv;
         for (int I = w.I0; I < w.I1 && ok; ++I) {
-          for (int b = w.b0; b < w.b1; ++b) {
+          for (int b = w.b0; b < w.b1; b += C::SB) {
             const int s = ndo % C::NS;
+            const int nb = min(C::SB, w.b1 - b);
             ok = mbar_wait(do_empty + s, ((ndo / C::NS) & 1) ^ 1, wc, G_DO_EMPTY);
             if (!ok) break;
-            mbar_expect_tx(do_full + s, C::TILE_BYTES);
-            for (int pn = 0; pn < C::NPANEL; ++pn)
-              tma_load_4d(smem + C::OFF_DO + s * C::TILE_BYTES + pn * C::PANEL_BYTES, &mdo, do_full + s, pn * 64,
-                          I * BLK, h, b);
+            mbar_expect_tx(do_full + s, nb * C::TILE_BYTES);
+            for (int e = 0; e < nb; ++e)
+              for (int pn = 0; pn < C::NPANEL; ++pn)
+                tma_load_4d(smem + C::OFF_DO + s * C::STAGE_BYTES + e * C::TILE_BYTES + pn * C::PANEL_BYTES, &mdo,
+                            do_full + s, pn * 64, I * BLK, h, b + e);
             ++ndo;
           }
         }
@@ -153,22 +163,25 @@ saf_pgrad_kernel(const __grid_constant__ CUtensorMap mv, const __grid_constant__
         const uint32_t gb = ng & 1;
         ok = mbar_wait_warp(g_free + gb, ((ng >> 1) & 1) ^ 1, wc, G_G_FREE);
         if (!ok) break;
-        for (int b = 0; b < nb; ++b) {
+        for (int b = 0; b < nb; b += C::SB) {
           const uint32_t s = ndo % C::NS;
+          const int ne = min(C::SB, nb - b);
           ok = mbar_wait_warp(do_full + s, (ndo / C::NS) & 1, wc, G_DO_FULL);
           if (!ok) break;
           ++ndo;
           tc_fence_after();
-          const uint32_t do_lo = lo_k + ((C::OFF_DO + s * C::TILE_BYTES) >> 4);
-          const uint32_t vb_lo = v_lo + ((b * C::TILE_BYTES) >> 4);
           if (leader) {
+            for (int e = 0; e < ne; ++e) {
+              const uint32_t do_lo = lo_k + ((C::OFF_DO + s * C::STAGE_BYTES + e * C::TILE_BYTES) >> 4);
+              const uint32_t vb_lo = v_lo + (((b + e) * C::TILE_BYTES) >> 4);
 #pragma unroll
-            for (int kc = 0; kc < D / 16; ++kc) {
-              const uint32_t off = ((kc >> 2) * C::PANEL_BYTES + (kc & 3) * 32) >> 4;
-              umma_ss2(tmem + 128 * gb, vb_lo + off, hi_k, do_lo + off, hi_k, idesc, (kc > 0) || (b > 0));
+              for (int kc = 0; kc < D / 16; ++kc) {
+                const uint32_t off = ((kc >> 2) * C::PANEL_BYTES + (kc & 3) * 32) >> 4;
+                umma_ss2(tmem + 128 * gb, vb_lo + off, hi_k, do_lo + off, hi_k, idesc, (kc > 0) || (b + e > 0));
+              }
             }
             umma_commit(do_empty + s);
-            if (b == nb - 1) {
+            if (b + ne >= nb) {
               umma_commit(g_full + gb);
               if (t == ntiles - 1) umma_commit(v_empty);
             }
