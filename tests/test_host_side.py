@@ -36,10 +36,29 @@ def test_library_exports_every_declared_symbol(lib):
     assert lib.status_string(0) == "ok" and "argument" in lib.status_string(1)
 
 
-def test_problem_struct_layout_matches_header(lib):
-    # 8 x 4-byte fields then 4 x 3 x int64
+def test_problem_struct_layout_matches_header(lib, tmp_path):
+    # ten 4-byte fields then 4 x 3 x int64
     assert ctypes.sizeof(lib.SafProblem) == 10 * 4 + 12 * 8
     assert lib.SafProblem.q_strides.offset == 40
+    # ... and the header itself, compiled as plain C: size and the offset of every field the binding names
+    import shutil
+    import subprocess
+    cc = shutil.which("gcc") or shutil.which("cc")
+    if cc is None:
+        pytest.skip("no C compiler")
+    fields = [name for name, _ in lib.SafProblem._fields_]
+    src = tmp_path / "layout.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "saf.h"\nint main(void) {\n'
+                   '  printf("%zu\\n", sizeof(saf_problem));\n'
+                   + "".join(f'  printf("%zu\\n", offsetof(saf_problem, {f}));\n' for f in fields)
+                   + '  printf("%d %d\\n", (int)SAF_BF16, (int)SAF_F32);\n  return 0;\n}\n')
+    exe = tmp_path / "layout"
+    subprocess.run([cc, "-std=c99", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
+    assert int(out[0]) == ctypes.sizeof(lib.SafProblem)
+    for f, off in zip(fields, out[1:1 + len(fields)]):
+        assert getattr(lib.SafProblem, f).offset == int(off), f
+    assert (int(out[-2]), int(out[-1])) == (lib.SAF_BF16, lib.SAF_F32)
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure mode")
