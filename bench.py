@@ -336,9 +336,9 @@ def run_ours(args):
     logZ = torch.zeros_like(alpha)
     O = torch.empty_like(Q)
     LSE = torch.empty(wl.B, wl.H, wl.T, device=dev)
-    dQ, dK, dV = (torch.empty(Q.shape, device=dev, dtype=torch.float32) for _ in range(3)) if bwd else (None,) * 3
+    dQ, dK, dV = (torch.empty(x.shape, device=dev, dtype=torch.float32) for x in (Q, K, V)) if bwd else (None,) * 3
     ctx = saf.Context(local_rank)
-    prob = saf.make_problem(Q, wl.stored_len)
+    prob = saf.make_problem(Q, wl.stored_len, k_like=K, v_like=V, kv_group=wl.kv_group)
     mask = inp.mask
     mask0 = np.zeros_like(mask)
 
@@ -516,15 +516,15 @@ def run_ours(args):
     hLSE = torch.empty(wl.B, wl.H, wl.T).pin_memory()
     nel = wl.B * wl.H * wl.T * wl.D
     if bwd:
-        hdQ, hdK, hdV = (torch.empty(Q.shape, dtype=torch.float32).pin_memory() for _ in range(3))
+        hdQ, hdK, hdV = (torch.empty(x.shape, dtype=torch.float32).pin_memory() for x in (Q, K, V))
         ctx2 = saf.Context(local_rank)
-        probh = saf.make_problem(hostQ, wl.stored_len)
+        probh = saf.make_problem(hostQ, wl.stored_len, k_like=hostK, v_like=hostV, kv_group=wl.kv_group)
 
         def step_host(prepare):
             ctx2.saf_hybrid_attn_step_host(probh, hostQ, hostK, hostV, hostdO, mask, alpha_h, rho_h, prepare, hO,
                                            hLSE, hdQ, hdK, hdV)
-        h2d = 4 * nel * 2
-        d2h = nel * 2 + wl.B * wl.H * wl.T * 4 + 3 * nel * 4
+        h2d = (2 * nel + K.numel() + V.numel()) * 2
+        d2h = nel * 2 + wl.B * wl.H * wl.T * 4 + (nel + K.numel() + V.numel()) * 4
     else:
         # forward-only workload: the device entry point between pinned-memory copies of Q, K, V in and O, LSE out
         def step_host(prepare):
@@ -534,7 +534,7 @@ def run_ours(args):
             ctx.saf_hybrid_attn_fwd(prob, Q, K, V, mask, alpha, rho, logZ, O, LSE)
             hO.copy_(O, non_blocking=True)
             hLSE.copy_(LSE, non_blocking=True)
-        h2d = 3 * nel * 2
+        h2d = (nel + K.numel() + V.numel()) * 2
         d2h = nel * 2 + wl.B * wl.H * wl.T * 4
 
     step_host(1)
@@ -622,7 +622,7 @@ def run_ours(args):
         "metric": METRIC if bwd else "hybrid_attn_fwd_tflops", "value": value, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl.name, "B_per_gpu": wl.B, "B": wl.B, "H": wl.H, "Hf": hf, "T": wl.T, "D": wl.D,
+        "config": {"workload": wl.name, "B_per_gpu": wl.B, "B": wl.B, "H": wl.H, "kv_heads": wl.H // wl.kv_group, "Hf": hf, "T": wl.T, "D": wl.D,
                    "pass": "fwd+bwd" if bwd else "fwd only",
                    "grad_dtype": "f32", "frozen_fraction": hf / wl.H,
                    "flops_per_step_per_gpu": flops_local,
@@ -703,7 +703,7 @@ def main():
     ap.add_argument("--repeats", type=int, default=5, help="how many times the K-step region is timed (median reported)")
     ap.add_argument("--region-gap", type=float, default=0.3, help="idle seconds before each timed region")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 4, 5, 6])
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 4, 5, 6, 7])
     ap.add_argument("--no-fit", action="store_true", help="skip the extra legs that time the one-time fitter and the calibration statistics")
     ap.add_argument("--ref-budget", type=float, default=12.0, help="seconds of CPU-oracle work per sample")
     ap.add_argument("--launcher-selftest", action="store_true", help=argparse.SUPPRESS)

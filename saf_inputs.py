@@ -87,7 +87,8 @@ def config(k: int, n_frozen: int | None = None, seed: int = 0) -> Workload:
     """The five benchmark/test configurations (k = 0..4).  `n_frozen` overrides the frozen count
     (config 3 is config 1's shape with n_frozen in {0,3,6,9,12}).  k = 5, 6 are two extra shapes for the wider
     head dimensions: config 1's layer at head dimension 128, and the layer of the paper's 1B model (16 heads of
-    dimension 96, batch 2 per rank, 8K context)."""
+    dimension 96, batch 2 per rank, 8K context); k = 7 is a grouped-query forward (32 query heads, 8 key/value heads of
+    dimension 128)."""
     if k == 0:
         nf = 1 if n_frozen is None else n_frozen
         return Workload("tiny", 1, 4, 256, 64, sweep_frozen_heads(4, nf, seed), -0.05, seed=seed)
@@ -108,6 +109,13 @@ def config(k: int, n_frozen: int | None = None, seed: int = 0) -> Workload:
     if k == 6:
         nf = 4 if n_frozen is None else n_frozen
         return Workload("1b-paper-8k-d96", 2, 16, 8192, 96, sweep_frozen_heads(16, nf, seed), -0.01, seed=seed)
+    if k == 7:
+        # grouped-query attention at the shape of the paper's GQA attention-operator timings (Appendix E.2): 32 query
+        # heads on 8 shared key/value heads of dimension 128, batch 4, 4K context, forward only; 30 % of the query
+        # heads replaced unless n_frozen says otherwise
+        nf = 10 if n_frozen is None else n_frozen
+        return Workload("gqa-32q-8kv-4k-d128", 4, 32, 4096, 128, sweep_frozen_heads(32, nf, seed), -0.01, seed=seed,
+                        kv_group=4, backward=False)
     raise ValueError(f"unknown config {k}")
 
 
