@@ -1098,8 +1098,10 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
                       static_cast<float*>(ctx->pg_delta.ptr), p->B, p->H, nf, p->T, p->D, st) != cudaSuccess)
       return SAF_ERR_CUDA;
   }
-  // Work list: (frozen-head ordinal, key block J, run of query blocks, run of batch entries), cut so that there are
-  // about four items per CTA, dealt longest first to the least loaded CTA.
+  // Work list: (frozen-head ordinal, key block J, run of query blocks, run of batch entries), dealt longest first to
+  // the least loaded CTA.  An item costs its tiles plus about 0.7 of a tile for loading its V tiles (which cannot
+  // start before the item in front of it has finished), so longer runs are cheaper but balance worse: the run
+  // length is the one of 1 .. 16 whose dealt list has the shortest longest CTA under that cost.
   const int nblk = (p->T + BLK - 1) / BLK;
   const int vb = pgrad_batch_chunk(p->D);
   const int nbc = (p->B + vb - 1) / vb;
@@ -1107,25 +1109,39 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
   const int grid = static_cast<int>(std::min<long long>(ctx->num_sms, total_tiles));
   const std::array<int, 5> key = {p->B, nf, p->T, p->D, grid};
   if (key != ctx->pg_key) {
-    const int run = static_cast<int>(std::max<long long>(1, std::min<long long>(8, total_tiles / (4LL * grid))));
-    std::vector<PgItem> items;
-    for (int hf = 0; hf < nf; ++hf)
-      for (int c = 0; c < nbc; ++c)
-        for (int J = 0; J < nblk; ++J)
-          for (int I0 = J; I0 < nblk; I0 += run)
-            items.push_back(PgItem{hf, J, I0, std::min(nblk, I0 + run), c * vb, std::min(p->B, (c + 1) * vb), 0, 0});
-    // cost of an item in tile loads: its dO tiles plus the V tile
-    auto cost = [](const PgItem& w) { return (w.I1 - w.I0) + 1; };
-    std::stable_sort(items.begin(), items.end(), [&](const PgItem& a, const PgItem& b) { return cost(a) > cost(b); });
-    std::vector<std::vector<PgItem>> per_cta(grid);
-    std::priority_queue<std::pair<long long, int>, std::vector<std::pair<long long, int>>, std::greater<>> load;
-    for (int c = 0; c < grid; ++c) load.push({0, c});
-    for (const PgItem& w : items) {
-      auto [l, c] = load.top();
-      load.pop();
-      per_cta[c].push_back(w);
-      load.push({l + cost(w), c});
+    auto cost = [](const PgItem& w) { return 10 * (w.I1 - w.I0) + 7; };
+    auto deal = [&](int run, std::vector<std::vector<PgItem>>* out) {
+      std::vector<PgItem> items;
+      for (int hf = 0; hf < nf; ++hf)
+        for (int c = 0; c < nbc; ++c)
+          for (int J = 0; J < nblk; ++J)
+            for (int I0 = J; I0 < nblk; I0 += run)
+              items.push_back(PgItem{hf, J, I0, std::min(nblk, I0 + run), c * vb, std::min(p->B, (c + 1) * vb), 0, 0});
+      std::stable_sort(items.begin(), items.end(), [&](const PgItem& a, const PgItem& b) { return cost(a) > cost(b); });
+      std::priority_queue<std::pair<long long, int>, std::vector<std::pair<long long, int>>, std::greater<>> load;
+      for (int c = 0; c < grid; ++c) load.push({0, c});
+      if (out) out->assign(grid, {});
+      long long longest = 0;
+      for (const PgItem& w : items) {
+        auto [l, c] = load.top();
+        load.pop();
+        if (out) (*out)[c].push_back(w);
+        load.push({l + cost(w), c});
+        longest = std::max(longest, l + cost(w));
+      }
+      return longest;
+    };
+    int run = 1;
+    long long best = -1;
+    for (int r = 1; r <= std::min(16, nblk); ++r) {
+      const long long m = deal(r, nullptr);
+      if (best < 0 || m < best) {
+        best = m;
+        run = r;
+      }
     }
+    std::vector<std::vector<PgItem>> per_cta;
+    deal(run, &per_cta);
     ctx->pg_items_host.clear();
     ctx->pg_offsets_host.assign(1, 0);
     for (int c = 0; c < grid; ++c) {
