@@ -125,12 +125,14 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // [B][H][T][D] bf16 tensor with element strides (batch, head, seq); box = 64 features x 128 rows,
 // 128-byte swizzle; rows beyond T read as zero.
 int make_map(saf_ctx* ctx, CUtensorMap* out, const void* base, const saf_problem* p, const int64_t* strides,
-             CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, int heads = 0, int box_rows = BLK) {
+             CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, int heads = 0, int box_rows = BLK,
+             int box_batch = 1) {
   cuuint64_t dims[4] = {static_cast<cuuint64_t>(p->D), static_cast<cuuint64_t>(p->T),
                         static_cast<cuuint64_t>(heads > 0 ? heads : p->H), static_cast<cuuint64_t>(p->B)};
   cuuint64_t gs[3] = {static_cast<cuuint64_t>(strides[2]) * 2, static_cast<cuuint64_t>(strides[1]) * 2,
                       static_cast<cuuint64_t>(strides[0]) * 2};
-  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(box_rows), 1, 1};
+  // (box_batch > 1: one copy brings the same tile of several consecutive batch entries, laid out one after the other)
+  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(box_rows), 1, static_cast<cuuint32_t>(box_batch)};
   cuuint32_t es[4] = {1, 1, 1, 1};
   CUresult r = ctx->encode(out, dtype, 4, const_cast<void*>(base), dims, gs, box, es,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1159,8 +1161,10 @@ int saf_pattern_grad(saf_ctx* ctx, const saf_problem* p, const void* V, const vo
     ctx->pg_key = key;
   }
   CUtensorMap mv, mdo;
-  if ((rc = make_map(ctx, &mv, V, p, p->v_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg))) return rc;
-  if ((rc = make_map(ctx, &mdo, dO, p, p->o_strides))) return rc;
+  // at D = 64 a tile is one 64-column panel, so one copy can bring the tiles of a whole batch run (V) or ring stage (dO)
+  const int vbox = p->D == 64 ? vb : 1, dobox = p->D == 64 ? pgrad_stage_entries(p->D) : 1;
+  if ((rc = make_map(ctx, &mv, V, p, p->v_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, p->H / kvg, BLK, vbox))) return rc;
+  if ((rc = make_map(ctx, &mdo, dO, p, p->o_strides, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 0, BLK, dobox))) return rc;
   PgradParams gp;
   gp.B = p->B; gp.H = p->H; gp.T = p->T; gp.Tp = p->Tp;
   gp.kv_group = kvg;

@@ -133,6 +133,8 @@ struct PgItem {
 };
 // Batch entries whose V tile stays in shared memory for the length of an item (the item's batch range is at most this).
 inline int pgrad_batch_chunk(int D) { return D == 64 ? 8 : 4; }
+// Batch entries (dO tiles) per stage of the kernel's dO ring.
+inline int pgrad_stage_entries(int D) { return D == 64 ? 2 : 1; }
 struct PgradParams {
   int B, H, T, Tp;
   int kv_group;

@@ -28,10 +28,6 @@
 #include "ptx.cuh"
 #include "saf_internal.h"
 
-// batch entries per ring stage at D = 64 (1, 2 or 4)
-#ifndef SAF_PG_SB
-#define SAF_PG_SB 2
-#endif
 
 namespace saf {
 
@@ -45,7 +41,7 @@ struct PgCfg {
   static constexpr int PANEL_BYTES = 128 * 64 * 2;
   static constexpr int TILE_BYTES = NPANEL * PANEL_BYTES;
   static constexpr int VB = (D == 64) ? 8 : 4;          // resident V tiles = batch entries per item (pgrad_batch_chunk)
-  static constexpr int SB = (D == 64) ? SAF_PG_SB : 1;  // batch entries (dO tiles) per ring stage
+  static constexpr int SB = (D == 64) ? 2 : 1;          // batch entries (dO tiles) per ring stage (pgrad_stage_entries)
   static constexpr int NS = (D == 64) ? 4 / SB : 2;     // dO ring depth (five single-tile stages measured the same)
   static constexpr int STAGE_BYTES = SB * TILE_BYTES;
   static constexpr int OFF_V = 0;
@@ -121,11 +117,17 @@ saf_pgrad_kernel(const __grid_constant__ CUtensorMap mv, const __grid_constant__
         const int h = p.hlist[w.hf];
         ok = mbar_wait(v_empty, (nv & 1) ^ 1, wc, G_V_EMPTY);
         if (!ok) break;
-        mbar_expect_tx(v_full, (w.b1 - w.b0) * C::TILE_BYTES);
-        for (int b = w.b0; b < w.b1; ++b)
-          for (int pn = 0; pn < C::NPANEL; ++pn)
-            tma_load_4d(smem + C::OFF_V + (b - w.b0) * C::TILE_BYTES + pn * C::PANEL_BYTES, &mv, v_full, pn * 64,
-                        w.J * BLK, h / p.kv_group, b);
+        if constexpr (C::NPANEL == 1) {
+          // one copy for the whole batch run (the map's box spans VB batch entries; entries beyond B arrive as zeros)
+          mbar_expect_tx(v_full, C::VB * C::TILE_BYTES);
+          tma_load_4d(smem + C::OFF_V, &mv, v_full, 0, w.J * BLK, h / p.kv_group, w.b0);
+        } else {
+          mbar_expect_tx(v_full, (w.b1 - w.b0) * C::TILE_BYTES);
+          for (int b = w.b0; b < w.b1; ++b)
+            for (int pn = 0; pn < C::NPANEL; ++pn)
+              tma_load_4d(smem + C::OFF_V + (b - w.b0) * C::TILE_BYTES + pn * C::PANEL_BYTES, &mv, v_full, pn * 64,
+                          w.J * BLK, h / p.kv_group, b);
+        }
         ++nv;
         for (int I = w.I0; I < w.I1 && ok; ++I) {
           for (int b = w.b0; b < w.b1; b += C::SB) {
@@ -133,11 +135,16 @@ saf_pgrad_kernel(const __grid_constant__ CUtensorMap mv, const __grid_constant__
             const int nb = min(C::SB, w.b1 - b);
             ok = mbar_wait(do_empty + s, ((ndo / C::NS) & 1) ^ 1, wc, G_DO_EMPTY);
             if (!ok) break;
-            mbar_expect_tx(do_full + s, nb * C::TILE_BYTES);
-            for (int e = 0; e < nb; ++e)
-              for (int pn = 0; pn < C::NPANEL; ++pn)
-                tma_load_4d(smem + C::OFF_DO + s * C::STAGE_BYTES + e * C::TILE_BYTES + pn * C::PANEL_BYTES, &mdo,
-                            do_full + s, pn * 64, I * BLK, h, b + e);
+            if constexpr (C::NPANEL == 1) {
+              mbar_expect_tx(do_full + s, C::STAGE_BYTES);   // (the map's box spans the stage's SB batch entries)
+              tma_load_4d(smem + C::OFF_DO + s * C::STAGE_BYTES, &mdo, do_full + s, 0, I * BLK, h, b);
+            } else {
+              mbar_expect_tx(do_full + s, nb * C::TILE_BYTES);
+              for (int e = 0; e < nb; ++e)
+                for (int pn = 0; pn < C::NPANEL; ++pn)
+                  tma_load_4d(smem + C::OFF_DO + s * C::STAGE_BYTES + e * C::TILE_BYTES + pn * C::PANEL_BYTES, &mdo,
+                              do_full + s, pn * 64, I * BLK, h, b + e);
+            }
             ++ndo;
           }
         }
