@@ -286,7 +286,7 @@ void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward,
 void sched_defaults(int wide, int backward, int* frozen_pct, int* overhead_pct) {
   if (backward) {
     *frozen_pct = 20;
-    *overhead_pct = wide ? 200 : 100;
+    *overhead_pct = wide ? 200 : 150;   // (a trace puts the item boundary of the 64-wide backward at ~1.6 tiles)
   } else {
     *frozen_pct = wide ? 50 : 30;
     *overhead_pct = wide ? 300 : 150;
