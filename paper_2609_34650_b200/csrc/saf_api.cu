@@ -235,7 +235,7 @@ int upload_mask(saf_ctx* ctx, const uint8_t* mask, int H, cudaStream_t st) {
 // end, and each item goes to the CTA that becomes free first (list scheduling, which is what a dynamic
 // queue would do); only the last items are ordered longest-first so that the tail stays short.
 void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward, int n_ctas, int frozen_pct,
-                         int overhead_pct, int second_wave_pct, std::vector<WorkItem>& items,
+                         int overhead_pct, int overhead_frozen_pct, int second_wave_pct, std::vector<WorkItem>& items,
                          std::vector<int>& offsets, std::vector<WorkItem>* order = nullptr) {
   const int nblk = (T + BLK - 1) / BLK;
   struct Cand { WorkItem w; long long cost; };
@@ -249,7 +249,9 @@ void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward,
         const int r = (z & 1) ? (nblk - 1 - z / 2) : (z / 2);        // rank by cost, 0 = most expensive
         const int k = backward ? r : (nblk - 1 - r);
         const long long tiles = backward ? (nblk - k) : (k + 1);
-        const long long cost = tiles * (kind == KIND_FROZEN ? frozen_pct : 100) + overhead_pct;   // + fixed per-item overhead
+        // + fixed per-item overhead
+        const long long cost = tiles * (kind == KIND_FROZEN ? frozen_pct : 100) +
+                               (kind == KIND_FROZEN ? overhead_frozen_pct : overhead_pct);
         cand.push_back({{b, h, k, kind}, cost});
       }
     }
@@ -283,13 +285,14 @@ void build_worklist_host(int B, int H, int T, const uint8_t* mask, int backward,
 }
 
 // Measured cost-model defaults: `wide` = the 128-wide kernels (head dimension 96 or 128), else the 64-wide ones.
-void sched_defaults(int wide, int backward, int* frozen_pct, int* overhead_pct) {
+void sched_defaults(int wide, int backward, int* frozen_pct, int* overhead_pct, int* overhead_frozen_pct) {
   if (backward) {
     *frozen_pct = 20;
     *overhead_pct = wide ? 200 : 150;   // (a trace puts the item boundary of the 64-wide backward at ~1.6 tiles)
+    *overhead_frozen_pct = wide ? 200 : 100;   // (a frozen item ends with half the epilogue: dV only)
   } else {
     *frozen_pct = wide ? 50 : 30;
-    *overhead_pct = wide ? 300 : 150;
+    *overhead_pct = *overhead_frozen_pct = wide ? 300 : 150;
   }
 }
 
@@ -310,16 +313,16 @@ int get_worklist(saf_ctx* ctx, int B, int H, int T, const uint8_t* mask, int bac
   }
   std::vector<WorkItem> items;
   std::vector<int> offsets;
-  int frozen_pct, overhead_pct;
-  sched_defaults(wide, backward, &frozen_pct, &overhead_pct);
+  int frozen_pct, overhead_pct, overhead_frozen_pct;
+  sched_defaults(wide, backward, &frozen_pct, &overhead_pct, &overhead_frozen_pct);
   const int fw = backward ? ctx->frozen_weight_bwd_pct : ctx->frozen_weight_pct;
   const int ov = backward ? ctx->item_overhead_bwd_pct : ctx->item_overhead_pct;
   if (fw > 0) frozen_pct = fw;
-  if (ov > 0) overhead_pct = ov;
+  if (ov > 0) overhead_pct = overhead_frozen_pct = ov;   // (the override sets both kinds)
   const int second_wave = backward ? 0 : (ctx->second_wave_pct >= 0 ? ctx->second_wave_pct : (wide ? 6 : 20));
   WorklistEntry e;
-  build_worklist_host(B, H, T, mask, backward, grid, frozen_pct, overhead_pct, second_wave, items, offsets,
-                      &e.order_host);
+  build_worklist_host(B, H, T, mask, backward, grid, frozen_pct, overhead_pct, overhead_frozen_pct, second_wave, items,
+                      offsets, &e.order_host);
   e.B = B; e.H = H; e.T = T; e.backward = backward; e.grid = grid; e.wide = wide;
   e.mask.assign(mask, mask + H);
   e.n_items = static_cast<int>(items.size());
@@ -1370,8 +1373,9 @@ int saf_build_worklist(int32_t B, int32_t H, int32_t T, const uint8_t* frozen_ma
     return SAF_ERR_INVALID_ARG;
   std::vector<WorkItem> items;
   std::vector<int> offsets;
-  build_worklist_host(B, H, T, frozen_mask_host, backward ? 1 : 0, n_ctas, frozen_weight_pct, backward ? 100 : 150, 0,
-                      items, offsets);
+  int fp_unused, ov, ovf;
+  sched_defaults(0, backward ? 1 : 0, &fp_unused, &ov, &ovf);      // the 64-wide kernels' per-item overheads
+  build_worklist_host(B, H, T, frozen_mask_host, backward ? 1 : 0, n_ctas, frozen_weight_pct, ov, ovf, 0, items, offsets);
   std::memcpy(items_out, items.data(), items.size() * sizeof(WorkItem));
   std::memcpy(offsets_out, offsets.data(), offsets.size() * sizeof(int));
   return SAF_OK;
